@@ -1,0 +1,165 @@
+/*
+ * attn_fp8.h -- C ABI of the FP8 Delta-Matching attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes causal / grouped-query softmax attention forward and backward with
+ * block-scaled FP8 operands in every attention-core matmul (paper Section 2.3:
+ * S = Q K^T * scale, P = softmax(S), O = P V, dV = P^T dO, dP = dO V^T, dS = P o (dP - delta),
+ * dQ = dS K * scale, dK = dS^T Q * scale).  The backward row correction delta is recomputed
+ * as rowsum(P o dP) from the unquantised probabilities and the FP32 product of the same FP8
+ * dO and V the gradient pass consumes ("Delta-Matching", paper Section 3.3, Eq. 4-5), so
+ * that dS keeps zero row sums; the saved-output shortcut rowsum(dO o O) ("stale delta",
+ * Section 3.2) is selectable as an ablation.
+ *
+ * Number format.  Operands are E4M3 codes (round to nearest even, saturating at +-448; paper
+ * Appendix "Operands, Scaling, and Accumulation") with one E8M0 scale byte (value 2^(byte-127))
+ * per 32 consecutive elements ALONG THE CONTRACTION DIMENSION of the matmul that consumes the
+ * operand.  Every input tensor therefore exists in up to two quantised copies:
+ *   "row" copy: blocks along the channel dim d      (used when the matmul contracts over d)
+ *   "col" copy: blocks along the token dim N, stored transposed (used when it contracts over N)
+ * The scale of a block is the smallest power of two that maps the block maximum to <= 448.
+ *
+ * Conventions.
+ *   - Every pointer is a DEVICE pointer unless stated otherwise; all tensors are contiguous.
+ *   - The caller owns every buffer.  The library allocates nothing and frees nothing.
+ *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*) and returns;
+ *     it never synchronises and never reads device memory from the host, except
+ *     attn_fp8_read_status, which says so.
+ *   - Errors are return codes; nothing aborts or traps.  Arguments are validated before any
+ *     launch.  attn_fp8_last_error() gives a thread-local message for the last failure.
+ *   - Results of quantize, fwd, bwd_delta and bwd are bitwise reproducible run to run.
+ *   - Changing delta_mode changes only `delta`, dQ and dK -- never O, LSE or dV.
+ *
+ * Supported shapes: seqlen a multiple of 128 (Nq == Nk, causal means key j <= query i);
+ * heads_q a multiple of heads_kv; head dims: (qk, v) in {(64,64), (128,128)} for the
+ * attention entry points; the quantiser accepts any d that is a multiple of 32 up to 256.
+ */
+#ifndef ATTN_FP8_H_
+#define ATTN_FP8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ATTN_OK = 0,
+  ATTN_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, heads_q % heads_kv != 0 ...  */
+  ATTN_ERR_UNSUPPORTED = 2,   /* shape / precision / mode outside the supported set             */
+  ATTN_ERR_ALIGNMENT = 3,     /* a pointer is not 16-byte aligned                               */
+  ATTN_ERR_WORKSPACE = 4,     /* workspace missing or smaller than attn_fp8_workspace_bytes()   */
+  ATTN_ERR_ARCH = 5,          /* current device is not compute capability 10.x                  */
+  ATTN_ERR_CUDA = 6,          /* a CUDA runtime / driver call failed; see attn_fp8_last_error   */
+  ATTN_ERR_TIMEOUT = 7        /* a bounded device-side wait expired (reported by read_status)   */
+} attn_status_t;
+
+typedef enum { ATTN_PREC_MXFP8 = 0, ATTN_PREC_BF16 = 1 } attn_precision_t;
+typedef enum { ATTN_DELTA_MATCHED = 0, ATTN_DELTA_STALE = 1 } attn_delta_mode_t;
+typedef enum { ATTN_SRC_BF16 = 0, ATTN_SRC_FP32 = 1 } attn_src_dtype_t;
+typedef enum { ATTN_WS_FWD = 0, ATTN_WS_BWD_DELTA = 1, ATTN_WS_BWD = 2 } attn_ws_kind_t;
+
+/* Problem description shared by the attention entry points.
+ * Tensors: Q, dO, O, dQ are [batch, heads_q, seqlen, dim]; K, V, dK, dV are
+ * [batch, heads_kv, seqlen, dim]; LSE, delta and the diagnostics are [batch, heads_q, seqlen].
+ * Query head h reads KV head h / (heads_q / heads_kv).                                        */
+typedef struct {
+  int32_t batch, seqlen, heads_q, heads_kv, head_dim_qk, head_dim_v;
+  int32_t causal;          /* 0 or 1                                                          */
+  float   softmax_scale;   /* multiplies the FP32 score accumulator; NOT folded into Q         */
+  int32_t precision;       /* attn_precision_t                                                 */
+  int32_t delta_mode;      /* attn_delta_mode_t (read by attn_fp8_bwd_delta only)              */
+} attn_params_t;
+
+/* One quantised tensor X [B, H, N, d] (caller-allocated device memory).
+ *
+ *   row_codes  uint8 [B, H, N, d]          E4M3 code of X[b,h,n,c], blocks = 32 channels
+ *   col_codes  uint8 [B, H, d, N]          E4M3 code of X[b,h,n,c] at [b,h,c,n], blocks = 32 tokens
+ *   row_scales uint8 [B, H, N/128, ceil(d/128), 512]
+ *   col_scales uint8 [B, H, ceil(d/128), N/128, 512]
+ *
+ * Scale bytes are stored in 512-byte tiles, the order in which the tensor cores take them
+ * from tensor memory.  A tile covers 128 rows x 4 blocks of the scaled matrix (row copy: rows
+ * are tokens, blocks run along d; col copy: rows are channels, blocks run along N).  Inside
+ * a tile, the byte of (row r, block k) sits at offset  (r % 32) * 16 + ((r % 128) / 32) * 4 + (k % 4);
+ * tiles are ordered [r / 128][k / 4].  Bytes of rows or blocks beyond the tensor are 0.
+ * attn_fp8_scale_offset() below returns this offset so that callers need not restate it.
+ *
+ * Either pair may be NULL when that orientation is not needed by the call.                    */
+typedef struct {
+  uint8_t *row_codes, *row_scales;
+  uint8_t *col_codes, *col_scales;
+} attn_qtensor_t;
+
+/* Byte offset, inside one (b, h) slab of a scale tensor, of the scale of (row, block) for a
+ * scaled matrix with `n_blocks` blocks per row.  Pure host arithmetic.                        */
+size_t attn_fp8_scale_offset(int64_t row, int64_t block, int64_t n_blocks);
+
+/* Bytes of one scale tensor (all B*H slabs) for a scaled matrix of `rows` x (`cols`/32 blocks):
+ * row copy: rows = N, cols = d; col copy: rows = d, cols = N.                                 */
+size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols);
+
+/* Block-scaling quantiser (paper Appendix "Operands, Scaling, and Accumulation", Eq.
+ * app_kernel_quantizer, with the FP32 scale amax/448 replaced by an E8M0 scale per 1x32 block).
+ *   src        [B, H, N, d] in `src_dtype` (BF16 or FP32), device memory, 16-byte aligned
+ *   out        the orientations whose pointers are non-NULL are written (codes AND scales of an
+ *              orientation must both be given); all 16-byte aligned
+ *   N % 128 == 0, d % 32 == 0, 32 <= d <= 256.
+ * Non-finite inputs do not trap: NaN encodes as 0x7F, +-Inf saturates to +-448.               */
+attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
+                                int32_t d, attn_qtensor_t out, void* stream);
+
+/* Forward (paper Appendix "Forward Probability Encoding"): per query row, online softmax of
+ * S = scale * Q^ K^^T over key tiles with a running INTEGER power-of-two shift, normaliser l
+ * taken from the exponentials BEFORE the FP8 cast, probabilities quantised in-register in
+ * blocks of 32 keys, O = (P^ V^) / l.
+ *   reads   q.row_*, k.row_*, v.col_*
+ *   writes  o_bf16 [B, Hq, N, dv] (BF16), lse [B, Hq, N] (FP32, natural log)                  */
+attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                           void* o_bf16, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Row correction (paper Section 3.3 Eq. 4; Appendix "Backward Correction and Gradient
+ * Computation", paragraph "Matched correction").
+ *   MATCHED: delta_i = sum_j P_ij dP^_ij with P_ij = exp(S_ij - LSE_i) unquantised FP32 and
+ *            dP^ = dO^ V^^T accumulated in FP32 from FP8 operands.
+ *            reads q.row_*, k.row_*, v.row_*, dO.row_*, lse.  dO_bf16 / o_bf16 are ignored.
+ *   STALE:   delta_i = sum_c dO_ic O_ic from BF16 dO and the saved BF16 O (both [B,Hq,N,dv]).
+ *            reads dO_bf16, o_bf16 only.
+ *   writes  delta [B, Hq, N] (FP32)                                                           */
+attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                 attn_qtensor_t dO, const void* dO_bf16, const void* o_bf16,
+                                 const float* lse, float* delta,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* Gradient pass (same Appendix, paragraphs "Score-gradient quantization" and "Query
+ * gradients"): recomputes S and dP^ from the FP8 operands, P = exp(S - LSE) and
+ * dS = P o (dP^ - delta) in FP32, quantises P and dS in-register along each contraction
+ * dimension and accumulates dV = P^^T dO^, dK = scale dS^^T Q^, dQ = scale dS^ K^; dK and dV are
+ * summed over the query heads of each KV group in FP32 before the BF16 store.
+ *   reads   q.row_*, q.col_*, k.row_*, k.col_*, v.row_*, dO.row_*, dO.col_*, lse, delta
+ *   writes  dq_bf16 [B,Hq,N,dqk], dk_bf16 [B,Hkv,N,dqk], dv_bf16 [B,Hkv,N,dv] (BF16)
+ *   diag_rowsum_ds / diag_rowsum_abs_ds: optional [B,Hq,N] FP32 outputs, sum_j dS_ij and
+ *   sum_j |dS_ij| taken before the FP8 cast (the paper's row-sum residual probe); may be NULL. */
+attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                           attn_qtensor_t dO, const float* lse, const float* delta,
+                           void* dq_bf16, void* dk_bf16, void* dv_bf16,
+                           float* diag_rowsum_ds, float* diag_rowsum_abs_ds,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of workspace the given entry point needs for `p` (attn_ws_kind_t).  The workspace is
+ * scratch: contents are undefined between calls, the library clears what it needs.  Its first
+ * word is the device-side status that attn_fp8_read_status returns.                           */
+size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which);
+
+/* Waits for `stream`, copies the status word of `workspace` to the host and returns it:
+ * ATTN_OK, or ATTN_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs of that
+ * call are then undefined).  This is the one call that synchronises.                          */
+attn_status_t attn_fp8_read_status(const void* workspace, void* stream);
+
+/* Message for the last non-OK return on this host thread (static storage; never NULL).        */
+const char* attn_fp8_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_FP8_H_ */

@@ -1,0 +1,242 @@
+"""ctypes binding of ``libattnfp8.so`` -- same entry-point names as ``include/attn_fp8.h``.
+
+Argument marshalling only: tensors are torch CUDA tensors whose device pointers
+are handed to the C ABI; every step of the attention path runs in the
+library's kernels.  Importing this module fails loudly when the library has
+not been built (``python -m paper_2609_37852_b200.build``): there is no
+fallback path.
+"""
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libattnfp8.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build the CUDA library first (python -m paper_2609_37852_b200.build); "
+        "this package has no CPU or eager fallback")
+_lib = ctypes.CDLL(LIB_PATH)
+
+ATTN_OK = 0
+STATUS_NAMES = {0: "ATTN_OK", 1: "ATTN_ERR_INVALID_ARG", 2: "ATTN_ERR_UNSUPPORTED", 3: "ATTN_ERR_ALIGNMENT",
+                4: "ATTN_ERR_WORKSPACE", 5: "ATTN_ERR_ARCH", 6: "ATTN_ERR_CUDA", 7: "ATTN_ERR_TIMEOUT"}
+ATTN_PREC_MXFP8, ATTN_PREC_BF16 = 0, 1
+ATTN_DELTA_MATCHED, ATTN_DELTA_STALE = 0, 1
+ATTN_SRC_BF16, ATTN_SRC_FP32 = 0, 1
+ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
+
+EXPORTED_SYMBOLS = (
+    "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta",
+    "attn_fp8_bwd", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
+)
+
+
+class AttnFp8Error(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("seqlen", ctypes.c_int32), ("heads_q", ctypes.c_int32),
+                ("heads_kv", ctypes.c_int32), ("head_dim_qk", ctypes.c_int32), ("head_dim_v", ctypes.c_int32),
+                ("causal", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("precision", ctypes.c_int32),
+                ("delta_mode", ctypes.c_int32)]
+
+
+class _QTensor(ctypes.Structure):
+    _fields_ = [("row_codes", ctypes.c_void_p), ("row_scales", ctypes.c_void_p),
+                ("col_codes", ctypes.c_void_p), ("col_scales", ctypes.c_void_p)]
+
+
+_vp, _i32, _sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+_lib.attn_fp8_scale_offset.restype = _sz
+_lib.attn_fp8_scale_offset.argtypes = [ctypes.c_int64] * 3
+_lib.attn_fp8_scale_bytes.restype = _sz
+_lib.attn_fp8_scale_bytes.argtypes = [ctypes.c_int64] * 4
+_lib.attn_fp8_quantize.restype = _i32
+_lib.attn_fp8_quantize.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _QTensor, _vp]
+_lib.attn_fp8_fwd.restype = _i32
+_lib.attn_fp8_fwd.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _vp, _vp, _vp, _sz, _vp]
+_lib.attn_fp8_bwd_delta.restype = _i32
+_lib.attn_fp8_bwd_delta.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp,
+                                    _vp, _vp, _sz, _vp]
+_lib.attn_fp8_bwd.restype = _i32
+_lib.attn_fp8_bwd.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp, _vp,
+                              _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.attn_fp8_workspace_bytes.restype = _sz
+_lib.attn_fp8_workspace_bytes.argtypes = [ctypes.POINTER(_Params), _i32]
+_lib.attn_fp8_read_status.restype = _i32
+_lib.attn_fp8_read_status.argtypes = [_vp, _vp]
+_lib.attn_fp8_last_error.restype = ctypes.c_char_p
+_lib.attn_fp8_last_error.argtypes = []
+
+
+def attn_fp8_last_error() -> str:
+    return _lib.attn_fp8_last_error().decode()
+
+
+def _check(status):
+    if status != ATTN_OK:
+        raise AttnFp8Error(status, attn_fp8_last_error())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+@dataclass
+class AttnParams:
+    batch: int
+    seqlen: int
+    heads_q: int
+    heads_kv: int
+    head_dim_qk: int
+    head_dim_v: int
+    causal: bool
+    softmax_scale: float
+    precision: int = ATTN_PREC_MXFP8
+    delta_mode: int = ATTN_DELTA_MATCHED
+
+    def c_struct(self) -> _Params:
+        return _Params(self.batch, self.seqlen, self.heads_q, self.heads_kv, self.head_dim_qk, self.head_dim_v,
+                       int(self.causal), float(self.softmax_scale), self.precision, self.delta_mode)
+
+
+@dataclass
+class QTensor:
+    """Device buffers of one quantised tensor [B, H, N, d] (see attn_qtensor_t)."""
+    shape: tuple
+    row_codes: Optional[torch.Tensor] = None
+    row_scales: Optional[torch.Tensor] = None
+    col_codes: Optional[torch.Tensor] = None
+    col_scales: Optional[torch.Tensor] = None
+
+    def c_struct(self) -> _QTensor:
+        return _QTensor(*(None if t is None else t.data_ptr()
+                          for t in (self.row_codes, self.row_scales, self.col_codes, self.col_scales)))
+
+
+def attn_fp8_scale_offset(row: int, block: int, n_blocks: int) -> int:
+    return int(_lib.attn_fp8_scale_offset(row, block, n_blocks))
+
+
+def attn_fp8_scale_bytes(B: int, H: int, rows: int, cols: int) -> int:
+    return int(_lib.attn_fp8_scale_bytes(B, H, rows, cols))
+
+
+def unpack_scales(scales: torch.Tensor, B: int, H: int, rows: int, cols: int) -> torch.Tensor:
+    """Reorders a tiled scale tensor into plain [B, H, rows, cols/32] (a pure index permutation,
+    the inverse of the offset rule documented for attn_qtensor_t)."""
+    nb = cols // 32
+    r = np.arange(rows)[:, None]
+    k = np.arange(nb)[None, :]
+    off = ((r // 128) * ((nb + 3) // 4) + k // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + (k % 4)
+    idx = torch.from_numpy(off.reshape(-1)).to(scales.device)
+    slab = scales.reshape(B * H, -1)
+    return slab[:, idx].reshape(B, H, rows, nb)
+
+
+def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None) -> QTensor:
+    """Quantise ``src`` [B, H, N, d] (BF16 or FP32, CUDA, contiguous) into the requested orientations."""
+    if not src.is_cuda or not src.is_contiguous() or src.dim() != 4:
+        raise ValueError("src must be a contiguous CUDA tensor [B, H, N, d]")
+    if src.dtype == torch.bfloat16:
+        dt = ATTN_SRC_BF16
+    elif src.dtype == torch.float32:
+        dt = ATTN_SRC_FP32
+    else:
+        raise ValueError("src must be bfloat16 or float32")
+    B, H, N, d = src.shape
+    out = QTensor(shape=(B, H, N, d))
+    u8 = dict(dtype=torch.uint8, device=src.device)
+    if want_row:
+        out.row_codes = torch.empty((B, H, N, d), **u8)
+        out.row_scales = torch.empty(attn_fp8_scale_bytes(B, H, N, d), **u8)
+    if want_col:
+        out.col_codes = torch.empty((B, H, d, N), **u8)
+        out.col_scales = torch.empty(attn_fp8_scale_bytes(B, H, d, N), **u8)
+    _check(_lib.attn_fp8_quantize(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
+    return out
+
+
+def attn_fp8_workspace_bytes(params: AttnParams, which: int) -> int:
+    c = params.c_struct()
+    return int(_lib.attn_fp8_workspace_bytes(ctypes.byref(c), which))
+
+
+def _workspace(params, which, workspace, device):
+    need = attn_fp8_workspace_bytes(params, which)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace
+
+
+def attn_fp8_read_status(workspace: torch.Tensor, stream=None) -> None:
+    """Synchronises ``stream`` and raises if a kernel of the last call reported a timeout."""
+    _check(_lib.attn_fp8_read_status(_ptr(workspace), _stream(stream)))
+
+
+def attn_fp8_fwd(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, o=None, lse=None, workspace=None,
+                 stream=None):
+    """Returns (O [B,Hq,N,dv] bf16, LSE [B,Hq,N] fp32, workspace)."""
+    dev = q.row_codes.device
+    if o is None:
+        o = torch.empty((params.batch, params.heads_q, params.seqlen, params.head_dim_v), dtype=torch.bfloat16, device=dev)
+    if lse is None:
+        lse = torch.empty((params.batch, params.heads_q, params.seqlen), dtype=torch.float32, device=dev)
+    workspace = _workspace(params, ATTN_WS_FWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_fwd(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), _ptr(o), _ptr(lse),
+                             _ptr(workspace), workspace.numel(), _stream(stream)))
+    return o, lse, workspace
+
+
+def attn_fp8_bwd_delta(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, dO_bf16=None,
+                       o_bf16=None, delta=None, workspace=None, stream=None):
+    """Returns (delta [B,Hq,N] fp32, workspace).  ``params.delta_mode`` selects matched / stale."""
+    dev = lse.device
+    if delta is None:
+        delta = torch.empty((params.batch, params.heads_q, params.seqlen), dtype=torch.float32, device=dev)
+    workspace = _workspace(params, ATTN_WS_BWD_DELTA, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd_delta(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),
+                                   _ptr(dO_bf16), _ptr(o_bf16), _ptr(lse), _ptr(delta), _ptr(workspace),
+                                   workspace.numel(), _stream(stream)))
+    return delta, workspace
+
+
+def attn_fp8_bwd(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dq=None, dk=None,
+                 dv=None, diagnostics: bool = False, workspace=None, stream=None):
+    """Returns (dQ, dK, dV, rowsum_dS or None, rowsum_abs_dS or None, workspace)."""
+    dev = lse.device
+    bf = dict(dtype=torch.bfloat16, device=dev)
+    B, N = params.batch, params.seqlen
+    if dq is None:
+        dq = torch.empty((B, params.heads_q, N, params.head_dim_qk), **bf)
+    if dk is None:
+        dk = torch.empty((B, params.heads_kv, N, params.head_dim_qk), **bf)
+    if dv is None:
+        dv = torch.empty((B, params.heads_kv, N, params.head_dim_v), **bf)
+    rs = ra = None
+    if diagnostics:
+        rs = torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev)
+        ra = torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev)
+    workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(), _ptr(lse),
+                             _ptr(delta), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(rs), _ptr(ra), _ptr(workspace),
+                             workspace.numel(), _stream(stream)))
+    return dq, dk, dv, rs, ra, workspace

@@ -1,0 +1,218 @@
+// C-ABI entry points: argument validation, workspace handling, dispatch to the kernel launchers.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace attnfp8 {
+
+static thread_local char g_last_error[512] = "no error";
+
+attn_status_t fail(attn_status_t code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+attn_status_t encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
+                                   uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {128, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return ATTN_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static attn_status_t check_device() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+  if (major != 10) return fail(ATTN_ERR_ARCH, "device compute capability %d.x is not 10.x (sm_100a)", major);
+  return ATTN_OK;
+}
+
+static attn_status_t check_params(const attn_params_t* p, AttnShape* s) {
+  if (!p) return fail(ATTN_ERR_INVALID_ARG, "params is NULL");
+  if (p->batch <= 0 || p->seqlen <= 0 || p->heads_q <= 0 || p->heads_kv <= 0)
+    return fail(ATTN_ERR_INVALID_ARG, "batch, seqlen and head counts must be positive");
+  if (p->heads_q % p->heads_kv) return fail(ATTN_ERR_INVALID_ARG, "heads_q must be a multiple of heads_kv");
+  if (p->causal != 0 && p->causal != 1) return fail(ATTN_ERR_INVALID_ARG, "causal must be 0 or 1");
+  if (!(p->softmax_scale > 0.f)) return fail(ATTN_ERR_INVALID_ARG, "softmax_scale must be positive");
+  if (p->precision != ATTN_PREC_MXFP8)
+    return fail(ATTN_ERR_UNSUPPORTED, "precision %d: only ATTN_PREC_MXFP8 is built", p->precision);
+  if (p->seqlen % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen must be a multiple of 128");
+  const bool dims_ok = (p->head_dim_qk == 64 && p->head_dim_v == 64) || (p->head_dim_qk == 128 && p->head_dim_v == 128);
+  if (!dims_ok)
+    return fail(ATTN_ERR_UNSUPPORTED, "head dims (%d, %d): supported are (64,64) and (128,128)", p->head_dim_qk,
+                p->head_dim_v);
+  *s = AttnShape{p->batch, p->seqlen, p->heads_q, p->heads_kv, p->head_dim_qk, p->head_dim_v, p->causal,
+                 p->softmax_scale};
+  return ATTN_OK;
+}
+
+static attn_status_t check_ptr(const void* p, const char* name) {
+  if (!p) return fail(ATTN_ERR_INVALID_ARG, "%s is NULL", name);
+  if (!aligned16(p)) return fail(ATTN_ERR_ALIGNMENT, "%s is not 16-byte aligned", name);
+  return ATTN_OK;
+}
+
+#define CHECK(x)                        \
+  do {                                  \
+    attn_status_t st_ = (x);            \
+    if (st_ != ATTN_OK) return st_;     \
+  } while (0)
+
+static attn_status_t prepare_workspace(void* ws, size_t ws_bytes, size_t need, cudaStream_t stream, int** status) {
+  if (!ws || ws_bytes < need) return fail(ATTN_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+  if (!aligned16(ws)) return fail(ATTN_ERR_ALIGNMENT, "workspace is not 16-byte aligned");
+  cudaError_t e = cudaMemsetAsync(ws, 0, kWorkspaceHeaderBytes, stream);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "cudaMemsetAsync(workspace): %s", cudaGetErrorString(e));
+  *status = static_cast<int*>(ws);
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8
+
+using namespace attnfp8;
+
+extern "C" {
+
+size_t attn_fp8_scale_offset(int64_t row, int64_t block, int64_t n_blocks) {
+  const int64_t tiles_per_row_tile = (n_blocks + 3) / 4;
+  const int64_t tile = (row / 128) * tiles_per_row_tile + block / 4;
+  return static_cast<size_t>(tile * 512 + (row % 32) * 16 + ((row % 128) / 32) * 4 + (block % 4));
+}
+
+size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols) {
+  return static_cast<size_t>(B * H) * scale_tiles_per_slab(rows, cols) * 512;
+}
+
+attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
+                                attn_qtensor_t out, void* stream) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return fail(ATTN_ERR_INVALID_ARG, "sizes must be positive");
+  if (src_dtype != ATTN_SRC_BF16 && src_dtype != ATTN_SRC_FP32)
+    return fail(ATTN_ERR_INVALID_ARG, "src_dtype %d is neither BF16 nor FP32", src_dtype);
+  if (N % 128 || d % 32 || d > 256)
+    return fail(ATTN_ERR_UNSUPPORTED, "quantize needs N %% 128 == 0 and d %% 32 == 0, d <= 256 (N=%d d=%d)", N, d);
+  CHECK(check_ptr(src, "src"));
+  if (!out.row_codes && !out.col_codes) return fail(ATTN_ERR_INVALID_ARG, "no output orientation requested");
+  if ((out.row_codes == nullptr) != (out.row_scales == nullptr) ||
+      (out.col_codes == nullptr) != (out.col_scales == nullptr))
+    return fail(ATTN_ERR_INVALID_ARG, "codes and scales of an orientation must be given together");
+  if (out.row_codes) { CHECK(check_ptr(out.row_codes, "row_codes")); CHECK(check_ptr(out.row_scales, "row_scales")); }
+  if (out.col_codes) { CHECK(check_ptr(out.col_codes, "col_codes")); CHECK(check_ptr(out.col_scales, "col_scales")); }
+  CHECK(check_device());
+  return launch_quantize(src, src_dtype, B, H, N, d, out, static_cast<cudaStream_t>(stream));
+}
+
+size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which) {
+  (void)p;
+  (void)which;
+  return kWorkspaceHeaderBytes;
+}
+
+attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                           void* o_bf16, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  AttnShape s;
+  CHECK(check_params(p, &s));
+  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
+  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
+  CHECK(check_ptr(v.col_codes, "v.col_codes")); CHECK(check_ptr(v.col_scales, "v.col_scales"));
+  CHECK(check_ptr(o_bf16, "o_bf16")); CHECK(check_ptr(lse, "lse"));
+  CHECK(check_device());
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_FWD), st, &status));
+  return launch_fwd(s, q, k, v, o_bf16, lse, status, st);
+}
+
+attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                 attn_qtensor_t dO, const void* dO_bf16, const void* o_bf16, const float* lse,
+                                 float* delta, void* workspace, size_t workspace_bytes, void* stream) {
+  AttnShape s;
+  CHECK(check_params(p, &s));
+  CHECK(check_ptr(delta, "delta"));
+  CHECK(check_device());
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD_DELTA), st, &status));
+  if (p->delta_mode == ATTN_DELTA_STALE) {
+    CHECK(check_ptr(dO_bf16, "dO_bf16")); CHECK(check_ptr(o_bf16, "o_bf16"));
+    return launch_stale_delta(s, dO_bf16, o_bf16, delta, st);
+  }
+  if (p->delta_mode != ATTN_DELTA_MATCHED) return fail(ATTN_ERR_INVALID_ARG, "delta_mode %d unknown", p->delta_mode);
+  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
+  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
+  CHECK(check_ptr(v.row_codes, "v.row_codes")); CHECK(check_ptr(v.row_scales, "v.row_scales"));
+  CHECK(check_ptr(dO.row_codes, "dO.row_codes")); CHECK(check_ptr(dO.row_scales, "dO.row_scales"));
+  CHECK(check_ptr(lse, "lse"));
+  return launch_bwd_delta(s, q, k, v, dO, lse, delta, status, st);
+}
+
+attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                           attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
+                           void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  AttnShape s;
+  CHECK(check_params(p, &s));
+  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
+  CHECK(check_ptr(q.col_codes, "q.col_codes")); CHECK(check_ptr(q.col_scales, "q.col_scales"));
+  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
+  CHECK(check_ptr(k.col_codes, "k.col_codes")); CHECK(check_ptr(k.col_scales, "k.col_scales"));
+  CHECK(check_ptr(v.row_codes, "v.row_codes")); CHECK(check_ptr(v.row_scales, "v.row_scales"));
+  CHECK(check_ptr(dO.row_codes, "dO.row_codes")); CHECK(check_ptr(dO.row_scales, "dO.row_scales"));
+  CHECK(check_ptr(dO.col_codes, "dO.col_codes")); CHECK(check_ptr(dO.col_scales, "dO.col_scales"));
+  CHECK(check_ptr(lse, "lse")); CHECK(check_ptr(delta, "delta"));
+  CHECK(check_ptr(dq_bf16, "dq_bf16")); CHECK(check_ptr(dk_bf16, "dk_bf16")); CHECK(check_ptr(dv_bf16, "dv_bf16"));
+  if ((diag_rowsum_ds == nullptr) != (diag_rowsum_abs_ds == nullptr))
+    return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
+  CHECK(check_device());
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD), st, &status));
+  CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, status, st));
+  return launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st);
+}
+
+attn_status_t attn_fp8_read_status(const void* workspace, void* stream) {
+  if (!workspace) return fail(ATTN_ERR_INVALID_ARG, "workspace is NULL");
+  int host = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "read_status: %s", cudaGetErrorString(e));
+  if (host != 0) return fail(ATTN_ERR_TIMEOUT, "a bounded device-side wait expired (status word %d)", host);
+  return ATTN_OK;
+}
+
+const char* attn_fp8_last_error(void) { return g_last_error; }
+
+}  // extern "C"

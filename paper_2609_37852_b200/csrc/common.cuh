@@ -1,0 +1,49 @@
+// Declarations shared by the kernels' translation units and the C-ABI layer.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/attn_fp8.h"
+
+namespace attnfp8 {
+
+// Records a message for attn_fp8_last_error() and returns `code`.
+attn_status_t fail(attn_status_t code, const char* fmt, ...);
+
+// Bytes at the head of every workspace reserved for the device status word.
+constexpr size_t kWorkspaceHeaderBytes = 256;
+
+// cuTensorMapEncodeTiled fetched through the runtime (no link-time dependency on libcuda).
+// Encodes a 2-D uint8 tensor [rows, row_bytes] (row pitch == row_bytes) with a
+// (box_rows x 128-byte) box and the 128-byte swizzle.
+attn_status_t encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
+                                   uint32_t box_rows);
+
+struct AttnShape {
+  int B, N, Hq, Hkv, dqk, dv, causal;
+  float scale;
+};
+
+// Kernel launchers (each validates nothing: the C-ABI layer has done so).
+attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
+                              cudaStream_t stream);
+attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
+                         float* lse, int* status, cudaStream_t stream);
+attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                               attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream);
+attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,
+                                 cudaStream_t stream);
+attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                            attn_qtensor_t dO, const float* lse, const float* delta, void* dq, float* rowsum,
+                            float* rowabs, int* status, cudaStream_t stream);
+attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                              attn_qtensor_t dO, const float* lse, const float* delta, void* dk, void* dv,
+                              int* status, cudaStream_t stream);
+
+inline size_t scale_tiles_per_slab(int64_t rows, int64_t cols) {
+  return static_cast<size_t>((rows + 127) / 128) * static_cast<size_t>((cols / 32 + 3) / 4);
+}
+
+}  // namespace attnfp8

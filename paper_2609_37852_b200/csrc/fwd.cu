@@ -1,0 +1,323 @@
+// Forward attention with block-scaled FP8 operands (paper Appendix "Forward Probability
+// Encoding", re-designed for tcgen05 / tensor memory).
+//
+// One CTA owns 128 query rows of one (batch, query head) and walks the key tiles (128 keys) up
+// to the causal diagonal.  Warp roles:
+//   warp 0      TMA producer: Q tile once, then K tiles and V tiles through two rings
+//   warp 1      MMA issuer (one elected lane): S = Q K^T and O += P V, both block-scaled,
+//               accumulating in tensor memory; S is double-buffered so that the scores of
+//               tile t+1 are computed while the softmax warps work on tile t
+//   warps 4..7  softmax: one query row per thread (thread <-> TMEM lane).  Scores are scaled
+//               into log2 units; the running shift M is an INTEGER, so rescaling is by exact
+//               powers of two and the E4M3 codes of the probabilities do not depend on the
+//               tile order; l accumulates the exponentials BEFORE the FP8 cast; probabilities
+//               are quantised in blocks of 32 keys in registers and written back to tensor
+//               memory (over the S buffer) as the A operand of the second MMA, their scale
+//               bytes going through shared memory into the scale-factor columns.
+// M is only raised when the tile maximum exceeds it by more than kLazyShift (the block scales
+// absorb the difference), so the accumulator in tensor memory is almost never rescaled.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "mxfp8_device.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;          // query rows per CTA and keys per tile
+constexpr int kStages = 3;          // K ring and V ring depth
+constexpr int kThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kLazyShift = 8;
+
+// tensor-memory columns
+constexpr uint32_t kColS = 0;        // two score buffers of 128 columns; P codes alias columns 0..31
+constexpr uint32_t kColO = 256;      // output accumulator, dv columns
+constexpr uint32_t kColSFQ = 384;    // scale factors: Q (4), K (2 x 4), V (2 x 4), P (2 x 4)
+constexpr uint32_t kColSFK = 388;
+constexpr uint32_t kColSFV = 396;
+constexpr uint32_t kColSFP = 404;
+constexpr uint32_t kTmemCols = 512;
+
+struct FwdSmem {
+  alignas(1024) uint8_t q[kTile * 128];
+  alignas(1024) uint8_t k[kStages][kTile * 128];
+  alignas(1024) uint8_t v[kStages][kTile * 128];
+  alignas(16) uint8_t sf_q[512];
+  alignas(16) uint8_t sf_k[kStages][512];
+  alignas(16) uint8_t sf_v[kStages][512];
+  alignas(16) uint8_t sf_p[2][512];
+  uint64_t q_full;
+  uint64_t k_full[kStages], k_empty[kStages];
+  uint64_t v_full[kStages], v_empty[kStages];
+  uint64_t s_full[2], p_full[2], pv_done[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct FwdParams {
+  const uint8_t* q_sf;      // row scales of Q
+  const uint8_t* k_sf;      // row scales of K
+  const uint8_t* v_sf;      // col scales of V
+  __nv_bfloat16* o;
+  float* lse;
+  int* status;
+  int N, Hq, Hkv, dqk, dv, causal;
+  float scale_log2;         // softmax_scale * log2(e)
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+           const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ uint8_t smem_raw[];
+  FwdSmem& sm = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // heavy (late) query tiles first
+  const int qt = p.causal ? (gridDim.x - 1 - blockIdx.x) : blockIdx.x;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.Hq / p.Hkv);
+  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
+  const int nk_qk = p.dqk / 32;                 // K blocks of the score MMA
+  volatile int* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_full[i], 128); mbar_init(&sm.pv_done[i], 1);
+    }
+    sm.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&sm.tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+      const int q_row = (b * p.Hq + h) * p.N + qt * kTile;
+      mbar_arrive_expect_tx(&sm.q_full, kTile * 128 + 512);
+      tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_row);
+      bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(b * p.Hq + h) * (p.N / kTile) + qt) * 512, 512, &sm.q_full);
+      const int kv_slab = b * p.Hkv + g;
+      int issued_k = 0, issued_v = 0;
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % kStages, u = t / kStages;
+        ok = mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
+        tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
+        bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * (p.N / kTile) + t) * 512, 512, &sm.k_full[s]);
+        ++issued_k;
+        ok = mbar_wait(&sm.v_empty[s], (u & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
+        tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * kTile, kv_slab * p.dv);
+        bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * (p.N / kTile) + t) * 512, 512, &sm.v_full[s]);
+        ++issued_v;
+      }
+      if (!ok) {
+        // let the copies already in flight land before the CTA gives its shared memory back
+        int dummy = 0;
+        for (int t = max(0, issued_k - kStages); t < issued_k; ++t)
+          mbar_wait(&sm.k_full[t % kStages], (t / kStages) & 1, &dummy);
+        for (int t = max(0, issued_v - kStages); t < issued_v; ++t)
+          mbar_wait(&sm.v_full[t % kStages], (t / kStages) & 1, &dummy);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
+      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+      }
+      auto issue_qk = [&](int t) -> bool {
+        const int s = t % kStages, u = t / kStages, buf = t & 1;
+        if (!mbar_wait(&sm.k_full[s], u & 1, abort_flag)) return false;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFK + 4 * buf, make_desc_sf(smem_u32(sm.sf_k[s])));
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s]));
+        for (int kb = 0; kb < nk_qk; ++kb)
+          mma_mxf8_ss(tmem + kColS + 128 * buf, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
+                      tmem + kColSFQ, tmem + kColSFK + 4 * buf, kb > 0);
+        mma_commit(&sm.k_empty[s]);
+        mma_commit(&sm.s_full[buf]);
+        return true;
+      };
+      auto issue_pv = [&](int t) -> bool {
+        const int s = t % kStages, u = t / kStages, buf = t & 1;
+        if (!mbar_wait(&sm.v_full[s], u & 1, abort_flag)) return false;
+        if (!mbar_wait(&sm.p_full[buf], (t >> 1) & 1, abort_flag)) return false;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFV + 4 * buf, make_desc_sf(smem_u32(sm.sf_v[s])));
+        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
+        for (int kb = 0; kb < 4; ++kb)
+          mma_mxf8_ts(tmem + kColO, tmem + kColS + 128 * buf + 8 * kb, desc_v + 2 * kb,
+                      make_idesc_mxf8(128, p.dv, kb, kb), tmem + kColSFP + 4 * buf, tmem + kColSFV + 4 * buf,
+                      (t > 0 || kb > 0));
+        mma_commit(&sm.v_empty[s]);
+        mma_commit(&sm.pv_done[buf]);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        if (t + 1 < n_tiles) ok = issue_qk(t + 1);
+        if (ok) ok = issue_pv(t);
+      }
+      if (!ok) {
+        // drain whatever was issued so that tensor memory can be released safely
+        int dummy = 0;
+        mma_commit(&sm.q_full);
+        mbar_wait(&sm.q_full, 1, &dummy);
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                 // row inside the tile == TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    float M = -INFINITY;                              // integer-valued running shift
+    float l = 0.f;
+    bool ok = true;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      ok = mbar_wait(&sm.s_full[buf], (t >> 1) & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after_sync();
+      float s2[128];
+      {
+        uint32_t* r = reinterpret_cast<uint32_t*>(s2);
+        const uint32_t a = tmem + kColS + 128 * buf + lane_addr;
+        tmem_ld32(a, r); tmem_ld32(a + 32, r + 32); tmem_ld32(a + 64, r + 64); tmem_ld32(a + 96, r + 96);
+        tmem_wait_ld();
+      }
+      const bool diag = p.causal && (t == qt);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 128; ++c) {
+        float x = s2[c] * p.scale_log2;
+        if (diag && c > row) x = -INFINITY;
+        s2[c] = x;
+        mx = fmaxf(mx, x);
+      }
+      const float m_new = ceilf(mx);
+      const bool raise = m_new > M + static_cast<float>(kLazyShift);   // always true on the first tile
+      if (__any_sync(0xffffffffu, raise)) {
+        const float factor = raise ? exp2f(M - m_new) : 1.f;            // exact power of two (0 on the first tile)
+        if (raise) { l *= factor; M = m_new; }
+        if (t > 0) {
+          // the previous P V product must have landed before the accumulator is touched
+          ok = mbar_wait(&sm.pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          for (int c0 = 0; c0 < p.dv; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem + kColO + lane_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
+            tmem_st32(tmem + kColO + lane_addr + c0, r);
+          }
+          tmem_wait_st();
+        }
+      }
+      uint32_t sf_word = 0;
+#pragma unroll
+      for (int blk = 0; blk < 4; ++blk) {
+        float pexp[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          pexp[c] = ex2_approx(s2[blk * 32 + c] - M);
+          l += pexp[c];
+        }
+        uint32_t words[8];
+        const uint32_t byte = quantize_block32(pexp, words);
+        sf_word |= byte << (8 * blk);
+        tmem_st8(tmem + kColS + 128 * buf + lane_addr + 8 * blk, words);
+      }
+      *reinterpret_cast<uint32_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = sf_word;
+      tmem_wait_st();
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.p_full[buf]);
+    }
+    if (ok) {
+      const int last = n_tiles - 1;
+      ok = mbar_wait(&sm.pv_done[last & 1], (last >> 1) & 1, abort_flag);
+    }
+    if (ok) {
+      tc_fence_after_sync();
+      const float inv_l = 1.f / l;
+      const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
+      __nv_bfloat16* o_row = p.o + grow * p.dv;
+      for (int c0 = 0; c0 < p.dv; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + kColO + lane_addr + c0, r);
+        tmem_wait_ld();
+        uint32_t packed[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(r[2 * c]) * inv_l, __uint_as_float(r[2 * c + 1]) * inv_l);
+          packed[c] = *reinterpret_cast<uint32_t*>(&v2);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(o_row + c0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+      }
+      p.lse[grow] = (M + log2f(l)) * kLn2;
+    }
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+
+}  // namespace
+
+attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
+                         int* status, cudaStream_t stream) {
+  CUtensorMap tm_q, tm_k, tm_v;
+  attn_status_t st;
+  st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
+  if (st != ATTN_OK) return st;
+  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, static_cast<uint64_t>(s.B) * s.Hkv * s.N, kTile);
+  if (st != ATTN_OK) return st;
+  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
+  if (st != ATTN_OK) return st;
+  FwdParams p;
+  p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
+  p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
+  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.scale_log2 = s.scale * kLog2e;
+  const size_t smem = sizeof(FwdSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  dim3 grid(s.N / kTile, s.Hq, s.B);
+  fwd_kernel<<<grid, kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8

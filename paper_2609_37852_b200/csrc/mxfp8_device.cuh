@@ -1,0 +1,50 @@
+// Device-side pieces of the block quantiser shared by the quantiser kernel and by the attention
+// kernels that quantise probabilities and score gradients in registers.
+#pragma once
+#include <cstdint>
+
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+
+// Scale of one block of 32 values with maximum magnitude `amax`: the smallest power of two 2^e
+// with amax * 2^-e <= 448 (448 = 1.75 * 2^8, so e = E - 8, one more when the mantissa of amax
+// exceeds 1.75).  Returns the stored byte e + 127 (0 for an all-zero block) and the exact
+// multiplier 2^-e.
+__device__ __forceinline__ void block_scale(float amax, uint32_t& byte, float& inv) {
+  const uint32_t bits = __float_as_uint(amax);
+  const int E = static_cast<int>((bits >> 23) & 0xFF);
+  const uint32_t mant = bits & 0x7FFFFF;
+  int eb;
+  if (E == 0) {
+    eb = 0;                                    // zero (or subnormal) block
+  } else if (E == 255) {
+    eb = 254;                                  // non-finite maximum
+  } else {
+    eb = E - 8 + (mant > 0x600000 ? 1 : 0);
+    eb = eb < 0 ? 0 : (eb > 254 ? 254 : eb);
+  }
+  byte = static_cast<uint32_t>(eb);
+  const int ib = 254 - eb;                     // biased exponent of 2^-e
+  inv = ib > 0 ? __uint_as_float(static_cast<uint32_t>(ib) << 23) : __uint_as_float(0x00400000u);
+}
+
+// Quantise 32 values held in registers: codes packed four per word (element 0 in the low byte)
+// and the block's scale byte.
+__device__ __forceinline__ uint32_t quantize_block32(const float* x, uint32_t* words) {
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(x[i]));
+  uint32_t byte;
+  float inv;
+  block_scale(amax, byte, inv);
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    words[i] = sm100::cvt_e4m3x4(x[4 * i] * inv, x[4 * i + 1] * inv, x[4 * i + 2] * inv, x[4 * i + 3] * inv);
+  return byte;
+}
+
+// offset of (row r of a 128-row tile, block k of 4) inside a 512-byte scale tile
+__device__ __forceinline__ int sf_tile_offset(int r, int k) { return (r & 31) * 16 + (r >> 5) * 4 + k; }
+
+}  // namespace attnfp8

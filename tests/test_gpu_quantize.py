@@ -1,0 +1,67 @@
+"""attn_fp8_quantize against the oracle quantiser: codes and scale bytes bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mxfp8
+from paper_2609_37852_b200 import workloads
+from tests.util import to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(x: torch.Tensor):
+    from paper_2609_37852_b200 import binding
+    B, H, N, d = x.shape
+    qt = binding.attn_fp8_quantize(x.cuda())
+    torch.cuda.synchronize()
+    xn = to_np(x)
+    rc, rs = mxfp8.quantize(xn, axis=-1)
+    cc, cs = mxfp8.quantize(xn, axis=-2)
+    assert np.array_equal(qt.row_codes.cpu().numpy(), rc)
+    assert np.array_equal(binding.unpack_scales(qt.row_scales, B, H, N, d).cpu().numpy(), rs)
+    assert np.array_equal(qt.col_codes.cpu().numpy(), np.swapaxes(cc, -1, -2))
+    assert np.array_equal(binding.unpack_scales(qt.col_scales, B, H, d, N).cpu().numpy(), np.swapaxes(cs, -1, -2))
+    # padding bytes of the scale tiles are zero
+    total = int(qt.row_scales.to(torch.int64).sum()) - int(rs.astype(np.int64).sum())
+    assert total == 0
+    total = int(qt.col_scales.to(torch.int64).sum()) - int(cs.astype(np.int64).sum())
+    assert total == 0
+
+
+@pytest.mark.parametrize("name,N", [("tiny", 256), ("gqa4k", 384), ("gqa8k_outlier", 256), ("mla8k", 256),
+                                    ("gqa8k_d256", 128), ("long64k", 256)])
+def test_quantize_workload_inputs_bit_exact(name, N):
+    w = workloads.WORKLOADS[name].scaled(seqlen=N, heads_q=min(4, workloads.WORKLOADS[name].heads_q),
+                                         heads_kv=min(2, workloads.WORKLOADS[name].heads_kv))
+    for x in workloads.make_inputs(w):
+        _check(x)
+
+
+def test_quantize_edge_values():
+    g = torch.Generator().manual_seed(7)
+    x = torch.randn(1, 2, 128, 64, generator=g)
+    x[0, 0, :32, :32] = 0.0                       # all-zero row and column blocks
+    x[0, 0, 5, 40] = -0.0
+    x[0, 1, 3, :] *= 2.0 ** 60                    # huge and tiny blocks
+    x[0, 1, 4, :] *= 2.0 ** -70
+    x[0, 1, 64:96, 7] = 448.0                     # exactly on the saturation edge
+    x[0, 1, 96:128, 9] = 1.75                     # mantissa exactly 1.75: no bump
+    x[0, 1, 96, 10] = 1.7500001
+    _check(x)
+    _check(x.to(torch.bfloat16))
+
+
+def test_quantize_single_orientation_and_errors():
+    from paper_2609_37852_b200 import binding
+    x = torch.randn(1, 1, 128, 96, device="cuda", dtype=torch.bfloat16)
+    full = binding.attn_fp8_quantize(x)
+    only_row = binding.attn_fp8_quantize(x, want_col=False)
+    only_col = binding.attn_fp8_quantize(x, want_row=False)
+    torch.cuda.synchronize()
+    assert only_row.col_codes is None and torch.equal(only_row.row_codes, full.row_codes)
+    assert only_col.row_codes is None and torch.equal(only_col.col_codes, full.col_codes)
+    assert torch.equal(only_col.col_scales, full.col_scales)
+    with pytest.raises(binding.AttnFp8Error) as e:
+        binding.attn_fp8_quantize(torch.randn(1, 1, 100, 64, device="cuda"))
+    assert e.value.status == 2
