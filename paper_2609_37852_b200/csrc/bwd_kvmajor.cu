@@ -1,0 +1,341 @@
+// Key-major backward kernel: dK and dV (paper Appendix "Backward Correction and Gradient
+// Computation", paragraph "Score-gradient quantization", merged with the GQA group reduction).
+//
+// One CTA owns 128 keys of one (batch, KV head).  It loops over the query heads of the group and,
+// for each, over the query tiles from the causal diagonal to the end, 64 query rows at a time.
+// Per sub-tile the tensor cores recompute the TRANSPOSED products
+//     S^T  = K^ Q^^T    (128 keys x 64 queries; row-blocked FP8 copies)
+//     dP^T = V^ dO^^T
+// so that a softmax thread owns one key (one TMEM lane) and sees 32 consecutive query rows in
+// its registers: exactly one quantisation block of the operands P^T and dS^T, whose matmuls
+// contract over the query index.  The thread rebuilds P = 2^(S*scale*log2e - LSE_i*log2e),
+// forms dS = P (dP - D_i) in FP32, quantises both in registers, and the tensor cores accumulate
+//     dV += P^^T dO^c      dK += dS^^T Q^c      (copies of dO, Q blocked along tokens)
+// in tensor memory across all query tiles and all query heads of the group: the group sum is
+// an FP32 sum, rounded to BF16 once at the end.
+//
+// Warp roles as in the query-major kernels: warp 0 TMA producer, warp 1 MMA issuer, warps 4..11
+// softmax (group w takes query columns 32w..32w+31 of each sub-tile).
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "mxfp8_device.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;
+constexpr int kSub = 64;
+constexpr int kStages = 2;
+constexpr int kThreads = 384;
+constexpr int kSoftmaxThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+
+constexpr uint32_t kColS = 0, kColdP = 64, kColP = 128 /* 2 x 16 */, kColdS = 160 /* 2 x 16 */;
+constexpr uint32_t kColdV = 192, kColdK = 320;
+constexpr uint32_t kColSFK = 448, kColSFV = 452, kColSFQ = 456 /* 2 x 4 */, kColSFdO = 464 /* 2 x 4 */,
+                   kColSFP = 472 /* 2 x 4 */, kColSFdS = 480 /* 2 x 4 */, kColSFdOc = 488 /* 2 x 4 */,
+                   kColSFQc = 496 /* 2 x 4 */;
+constexpr uint32_t kTmemCols = 512;
+
+struct KvStage {
+  alignas(1024) uint8_t q[kTile * 128];       // Q row copy  [128 queries][dqk]
+  alignas(1024) uint8_t dO[kTile * 128];      // dO row copy [128 queries][dv]
+  alignas(1024) uint8_t qc[kTile * 128];      // Q col copy  [dqk][128 queries]
+  alignas(1024) uint8_t dOc[kTile * 128];     // dO col copy [dv][128 queries]
+  alignas(16) uint8_t sf_q[512];
+  alignas(16) uint8_t sf_dO[512];
+  alignas(16) uint8_t sf_qc[512];
+  alignas(16) uint8_t sf_dOc[512];
+  alignas(16) float lse[kTile];
+  alignas(16) float delta[kTile];
+};
+
+struct KvSmem {
+  alignas(1024) uint8_t k[kTile * 128];
+  alignas(1024) uint8_t v[kTile * 128];
+  KvStage st[kStages];
+  alignas(16) uint8_t sf_k[512];
+  alignas(16) uint8_t sf_v[512];
+  alignas(16) uint8_t sf_p[2][512];
+  alignas(16) uint8_t sf_ds[2][512];
+  uint64_t kv_full;
+  uint64_t q_full[kStages], q_empty[kStages];
+  uint64_t sdp_full, sdp_free;
+  uint64_t pds_full[2];
+  uint64_t done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct KvParams {
+  const uint8_t *k_sf, *v_sf, *q_sf, *dO_sf, *qc_sf, *dOc_sf;
+  const float* lse;
+  const float* delta;
+  __nv_bfloat16* dk;
+  __nv_bfloat16* dv_out;
+  int* status;
+  int N, Hq, Hkv, dqk, dv, causal;
+  float scale, scale_log2;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+               const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
+               const __grid_constant__ CUtensorMap tm_qc, const __grid_constant__ CUtensorMap tm_dOc) {
+  extern __shared__ uint8_t smem_raw[];
+  KvSmem& sm = *reinterpret_cast<KvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int jt = blockIdx.x;                        // key tile; tile 0 has the most work under the causal mask
+  const int g = blockIdx.y, b = blockIdx.z;
+  const int G = p.Hq / p.Hkv;
+  const int tiles_n = p.N / kTile;
+  const int it0 = p.causal ? jt : 0;                // first query tile that sees these keys
+  const int tiles_per_head = tiles_n - it0;
+  const int n_qtiles = G * tiles_per_head;          // query tiles this CTA walks
+  const int n_sub = 2 * n_qtiles;
+  const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
+  volatile int* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    mbar_init(&sm.kv_full, 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
+    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.sdp_free, kSoftmaxThreads);
+    mbar_init(&sm.pds_full[0], kSoftmaxThreads); mbar_init(&sm.pds_full[1], kSoftmaxThreads);
+    mbar_init(&sm.done, 1);
+    sm.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&sm.tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO);
+      prefetch_tmap(&tm_qc); prefetch_tmap(&tm_dOc);
+      const int kv_slab = b * p.Hkv + g;
+      mbar_arrive_expect_tx(&sm.kv_full, 2 * (kTile * 128 + 512));
+      tma_load_2d(sm.k, &tm_k, &sm.kv_full, 0, kv_slab * p.N + jt * kTile);
+      tma_load_2d(sm.v, &tm_v, &sm.kv_full, 0, kv_slab * p.N + jt * kTile);
+      bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
+      bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
+      int issued = 0;
+      bool ok = true;
+      for (int n = 0; n < n_qtiles && ok; ++n) {
+        const int s = n % kStages, u = n / kStages;
+        const int h = g * G + n / tiles_per_head, it = it0 + n % tiles_per_head;
+        const int q_slab = b * p.Hq + h;
+        ok = mbar_wait(&sm.q_empty[s], (u & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        KvStage& st = sm.st[s];
+        mbar_arrive_expect_tx(&sm.q_full[s], 2 * kTile * 128 + (p.dqk + p.dv) * 128 + 4 * 512 + 2 * kTile * 4);
+        tma_load_2d(st.q, &tm_q, &sm.q_full[s], 0, q_slab * p.N + it * kTile);
+        tma_load_2d(st.dO, &tm_dO, &sm.q_full[s], 0, q_slab * p.N + it * kTile);
+        tma_load_2d(st.qc, &tm_qc, &sm.q_full[s], it * kTile, q_slab * p.dqk);
+        tma_load_2d(st.dOc, &tm_dOc, &sm.q_full[s], it * kTile, q_slab * p.dv);
+        const size_t sf_tile = (static_cast<size_t>(q_slab) * tiles_n + it) * 512;
+        bulk_load_1d(st.sf_q, p.q_sf + sf_tile, 512, &sm.q_full[s]);
+        bulk_load_1d(st.sf_dO, p.dO_sf + sf_tile, 512, &sm.q_full[s]);
+        bulk_load_1d(st.sf_qc, p.qc_sf + sf_tile, 512, &sm.q_full[s]);
+        bulk_load_1d(st.sf_dOc, p.dOc_sf + sf_tile, 512, &sm.q_full[s]);
+        const size_t row0 = static_cast<size_t>(q_slab) * p.N + it * kTile;
+        bulk_load_1d(st.lse, p.lse + row0, kTile * 4, &sm.q_full[s]);
+        bulk_load_1d(st.delta, p.delta + row0, kTile * 4, &sm.q_full[s]);
+        ++issued;
+      }
+      if (!ok) {
+        int dummy = 0;
+        for (int n = max(0, issued - kStages); n < issued; ++n)
+          mbar_wait(&sm.q_full[n % kStages], (n / kStages) & 1, &dummy);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k));
+      const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v));
+      bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
+        sf_copy(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
+      }
+      auto issue_sdp = [&](int u) -> bool {
+        const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
+        KvStage& st = sm.st[s];
+        if (half == 0) {
+          if (!mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag)) return false;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
+          sf_copy(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
+        }
+        if (u > 0) {
+          if (!mbar_wait(&sm.sdp_free, (u - 1) & 1, abort_flag)) return false;
+          tc_fence_after_sync();
+        }
+        const uint64_t desc_q = make_desc_sw128(smem_u32(st.q)) + half * (kSub * 128 / 16);
+        const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO)) + half * (kSub * 128 / 16);
+        for (int kb = 0; kb < nk_qk; ++kb)
+          mma_mxf8_ss(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+                      tmem + kColSFK, tmem + kColSFQ + 4 * slot + 2 * half, kb > 0);
+        for (int kb = 0; kb < nk_v; ++kb)
+          mma_mxf8_ss(tmem + kColdP, desc_v + 2 * kb, desc_dO + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+                      tmem + kColSFV, tmem + kColSFdO + 4 * slot + 2 * half, kb > 0);
+        mma_commit(&sm.sdp_full);
+        return true;
+      };
+      auto issue_dkv = [&](int u) -> bool {
+        const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1, buf = u & 1;
+        KvStage& st = sm.st[s];
+        if (!mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag)) return false;
+        tc_fence_after_sync();
+        if (half == 0) {
+          sf_copy(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
+          sf_copy(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
+        }
+        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        const uint64_t desc_dOc = make_desc_sw128(smem_u32(st.dOc));
+        const uint64_t desc_qc = make_desc_sw128(smem_u32(st.qc));
+        for (int kb = 0; kb < 2; ++kb)
+          mma_mxf8_ts(tmem + kColdV, tmem + kColP + 16 * buf + 8 * kb, desc_dOc + 2 * (2 * half + kb),
+                      make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
+                      tmem + kColSFdOc + 4 * slot, (u > 0 || kb > 0));
+        for (int kb = 0; kb < 2; ++kb)
+          mma_mxf8_ts(tmem + kColdK, tmem + kColdS + 16 * buf + 8 * kb, desc_qc + 2 * (2 * half + kb),
+                      make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
+                      tmem + kColSFQc + 4 * slot, (u > 0 || kb > 0));
+        if (half == 1) mma_commit(&sm.q_empty[s]);
+        if (u == n_sub - 1) mma_commit(&sm.done);
+        return true;
+      };
+      if (ok) ok = issue_sdp(0);
+      for (int u = 0; u < n_sub && ok; ++u) {
+        if (u + 1 < n_sub) ok = issue_sdp(u + 1);
+        if (ok) ok = issue_dkv(u);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.kv_full);
+        mbar_wait(&sm.kv_full, 1, &dummy);
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax
+    const int grp = (warp - 4) >> 2;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                 // key inside the tile == TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    bool ok = true;
+    for (int u = 0; u < n_sub; ++u) {
+      const int n = u >> 1, half = u & 1, buf = u & 1, s = n % kStages;
+      const int it = it0 + n % tiles_per_head;
+      ok = mbar_wait(&sm.sdp_full, u & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after_sync();
+      uint32_t sr[32], dpr[32];
+      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
+      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.sdp_free);
+      const bool diag = p.causal && (it == jt);
+      const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
+      const float* s_lse = sm.st[s].lse + col0;
+      const float* s_delta = sm.st[s].delta + col0;
+      float pr[32], ds[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -s_lse[c] * kLog2e);
+        if (diag && (row > col0 + c)) x = -INFINITY;   // key after the query
+        const float pv = ex2_approx(x);
+        pr[c] = pv;
+        ds[c] = pv * (__uint_as_float(dpr[c]) - s_delta[c]);
+      }
+      uint32_t words[8];
+      const uint32_t byte_p = quantize_block32(pr, words);
+      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
+      const uint32_t byte_s = quantize_block32(ds, words);
+      tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
+      const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
+      sm.sf_p[buf][sf_at] = static_cast<uint8_t>(byte_p);
+      sm.sf_ds[buf][sf_at] = static_cast<uint8_t>(byte_s);
+      tmem_wait_st();
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.pds_full[buf]);
+    }
+    if (ok) ok = mbar_wait(&sm.done, 0, abort_flag);
+    if (ok) {
+      tc_fence_after_sync();
+      const size_t grow = static_cast<size_t>(b * p.Hkv + g) * p.N + jt * kTile + row;
+      // group 0 stores dV, group 1 stores dK (scaled)
+      const uint32_t col = grp == 0 ? kColdV : kColdK;
+      const int width = grp == 0 ? p.dv : p.dqk;
+      const float mul = grp == 0 ? 1.f : p.scale;
+      __nv_bfloat16* out_row = (grp == 0 ? p.dv_out : p.dk) + grow * width;
+      for (int c0 = 0; c0 < width; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + col + lane_addr + c0, r);
+        tmem_wait_ld();
+        uint32_t packed[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(r[2 * c]) * mul, __uint_as_float(r[2 * c + 1]) * mul);
+          packed[c] = *reinterpret_cast<uint32_t*>(&v2);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(out_row + c0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+      }
+    }
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+
+}  // namespace
+
+attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                              const float* lse, const float* delta, void* dk, void* dv, int* status,
+                              cudaStream_t stream) {
+  CUtensorMap tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc;
+  attn_status_t st;
+  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
+  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, s.dqk)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dOc, dO.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hq * s.dv, s.dv)) != ATTN_OK) return st;
+  KvParams p;
+  p.k_sf = k.row_scales; p.v_sf = v.row_scales; p.q_sf = q.row_scales; p.dO_sf = dO.row_scales;
+  p.qc_sf = q.col_scales; p.dOc_sf = dO.col_scales;
+  p.lse = lse; p.delta = delta;
+  p.dk = static_cast<__nv_bfloat16*>(dk); p.dv_out = static_cast<__nv_bfloat16*>(dv); p.status = status;
+  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
+  const size_t smem = sizeof(KvSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  dim3 grid(s.N / kTile, s.Hkv, s.B);
+  kvmajor_kernel<<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8

@@ -1,0 +1,409 @@
+// Query-major backward kernels: the matched row correction (Delta-Matching, paper Section 3.3
+// Eq. 4) and the query gradient (paper Appendix "Backward Correction and Gradient Computation").
+//
+// One CTA owns 128 query rows of one (batch, query head) and sweeps the key tiles up to the
+// causal diagonal, 64 keys at a time.  For every 64-key sub-tile the tensor cores recompute
+//     S  = Q^ K^^T   (row-blocked FP8 copies, contraction over the qk channels)
+//     dP = dO^ V^^T  (row-blocked FP8 copies, contraction over the v channels)
+// into tensor memory; the softmax warps rebuild P = 2^(S*scale*log2e - LSE*log2e) in FP32 from
+// the saved LSE (not renormalised, not quantised) and then either
+//   kDelta: accumulate D_i = sum_j P_ij dP_ij, or
+//   kDQ:    form dS = P (dP - D), record the pre-cast row statistics, quantise dS in blocks of
+//           32 keys in registers, hand the codes back through tensor memory and let the tensor
+//           cores accumulate dQ += dS^ K^c (K copy blocked along keys).
+// Both modes run the same instruction sequence for P and dP, so the correction the first
+// produces is the one that zeroes the row sums of the second up to FP32 rounding.
+//
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 4..11 softmax (two groups of four
+// warps; group w takes columns 32w..32w+31 of each sub-tile, warp % 4 selects the 32 TMEM lanes).
+// S and dP are single-buffered: the softmax warps pull them into registers and release the
+// buffers at once, so the next sub-tile's MMAs overlap the exponentials of this one.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "mxfp8_device.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;
+constexpr int kSub = 64;
+constexpr int kStages = 2;
+constexpr int kThreads = 384;
+constexpr int kSoftmaxThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
+
+constexpr uint32_t kColS = 0, kColdP = 64, kColdS = 128 /* 2 x 16 */, kColdQ = 256;
+constexpr uint32_t kColSFQ = 384, kColSFdO = 388, kColSFK = 392 /* 2 x 4 */, kColSFV = 400 /* 2 x 4 */,
+                   kColSFdS = 408 /* 2 x 4 */, kColSFKc = 416 /* 2 x 4 */;
+constexpr uint32_t kTmemCols = 512;
+
+struct QmSmem {
+  alignas(1024) uint8_t q[kTile * 128];
+  alignas(1024) uint8_t dO[kTile * 128];
+  alignas(1024) uint8_t k[kStages][kTile * 128];
+  alignas(1024) uint8_t v[kStages][kTile * 128];
+  alignas(1024) uint8_t kc[kStages][kTile * 128];
+  alignas(16) uint8_t sf_q[512];
+  alignas(16) uint8_t sf_dO[512];
+  alignas(16) uint8_t sf_k[kStages][512];
+  alignas(16) uint8_t sf_v[kStages][512];
+  alignas(16) uint8_t sf_kc[kStages][512];
+  alignas(16) uint8_t sf_ds[2][512];
+  alignas(16) float red[3][kTile];          // cross-group reduction of row sums
+  uint64_t q_full;
+  uint64_t kv_full[kStages], kv_empty[kStages];
+  uint64_t kc_full[kStages], kc_empty[kStages];
+  uint64_t sdp_full, sdp_free;
+  uint64_t ds_full[2];
+  uint64_t dq_done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct QmParams {
+  const uint8_t *q_sf, *dO_sf, *k_sf, *v_sf, *kc_sf;
+  const float* lse;
+  const float* delta_in;
+  float* delta_out;
+  __nv_bfloat16* dq;
+  float* rowsum;
+  float* rowabs;
+  int* status;
+  int N, Hq, Hkv, dqk, dv, causal;
+  float scale, scale_log2;
+};
+
+template <bool kDQ>
+__global__ void __launch_bounds__(kThreads, 1)
+qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
+              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+              const __grid_constant__ CUtensorMap tm_kc) {
+  extern __shared__ uint8_t smem_raw[];
+  QmSmem& sm = *reinterpret_cast<QmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qt = p.causal ? (gridDim.x - 1 - blockIdx.x) : blockIdx.x;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.Hq / p.Hkv);
+  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
+  const int n_sub = 2 * n_tiles;
+  const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
+  volatile int* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1);
+      mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1);
+    }
+    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.sdp_free, kSoftmaxThreads);
+    mbar_init(&sm.ds_full[0], kSoftmaxThreads); mbar_init(&sm.ds_full[1], kSoftmaxThreads);
+    mbar_init(&sm.dq_done, 1);
+    sm.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&sm.tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+      if (kDQ) prefetch_tmap(&tm_kc);
+      const int q_slab = b * p.Hq + h, kv_slab = b * p.Hkv + g;
+      const int tiles_n = p.N / kTile;
+      mbar_arrive_expect_tx(&sm.q_full, 2 * (kTile * 128 + 512));
+      tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_slab * p.N + qt * kTile);
+      tma_load_2d(sm.dO, &tm_dO, &sm.q_full, 0, q_slab * p.N + qt * kTile);
+      bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * 512, 512, &sm.q_full);
+      bulk_load_1d(sm.sf_dO, p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * 512, 512, &sm.q_full);
+      int issued_kv = 0, issued_kc = 0;
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % kStages, u = t / kStages;
+        ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&sm.kv_full[s], 2 * (kTile * 128 + 512));
+        tma_load_2d(sm.k[s], &tm_k, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
+        tma_load_2d(sm.v[s], &tm_v, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
+        bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kv_full[s]);
+        bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kv_full[s]);
+        ++issued_kv;
+        if (kDQ) {
+          ok = mbar_wait(&sm.kc_empty[s], (u & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sm.kc_full[s], p.dqk * 128 + 512);
+          tma_load_2d(sm.kc[s], &tm_kc, &sm.kc_full[s], t * kTile, kv_slab * p.dqk);
+          bulk_load_1d(sm.sf_kc[s], p.kc_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kc_full[s]);
+          ++issued_kc;
+        }
+      }
+      if (!ok) {
+        int dummy = 0;
+        for (int t = max(0, issued_kv - kStages); t < issued_kv; ++t)
+          mbar_wait(&sm.kv_full[t % kStages], (t / kStages) & 1, &dummy);
+        for (int t = max(0, issued_kc - kStages); t < issued_kc; ++t)
+          mbar_wait(&sm.kc_full[t % kStages], (t / kStages) & 1, &dummy);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
+      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO));
+      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+        sf_copy(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
+      }
+      auto issue_sdp = [&](int u) -> bool {
+        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
+        if (half == 0) {
+          if (!mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag)) return false;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        }
+        if (u > 0) {
+          if (!mbar_wait(&sm.sdp_free, (u - 1) & 1, abort_flag)) return false;
+          tc_fence_after_sync();
+        }
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s])) + half * (kSub * 128 / 16);
+        for (int kb = 0; kb < nk_qk; ++kb)
+          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+                      tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
+        for (int kb = 0; kb < nk_v; ++kb)
+          mma_mxf8_ss(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+                      tmem + kColSFdO, tmem + kColSFV + 4 * slot + 2 * half, kb > 0);
+        mma_commit(&sm.sdp_full);
+        if (half == 1) mma_commit(&sm.kv_empty[s]);
+        return true;
+      };
+      auto issue_dq = [&](int u) -> bool {
+        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
+        if (half == 0) {
+          if (!mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag)) return false;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+        }
+        if (!mbar_wait(&sm.ds_full[buf], (u >> 1) & 1, abort_flag)) return false;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
+        for (int kb = 0; kb < 2; ++kb)
+          mma_mxf8_ts(tmem + kColdQ, tmem + kColdS + 16 * buf + 8 * kb, desc_kc + 2 * (2 * half + kb),
+                      make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
+                      tmem + kColSFKc + 4 * slot, (u > 0 || kb > 0));
+        if (half == 1) mma_commit(&sm.kc_empty[s]);
+        if (u == n_sub - 1) mma_commit(&sm.dq_done);
+        return true;
+      };
+      if (kDQ) {
+        if (ok) ok = issue_sdp(0);
+        for (int u = 0; u < n_sub && ok; ++u) {
+          if (u + 1 < n_sub) ok = issue_sdp(u + 1);
+          if (ok) ok = issue_dq(u);
+        }
+      } else {
+        for (int u = 0; u < n_sub && ok; ++u) ok = issue_sdp(u);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.q_full);
+        mbar_wait(&sm.q_full, 1, &dummy);
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax
+    const int grp = (warp - 4) >> 2;                  // column half of each sub-tile
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
+    // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
+    // to the half ulp the FP32 storage of LSE already carries
+    const float lse_nat = p.lse[grow];
+    const float lse2 = lse_nat * kLog2e;
+    const float lse2_lo = fmaf(lse_nat, kLog2e, -lse2) + lse_nat * kLog2eLo;
+    const float D = kDQ ? p.delta_in[grow] : 0.f;
+    float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
+    bool ok = true;
+    for (int u = 0; u < n_sub; ++u) {
+      const int t = u >> 1, half = u & 1, buf = u & 1;
+      ok = mbar_wait(&sm.sdp_full, u & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after_sync();
+      uint32_t sr[32], dpr[32];
+      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
+      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.sdp_free);
+      const bool diag = p.causal && (t == qt);
+      const int col0 = half * kSub + 32 * grp;        // column of this thread's first element inside the key tile
+      float ds[32];
+      float part = 0.f;
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -lse2) - lse2_lo;
+        if (diag && (col0 + c > row)) x = -INFINITY;
+        const float pr = ex2_approx(x);
+        const float dp = __uint_as_float(dpr[c]);
+        if (kDQ) {
+          const float d = pr * (dp - D);
+          ds[c] = d;
+          acc0 += d;
+          acc1 += fabsf(d);
+        } else {
+          part = fmaf(pr, dp, part);
+        }
+      }
+      if (!kDQ) {
+        acc0 += part;
+      } else {
+        uint32_t words[8];
+        const uint32_t byte = quantize_block32(ds, words);
+        tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
+        sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&sm.ds_full[buf]);
+      }
+    }
+    // combine the two column groups' row sums
+    if (grp == 1) {
+      sm.red[0][row] = acc0;
+      sm.red[1][row] = acc1;
+    }
+    named_barrier_sync(1, kSoftmaxThreads);
+    if (ok && grp == 0) {
+      acc0 += sm.red[0][row];
+      acc1 += sm.red[1][row];
+      if (!kDQ) {
+        p.delta_out[grow] = acc0;
+      } else if (p.rowsum) {
+        p.rowsum[grow] = acc0;
+        p.rowabs[grow] = acc1;
+      }
+    }
+    if (kDQ && ok) {
+      ok = mbar_wait(&sm.dq_done, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        __nv_bfloat16* out_row = p.dq + grow * p.dqk;
+        const int half_cols = p.dqk / 2;
+        for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(tmem + kColdQ + lane_addr + c0, r);
+          tmem_wait_ld();
+          uint32_t packed[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(r[2 * c]) * p.scale, __uint_as_float(r[2 * c + 1]) * p.scale);
+            packed[c] = *reinterpret_cast<uint32_t*>(&v2);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(out_row + c0);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+        }
+      }
+    }
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+
+template <bool kDQ>
+attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                            const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
+                            float* rowabs, int* status, cudaStream_t stream) {
+  CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
+  attn_status_t st;
+  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
+  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv, kv_rows, kTile)) != ATTN_OK) return st;
+  if (kDQ) {
+    if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk, s.dqk)) != ATTN_OK)
+      return st;
+  } else {
+    tm_kc = tm_k;
+  }
+  QmParams p;
+  p.q_sf = q.row_scales; p.dO_sf = dO.row_scales; p.k_sf = k.row_scales; p.v_sf = v.row_scales;
+  p.kc_sf = kDQ ? k.col_scales : nullptr;
+  p.lse = lse; p.delta_in = delta_in; p.delta_out = delta_out;
+  p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.status = status;
+  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
+  const size_t smem = sizeof(QmSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<kDQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  dim3 grid(s.N / kTile, s.Hq, s.B);
+  qmajor_kernel<kDQ><<<grid, kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+// Stale delta: D_i = sum_c dO_ic O_ic from the BF16 tensors (paper Section 3.2).  One warp per row.
+__global__ void stale_delta_kernel(const __nv_bfloat16* __restrict__ dO, const __nv_bfloat16* __restrict__ o,
+                                   float* __restrict__ delta, size_t rows, int dv) {
+  const size_t row = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float acc = 0.f;
+  for (int c = lane * 2; c < dv; c += 64) {
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(dO + row * dv + c);
+    const __nv_bfloat162 bb = *reinterpret_cast<const __nv_bfloat162*>(o + row * dv + c);
+    acc = fmaf(__bfloat162float(a.x), __bfloat162float(bb.x), acc);
+    acc = fmaf(__bfloat162float(a.y), __bfloat162float(bb.y), acc);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) delta[row] = acc;
+}
+
+}  // namespace
+
+attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                               attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream) {
+  return launch_qmajor<false>(s, q, k, v, dO, lse, nullptr, delta, nullptr, nullptr, nullptr, status, stream);
+}
+
+attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                            const float* lse, const float* delta, void* dq, float* rowsum, float* rowabs, int* status,
+                            cudaStream_t stream) {
+  return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, status, stream);
+}
+
+attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,
+                                 cudaStream_t stream) {
+  const size_t rows = static_cast<size_t>(s.B) * s.Hq * s.N;
+  const int threads = 256;
+  const size_t blocks = (rows * 32 + threads - 1) / threads;
+  stale_delta_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+      static_cast<const __nv_bfloat16*>(dO_bf16), static_cast<const __nv_bfloat16*>(o_bf16), delta, rows, s.dv);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "stale delta: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8

@@ -31,7 +31,8 @@ constexpr int kTile = 128;          // query rows per CTA and keys per tile
 constexpr int kStages = 3;          // K ring and V ring depth
 constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
+constexpr float kLn2Lo = -2.12194440054690583e-4f;
 constexpr int kLazyShift = 8;
 
 // tensor-memory columns
@@ -241,19 +242,25 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         }
       }
       uint32_t sf_word = 0;
+      float tile_sum = 0.f;                     // summed per block, per tile, then into l: short chains
 #pragma unroll
       for (int blk = 0; blk < 4; ++blk) {
         float pexp[32];
+        float bs0 = 0.f, bs1 = 0.f;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
+        for (int c = 0; c < 32; c += 2) {
           pexp[c] = ex2_approx(s2[blk * 32 + c] - M);
-          l += pexp[c];
+          pexp[c + 1] = ex2_approx(s2[blk * 32 + c + 1] - M);
+          bs0 += pexp[c];
+          bs1 += pexp[c + 1];
         }
+        tile_sum += bs0 + bs1;
         uint32_t words[8];
         const uint32_t byte = quantize_block32(pexp, words);
         sf_word |= byte << (8 * blk);
         tmem_st8(tmem + kColS + 128 * buf + lane_addr + 8 * blk, words);
       }
+      l += tile_sum;
       *reinterpret_cast<uint32_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = sf_word;
       tmem_wait_st();
       fence_proxy_async_smem();
@@ -283,7 +290,8 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
 #pragma unroll
         for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
       }
-      p.lse[grow] = (M + log2f(l)) * kLn2;
+      // LSE = M ln2 + ln l with ln2 split so that M * ln2_hi is exact: one rounding at the end
+      p.lse[grow] = fmaf(M, kLn2Hi, fmaf(M, kLn2Lo, logf(l)));
     }
   }
   __syncwarp();
