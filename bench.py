@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 Delta-Matching attention path on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+quantise Q, K, V, dO (both block orientations), forward, matched row
+correction, gradient pass (dQ, then dK/dV).  The metric is causal-adjusted
+TFLOP/s of forward + backward in the paper's FLOP convention (the correction
+pass and the quantiser earn no credit).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched under torchrun) every rank
+runs an independent replica of the workload on its own GPU -- the path has no
+exchange step -- and the value is the aggregate over ranks.
+``--impl reference`` times the CPU oracle on a bounded causal prefix of the
+same workload instead (host cores; rank 0 only).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD = "gqa8k_outlier"          # B=1, Hq=32, Hkv=8, N=8192, d=128, causal: the configuration the metric is quoted on
+METRIC = "fp8_attn_fwd_bwd_causal_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_FP8_TFLOPS = 4500.0
+FP8_OVER_BF16 = 2.0                 # nominal dense FP8 : BF16 tensor ratio on B200
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on WORKLOAD, from
+# the ncu captures summarised under profiles/; None where no capture has been taken.
+NCU_TRAFFIC_BYTES = {"quantize": None, "fwd": None, "bwd_delta": None, "bwd_dq": None, "bwd_dkdv": None}
+
+# executed matmul products per kernel (each 2*d FLOPs per unmasked (i, j) pair and query head)
+PRODUCTS = {"fwd": 2, "bwd_delta": 2, "bwd_dq": 3, "bwd_dkdv": 4}
+
+
+def _measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"], hbm=p["hbm_gbs"],
+                    source="measured")
+    return dict(bf16_burst=1590.0, bf16_sustained=1400.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            # samples under load are the upper half of the distribution when the region is short
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_step(w, sample_tokens, q, k, v, dO):
+    """One pass of the oracle (forward, matched correction, gradient pass) on the causal prefix of
+    ``sample_tokens`` tokens of one KV group.  Returns credited FLOPs."""
+    import numpy as np
+    from oracle import attention as A
+    G = w.heads_q // w.heads_kv
+    qs, ks, vs, dOs = (x[:1, :hh, :sample_tokens].float().numpy().astype(np.float64)
+                       for x, hh in ((q, G), (k, 1), (v, 1), (dO, G)))
+    O, LSE = A.emu_forward(qs, ks, vs, w.softmax_scale, w.causal)
+    D = A.emu_delta(qs, ks, vs, dOs, LSE, w.softmax_scale, w.causal)
+    A.emu_backward(qs, ks, vs, dOs, LSE, D, w.softmax_scale, w.causal)
+    sub = w.scaled(batch=1, heads_q=G, heads_kv=1, seqlen=sample_tokens)
+    return sum(sub.credited_flops())
+
+
+def _cores_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle, as it stands, on the host cores."""
+    from paper_2609_37852_b200 import workloads
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_tokens = 512
+    small = w.scaled(heads_q=w.heads_q // w.heads_kv, heads_kv=1, seqlen=sample_tokens)
+    q, k, v, dO = workloads.make_inputs(small)
+    for _ in range(args.warmup):
+        oracle_step(w, sample_tokens, q, k, v, dO)
+    t0 = time.perf_counter()
+    flops = 0
+    for _ in range(args.steps):
+        flops += oracle_step(w, sample_tokens, q, k, v, dO)
+    dt = time.perf_counter() - t0
+    value = flops / dt / 1e12
+    sample = (f"causal prefix of {sample_tokens} tokens of one KV group ({small.heads_q} query heads) of {w.name}, "
+              f"fwd + matched correction + gradient pass per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2609_37852_b200 import workloads
+    w = workloads.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_2609_37852_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    warmup = max(args.warmup, 3)
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                          w.softmax_scale)
+    host = [x.pin_memory() for x in workloads.make_inputs(w)]
+    q, k, v, dO = (x.to(dev, non_blocking=True) for x in host)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    # pre-allocated operands, outputs and workspaces (device memory is PyTorch's job; the path is the library's)
+    qq, kq, vq, dOq = (B.attn_fp8_quantize(x) for x in (q, k, v, dO))
+    bf = dict(dtype=torch.bfloat16, device=dev)
+    o = torch.empty((w.batch, w.heads_q, w.seqlen, w.head_dim_v), **bf)
+    lse = torch.empty((w.batch, w.heads_q, w.seqlen), dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    dq = torch.empty((w.batch, w.heads_q, w.seqlen, w.head_dim_qk), **bf)
+    dk = torch.empty((w.batch, w.heads_kv, w.seqlen, w.head_dim_qk), **bf)
+    dv = torch.empty((w.batch, w.heads_kv, w.seqlen, w.head_dim_v), **bf)
+    ws = torch.empty(max(B.attn_fp8_workspace_bytes(params, i) for i in range(3)), dtype=torch.uint8, device=dev)
+
+    stage_names = ("quantize", "fwd", "bwd_delta", "bwd_dq", "bwd_dkdv")
+
+    def step(events=None):
+        def mark(i):
+            if events is not None:
+                events[i].record(stream)
+        mark(0)
+        B.attn_fp8_quantize(q, out=qq); B.attn_fp8_quantize(k, out=kq)
+        B.attn_fp8_quantize(v, out=vq); B.attn_fp8_quantize(dO, out=dOq)
+        mark(1)
+        B.attn_fp8_fwd(params, qq, kq, vq, o=o, lse=lse, workspace=ws)
+        mark(2)
+        B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, delta=delta, workspace=ws)
+        mark(3)
+        B.attn_fp8_bwd_dq(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
+        mark(4)
+        B.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, dk=dk, dv=dv, workspace=ws)
+        mark(5)
+
+    kernels_per_step = 8            # 4 quantiser launches + fwd + delta + dQ + dK/dV
+
+    # ---- device-resident timing -------------------------------------------------------------
+    for _ in range(warmup):
+        step()
+    B.attn_fp8_read_status(ws)
+    sampler = ClockSampler(local_rank)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    barrier()
+    sampler.start()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(events[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    B.attn_fp8_read_status(ws)
+    total_ms = t_start.elapsed_time(t_end)
+    stage_ms = {n: statistics.mean(events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps))
+                for j, n in enumerate(stage_names)}
+
+    # ---- end to end through the library with host buffers --------------------------------------
+    outs_host = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)]
+
+    def e2e_step():
+        for src, dst in zip(host, (q, k, v, dO)):
+            dst.copy_(src, non_blocking=True)
+        step()
+        for src, dst in zip((o, lse, dq, dk, dv), outs_host):
+            dst.copy_(src, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e_start = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+    e_start.record(stream)
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(e2e_steps):
+        e2e_step()
+    e_end.record(stream)
+    barrier()
+    e2e_ms = e_start.elapsed_time(e_end)
+    h2d = sum(t.numel() * t.element_size() for t in host)
+    d2h = sum(t.numel() * t.element_size() for t in outs_host)
+
+    # ---- max over ranks -----------------------------------------------------------------------
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = (float(x) for x in times.cpu())
+
+    fwd_flops, bwd_flops = w.credited_flops()
+    credited = fwd_flops + bwd_flops
+    value = world * credited * args.steps / (total_ms * 1e-3) / 1e12
+    e2e_value = world * credited * e2e_steps / (e2e_ms * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel ------------------------------------------------------
+    peaks = _measured_peaks()
+    attn_stages = {n: stage_ms[n] for n in PRODUCTS}
+    dominant = max(attn_stages, key=attn_stages.get)
+    c = 1 if w.causal else 2
+    pair_flops = c * w.batch * w.heads_q * w.seqlen * w.seqlen * w.head_dim_qk     # 2*d flops x N^2/2 pairs per head
+    kernel_flops = PRODUCTS[dominant] * pair_flops
+    achieved = kernel_flops / (stage_ms[dominant] * 1e-3) / 1e12
+    peak = peaks["bf16_sustained"] * FP8_OVER_BF16
+    roofline = {
+        "kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+        "frac": achieved / peak,
+        "peak_source": f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x {FP8_OVER_BF16} (nominal fp8:bf16)",
+        "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8_e4m3", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "heads_q": w.heads_q, "heads_kv": w.heads_kv,
+                   "seqlen": w.seqlen, "head_dim": w.head_dim_qk, "causal": w.causal, "delta_mode": "matched",
+                   "l2": "working set per step (>500 MB) exceeds the 126 MB L2", "parallelism": f"replicas x{world}",
+                   "step": "quantize(Q,K,V,dO) + fwd + matched delta + dQ + dK/dV"},
+        "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
+        "stage_ms": stage_ms,
+        "attn_only_tflops": credited / ((sum(attn_stages.values())) * 1e-3) / 1e12,
+        "fwd_tflops": fwd_flops / (stage_ms["fwd"] * 1e-3) / 1e12,
+        "bwd_tflops": bwd_flops / ((stage_ms["bwd_delta"] + stage_ms["bwd_dq"] + stage_ms["bwd_dkdv"]) * 1e-3) / 1e12,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": kernels_per_step * args.steps,
+        "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample_tokens = 2048
+        small = w.scaled(heads_q=w.heads_q // w.heads_kv, heads_kv=1, seqlen=sample_tokens)
+        sq, sk, sv, sdO = workloads.make_inputs(small)
+        t0 = time.perf_counter()
+        flops = oracle_step(w, sample_tokens, sq, sk, sv, sdO)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": flops / dt / 1e12, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "seconds": dt,
+            "sample": f"causal prefix of {sample_tokens} tokens of one KV group ({small.heads_q} query heads) of {w.name}",
+        }
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

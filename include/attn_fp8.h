@@ -146,6 +146,22 @@ attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtenso
                            float* diag_rowsum_ds, float* diag_rowsum_abs_ds,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* The two halves of attn_fp8_bwd, for callers that need only one of them (frozen keys/values,
+ * or timing the two kernels separately).  Same arguments and meaning as attn_fp8_bwd:
+ *   attn_fp8_bwd_dq    the query-major pass: dQ (and the optional row statistics);
+ *                      reads q.row_*, k.row_*, k.col_*, v.row_*, dO.row_*, lse, delta
+ *   attn_fp8_bwd_dkdv  the key-major pass: dK and dV;
+ *                      reads q.row_*, q.col_*, k.row_*, v.row_*, dO.row_*, dO.col_*, lse, delta
+ * attn_fp8_bwd is exactly the first followed by the second on the same stream.               */
+attn_status_t attn_fp8_bwd_dq(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                              attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                              float* diag_rowsum_ds, float* diag_rowsum_abs_ds,
+                              void* workspace, size_t workspace_bytes, void* stream);
+attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                attn_qtensor_t dO, const float* lse, const float* delta,
+                                void* dk_bf16, void* dv_bf16,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of workspace the given entry point needs for `p` (attn_ws_kind_t).  The workspace is
  * scratch: contents are undefined between calls, the library clears what it needs.  Its first
  * word is the device-side status that attn_fp8_read_status returns.                           */

@@ -33,7 +33,7 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta",
-    "attn_fp8_bwd", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
+    "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
 )
 
 
@@ -70,6 +70,12 @@ _lib.attn_fp8_bwd_delta.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor,
 _lib.attn_fp8_bwd.restype = _i32
 _lib.attn_fp8_bwd.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp, _vp,
                               _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.attn_fp8_bwd_dq.restype = _i32
+_lib.attn_fp8_bwd_dq.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp, _vp,
+                                 _vp, _vp, _sz, _vp]
+_lib.attn_fp8_bwd_dkdv.restype = _i32
+_lib.attn_fp8_bwd_dkdv.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp,
+                                   _vp, _vp, _sz, _vp]
 _lib.attn_fp8_workspace_bytes.restype = _sz
 _lib.attn_fp8_workspace_bytes.argtypes = [ctypes.POINTER(_Params), _i32]
 _lib.attn_fp8_read_status.restype = _i32
@@ -149,8 +155,10 @@ def unpack_scales(scales: torch.Tensor, B: int, H: int, rows: int, cols: int) ->
     return slab[:, idx].reshape(B, H, rows, nb)
 
 
-def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None) -> QTensor:
-    """Quantise ``src`` [B, H, N, d] (BF16 or FP32, CUDA, contiguous) into the requested orientations."""
+def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None,
+                      out: Optional[QTensor] = None) -> QTensor:
+    """Quantise ``src`` [B, H, N, d] (BF16 or FP32, CUDA, contiguous) into the requested orientations.
+    ``out`` reuses the buffers of an earlier call of the same shape (its non-None orientations are written)."""
     if not src.is_cuda or not src.is_contiguous() or src.dim() != 4:
         raise ValueError("src must be a contiguous CUDA tensor [B, H, N, d]")
     if src.dtype == torch.bfloat16:
@@ -160,14 +168,17 @@ def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool =
     else:
         raise ValueError("src must be bfloat16 or float32")
     B, H, N, d = src.shape
-    out = QTensor(shape=(B, H, N, d))
-    u8 = dict(dtype=torch.uint8, device=src.device)
-    if want_row:
-        out.row_codes = torch.empty((B, H, N, d), **u8)
-        out.row_scales = torch.empty(attn_fp8_scale_bytes(B, H, N, d), **u8)
-    if want_col:
-        out.col_codes = torch.empty((B, H, d, N), **u8)
-        out.col_scales = torch.empty(attn_fp8_scale_bytes(B, H, d, N), **u8)
+    if out is None:
+        out = QTensor(shape=(B, H, N, d))
+        u8 = dict(dtype=torch.uint8, device=src.device)
+        if want_row:
+            out.row_codes = torch.empty((B, H, N, d), **u8)
+            out.row_scales = torch.empty(attn_fp8_scale_bytes(B, H, N, d), **u8)
+        if want_col:
+            out.col_codes = torch.empty((B, H, d, N), **u8)
+            out.col_scales = torch.empty(attn_fp8_scale_bytes(B, H, d, N), **u8)
+    elif tuple(out.shape) != (B, H, N, d):
+        raise ValueError("out was allocated for another shape")
     _check(_lib.attn_fp8_quantize(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
     return out
 
@@ -240,3 +251,40 @@ def attn_fp8_bwd(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTe
                              _ptr(delta), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(rs), _ptr(ra), _ptr(workspace),
                              workspace.numel(), _stream(stream)))
     return dq, dk, dv, rs, ra, workspace
+
+
+def attn_fp8_bwd_dq(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dq=None,
+                    diagnostics: bool = False, workspace=None, stream=None):
+    """Query-major half of the gradient pass.  Returns (dQ, rowsum_dS or None, rowsum_abs_dS or None, workspace)."""
+    dev = lse.device
+    B, N = params.batch, params.seqlen
+    if dq is None:
+        dq = torch.empty((B, params.heads_q, N, params.head_dim_qk), dtype=torch.bfloat16, device=dev)
+    rs = ra = None
+    if diagnostics:
+        rs = torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev)
+        ra = torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev)
+    workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd_dq(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(), _ptr(lse),
+                                _ptr(delta), _ptr(dq), _ptr(rs), _ptr(ra), _ptr(workspace), workspace.numel(),
+                                _stream(stream)))
+    return dq, rs, ra, workspace
+
+
+def attn_fp8_bwd_dkdv(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dk=None,
+                      dv=None, workspace=None, stream=None):
+    """Key-major half of the gradient pass.  Returns (dK, dV, workspace)."""
+    dev = lse.device
+    bf = dict(dtype=torch.bfloat16, device=dev)
+    B, N = params.batch, params.seqlen
+    if dk is None:
+        dk = torch.empty((B, params.heads_kv, N, params.head_dim_qk), **bf)
+    if dv is None:
+        dv = torch.empty((B, params.heads_kv, N, params.head_dim_v), **bf)
+    workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd_dkdv(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),
+                                  _ptr(lse), _ptr(delta), _ptr(dk), _ptr(dv), _ptr(workspace), workspace.numel(),
+                                  _stream(stream)))
+    return dk, dv, workspace

@@ -177,29 +177,59 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
   return launch_bwd_delta(s, q, k, v, dO, lse, delta, status, st);
 }
 
-attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
-                           attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
-                           void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
-                           size_t workspace_bytes, void* stream) {
+static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                              attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
+                              void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
+                              size_t workspace_bytes, void* stream, bool want_dq, bool want_dkdv) {
   AttnShape s;
   CHECK(check_params(p, &s));
   CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
-  CHECK(check_ptr(q.col_codes, "q.col_codes")); CHECK(check_ptr(q.col_scales, "q.col_scales"));
   CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
-  CHECK(check_ptr(k.col_codes, "k.col_codes")); CHECK(check_ptr(k.col_scales, "k.col_scales"));
   CHECK(check_ptr(v.row_codes, "v.row_codes")); CHECK(check_ptr(v.row_scales, "v.row_scales"));
   CHECK(check_ptr(dO.row_codes, "dO.row_codes")); CHECK(check_ptr(dO.row_scales, "dO.row_scales"));
-  CHECK(check_ptr(dO.col_codes, "dO.col_codes")); CHECK(check_ptr(dO.col_scales, "dO.col_scales"));
   CHECK(check_ptr(lse, "lse")); CHECK(check_ptr(delta, "delta"));
-  CHECK(check_ptr(dq_bf16, "dq_bf16")); CHECK(check_ptr(dk_bf16, "dk_bf16")); CHECK(check_ptr(dv_bf16, "dv_bf16"));
-  if ((diag_rowsum_ds == nullptr) != (diag_rowsum_abs_ds == nullptr))
-    return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
+  if (want_dq) {
+    CHECK(check_ptr(k.col_codes, "k.col_codes")); CHECK(check_ptr(k.col_scales, "k.col_scales"));
+    CHECK(check_ptr(dq_bf16, "dq_bf16"));
+    if ((diag_rowsum_ds == nullptr) != (diag_rowsum_abs_ds == nullptr))
+      return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
+  }
+  if (want_dkdv) {
+    CHECK(check_ptr(q.col_codes, "q.col_codes")); CHECK(check_ptr(q.col_scales, "q.col_scales"));
+    CHECK(check_ptr(dO.col_codes, "dO.col_codes")); CHECK(check_ptr(dO.col_scales, "dO.col_scales"));
+    CHECK(check_ptr(dk_bf16, "dk_bf16")); CHECK(check_ptr(dv_bf16, "dv_bf16"));
+  }
   CHECK(check_device());
   int* status = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD), st, &status));
-  CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, status, st));
-  return launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st);
+  if (want_dq)
+    CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, status, st));
+  if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));
+  return ATTN_OK;
+}
+
+attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                           attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
+                           void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, dk_bf16, dv_bf16, diag_rowsum_ds, diag_rowsum_abs_ds,
+                  workspace, workspace_bytes, stream, true, true);
+}
+
+attn_status_t attn_fp8_bwd_dq(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                              attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                              float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, nullptr, nullptr, diag_rowsum_ds, diag_rowsum_abs_ds,
+                  workspace, workspace_bytes, stream, true, false);
+}
+
+attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                attn_qtensor_t dO, const float* lse, const float* delta, void* dk_bf16,
+                                void* dv_bf16, void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, q, k, v, dO, lse, delta, nullptr, dk_bf16, dv_bf16, nullptr, nullptr, workspace,
+                  workspace_bytes, stream, false, true);
 }
 
 attn_status_t attn_fp8_read_status(const void* workspace, void* stream) {
