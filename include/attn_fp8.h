@@ -162,6 +162,31 @@ attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_q
                                 void* dk_bf16, void* dv_bf16,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* Forward without a workspace argument (the paper has no counterpart; this is a packaging variant
+ * of attn_fp8_fwd and computes exactly the same O and LSE).
+ *
+ * It is meant for callers that have no way to produce device scratch at the call site: code that
+ * runs inside a host framework which owns all device memory and forbids allocation from within
+ * an operator, services whose device memory is carved up once at start-up and must not grow, and
+ * similar set-ups where cudaMalloc (or any allocating library routine) is off limits.  The scratch
+ * the forward kernel needs is therefore a fixed 4096-byte array compiled into the library; every
+ * GPU that loads the library holds those bytes until the process exits.  The call itself performs
+ * no allocation and no free of any kind.
+ *
+ *   - Problems whose scratch need (attn_fp8_workspace_bytes(p, ATTN_WS_FWD)) exceeds 4096 bytes are
+ *     rejected with ATTN_ERR_WORKSPACE and a message naming both sizes.
+ *   - The first call on each device looks up the array's device address (a one-time runtime query
+ *     made with that device current); make that first call outside of any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; the
+ *     call clears the part that has to start at zero.  Two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them, or use attn_fp8_fwd
+ *     with separate workspaces.
+ *   - The device status word lands in the built-in array and is not reported by
+ *     attn_fp8_read_status; callers that want the time-out report use attn_fp8_fwd.
+ * Arguments, layouts and error codes are otherwise those of attn_fp8_fwd.                       */
+attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                   void* o_bf16, float* lse, void* stream);
+
 /* Bytes of workspace the given entry point needs for `p` (attn_ws_kind_t).  The workspace is
  * scratch: contents are undefined between calls, the library clears what it needs.  Its first
  * word is the device-side status that attn_fp8_read_status returns.                           */

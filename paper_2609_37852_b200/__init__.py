@@ -7,7 +7,7 @@ only) and raises at import when the library has not been built.
 from the compute path.
 """
 _EXPORTS = (
-    "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta", "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv",
+    "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta", "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_workspace_bytes", "attn_fp8_last_error", "QTensor", "AttnParams",
 )
 

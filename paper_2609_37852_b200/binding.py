@@ -33,7 +33,8 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta",
-    "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
+    "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
+    "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
 )
 
 
@@ -288,3 +289,18 @@ def attn_fp8_bwd_dkdv(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO
                                   _ptr(lse), _ptr(delta), _ptr(dk), _ptr(dv), _ptr(workspace), workspace.numel(),
                                   _stream(stream)))
     return dk, dv, workspace
+
+
+_lib.attn_fp8_fwd_noalloc.restype = _i32
+_lib.attn_fp8_fwd_noalloc.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _vp, _vp, _vp]
+
+
+def attn_fp8_fwd_noalloc(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, o: torch.Tensor, lse: torch.Tensor,
+                         stream=None) -> None:
+    """Forward for call sites that may not allocate: the caller passes the outputs ``o`` and ``lse``
+    (already allocated, like the inputs) and no workspace; the library uses its built-in 4096-byte
+    scratch array.  This wrapper allocates nothing either.  Calls that overlap on the GPU share that
+    array and race; see the header for the remaining rules."""
+    c = params.c_struct()
+    _check(_lib.attn_fp8_fwd_noalloc(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), _ptr(o), _ptr(lse),
+                                     _stream(stream)))

@@ -2,6 +2,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -246,3 +247,61 @@ attn_status_t attn_fp8_read_status(const void* workspace, void* stream) {
 const char* attn_fp8_last_error(void) { return g_last_error; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Forward for callers that cannot hand over a workspace.
+//
+// The scratch the forward kernel needs (today: its status header) lives in a fixed array that is
+// part of the library image, so every GPU that loads the library carries these bytes until the
+// process exits.  In host code the array's name is only a handle: the device address has to be
+// asked for, per device, with that device current.
+namespace attnfp8 {
+
+constexpr size_t kBuiltinScratchBytes = 4096;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_builtin_scratch_addr[kMaxDevices];   // device address of the array, per device ordinal
+static std::mutex g_builtin_scratch_mutex;
+
+static attn_status_t builtin_scratch_for_current_device(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device ordinal %d is outside 0..%d", dev, kMaxDevices - 1);
+  std::lock_guard<std::mutex> lock(g_builtin_scratch_mutex);
+  if (!g_builtin_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_builtin_scratch);
+    if (e != cudaSuccess || !ptr)
+      return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress(built-in scratch) on device %d: %s", dev, cudaGetErrorString(e));
+    g_builtin_scratch_addr[dev] = ptr;
+  }
+  *out = g_builtin_scratch_addr[dev];
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8
+
+extern "C" attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k,
+                                              attn_qtensor_t v, void* o_bf16, float* lse, void* stream) {
+  AttnShape s;
+  CHECK(check_params(p, &s));
+  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
+  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
+  CHECK(check_ptr(v.col_codes, "v.col_codes")); CHECK(check_ptr(v.col_scales, "v.col_scales"));
+  CHECK(check_ptr(o_bf16, "o_bf16")); CHECK(check_ptr(lse, "lse"));
+  const size_t need = attn_fp8_workspace_bytes(p, ATTN_WS_FWD);
+  if (need > kBuiltinScratchBytes)
+    return fail(ATTN_ERR_WORKSPACE,
+                "attn_fp8_fwd_noalloc: this problem needs %zu bytes of scratch but the built-in array holds %zu; "
+                "use attn_fp8_fwd with a caller workspace", need, kBuiltinScratchBytes);
+  CHECK(check_device());
+  void* scratch = nullptr;
+  CHECK(builtin_scratch_for_current_device(&scratch));
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the previous call left: clear the part that must start at zero
+  CHECK(prepare_workspace(scratch, kBuiltinScratchBytes, need, st, &status));
+  return launch_fwd(s, q, k, v, o_bf16, lse, status, st);
+}
