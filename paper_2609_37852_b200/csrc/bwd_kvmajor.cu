@@ -14,9 +14,13 @@
 // in tensor memory across all query tiles and all query heads of the group: the group sum is
 // an FP32 sum, rounded to BF16 once at the end.
 //
-// Warp roles as in the query-major kernels: warp 0 TMA producer, warp 1 MMA issuer, warps 4..11
-// softmax (group w takes query columns 32w..32w+31 of each sub-tile).
+// Warp roles: warp 0 TMA producer; warps 1, 2, 3 issue the S^T, dP^T and dV/dK MMAs (one warp
+// cannot issue tcgen05.mma fast enough for small tiles); warps 4..19 are two softmax teams that
+// take alternate sub-tiles (within a team, warp % 4 selects the 32 TMEM lanes and the column
+// group w takes query columns 32w..32w+31).
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "mxfp8_device.cuh"
@@ -30,8 +34,10 @@ using namespace sm100;
 constexpr int kTile = 128;
 constexpr int kSub = 64;
 constexpr int kStages = 2;
-constexpr int kThreads = 384;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
+constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
+constexpr int kThreads = 128 + kTeams * kTeamThreads;
+constexpr int kPrepThreads = 32;                // warp 2 turns LSE into -LSE*log2(e) once per query tile
 constexpr float kLog2e = 1.4426950408889634f;
 
 constexpr uint32_t kColS = 0, kColdP = 64, kColP = 128 /* 2 x 16 */, kColdS = 160 /* 2 x 16 */;
@@ -52,6 +58,7 @@ struct KvStage {
   alignas(16) uint8_t sf_dOc[512];
   alignas(16) float lse[kTile];
   alignas(16) float delta[kTile];
+  alignas(16) float neg_lse2[kTile];          // -LSE * log2(e), written by the prep warps
 };
 
 struct KvSmem {
@@ -64,9 +71,11 @@ struct KvSmem {
   alignas(16) uint8_t sf_ds[2][512];
   uint64_t kv_full;
   uint64_t q_full[kStages], q_empty[kStages];
-  uint64_t sdp_full, sdp_free;
-  uint64_t pds_full[2];
+  uint64_t lse_ready[kStages];
+  uint64_t sdp_full[kTeams], sdp_free[kTeams];
+  uint64_t pds_full[2], pds_free[2];
   uint64_t done;
+  uint64_t drain[3];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -103,8 +112,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
-    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.sdp_free, kSoftmaxThreads);
-    mbar_init(&sm.pds_full[0], kSoftmaxThreads); mbar_init(&sm.pds_full[1], kSoftmaxThreads);
+    for (int s = 0; s < kStages; ++s) mbar_init(&sm.lse_ready[s], kPrepThreads);
+    for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); }
+    for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     mbar_init(&sm.done, 1);
     sm.abort_flag = 0;
     fence_mbar_init();
@@ -160,49 +171,103 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ S^T issuer
+    // One tcgen05.mma can be issued per ~130 cycles from one warp whatever its size, so the
+    // products are spread over three issuing warps; orderings that a single issuer would give
+    // for free are carried by mbarriers instead.
     if (lane == 0) {
       const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k));
-      const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v));
       bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
         sf_copy(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
-        sf_copy(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
       }
-      auto issue_sdp = [&](int u) -> bool {
+      for (int u = 0; u < n_sub && ok; ++u) {
         const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
         KvStage& st = sm.st[s];
         if (half == 0) {
-          if (!mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag)) return false;
+          ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after_sync();
           sf_copy(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
-          sf_copy(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
         }
         if (u > 0) {
-          if (!mbar_wait(&sm.sdp_free, (u - 1) & 1, abort_flag)) return false;
+          // the team of the previous sub-tile has pulled S and dP into registers
+          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after_sync();
         }
         const uint64_t desc_q = make_desc_sw128(smem_u32(st.q)) + half * (kSub * 128 / 16);
-        const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO)) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
           mma_mxf8_ss(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFK, tmem + kColSFQ + 4 * slot + 2 * half, kb > 0);
+        mma_commit(&sm.sdp_full[u % kTeams]);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.drain[0]);
+        mbar_wait(&sm.drain[0], 0, &dummy);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ dP^T issuer + LSE preparation
+    const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v));
+    bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
+    if (ok && lane == 0) {
+      tc_fence_after_sync();
+      sf_copy(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
+    }
+    for (int u = 0; u < n_sub && ok; ++u) {
+      const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
+      KvStage& st = sm.st[s];
+      if (half == 0) {
+        ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+        if (!ok) break;
+        // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
+        const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
+        *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
+            make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
+        mbar_arrive(&sm.lse_ready[s]);
+        if (lane == 0) {
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
+        }
+      }
+      if (u > 0) {
+        ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+        if (!ok) break;
+      }
+      if (lane == 0) {
+        tc_fence_after_sync();
+        const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO)) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_v; ++kb)
           mma_mxf8_ss(tmem + kColdP, desc_v + 2 * kb, desc_dO + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFV, tmem + kColSFdO + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full);
-        return true;
-      };
-      auto issue_dkv = [&](int u) -> bool {
+        mma_commit(&sm.sdp_full[u % kTeams]);
+      }
+    }
+    if (!ok && lane == 0) {
+      int dummy = 0;
+      mma_commit(&sm.drain[1]);
+      mbar_wait(&sm.drain[1], 0, &dummy);
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ dV / dK issuer
+    if (lane == 0) {
+      bool ok = true;
+      for (int u = 0; u < n_sub && ok; ++u) {
         const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1, buf = u & 1;
         KvStage& st = sm.st[s];
-        if (!mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag)) return false;
-        tc_fence_after_sync();
         if (half == 0) {
+          ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
           sf_copy(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
           sf_copy(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
         }
+        ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
         sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_dOc = make_desc_sw128(smem_u32(st.dOc));
@@ -215,57 +280,87 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           mma_mxf8_ts(tmem + kColdK, tmem + kColdS + 16 * buf + 8 * kb, desc_qc + 2 * (2 * half + kb),
                       make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
                       tmem + kColSFQc + 4 * slot, (u > 0 || kb > 0));
+        // codes and scale bytes of this buffer may be overwritten once these MMAs have run; the
+        // stage may be refilled after the second half (the S^T / dP^T MMAs that read it finished
+        // before the softmax team could even start on this sub-tile)
+        mma_commit(&sm.pds_free[buf]);
         if (half == 1) mma_commit(&sm.q_empty[s]);
         if (u == n_sub - 1) mma_commit(&sm.done);
-        return true;
-      };
-      if (ok) ok = issue_sdp(0);
-      for (int u = 0; u < n_sub && ok; ++u) {
-        if (u + 1 < n_sub) ok = issue_sdp(u + 1);
-        if (ok) ok = issue_dkv(u);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.kv_full);
-        mbar_wait(&sm.kv_full, 1, &dummy);
+        mma_commit(&sm.drain[2]);
+        mbar_wait(&sm.drain[2], 0, &dummy);
       }
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax
-    const int grp = (warp - 4) >> 2;
+    const int team = (warp - 4) >> 3;
+    const int grp = ((warp - 4) >> 2) & 1;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                 // key inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
     bool ok = true;
-    for (int u = 0; u < n_sub; ++u) {
+    for (int u = team; u < n_sub; u += kTeams) {
       const int n = u >> 1, half = u & 1, buf = u & 1, s = n % kStages;
       const int it = it0 + n % tiles_per_head;
-      ok = mbar_wait(&sm.sdp_full, u & 1, abort_flag);
+      ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
-      uint32_t sr[32], dpr[32];
+      uint32_t sr[32], dpr[32];                       // S then P; dP then dS (in place)
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
       tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(&sm.sdp_free);
-      const bool diag = p.causal && (it == jt);
+      mbar_arrive(&sm.sdp_free[team]);
+      ok = mbar_wait(&sm.lse_ready[s], (n / kStages) & 1, abort_flag);
+      if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
-      const float* s_lse = sm.st[s].lse + col0;
-      const float* s_delta = sm.st[s].delta + col0;
-      float pr[32], ds[32];
+      const KvStage& st = sm.st[s];
+      float amax_p = 0.f, amax_s = 0.f;
+      auto body = [&](auto diag_tag) {
+        constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -s_lse[c] * kLog2e);
-        if (diag && (row > col0 + c)) x = -INFINITY;   // key after the query
-        const float pv = ex2_approx(x);
-        pr[c] = pv;
-        ds[c] = pv * (__uint_as_float(dpr[c]) - s_delta[c]);
+        for (int c4 = 0; c4 < 32; c4 += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(&st.neg_lse2[col0 + c4]);
+          const float4 d4 = *reinterpret_cast<const float4*>(&st.delta[col0 + c4]);
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+          const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = c4 + e;
+            float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, lv[e]);
+            if (kDiag && (row > col0 + c)) x = -INFINITY;      // key after the query
+            const float pv = ex2_approx(x);
+            const float dsv = pv * (__uint_as_float(dpr[c]) - dv4[e]);
+            sr[c] = __float_as_uint(pv);
+            dpr[c] = __float_as_uint(dsv);
+            amax_p = fmaxf(amax_p, pv);
+            amax_s = fmaxf(amax_s, fabsf(dsv));
+          }
+        }
+      };
+      if (p.causal && it == jt) body(std::true_type{}); else body(std::false_type{});
+      uint32_t byte_p, byte_s;
+      float inv_p, inv_s;
+      block_scale(amax_p, byte_p, inv_p);
+      block_scale(amax_s, byte_s, inv_s);
+      if (u >= 2) {
+        // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+        ok = mbar_wait(&sm.pds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
       }
       uint32_t words[8];
-      const uint32_t byte_p = quantize_block32(pr, words);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        words[i] = cvt_e4m3x4(__uint_as_float(sr[4 * i]) * inv_p, __uint_as_float(sr[4 * i + 1]) * inv_p,
+                              __uint_as_float(sr[4 * i + 2]) * inv_p, __uint_as_float(sr[4 * i + 3]) * inv_p);
       tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
-      const uint32_t byte_s = quantize_block32(ds, words);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        words[i] = cvt_e4m3x4(__uint_as_float(dpr[4 * i]) * inv_s, __uint_as_float(dpr[4 * i + 1]) * inv_s,
+                              __uint_as_float(dpr[4 * i + 2]) * inv_s, __uint_as_float(dpr[4 * i + 3]) * inv_s);
       tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
       const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
       sm.sf_p[buf][sf_at] = static_cast<uint8_t>(byte_p);
@@ -275,6 +370,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tc_fence_before_sync();
       mbar_arrive(&sm.pds_full[buf]);
     }
+    // the epilogue is done by team 0 (group 0 stores dV, group 1 stores dK)
+    if (team != 0) ok = false;
     if (ok) ok = mbar_wait(&sm.done, 0, abort_flag);
     if (ok) {
       tc_fence_after_sync();
