@@ -129,6 +129,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_base;
 
+
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
@@ -317,13 +318,15 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
       const KvStage& st = sm.st[s];
-      float amax_p = 0.f, amax_s = 0.f;
+      float amax_p = 0.f, max_s = 0.f, min_s = 0.f;   // |dS| maximum from a running max and min
+      const float* s_lse = &st.neg_lse2[col0];
+      const float* s_delta = &st.delta[col0];
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
         for (int c4 = 0; c4 < 32; c4 += 4) {
-          const float4 l4 = *reinterpret_cast<const float4*>(&st.neg_lse2[col0 + c4]);
-          const float4 d4 = *reinterpret_cast<const float4*>(&st.delta[col0 + c4]);
+          const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[c4]);
+          const float4 d4 = *reinterpret_cast<const float4*>(&s_delta[c4]);
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
           const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
@@ -336,7 +339,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             sr[c] = __float_as_uint(pv);
             dpr[c] = __float_as_uint(dsv);
             amax_p = fmaxf(amax_p, pv);
-            amax_s = fmaxf(amax_s, fabsf(dsv));
+            max_s = fmaxf(max_s, dsv);
+            min_s = fminf(min_s, dsv);
           }
         }
       };
@@ -344,7 +348,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       uint32_t byte_p, byte_s;
       float inv_p, inv_s;
       block_scale(amax_p, byte_p, inv_p);
-      block_scale(amax_s, byte_s, inv_s);
+      block_scale(fmaxf(max_s, -min_s), byte_s, inv_s);
       if (u >= 2) {
         // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
         ok = mbar_wait(&sm.pds_free[buf], ((u - 2) >> 1) & 1, abort_flag);

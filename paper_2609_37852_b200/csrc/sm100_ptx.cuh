@@ -39,22 +39,51 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity
   return ok;
 }
 
+// Same test, but the hardware may park the thread for up to `ns` nanoseconds while the phase is
+// still open (it is woken as soon as the phase completes), which keeps waiting warps out of the
+// issue slots.
+__device__ __forceinline__ uint32_t mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok;
+}
+
 // Bounded wait: gives up after about `kWaitLimitCycles` SM cycles or as soon as another thread
 // of the CTA has raised `*abort_flag`.  Returns false on give-up (and raises the flag).
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at 2 GHz
+constexpr uint32_t kParkNs = 20000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
+  long long t0 = 0;
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 0x3FF) == 0) {
-      if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+  while (!mbar_try_wait_parked(bar, parity, kParkNs)) {
+    // the clock and the abort flag are looked at once every 64 polls to keep the loop short
+    if ((++spins & 63) == 0) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (*abort_flag || now - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
         return false;
       }
     }
   }
   return true;
+}
+
+// 16-byte load from shared memory (the address space is stated, so no generic load is emitted).
+__device__ __forceinline__ float4 lds_f4(const void* p) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(smem_u32(p)));
+  return v;
 }
 
 // ------------------------------------------------------------------ proxies / fences
@@ -72,6 +101,16 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t nthread
 }
 __device__ __forceinline__ void named_barrier_arrive(uint32_t id, uint32_t nthreads) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Register re-allocation between warpgroups (all four warps of a warpgroup must execute it).
+template <int N>
+__device__ __forceinline__ void reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // ------------------------------------------------------------------ TMA
