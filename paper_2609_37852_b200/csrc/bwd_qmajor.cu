@@ -14,8 +14,9 @@
 // Both modes run the same instruction sequence for P and dP, so the correction the first
 // produces is the one that zeroes the row sums of the second up to FP32 rounding.
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 4..11 softmax (two groups of four
-// warps; group w takes columns 32w..32w+31 of each sub-tile, warp % 4 selects the 32 TMEM lanes).
+// Warp roles: warp 0 TMA producer; warps 1, 2, 3 issue the S, dP and dQ MMAs; warps 4..19 are two
+// softmax teams that take alternate sub-tiles (inside a team, column group w takes columns
+// 32w..32w+31 of the sub-tile and warp % 4 selects the 32 TMEM lanes).
 // S and dP are single-buffered: the softmax warps pull them into registers and release the
 // buffers at once, so the next sub-tile's MMAs overlap the exponentials of this one.
 #include <cuda_bf16.h>
@@ -32,8 +33,9 @@ using namespace sm100;
 constexpr int kTile = 128;
 constexpr int kSub = 64;
 constexpr int kStages = 2;
-constexpr int kThreads = 384;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
+constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
+constexpr int kThreads = 128 + kTeams * kTeamThreads;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
 
@@ -54,13 +56,14 @@ struct QmSmem {
   alignas(16) uint8_t sf_v[kStages][512];
   alignas(16) uint8_t sf_kc[kStages][512];
   alignas(16) uint8_t sf_ds[2][512];
-  alignas(16) float red[3][kTile];          // cross-group reduction of row sums
+  alignas(16) float red[2 * kTeams][2][kTile];   // partial row sums of every (team, column group)
   uint64_t q_full;
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[kStages], kc_empty[kStages];
-  uint64_t sdp_full, sdp_free;
-  uint64_t ds_full[2];
+  uint64_t sdp_full[kTeams], sdp_free[kTeams];
+  uint64_t ds_full[2], ds_free[2];
   uint64_t dq_done;
+  uint64_t drain[3];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -97,12 +100,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1);
+      mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 2);   // released by the S and the dP issuer
       mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1);
     }
-    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.sdp_free, kSoftmaxThreads);
-    mbar_init(&sm.ds_full[0], kSoftmaxThreads); mbar_init(&sm.ds_full[1], kSoftmaxThreads);
+    for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kTeamThreads); mbar_init(&sm.ds_free[i], 1); }
     mbar_init(&sm.dq_done, 1);
+    for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     sm.abort_flag = 0;
     fence_mbar_init();
   }
@@ -157,48 +161,93 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ S issuer
+    // One warp can issue one tcgen05.mma per ~130 cycles whatever its size, so the three products
+    // have an issuing warp each; orderings a single issuer would give for free are carried by
+    // mbarriers instead.
     if (lane == 0) {
       const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
-      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
         sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
-        sf_copy(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
       }
-      auto issue_sdp = [&](int u) -> bool {
+      for (int u = 0; u < n_sub && ok; ++u) {
         const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
         if (half == 0) {
-          if (!mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag)) return false;
+          ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after_sync();
           sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
-          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
         }
         if (u > 0) {
-          if (!mbar_wait(&sm.sdp_free, (u - 1) & 1, abort_flag)) return false;
+          // the team of the previous sub-tile has pulled S and dP into registers
+          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after_sync();
         }
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
           mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
+        mma_commit(&sm.sdp_full[u % kTeams]);
+        if (half == 1) mma_commit(&sm.kv_empty[s]);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.drain[0]);
+        mbar_wait(&sm.drain[0], 0, &dummy);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ dP issuer
+    if (lane == 0) {
+      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO));
+      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
+      }
+      for (int u = 0; u < n_sub && ok; ++u) {
+        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
+        if (half == 0) {
+          ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        }
+        if (u > 0) {
+          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_v; ++kb)
           mma_mxf8_ss(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFdO, tmem + kColSFV + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full);
+        mma_commit(&sm.sdp_full[u % kTeams]);
         if (half == 1) mma_commit(&sm.kv_empty[s]);
-        return true;
-      };
-      auto issue_dq = [&](int u) -> bool {
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.drain[1]);
+        mbar_wait(&sm.drain[1], 0, &dummy);
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ dQ issuer
+    if (kDQ && lane == 0) {
+      bool ok = true;
+      for (int u = 0; u < n_sub && ok; ++u) {
         const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
         if (half == 0) {
-          if (!mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag)) return false;
+          ok = mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after_sync();
           sf_copy(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
         }
-        if (!mbar_wait(&sm.ds_full[buf], (u >> 1) & 1, abort_flag)) return false;
+        ok = mbar_wait(&sm.ds_full[buf], (u >> 1) & 1, abort_flag);
+        if (!ok) break;
         tc_fence_after_sync();
         sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
@@ -206,28 +255,20 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           mma_mxf8_ts(tmem + kColdQ, tmem + kColdS + 16 * buf + 8 * kb, desc_kc + 2 * (2 * half + kb),
                       make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
                       tmem + kColSFKc + 4 * slot, (u > 0 || kb > 0));
+        mma_commit(&sm.ds_free[buf]);            // codes and scale bytes of this buffer may be overwritten
         if (half == 1) mma_commit(&sm.kc_empty[s]);
         if (u == n_sub - 1) mma_commit(&sm.dq_done);
-        return true;
-      };
-      if (kDQ) {
-        if (ok) ok = issue_sdp(0);
-        for (int u = 0; u < n_sub && ok; ++u) {
-          if (u + 1 < n_sub) ok = issue_sdp(u + 1);
-          if (ok) ok = issue_dq(u);
-        }
-      } else {
-        for (int u = 0; u < n_sub && ok; ++u) ok = issue_sdp(u);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.q_full);
-        mbar_wait(&sm.q_full, 1, &dummy);
+        mma_commit(&sm.drain[2]);
+        mbar_wait(&sm.drain[2], 0, &dummy);
       }
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax
-    const int grp = (warp - 4) >> 2;                  // column half of each sub-tile
+    const int team = (warp - 4) >> 3;
+    const int grp = ((warp - 4) >> 2) & 1;            // column half of each sub-tile
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
@@ -240,9 +281,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float D = kDQ ? p.delta_in[grow] : 0.f;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
     bool ok = true;
-    for (int u = 0; u < n_sub; ++u) {
+    for (int u = team; u < n_sub; u += kTeams) {
       const int t = u >> 1, half = u & 1, buf = u & 1;
-      ok = mbar_wait(&sm.sdp_full, u & 1, abort_flag);
+      ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
@@ -250,7 +291,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(&sm.sdp_free);
+      mbar_arrive(&sm.sdp_free[team]);
       const bool diag = p.causal && (t == qt);
       const int col0 = half * kSub + 32 * grp;        // column of this thread's first element inside the key tile
       float ds[32];
@@ -275,6 +316,12 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       } else {
         uint32_t words[8];
         const uint32_t byte = quantize_block32(ds, words);
+        if (u >= 2) {
+          // the dQ MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+          ok = mbar_wait(&sm.ds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
         tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
         sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
         tmem_wait_st();
@@ -283,15 +330,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
-    // combine the two column groups' row sums
-    if (grp == 1) {
-      sm.red[0][row] = acc0;
-      sm.red[1][row] = acc1;
-    }
-    named_barrier_sync(1, kSoftmaxThreads);
-    if (ok && grp == 0) {
-      acc0 += sm.red[0][row];
-      acc1 += sm.red[1][row];
+    // combine the row sums of the teams and column groups (fixed order: reproducible)
+    sm.red[team * 2 + grp][0][row] = acc0;
+    sm.red[team * 2 + grp][1][row] = acc1;
+    named_barrier_sync(1, kTeams * kTeamThreads);
+    if (ok && team == 0 && grp == 0) {
+      acc0 = 0.f; acc1 = 0.f;
+      for (int i = 0; i < 2 * kTeams; ++i) { acc0 += sm.red[i][0][row]; acc1 += sm.red[i][1][row]; }
       if (!kDQ) {
         p.delta_out[grow] = acc0;
       } else if (p.rowsum) {
@@ -299,7 +344,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         p.rowabs[grow] = acc1;
       }
     }
-    if (kDQ && ok) {
+    if (kDQ && ok && team == 0) {
       ok = mbar_wait(&sm.dq_done, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
