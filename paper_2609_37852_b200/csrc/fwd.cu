@@ -1,22 +1,26 @@
 // Forward attention with block-scaled FP8 operands (paper Appendix "Forward Probability
 // Encoding", re-designed for tcgen05 / tensor memory).
 //
-// One CTA owns 128 query rows of one (batch, query head) and walks the key tiles (128 keys) up
-// to the causal diagonal.  Warp roles:
-//   warp 0      TMA producer: Q tile once, then K tiles and V tiles through two rings
-//   warp 1      MMA issuer (one elected lane): S = Q K^T and O += P V, both block-scaled,
-//               accumulating in tensor memory; S is double-buffered so that the scores of
-//               tile t+1 are computed while the softmax warps work on tile t
-//   warps 4..7  softmax: one query row per thread (thread <-> TMEM lane).  Scores are scaled
-//               into log2 units; the running shift M is an INTEGER, so rescaling is by exact
-//               powers of two and the E4M3 codes of the probabilities do not depend on the
-//               tile order; l accumulates the exponentials BEFORE the FP8 cast; probabilities
-//               are quantised in blocks of 32 keys in registers and written back to tensor
-//               memory (over the S buffer) as the A operand of the second MMA, their scale
-//               bytes going through shared memory into the scale-factor columns.
-// M is only raised when the tile maximum exceeds it by more than kLazyShift (the block scales
+// One CTA owns 128 query rows of one (batch, query head) and walks the keys up to the causal
+// diagonal, 64 keys at a time; it uses 256 of the 512 tensor-memory columns and under half of the
+// shared memory, so two CTAs share an SM and each fills the other's stalls.  Warp roles:
+//   warp 0      TMA producer: Q tile once, then K tiles [128 keys x d] and V tiles [dv x 128 keys]
+//   warp 1      issues S = Q K^T (block-scaled, 128 x 64 per sub-tile)
+//   warp 2      issues O += P V (A operand = quantised probabilities read from tensor memory)
+//   warps 4..7  softmax: one query row per thread (thread <-> TMEM lane).  A thread pulls its 64
+//               scores into registers and releases the score buffer at once, so the next S is
+//               computed while it works.  Scores go to log2 units; the running shift M is an
+//               INTEGER, so rescaling is by exact powers of two and the E4M3 codes of the
+//               probabilities do not depend on the tile order; l accumulates the exponentials
+//               BEFORE the FP8 cast; probabilities are quantised in blocks of 32 keys in
+//               registers and written to tensor memory as the A operand of the second MMA, their
+//               scale bytes going through shared memory into the scale-factor columns.
+// M is only raised when the sub-tile maximum exceeds it by more than kLazyShift (the block scales
 // absorb the difference), so the accumulator in tensor memory is almost never rescaled.
+// Two MMA-issuing warps because one warp issues at most one tcgen05.mma per ~130 cycles.
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "mxfp8_device.cuh"
@@ -27,22 +31,25 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kTile = 128;          // query rows per CTA and keys per tile
-constexpr int kStages = 3;          // K ring and V ring depth
+constexpr int kTile = 128;          // query rows per CTA; keys per K / V tile in shared memory
+constexpr int kSub = 64;            // keys per softmax step
+constexpr int kStages = 2;          // K ring and V ring depth
 constexpr int kThreads = 256;
+constexpr int kSoftmaxThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
 constexpr int kLazyShift = 8;
 
-// tensor-memory columns
-constexpr uint32_t kColS = 0;        // two score buffers of 128 columns; P codes alias columns 0..31
-constexpr uint32_t kColO = 256;      // output accumulator, dv columns
-constexpr uint32_t kColSFQ = 384;    // scale factors: Q (4), K (2 x 4), V (2 x 4), P (2 x 4)
-constexpr uint32_t kColSFK = 388;
-constexpr uint32_t kColSFV = 396;
-constexpr uint32_t kColSFP = 404;
-constexpr uint32_t kTmemCols = 512;
+// tensor-memory columns (256 allocated)
+constexpr uint32_t kColS = 0;        // scores of the current sub-tile, 64 columns
+constexpr uint32_t kColP = 64;       // probability codes, two buffers of 16 columns
+constexpr uint32_t kColO = 96;       // output accumulator, dv (<= 128) columns
+constexpr uint32_t kColSFQ = 224;    // scale factors: Q (4), K (2 x 4), V (2 x 4), P (2 x 4)
+constexpr uint32_t kColSFK = 228;
+constexpr uint32_t kColSFV = 236;
+constexpr uint32_t kColSFP = 244;
+constexpr uint32_t kTmemCols = 256;
 
 struct FwdSmem {
   alignas(1024) uint8_t q[kTile * 128];
@@ -55,7 +62,10 @@ struct FwdSmem {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages];
   uint64_t v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], p_full[2], pv_done[2];
+  uint64_t s_full, s_free;
+  uint64_t p_full[2], p_free[2];
+  uint64_t o_done;
+  uint64_t drain[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -71,7 +81,7 @@ struct FwdParams {
   float scale_log2;         // softmax_scale * log2(e)
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ uint8_t smem_raw[];
@@ -82,6 +92,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
+  const int n_sub = 2 * n_tiles;
   const int nk_qk = p.dqk / 32;                 // K blocks of the score MMA
   volatile int* abort_flag = &sm.abort_flag;
 
@@ -91,9 +102,10 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_full[i], 128); mbar_init(&sm.pv_done[i], 1);
-    }
+    mbar_init(&sm.s_full, 1); mbar_init(&sm.s_free, kSoftmaxThreads);
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.p_full[i], kSoftmaxThreads); mbar_init(&sm.p_free[i], 1); }
+    mbar_init(&sm.o_done, 1);
+    mbar_init(&sm.drain[0], 1); mbar_init(&sm.drain[1], 1);
     sm.abort_flag = 0;
     fence_mbar_init();
   }
@@ -142,7 +154,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ S = Q K^T issuer
     if (lane == 0) {
       const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
@@ -150,45 +162,62 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         tc_fence_after_sync();
         sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
       }
-      auto issue_qk = [&](int t) -> bool {
-        const int s = t % kStages, u = t / kStages, buf = t & 1;
-        if (!mbar_wait(&sm.k_full[s], u & 1, abort_flag)) return false;
-        tc_fence_after_sync();
-        sf_copy(tmem + kColSFK + 4 * buf, make_desc_sf(smem_u32(sm.sf_k[s])));
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s]));
+      for (int u = 0; u < n_sub && ok; ++u) {
+        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
+        if (half == 0) {
+          ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+        }
+        if (u > 0) {
+          // the softmax threads have pulled the previous scores into registers
+          ok = mbar_wait(&sm.s_free, (u - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS + 128 * buf, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
-                      tmem + kColSFQ, tmem + kColSFK + 4 * buf, kb > 0);
-        mma_commit(&sm.k_empty[s]);
-        mma_commit(&sm.s_full[buf]);
-        return true;
-      };
-      auto issue_pv = [&](int t) -> bool {
-        const int s = t % kStages, u = t / kStages, buf = t & 1;
-        if (!mbar_wait(&sm.v_full[s], u & 1, abort_flag)) return false;
-        if (!mbar_wait(&sm.p_full[buf], (t >> 1) & 1, abort_flag)) return false;
-        tc_fence_after_sync();
-        sf_copy(tmem + kColSFV + 4 * buf, make_desc_sf(smem_u32(sm.sf_v[s])));
-        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
-        for (int kb = 0; kb < 4; ++kb)
-          mma_mxf8_ts(tmem + kColO, tmem + kColS + 128 * buf + 8 * kb, desc_v + 2 * kb,
-                      make_idesc_mxf8(128, p.dv, kb, kb), tmem + kColSFP + 4 * buf, tmem + kColSFV + 4 * buf,
-                      (t > 0 || kb > 0));
-        mma_commit(&sm.v_empty[s]);
-        mma_commit(&sm.pv_done[buf]);
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        if (t + 1 < n_tiles) ok = issue_qk(t + 1);
-        if (ok) ok = issue_pv(t);
+          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+                      tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
+        mma_commit(&sm.s_full);
+        if (half == 1) mma_commit(&sm.k_empty[s]);
       }
       if (!ok) {
-        // drain whatever was issued so that tensor memory can be released safely
         int dummy = 0;
-        mma_commit(&sm.q_full);
-        mbar_wait(&sm.q_full, 1, &dummy);
+        mma_commit(&sm.drain[0]);
+        mbar_wait(&sm.drain[0], 0, &dummy);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ O += P V issuer
+    if (lane == 0) {
+      bool ok = true;
+      for (int u = 0; u < n_sub && ok; ++u) {
+        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
+        if (half == 0) {
+          ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        }
+        ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
+        for (int kb = 0; kb < 2; ++kb)
+          mma_mxf8_ts(tmem + kColO, tmem + kColP + 16 * buf + 8 * kb, desc_v + 2 * (2 * half + kb),
+                      make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
+                      tmem + kColSFV + 4 * slot, (u > 0 || kb > 0));
+        mma_commit(&sm.p_free[buf]);              // codes / scale bytes of this buffer consumed; O updated
+        if (half == 1) mma_commit(&sm.v_empty[s]);
+        if (u == n_sub - 1) mma_commit(&sm.o_done);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit(&sm.drain[1]);
+        mbar_wait(&sm.drain[1], 0, &dummy);
       }
     }
   } else if (warp >= 4) {
@@ -196,38 +225,46 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                 // row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-    float M = -INFINITY;                              // integer-valued running shift
+    float M = -INFINITY;                              // integer-valued running shift (log2 units)
     float l = 0.f;
     bool ok = true;
-    for (int t = 0; t < n_tiles; ++t) {
-      const int buf = t & 1;
-      ok = mbar_wait(&sm.s_full[buf], (t >> 1) & 1, abort_flag);
+    for (int u = 0; u < n_sub; ++u) {
+      const int t = u >> 1, half = u & 1, buf = u & 1;
+      ok = mbar_wait(&sm.s_full, u & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
-      float s2[128];
+      float sv[kSub];
       {
-        uint32_t* r = reinterpret_cast<uint32_t*>(s2);
-        const uint32_t a = tmem + kColS + 128 * buf + lane_addr;
-        tmem_ld32(a, r); tmem_ld32(a + 32, r + 32); tmem_ld32(a + 64, r + 64); tmem_ld32(a + 96, r + 96);
+        uint32_t* r = reinterpret_cast<uint32_t*>(sv);
+        tmem_ld32(tmem + kColS + lane_addr, r);
+        tmem_ld32(tmem + kColS + lane_addr + 32, r + 32);
         tmem_wait_ld();
       }
-      const bool diag = p.causal && (t == qt);
+      tc_fence_before_sync();
+      mbar_arrive(&sm.s_free);
+      // maximum of the raw accumulators (the scale is positive), masked on the diagonal tile
       float mx = -INFINITY;
+      if (p.causal && t == qt) {
+        const int col0 = half * kSub;
 #pragma unroll
-      for (int c = 0; c < 128; ++c) {
-        float x = s2[c] * p.scale_log2;
-        if (diag && c > row) x = -INFINITY;
-        s2[c] = x;
-        mx = fmaxf(mx, x);
+        for (int c = 0; c < kSub; ++c) {
+          if (col0 + c > row) sv[c] = -INFINITY;
+          mx = fmaxf(mx, sv[c]);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < kSub; ++c) mx = fmaxf(mx, sv[c]);
       }
-      const float m_new = ceilf(mx);
-      const bool raise = m_new > M + static_cast<float>(kLazyShift);   // always true on the first tile
+      // a fully masked sub-tile (second half of the diagonal tile for the first 64 rows) gives -inf:
+      // it never raises M and contributes zeros
+      const float m_new = ceilf(mx * p.scale_log2);
+      const bool raise = m_new > M + static_cast<float>(kLazyShift);   // true on the first sub-tile
       if (__any_sync(0xffffffffu, raise)) {
-        const float factor = raise ? exp2f(M - m_new) : 1.f;            // exact power of two (0 on the first tile)
+        const float factor = raise ? exp2f(M - m_new) : 1.f;            // exact power of two (0 at the start)
         if (raise) { l *= factor; M = m_new; }
-        if (t > 0) {
+        if (u > 0) {
           // the previous P V product must have landed before the accumulator is touched
-          ok = mbar_wait(&sm.pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, abort_flag);
+          ok = mbar_wait(&sm.p_free[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           for (int c0 = 0; c0 < p.dv; c0 += 32) {
@@ -241,36 +278,49 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tmem_wait_st();
         }
       }
-      uint32_t sf_word = 0;
-      float tile_sum = 0.f;                     // summed per block, per tile, then into l: short chains
+      const float neg_m = -M;
+      uint32_t words[16];
+      uint32_t sf_half = 0;
+      float sub_sum = 0.f;                            // per block, per sub-tile, then into l: short chains
 #pragma unroll
-      for (int blk = 0; blk < 4; ++blk) {
-        float pexp[32];
-        float bs0 = 0.f, bs1 = 0.f;
+      for (int blk = 0; blk < 2; ++blk) {
+        float bs0 = 0.f, bs1 = 0.f, amax = 0.f;
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          pexp[c] = ex2_approx(s2[blk * 32 + c] - M);
-          pexp[c + 1] = ex2_approx(s2[blk * 32 + c + 1] - M);
-          bs0 += pexp[c];
-          bs1 += pexp[c + 1];
+          const float p0 = ex2_approx(fmaf(sv[blk * 32 + c], p.scale_log2, neg_m));
+          const float p1 = ex2_approx(fmaf(sv[blk * 32 + c + 1], p.scale_log2, neg_m));
+          sv[blk * 32 + c] = p0;
+          sv[blk * 32 + c + 1] = p1;
+          bs0 += p0;
+          bs1 += p1;
+          amax = fmaxf(amax, fmaxf(p0, p1));
         }
-        tile_sum += bs0 + bs1;
-        uint32_t words[8];
-        const uint32_t byte = quantize_block32(pexp, words);
-        sf_word |= byte << (8 * blk);
-        tmem_st8(tmem + kColS + 128 * buf + lane_addr + 8 * blk, words);
+        sub_sum += bs0 + bs1;
+        uint32_t byte;
+        float inv;
+        block_scale(amax, byte, inv);
+        sf_half |= byte << (8 * blk);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          words[blk * 8 + i] = cvt_e4m3x4(sv[blk * 32 + 4 * i] * inv, sv[blk * 32 + 4 * i + 1] * inv,
+                                          sv[blk * 32 + 4 * i + 2] * inv, sv[blk * 32 + 4 * i + 3] * inv);
       }
-      l += tile_sum;
-      *reinterpret_cast<uint32_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = sf_word;
+      l += sub_sum;
+      if (u >= 2) {
+        // the P V MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+        ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+      }
+      tmem_st8(tmem + kColP + 16 * buf + lane_addr, words);
+      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8, words + 8);
+      *reinterpret_cast<uint16_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = static_cast<uint16_t>(sf_half);
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.p_full[buf]);
     }
-    if (ok) {
-      const int last = n_tiles - 1;
-      ok = mbar_wait(&sm.pv_done[last & 1], (last >> 1) & 1, abort_flag);
-    }
+    if (ok) ok = mbar_wait(&sm.o_done, 0, abort_flag);
     if (ok) {
       tc_fence_after_sync();
       const float inv_l = 1.f / l;
