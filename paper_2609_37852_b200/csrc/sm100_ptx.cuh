@@ -60,19 +60,39 @@ __device__ __forceinline__ uint32_t mbar_try_wait_parked(uint64_t* bar, uint32_t
 // of the CTA has raised `*abort_flag`.  Returns false on give-up (and raises the flag).
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at 2 GHz
 constexpr uint32_t kParkNs = 20000;
+// The poll loop is written in PTX so that an iteration is a handful of instructions: waiting
+// warps share issue slots with the warps that do the arithmetic.  Each poll parks the thread for
+// up to kParkNs (the hardware wakes it when the phase completes); after kPollsPerCheck polls the
+// clock and the CTA's abort flag are looked at.
+constexpr uint32_t kPollsPerCheck = 4096;
+__device__ __forceinline__ uint32_t mbar_poll(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      ".reg .u32 n;\n"
+      "mov.u32 n, 0;\n"
+      "WAIT_LOOP:\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "@p bra WAIT_DONE;\n"
+      "add.u32 n, n, 1;\n"
+      "setp.lt.u32 q, n, %4;\n"
+      "@q bra WAIT_LOOP;\n"
+      "WAIT_DONE:\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kParkNs), "r"(max_polls)
+      : "memory");
+  return ok;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  long long t0 = 0;
-  uint32_t spins = 0;
-  while (!mbar_try_wait_parked(bar, parity, kParkNs)) {
-    // the clock and the abort flag are looked at once every 64 polls to keep the loop short
-    if ((++spins & 63) == 0) {
-      const long long now = clock64();
-      if (t0 == 0) t0 = now;
-      if (*abort_flag || now - t0 > kWaitLimitCycles) {
-        *abort_flag = 1;
-        return false;
-      }
+  const long long t0 = clock64();
+  while (!mbar_poll(bar, parity, kPollsPerCheck)) {
+    if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      return false;
     }
   }
   return true;
@@ -159,6 +179,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
 }
