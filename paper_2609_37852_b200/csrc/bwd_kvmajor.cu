@@ -112,7 +112,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
-    for (int s = 0; s < kStages; ++s) mbar_init(&sm.lse_ready[s], kPrepThreads);
+    for (int s = 0; s < kStages; ++s) mbar_init(&sm.lse_ready[s], 1);
     for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); }
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
@@ -228,7 +228,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
         *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
             make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
-        mbar_arrive(&sm.lse_ready[s]);
+        mbar_arrive_warp(&sm.lse_ready[s]);
         if (lane == 0) {
           tc_fence_after_sync();
           sf_copy(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));

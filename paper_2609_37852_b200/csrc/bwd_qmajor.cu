@@ -17,8 +17,8 @@
 // Warp roles: warp 0 TMA producer; warps 1, 2, 3 issue the S, dP and dQ MMAs; warps 4..19 are two
 // softmax teams that take alternate sub-tiles (inside a team, column group w takes columns
 // 32w..32w+31 of the sub-tile and warp % 4 selects the 32 TMEM lanes).
-// S and dP are single-buffered: the softmax warps pull them into registers and release the
-// buffers at once, so the next sub-tile's MMAs overlap the exponentials of this one.
+// S and dP have one buffer per team; a team pulls them into registers and releases its buffer at
+// once, so the MMAs run ahead of the exponentials.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -32,24 +32,29 @@ using namespace sm100;
 
 constexpr int kTile = 128;
 constexpr int kSub = 64;
-constexpr int kStages = 2;
+// K/V ring depth: deep enough to cover the L2 -> shared-memory latency of a tile (what fits)
+template <bool kDQ> constexpr int kStagesFor = kDQ ? 3 : 4;
 constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
 constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
 constexpr int kThreads = 128 + kTeams * kTeamThreads;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
 
-constexpr uint32_t kColS = 0, kColdP = 64, kColdS = 128 /* 2 x 16 */, kColdQ = 256;
-constexpr uint32_t kColSFQ = 384, kColSFdO = 388, kColSFK = 392 /* 2 x 4 */, kColSFV = 400 /* 2 x 4 */,
-                   kColSFdS = 408 /* 2 x 4 */, kColSFKc = 416 /* 2 x 4 */;
+// S and dP have one 64-column buffer per softmax team, so the MMAs of the next sub-tile never
+// wait for the team that works on the current one.
+constexpr uint32_t kColS = 0 /* 2 x 64 */, kColdP = 128 /* 2 x 64 */, kColdS = 256 /* 2 x 16 */, kColdQ = 288;
+constexpr uint32_t kColSFQ = 416, kColSFdO = 420, kColSFK = 424 /* 2 x 4 */, kColSFV = 432 /* 2 x 4 */,
+                   kColSFdS = 440 /* 2 x 4 */, kColSFKc = 448 /* 2 x 4 */;
 constexpr uint32_t kTmemCols = 512;
 
+template <bool kDQ>
 struct QmSmem {
+  static constexpr int kStages = kStagesFor<kDQ>;
   alignas(1024) uint8_t q[kTile * 128];
   alignas(1024) uint8_t dO[kTile * 128];
   alignas(1024) uint8_t k[kStages][kTile * 128];
   alignas(1024) uint8_t v[kStages][kTile * 128];
-  alignas(1024) uint8_t kc[kStages][kTile * 128];
+  alignas(1024) uint8_t kc[kDQ ? kStages : 1][kTile * 128];
   alignas(16) uint8_t sf_q[512];
   alignas(16) uint8_t sf_dO[512];
   alignas(16) uint8_t sf_k[kStages][512];
@@ -87,7 +92,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
               const __grid_constant__ CUtensorMap tm_kc) {
   extern __shared__ uint8_t smem_raw[];
-  QmSmem& sm = *reinterpret_cast<QmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kStages = kStagesFor<kDQ>;
+  QmSmem<kDQ>& sm = *reinterpret_cast<QmSmem<kDQ>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qt = p.causal ? (gridDim.x - 1 - blockIdx.x) : blockIdx.x;
   const int h = blockIdx.y, b = blockIdx.z;
@@ -180,15 +186,15 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           tc_fence_after_sync();
           sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
         }
-        if (u > 0) {
-          // the team of the previous sub-tile has pulled S and dP into registers
-          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+        if (u >= kTeams) {
+          // this buffer's team has pulled its previous S and dP into registers
+          ok = mbar_wait(&sm.sdp_free[u % kTeams], ((u - kTeams) / kTeams) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+          mma_mxf8_ss(tmem + kColS + kSub * (u % kTeams), desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
         mma_commit(&sm.sdp_full[u % kTeams]);
         if (half == 1) mma_commit(&sm.kv_empty[s]);
@@ -216,14 +222,14 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           tc_fence_after_sync();
           sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
         }
-        if (u > 0) {
-          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+        if (u >= kTeams) {
+          ok = mbar_wait(&sm.sdp_free[u % kTeams], ((u - kTeams) / kTeams) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
         const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+          mma_mxf8_ss(tmem + kColdP + kSub * (u % kTeams), desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFdO, tmem + kColSFV + 4 * slot + 2 * half, kb > 0);
         mma_commit(&sm.sdp_full[u % kTeams]);
         if (half == 1) mma_commit(&sm.kv_empty[s]);
@@ -287,8 +293,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       if (!ok) break;
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
-      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
-      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
+      tmem_ld32(tmem + kColS + kSub * team + lane_addr + 32 * grp, sr);
+      tmem_ld32(tmem + kColdP + kSub * team + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
@@ -398,7 +404,7 @@ attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t
   p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
-  const size_t smem = sizeof(QmSmem) + 1024;
+  const size_t smem = sizeof(QmSmem<kDQ>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<kDQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(s.N / kTile, s.Hq, s.B);
