@@ -1,8 +1,8 @@
 // Query-major backward kernels: the matched row correction (Delta-Matching, paper Section 3.3
 // Eq. 4) and the query gradient (paper Appendix "Backward Correction and Gradient Computation").
 //
-// One CTA owns 128 query rows of one (batch, query head) and sweeps the key tiles up to the
-// causal diagonal, 64 keys at a time.  For every 64-key sub-tile the tensor cores recompute
+// One CTA owns 128 query rows of one (batch, query head) and sweeps the key tiles (128 keys) up to
+// the causal diagonal.  For every key tile the tensor cores recompute
 //     S  = Q^ K^^T   (row-blocked FP8 copies, contraction over the qk channels)
 //     dP = dO^ V^^T  (row-blocked FP8 copies, contraction over the v channels)
 // into tensor memory; the softmax warps rebuild P = 2^(S*scale*log2e - LSE*log2e) in FP32 from
@@ -14,11 +14,11 @@
 // Both modes run the same instruction sequence for P and dP, so the correction the first
 // produces is the one that zeroes the row sums of the second up to FP32 rounding.
 //
-// Warp roles: warp 0 TMA producer; warps 1, 2, 3 issue the S, dP and dQ MMAs; warps 4..19 are two
-// softmax teams that take alternate sub-tiles (inside a team, column group w takes columns
-// 32w..32w+31 of the sub-tile and warp % 4 selects the 32 TMEM lanes).
-// S and dP have one buffer per team; a team pulls them into registers and releases its buffer at
-// once, so the MMAs run ahead of the exponentials.
+// Warp roles: warp 0 TMA producer; warps 1, 2, 3 issue the S, dP and dQ MMAs (an issuing warp
+// spends ~130 cycles per tcgen05 instruction whatever its size, so the MMAs are 128 keys wide and
+// spread over three warps); warps 4..19 softmax: warp % 4 selects the 32 TMEM lanes (query rows),
+// (warp - 4) / 4 the 32-key column group.  The softmax threads pull S and dP into registers and
+// release the buffers at once, so the next tile's MMAs overlap the exponentials of this one.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -31,20 +31,17 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
-constexpr int kSub = 64;
 // K/V ring depth: deep enough to cover the L2 -> shared-memory latency of a tile (what fits)
 template <bool kDQ> constexpr int kStagesFor = kDQ ? 3 : 4;
-constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
-constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
-constexpr int kThreads = 128 + kTeams * kTeamThreads;
+constexpr int kGroups = 4;                      // 32-key column groups of a tile
+constexpr int kSoftmaxThreads = 128 * kGroups;  // 16 warps: 4 TMEM lane quadrants x 4 column groups
+constexpr int kThreads = 128 + kSoftmaxThreads;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
 
-// S and dP have one 64-column buffer per softmax team, so the MMAs of the next sub-tile never
-// wait for the team that works on the current one.
-constexpr uint32_t kColS = 0 /* 2 x 64 */, kColdP = 128 /* 2 x 64 */, kColdS = 256 /* 2 x 16 */, kColdQ = 288;
-constexpr uint32_t kColSFQ = 416, kColSFdO = 420, kColSFK = 424 /* 2 x 4 */, kColSFV = 432 /* 2 x 4 */,
-                   kColSFdS = 440 /* 2 x 4 */, kColSFKc = 448 /* 2 x 4 */;
+constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* 2 x 32 */, kColdQ = 320;
+constexpr uint32_t kColSFQ = 448, kColSFdO = 452, kColSFK = 456 /* 2 x 4 */, kColSFV = 464 /* 2 x 4 */,
+                   kColSFdS = 472 /* 2 x 4 */, kColSFKc = 480 /* 2 x 4 */;
 constexpr uint32_t kTmemCols = 512;
 
 template <bool kDQ>
@@ -61,11 +58,11 @@ struct QmSmem {
   alignas(16) uint8_t sf_v[kStages][512];
   alignas(16) uint8_t sf_kc[kStages][512];
   alignas(16) uint8_t sf_ds[2][512];
-  alignas(16) float red[2 * kTeams][2][kTile];   // partial row sums of every (team, column group)
+  alignas(16) float red[kGroups][2][kTile];      // partial row sums of every column group
   uint64_t q_full;
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[kStages], kc_empty[kStages];
-  uint64_t sdp_full[kTeams], sdp_free[kTeams];
+  uint64_t sdp_full, sdp_free;
   uint64_t ds_full[2], ds_free[2];
   uint64_t dq_done;
   uint64_t drain[3];
@@ -99,7 +96,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
-  const int n_sub = 2 * n_tiles;
   const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
   volatile int* abort_flag = &sm.abort_flag;
 
@@ -109,8 +105,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 2);   // released by the S and the dP issuer
       mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1);
     }
-    for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kTeamThreads); mbar_init(&sm.ds_free[i], 1); }
+    mbar_init(&sm.sdp_full, 2); mbar_init(&sm.sdp_free, kSoftmaxThreads);
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kSoftmaxThreads); mbar_init(&sm.ds_free[i], 1); }
     mbar_init(&sm.dq_done, 1);
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     sm.abort_flag = 0;
@@ -168,9 +164,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S issuer
-    // One warp can issue one tcgen05.mma per ~130 cycles whatever its size, so the three products
-    // have an issuing warp each; orderings a single issuer would give for free are carried by
-    // mbarriers instead.
     if (lane == 0) {
       const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
@@ -178,26 +171,24 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         tc_fence_after_sync();
         sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
       }
-      for (int u = 0; u < n_sub && ok; ++u) {
-        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
-        if (half == 0) {
-          ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
-        }
-        if (u >= kTeams) {
-          // this buffer's team has pulled its previous S and dP into registers
-          ok = mbar_wait(&sm.sdp_free[u % kTeams], ((u - kTeams) / kTeams) & 1, abort_flag);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % kStages, slot = t & 1;
+        ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+        if (t > 0) {
+          // the softmax threads have pulled the previous S and dP into registers
+          ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s]));
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS + kSub * (u % kTeams), desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
-                      tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full[u % kTeams]);
-        if (half == 1) mma_commit(&sm.kv_empty[s]);
+          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
+                      tmem + kColSFQ, tmem + kColSFK + 4 * slot, kb > 0);
+        mma_commit(&sm.sdp_full);
+        mma_commit(&sm.kv_empty[s]);
       }
       if (!ok) {
         int dummy = 0;
@@ -214,25 +205,23 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         tc_fence_after_sync();
         sf_copy(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
       }
-      for (int u = 0; u < n_sub && ok; ++u) {
-        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
-        if (half == 0) {
-          ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
-        }
-        if (u >= kTeams) {
-          ok = mbar_wait(&sm.sdp_free[u % kTeams], ((u - kTeams) / kTeams) & 1, abort_flag);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % kStages, slot = t & 1;
+        ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        if (t > 0) {
+          ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s])) + half * (kSub * 128 / 16);
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
         for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss(tmem + kColdP + kSub * (u % kTeams), desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
-                      tmem + kColSFdO, tmem + kColSFV + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full[u % kTeams]);
-        if (half == 1) mma_commit(&sm.kv_empty[s]);
+          mma_mxf8_ss(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
+                      tmem + kColSFdO, tmem + kColSFV + 4 * slot, kb > 0);
+        mma_commit(&sm.sdp_full);
+        mma_commit(&sm.kv_empty[s]);
       }
       if (!ok) {
         int dummy = 0;
@@ -244,26 +233,24 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     // ------------------------------------------------------------------ dQ issuer
     if (kDQ && lane == 0) {
       bool ok = true;
-      for (int u = 0; u < n_sub && ok; ++u) {
-        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
-        if (half == 0) {
-          ok = mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          sf_copy(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
-        }
-        ok = mbar_wait(&sm.ds_full[buf], (u >> 1) & 1, abort_flag);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % kStages, slot = t & 1, buf = t & 1;
+        ok = mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        sf_copy(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+        ok = mbar_wait(&sm.ds_full[buf], (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
         sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
-        for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts(tmem + kColdQ, tmem + kColdS + 16 * buf + 8 * kb, desc_kc + 2 * (2 * half + kb),
-                      make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
-                      tmem + kColSFKc + 4 * slot, (u > 0 || kb > 0));
+        for (int kb = 0; kb < 4; ++kb)
+          mma_mxf8_ts(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+                      make_idesc_mxf8(128, p.dqk, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
+                      (t > 0 || kb > 0));
         mma_commit(&sm.ds_free[buf]);            // codes and scale bytes of this buffer may be overwritten
-        if (half == 1) mma_commit(&sm.kc_empty[s]);
-        if (u == n_sub - 1) mma_commit(&sm.dq_done);
+        mma_commit(&sm.kc_empty[s]);
+        if (t == n_tiles - 1) mma_commit(&sm.dq_done);
       }
       if (!ok) {
         int dummy = 0;
@@ -273,8 +260,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax
-    const int team = (warp - 4) >> 3;
-    const int grp = ((warp - 4) >> 2) & 1;            // column half of each sub-tile
+    const int grp = (warp - 4) >> 2;                  // 32-key column group of the tile
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
@@ -287,19 +273,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float D = kDQ ? p.delta_in[grow] : 0.f;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
     bool ok = true;
-    for (int u = team; u < n_sub; u += kTeams) {
-      const int t = u >> 1, half = u & 1, buf = u & 1;
-      ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      ok = mbar_wait(&sm.sdp_full, t & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
-      tmem_ld32(tmem + kColS + kSub * team + lane_addr + 32 * grp, sr);
-      tmem_ld32(tmem + kColdP + kSub * team + lane_addr + 32 * grp, dpr);
+      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
+      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(&sm.sdp_free[team]);
+      mbar_arrive(&sm.sdp_free);
       const bool diag = p.causal && (t == qt);
-      const int col0 = half * kSub + 32 * grp;        // column of this thread's first element inside the key tile
+      const int col0 = 32 * grp;                      // column of this thread's first element inside the key tile
       float ds[32];
       float part = 0.f;
 #pragma unroll
@@ -322,13 +308,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       } else {
         uint32_t words[8];
         const uint32_t byte = quantize_block32(ds, words);
-        if (u >= 2) {
-          // the dQ MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
-          ok = mbar_wait(&sm.ds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+        if (t >= 2) {
+          // the dQ MMAs of tile t-2 have consumed this buffer's codes and scale bytes
+          ok = mbar_wait(&sm.ds_free[buf], ((t - 2) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
+        tmem_st8(tmem + kColdS + 32 * buf + lane_addr + 8 * grp, words);
         sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
         tmem_wait_st();
         fence_proxy_async_smem();
@@ -336,13 +322,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
-    // combine the row sums of the teams and column groups (fixed order: reproducible)
-    sm.red[team * 2 + grp][0][row] = acc0;
-    sm.red[team * 2 + grp][1][row] = acc1;
-    named_barrier_sync(1, kTeams * kTeamThreads);
-    if (ok && team == 0 && grp == 0) {
+    // combine the row sums of the column groups (fixed order: reproducible)
+    sm.red[grp][0][row] = acc0;
+    sm.red[grp][1][row] = acc1;
+    named_barrier_sync(1, kSoftmaxThreads);
+    if (ok && grp == 0) {
       acc0 = 0.f; acc1 = 0.f;
-      for (int i = 0; i < 2 * kTeams; ++i) { acc0 += sm.red[i][0][row]; acc1 += sm.red[i][1][row]; }
+      for (int i = 0; i < kGroups; ++i) { acc0 += sm.red[i][0][row]; acc1 += sm.red[i][1][row]; }
       if (!kDQ) {
         p.delta_out[grow] = acc0;
       } else if (p.rowsum) {
@@ -350,13 +336,12 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         p.rowabs[grow] = acc1;
       }
     }
-    if (kDQ && ok && team == 0) {
+    if (kDQ && ok) {
       ok = mbar_wait(&sm.dq_done, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
         __nv_bfloat16* out_row = p.dq + grow * p.dqk;
-        const int half_cols = p.dqk / 2;
-        for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 32) {
+        for (int c0 = grp * 32; c0 < p.dqk; c0 += 32 * kGroups) {
           uint32_t r[32];
           tmem_ld32(tmem + kColdQ + lane_addr + c0, r);
           tmem_wait_ld();
