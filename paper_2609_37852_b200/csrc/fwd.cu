@@ -267,19 +267,25 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.p_free[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          for (int c0 = 0; c0 < p.dv; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tmem + kColO + lane_addr + c0, r);
+          // rare path: small chunks keep the scores of this sub-tile in registers
+          for (int c0 = 0; c0 < p.dv; c0 += 8) {
+            uint32_t r[8];
+            tmem_ld8(tmem + kColO + lane_addr + c0, r);
             tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
-            tmem_st32(tmem + kColO + lane_addr + c0, r);
+            for (int c = 0; c < 8; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
+            tmem_st8(tmem + kColO + lane_addr + c0, r);
           }
           tmem_wait_st();
         }
       }
       const float neg_m = -M;
-      uint32_t words[16];
+      if (u >= 2) {
+        // the P V MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+        ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+      }
       uint32_t sf_half = 0;
       float sub_sum = 0.f;                            // per block, per sub-tile, then into l: short chains
 #pragma unroll
@@ -300,20 +306,14 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         float inv;
         block_scale(amax, byte, inv);
         sf_half |= byte << (8 * blk);
+        uint32_t words[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          words[blk * 8 + i] = cvt_e4m3x4(sv[blk * 32 + 4 * i] * inv, sv[blk * 32 + 4 * i + 1] * inv,
-                                          sv[blk * 32 + 4 * i + 2] * inv, sv[blk * 32 + 4 * i + 3] * inv);
+          words[i] = cvt_e4m3x4(sv[blk * 32 + 4 * i] * inv, sv[blk * 32 + 4 * i + 1] * inv,
+                                sv[blk * 32 + 4 * i + 2] * inv, sv[blk * 32 + 4 * i + 3] * inv);
+        tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * blk, words);
       }
       l += sub_sum;
-      if (u >= 2) {
-        // the P V MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
-        ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-      }
-      tmem_st8(tmem + kColP + 16 * buf + lane_addr, words);
-      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8, words + 8);
       *reinterpret_cast<uint16_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = static_cast<uint16_t>(sf_half);
       tmem_wait_st();
       fence_proxy_async_smem();
