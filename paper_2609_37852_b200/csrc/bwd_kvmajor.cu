@@ -176,12 +176,12 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // One tcgen05.mma can be issued per ~130 cycles from one warp whatever its size, so the
     // products are spread over three issuing warps; orderings that a single issuer would give
     // for free are carried by mbarriers instead.
-    if (lane == 0) {
+    {
       const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k));
       bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
+        sf_copy_elect(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
       }
       for (int u = 0; u < n_sub && ok; ++u) {
         const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
@@ -190,7 +190,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
+          sf_copy_elect(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
         }
         if (u > 0) {
           // the team of the previous sub-tile has pulled S and dP into registers
@@ -200,13 +200,13 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         }
         const uint64_t desc_q = make_desc_sw128(smem_u32(st.q)) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+          mma_mxf8_ss_elect(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFK, tmem + kColSFQ + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full[u % kTeams]);
+        mma_commit_elect(&sm.sdp_full[u % kTeams]);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[0]);
+        mma_commit_elect(&sm.drain[0]);
         mbar_wait(&sm.drain[0], 0, &dummy);
       }
     }
@@ -214,9 +214,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // ------------------------------------------------------------------ dP^T issuer + LSE preparation
     const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v));
     bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-    if (ok && lane == 0) {
+    if (ok) {
       tc_fence_after_sync();
-      sf_copy(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
+      sf_copy_elect(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
     }
     for (int u = 0; u < n_sub && ok; ++u) {
       const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
@@ -229,32 +229,32 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
             make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
         mbar_arrive_warp(&sm.lse_ready[s]);
-        if (lane == 0) {
+        {
           tc_fence_after_sync();
-          sf_copy(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
+          sf_copy_elect(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
         }
       }
       if (u > 0) {
         ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
         if (!ok) break;
       }
-      if (lane == 0) {
+      {
         tc_fence_after_sync();
         const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO)) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss(tmem + kColdP, desc_v + 2 * kb, desc_dO + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+          mma_mxf8_ss_elect(tmem + kColdP, desc_v + 2 * kb, desc_dO + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFV, tmem + kColSFdO + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.sdp_full[u % kTeams]);
+        mma_commit_elect(&sm.sdp_full[u % kTeams]);
       }
     }
-    if (!ok && lane == 0) {
+    if (!ok) {
       int dummy = 0;
-      mma_commit(&sm.drain[1]);
+      mma_commit_elect(&sm.drain[1]);
       mbar_wait(&sm.drain[1], 0, &dummy);
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------------ dV / dK issuer
-    if (lane == 0) {
+    {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
         const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1, buf = u & 1;
@@ -263,34 +263,34 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
-          sf_copy(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
+          sf_copy_elect(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
+          sf_copy_elect(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
         }
         ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
-        sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_dOc = make_desc_sw128(smem_u32(st.dOc));
         const uint64_t desc_qc = make_desc_sw128(smem_u32(st.qc));
         for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts(tmem + kColdV, tmem + kColP + 16 * buf + 8 * kb, desc_dOc + 2 * (2 * half + kb),
+          mma_mxf8_ts_elect(tmem + kColdV, tmem + kColP + 16 * buf + 8 * kb, desc_dOc + 2 * (2 * half + kb),
                       make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
                       tmem + kColSFdOc + 4 * slot, (u > 0 || kb > 0));
         for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts(tmem + kColdK, tmem + kColdS + 16 * buf + 8 * kb, desc_qc + 2 * (2 * half + kb),
+          mma_mxf8_ts_elect(tmem + kColdK, tmem + kColdS + 16 * buf + 8 * kb, desc_qc + 2 * (2 * half + kb),
                       make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
                       tmem + kColSFQc + 4 * slot, (u > 0 || kb > 0));
         // codes and scale bytes of this buffer may be overwritten once these MMAs have run; the
         // stage may be refilled after the second half (the S^T / dP^T MMAs that read it finished
         // before the softmax team could even start on this sub-tile)
-        mma_commit(&sm.pds_free[buf]);
-        if (half == 1) mma_commit(&sm.q_empty[s]);
-        if (u == n_sub - 1) mma_commit(&sm.done);
+        mma_commit_elect(&sm.pds_free[buf]);
+        if (half == 1) mma_commit_elect(&sm.q_empty[s]);
+        if (u == n_sub - 1) mma_commit_elect(&sm.done);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[2]);
+        mma_commit_elect(&sm.drain[2]);
         mbar_wait(&sm.drain[2], 0, &dummy);
       }
     }

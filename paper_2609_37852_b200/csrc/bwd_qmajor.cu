@@ -26,6 +26,18 @@
 #include "sm100_ptx.cuh"
 
 namespace attnfp8 {
+
+#ifdef ATTN_TRACE
+// Debug build only: clock stamps of one CTA (roles x tiles x events), read back by the host.
+__device__ long long g_qm_trace[4][128][4];
+#define QM_TRACE(role, tile, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (tile) < 128) g_qm_trace[role][tile][ev] = clock64(); } while (0)
+extern "C" int attn_fp8_debug_qm_trace(long long* host_out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_qm_trace, sizeof(g_qm_trace)));
+}
+#else
+#define QM_TRACE(role, tile, ev) do { } while (0)
+#endif
+
 namespace {
 
 using namespace sm100;
@@ -139,6 +151,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         const int s = t % kStages, u = t / kStages;
         ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
+        QM_TRACE(0, t, 0);
         mbar_arrive_expect_tx(&sm.kv_full[s], 2 * (kTile * 128 + 512));
         tma_load_2d(sm.k[s], &tm_k, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
         tma_load_2d(sm.v[s], &tm_v, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
@@ -164,53 +177,57 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S issuer
-    if (lane == 0) {
+    {
       const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+        sf_copy_elect(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kStages, slot = t & 1;
         ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
         if (!ok) break;
+        QM_TRACE(1, t, 0);
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+        sf_copy_elect(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+        QM_TRACE(1, t, 1);
         if (t > 0) {
           // the softmax threads have pulled the previous S and dP into registers
           ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
+        QM_TRACE(1, t, 2);
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s]));
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
+          mma_mxf8_ss_elect(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
                       tmem + kColSFQ, tmem + kColSFK + 4 * slot, kb > 0);
-        mma_commit(&sm.sdp_full);
-        mma_commit(&sm.kv_empty[s]);
+        mma_commit_elect(&sm.sdp_full);
+        mma_commit_elect(&sm.kv_empty[s]);
+        QM_TRACE(1, t, 3);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[0]);
+        mma_commit_elect(&sm.drain[0]);
         mbar_wait(&sm.drain[0], 0, &dummy);
       }
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ dP issuer
-    if (lane == 0) {
+    {
       const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
+        sf_copy_elect(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kStages, slot = t & 1;
         ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        sf_copy_elect(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
         if (t > 0) {
           ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
@@ -218,43 +235,43 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
         for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
+          mma_mxf8_ss_elect(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
                       tmem + kColSFdO, tmem + kColSFV + 4 * slot, kb > 0);
-        mma_commit(&sm.sdp_full);
-        mma_commit(&sm.kv_empty[s]);
+        mma_commit_elect(&sm.sdp_full);
+        mma_commit_elect(&sm.kv_empty[s]);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[1]);
+        mma_commit_elect(&sm.drain[1]);
         mbar_wait(&sm.drain[1], 0, &dummy);
       }
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------------ dQ issuer
-    if (kDQ && lane == 0) {
+    if (kDQ) {
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kStages, slot = t & 1, buf = t & 1;
         ok = mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+        sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
         ok = mbar_wait(&sm.ds_full[buf], (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
         for (int kb = 0; kb < 4; ++kb)
-          mma_mxf8_ts(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+          mma_mxf8_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
                       make_idesc_mxf8(128, p.dqk, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
                       (t > 0 || kb > 0));
-        mma_commit(&sm.ds_free[buf]);            // codes and scale bytes of this buffer may be overwritten
-        mma_commit(&sm.kc_empty[s]);
-        if (t == n_tiles - 1) mma_commit(&sm.dq_done);
+        mma_commit_elect(&sm.ds_free[buf]);            // codes and scale bytes of this buffer may be overwritten
+        mma_commit_elect(&sm.kc_empty[s]);
+        if (t == n_tiles - 1) mma_commit_elect(&sm.dq_done);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[2]);
+        mma_commit_elect(&sm.drain[2]);
         mbar_wait(&sm.drain[2], 0, &dummy);
       }
     }
@@ -275,8 +292,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     bool ok = true;
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
+      if (warp == 4 && lane == 0) QM_TRACE(2, t, 0);
       ok = mbar_wait(&sm.sdp_full, t & 1, abort_flag);
       if (!ok) break;
+      if (warp == 4 && lane == 0) QM_TRACE(2, t, 1);
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
@@ -284,6 +303,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free);
+      if (warp == 4 && lane == 0) QM_TRACE(2, t, 2);
       const bool diag = p.causal && (t == qt);
       const int col0 = 32 * grp;                      // column of this thread's first element inside the key tile
       float ds[32];

@@ -155,12 +155,12 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S = Q K^T issuer
-    if (lane == 0) {
+    {
       const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+        sf_copy_elect(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
       }
       for (int u = 0; u < n_sub && ok; ++u) {
         const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
@@ -168,7 +168,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+          sf_copy_elect(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
         }
         if (u > 0) {
           // the softmax threads have pulled the previous scores into registers
@@ -178,20 +178,20 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         }
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
+          mma_mxf8_ss_elect(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
-        mma_commit(&sm.s_full);
-        if (half == 1) mma_commit(&sm.k_empty[s]);
+        mma_commit_elect(&sm.s_full);
+        if (half == 1) mma_commit_elect(&sm.k_empty[s]);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[0]);
+        mma_commit_elect(&sm.drain[0]);
         mbar_wait(&sm.drain[0], 0, &dummy);
       }
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ O += P V issuer
-    if (lane == 0) {
+    {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
         const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
@@ -199,24 +199,24 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+          sf_copy_elect(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
         }
         ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
         for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts(tmem + kColO, tmem + kColP + 16 * buf + 8 * kb, desc_v + 2 * (2 * half + kb),
+          mma_mxf8_ts_elect(tmem + kColO, tmem + kColP + 16 * buf + 8 * kb, desc_v + 2 * (2 * half + kb),
                       make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
                       tmem + kColSFV + 4 * slot, (u > 0 || kb > 0));
-        mma_commit(&sm.p_free[buf]);              // codes / scale bytes of this buffer consumed; O updated
-        if (half == 1) mma_commit(&sm.v_empty[s]);
-        if (u == n_sub - 1) mma_commit(&sm.o_done);
+        mma_commit_elect(&sm.p_free[buf]);              // codes / scale bytes of this buffer consumed; O updated
+        if (half == 1) mma_commit_elect(&sm.v_empty[s]);
+        if (u == n_sub - 1) mma_commit_elect(&sm.o_done);
       }
       if (!ok) {
         int dummy = 0;
-        mma_commit(&sm.drain[1]);
+        mma_commit_elect(&sm.drain[1]);
         mbar_wait(&sm.drain[1], 0, &dummy);
       }
     }

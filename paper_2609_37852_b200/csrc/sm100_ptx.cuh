@@ -290,6 +290,53 @@ __device__ __forceinline__ void sf_copy(uint32_t tmem_dst, uint64_t sf_desc) {
   asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_dst), "l"(sf_desc) : "memory");
 }
 
+// Warp-convergent variants: the whole warp executes the call, one elected lane issues.  Keeping
+// the issuing loop convergent lets descriptors and addresses live in uniform registers, which
+// makes the loop far shorter than a single-lane (divergent) one -- it matters because the issuing
+// warp shares its scheduler with arithmetic warps.
+__device__ __forceinline__ void mma_mxf8_ss_elect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %6, 0;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%4], [%5], p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_mxf8_ts_elect(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %6, 0;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], [%1], %2, %3, [%4], [%5], p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit_elect(uint64_t* bar) {
+  asm volatile(
+      "{\n"
+      ".reg .pred q;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+      "}\n"
+      ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void sf_copy_elect(uint32_t tmem_dst, uint64_t sf_desc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred q;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;\n"
+      "}\n"
+      ::"r"(tmem_dst), "l"(sf_desc) : "memory");
+}
+
 // ------------------------------------------------------------------ conversions
 // Two floats -> two E4M3 codes (lo in bits 0..7), round to nearest even, saturating.
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
