@@ -7,9 +7,9 @@
 //   warp 0      TMA producer: Q tile once, then K tiles [128 keys x d] and V tiles [dv x 128 keys]
 //   warp 1      issues S = Q K^T (block-scaled, 128 x 64 per sub-tile)
 //   warp 2      issues O += P V (A operand = quantised probabilities read from tensor memory)
-//   warps 4..7  softmax: one query row per thread (thread <-> TMEM lane).  A thread pulls its 64
-//               scores into registers and releases the score buffer at once, so the next S is
-//               computed while it works.  Scores go to log2 units; the running shift M is an
+//   warps 4..11 softmax: two threads per query row (thread <-> TMEM lane x 32-key column group).
+//               A thread pulls its 32 scores into registers and releases the score buffer at
+//               once, so the next S is computed while it works.  Scores go to log2 units; the running shift M is an
 //               INTEGER, so rescaling is by exact powers of two and the E4M3 codes of the
 //               probabilities do not depend on the tile order; l accumulates the exponentials
 //               BEFORE the FP8 cast; probabilities are quantised in blocks of 32 keys in
@@ -34,8 +34,8 @@ using namespace sm100;
 constexpr int kTile = 128;          // query rows per CTA; keys per K / V tile in shared memory
 constexpr int kSub = 64;            // keys per softmax step
 constexpr int kStages = 2;          // K ring and V ring depth
-constexpr int kThreads = 256;
-constexpr int kSoftmaxThreads = 128;
+constexpr int kThreads = 384;
+constexpr int kSoftmaxThreads = 256;      // two threads per query row
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
@@ -59,12 +59,14 @@ struct FwdSmem {
   alignas(16) uint8_t sf_k[kStages][512];
   alignas(16) uint8_t sf_v[kStages][512];
   alignas(16) uint8_t sf_p[2][512];
+  alignas(16) float xch[2][2][kTile];       // row maxima (and at the end normaliser shares) of the thread pairs
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages];
   uint64_t v_full[kStages], v_empty[kStages];
   uint64_t s_full, s_free;
   uint64_t p_full[2], p_free[2];
   uint64_t o_done;
+  uint64_t pair[4];                         // one per TMEM lane quadrant: the two warps of a thread pair
   uint64_t drain[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -105,6 +107,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     mbar_init(&sm.s_full, 1); mbar_init(&sm.s_free, kSoftmaxThreads);
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.p_full[i], kSoftmaxThreads); mbar_init(&sm.p_free[i], 1); }
     mbar_init(&sm.o_done, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[i], 64);
     mbar_init(&sm.drain[0], 1); mbar_init(&sm.drain[1], 1);
     sm.abort_flag = 0;
     fence_mbar_init();
@@ -222,44 +225,49 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax
+    // Two threads per query row: column group `grp` owns keys 32*grp .. 32*grp+31 of the sub-tile
+    // (one quantisation block).  The pair lives in two warps with the same TMEM lane quadrant and
+    // exchanges its block maxima through shared memory, so that both use the same shift M.
+    const int grp = (warp - 4) >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                 // row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
     float M = -INFINITY;                              // integer-valued running shift (log2 units)
-    float l = 0.f;
+    float l = 0.f;                                    // this thread's share of the normaliser
     bool ok = true;
     for (int u = 0; u < n_sub; ++u) {
       const int t = u >> 1, half = u & 1, buf = u & 1;
       ok = mbar_wait(&sm.s_full, u & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
-      float sv[kSub];
-      {
-        uint32_t* r = reinterpret_cast<uint32_t*>(sv);
-        tmem_ld32(tmem + kColS + lane_addr, r);
-        tmem_ld32(tmem + kColS + lane_addr + 32, r + 32);
-        tmem_wait_ld();
-      }
+      float sv[32];
+      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, reinterpret_cast<uint32_t*>(sv));
+      tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.s_free);
       // maximum of the raw accumulators (the scale is positive), masked on the diagonal tile
       float mx = -INFINITY;
       if (p.causal && t == qt) {
-        const int col0 = half * kSub;
+        const int col0 = half * kSub + 32 * grp;
 #pragma unroll
-        for (int c = 0; c < kSub; ++c) {
+        for (int c = 0; c < 32; ++c) {
           if (col0 + c > row) sv[c] = -INFINITY;
           mx = fmaxf(mx, sv[c]);
         }
       } else {
 #pragma unroll
-        for (int c = 0; c < kSub; ++c) mx = fmaxf(mx, sv[c]);
+        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, sv[c]);
       }
+      sm.xch[u & 1][grp][row] = mx;
+      mbar_arrive(&sm.pair[quad]);                    // the two warps that share these 32 rows
+      ok = mbar_wait(&sm.pair[quad], u & 1, abort_flag);
+      if (!ok) break;
+      mx = fmaxf(mx, sm.xch[u & 1][grp ^ 1][row]);
       // a fully masked sub-tile (second half of the diagonal tile for the first 64 rows) gives -inf:
       // it never raises M and contributes zeros
       const float m_new = ceilf(mx * p.scale_log2);
       const bool raise = m_new > M + static_cast<float>(kLazyShift);   // true on the first sub-tile
-      if (__any_sync(0xffffffffu, raise)) {
+      if (__any_sync(0xffffffffu, raise)) {             // same rows, same decision in both warps of the pair
         const float factor = raise ? exp2f(M - m_new) : 1.f;            // exact power of two (0 at the start)
         if (raise) { l *= factor; M = m_new; }
         if (u > 0) {
@@ -267,8 +275,9 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.p_free[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          // rare path: small chunks keep the scores of this sub-tile in registers
-          for (int c0 = 0; c0 < p.dv; c0 += 8) {
+          // rare path; each thread of the pair rescales its half of the output columns
+          const int half_cols = p.dv / 2;
+          for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 8) {
             uint32_t r[8];
             tmem_ld8(tmem + kColO + lane_addr + c0, r);
             tmem_wait_ld();
@@ -280,45 +289,44 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         }
       }
       const float neg_m = -M;
+      float bs0 = 0.f, bs1 = 0.f, amax = 0.f;          // two short chains for the block sum
+#pragma unroll
+      for (int c = 0; c < 32; c += 2) {
+        const float p0 = ex2_approx(fmaf(sv[c], p.scale_log2, neg_m));
+        const float p1 = ex2_approx(fmaf(sv[c + 1], p.scale_log2, neg_m));
+        sv[c] = p0;
+        sv[c + 1] = p1;
+        bs0 += p0;
+        bs1 += p1;
+        amax = fmaxf(amax, fmaxf(p0, p1));
+      }
+      l += bs0 + bs1;
+      uint32_t byte;
+      float inv;
+      block_scale(amax, byte, inv);
+      uint32_t words[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        words[i] = cvt_e4m3x4(sv[4 * i] * inv, sv[4 * i + 1] * inv, sv[4 * i + 2] * inv, sv[4 * i + 3] * inv);
       if (u >= 2) {
         // the P V MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
         ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
-      uint32_t sf_half = 0;
-      float sub_sum = 0.f;                            // per block, per sub-tile, then into l: short chains
-#pragma unroll
-      for (int blk = 0; blk < 2; ++blk) {
-        float bs0 = 0.f, bs1 = 0.f, amax = 0.f;
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float p0 = ex2_approx(fmaf(sv[blk * 32 + c], p.scale_log2, neg_m));
-          const float p1 = ex2_approx(fmaf(sv[blk * 32 + c + 1], p.scale_log2, neg_m));
-          sv[blk * 32 + c] = p0;
-          sv[blk * 32 + c + 1] = p1;
-          bs0 += p0;
-          bs1 += p1;
-          amax = fmaxf(amax, fmaxf(p0, p1));
-        }
-        sub_sum += bs0 + bs1;
-        uint32_t byte;
-        float inv;
-        block_scale(amax, byte, inv);
-        sf_half |= byte << (8 * blk);
-        uint32_t words[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          words[i] = cvt_e4m3x4(sv[blk * 32 + 4 * i] * inv, sv[blk * 32 + 4 * i + 1] * inv,
-                                sv[blk * 32 + 4 * i + 2] * inv, sv[blk * 32 + 4 * i + 3] * inv);
-        tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * blk, words);
-      }
-      l += sub_sum;
-      *reinterpret_cast<uint16_t*>(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4]) = static_cast<uint16_t>(sf_half);
+      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
+      sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.p_full[buf]);
+    }
+    // total normaliser of the row = sum of the pair's shares
+    if (ok) {
+      sm.xch[0][grp][row] = l;
+      mbar_arrive(&sm.pair[quad]);
+      ok = mbar_wait(&sm.pair[quad], n_sub & 1, abort_flag);
+      if (ok) l += sm.xch[0][grp ^ 1][row];
     }
     if (ok) ok = mbar_wait(&sm.o_done, 0, abort_flag);
     if (ok) {
@@ -326,7 +334,8 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       const float inv_l = 1.f / l;
       const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
       __nv_bfloat16* o_row = p.o + grow * p.dv;
-      for (int c0 = 0; c0 < p.dv; c0 += 32) {
+      const int half_cols = p.dv / 2;                 // each thread of the pair stores half of the row
+      for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem + kColO + lane_addr + c0, r);
         tmem_wait_ld();
@@ -341,7 +350,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
       }
       // LSE = M ln2 + ln l with ln2 split so that M * ln2_hi is exact: one rounding at the end
-      p.lse[grow] = fmaf(M, kLn2Hi, fmaf(M, kLn2Lo, logf(l)));
+      if (grp == 0) p.lse[grow] = fmaf(M, kLn2Hi, fmaf(M, kLn2Lo, logf(l)));
     }
   }
   __syncwarp();
