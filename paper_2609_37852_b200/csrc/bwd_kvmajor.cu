@@ -27,13 +27,30 @@
 #include "sm100_ptx.cuh"
 
 namespace attnfp8 {
+
+#ifdef ATTN_TRACE
+// Debug build only: clock stamps of one CTA (roles x steps x events), read back by the host.
+__device__ long long g_kv_trace[4][256][4];
+#define KV_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_kv_trace[role][step][ev] = clock64(); } while (0)
+extern "C" int attn_fp8_debug_kv_trace(long long* host_out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_kv_trace, sizeof(g_kv_trace)));
+}
+#else
+#define KV_TRACE(role, step, ev) do { } while (0)
+#endif
+
 namespace {
 
 using namespace sm100;
 
 constexpr int kTile = 128;
 constexpr int kSub = 64;
-constexpr int kStages = 2;
+// Per query tile the CTA streams a 'row' set (Q and dO row copies, their scales, LSE, D: read by
+// the S^T / dP^T MMAs and the softmax) and a 'col' set (Q and dO column copies: read by the dV / dK
+// MMAs).  The row set is released early and has three stages, so that a reload never sits between
+// the end of one tile's gradient MMAs and the start of the next tile's scores.
+constexpr int kRowStages = 3;
+constexpr int kColStages = 2;
 constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
 constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
 constexpr int kThreads = 128 + kTeams * kTeamThreads;
@@ -47,31 +64,35 @@ constexpr uint32_t kColSFK = 448, kColSFV = 452, kColSFQ = 456 /* 2 x 4 */, kCol
                    kColSFQc = 496 /* 2 x 4 */;
 constexpr uint32_t kTmemCols = 512;
 
-struct KvStage {
+struct KvRowStage {
   alignas(1024) uint8_t q[kTile * 128];       // Q row copy  [128 queries][dqk]
   alignas(1024) uint8_t dO[kTile * 128];      // dO row copy [128 queries][dv]
-  alignas(1024) uint8_t qc[kTile * 128];      // Q col copy  [dqk][128 queries]
-  alignas(1024) uint8_t dOc[kTile * 128];     // dO col copy [dv][128 queries]
   alignas(16) uint8_t sf_q[512];
   alignas(16) uint8_t sf_dO[512];
-  alignas(16) uint8_t sf_qc[512];
-  alignas(16) uint8_t sf_dOc[512];
   alignas(16) float lse[kTile];
   alignas(16) float delta[kTile];
-  alignas(16) float neg_lse2[kTile];          // -LSE * log2(e), written by the prep warps
+  alignas(16) float neg_lse2[kTile];          // -LSE * log2(e), written by the prep warp
+};
+struct KvColStage {
+  alignas(1024) uint8_t qc[kTile * 128];      // Q col copy  [dqk][128 queries]
+  alignas(1024) uint8_t dOc[kTile * 128];     // dO col copy [dv][128 queries]
+  alignas(16) uint8_t sf_qc[512];
+  alignas(16) uint8_t sf_dOc[512];
 };
 
 struct KvSmem {
   alignas(1024) uint8_t k[kTile * 128];
   alignas(1024) uint8_t v[kTile * 128];
-  KvStage st[kStages];
+  KvRowStage rst[kRowStages];
+  KvColStage cst[kColStages];
   alignas(16) uint8_t sf_k[512];
   alignas(16) uint8_t sf_v[512];
   alignas(16) uint8_t sf_p[2][512];
   alignas(16) uint8_t sf_ds[2][512];
   uint64_t kv_full;
-  uint64_t q_full[kStages], q_empty[kStages];
-  uint64_t lse_ready[kStages];
+  uint64_t row_full[kRowStages], row_empty[kRowStages];
+  uint64_t col_full[kColStages], col_empty[kColStages];
+  uint64_t lse_ready[kRowStages];
   uint64_t sdp_full[kTeams], sdp_free[kTeams];
   uint64_t pds_full[2], pds_free[2];
   uint64_t done;
@@ -111,8 +132,11 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
-    for (int s = 0; s < kStages; ++s) mbar_init(&sm.lse_ready[s], 1);
+    for (int s = 0; s < kRowStages; ++s) {
+      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], 1);      // released once both softmax teams are done with the tile
+      mbar_init(&sm.lse_ready[s], 1);                 // one arrival by the prep warp
+    }
+    for (int s = 0; s < kColStages; ++s) { mbar_init(&sm.col_full[s], 1); mbar_init(&sm.col_empty[s], 1); }
     for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); }
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
@@ -141,34 +165,41 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tma_load_2d(sm.v, &tm_v, &sm.kv_full, 0, kv_slab * p.N + jt * kTile);
       bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
       bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
-      int issued = 0;
+      int issued_row = 0, issued_col = 0;
       bool ok = true;
       for (int n = 0; n < n_qtiles && ok; ++n) {
-        const int s = n % kStages, u = n / kStages;
+        const int rs = n % kRowStages, cs = n % kColStages;
         const int h = g * G + n / tiles_per_head, it = it0 + n % tiles_per_head;
         const int q_slab = b * p.Hq + h;
-        ok = mbar_wait(&sm.q_empty[s], (u & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        KvStage& st = sm.st[s];
-        mbar_arrive_expect_tx(&sm.q_full[s], 2 * kTile * 128 + (p.dqk + p.dv) * 128 + 4 * 512 + 2 * kTile * 4);
-        tma_load_2d(st.q, &tm_q, &sm.q_full[s], 0, q_slab * p.N + it * kTile);
-        tma_load_2d(st.dO, &tm_dO, &sm.q_full[s], 0, q_slab * p.N + it * kTile);
-        tma_load_2d(st.qc, &tm_qc, &sm.q_full[s], it * kTile, q_slab * p.dqk);
-        tma_load_2d(st.dOc, &tm_dOc, &sm.q_full[s], it * kTile, q_slab * p.dv);
         const size_t sf_tile = (static_cast<size_t>(q_slab) * tiles_n + it) * 512;
-        bulk_load_1d(st.sf_q, p.q_sf + sf_tile, 512, &sm.q_full[s]);
-        bulk_load_1d(st.sf_dO, p.dO_sf + sf_tile, 512, &sm.q_full[s]);
-        bulk_load_1d(st.sf_qc, p.qc_sf + sf_tile, 512, &sm.q_full[s]);
-        bulk_load_1d(st.sf_dOc, p.dOc_sf + sf_tile, 512, &sm.q_full[s]);
         const size_t row0 = static_cast<size_t>(q_slab) * p.N + it * kTile;
-        bulk_load_1d(st.lse, p.lse + row0, kTile * 4, &sm.q_full[s]);
-        bulk_load_1d(st.delta, p.delta + row0, kTile * 4, &sm.q_full[s]);
-        ++issued;
+        ok = mbar_wait(&sm.row_empty[rs], ((n / kRowStages) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        KvRowStage& r = sm.rst[rs];
+        mbar_arrive_expect_tx(&sm.row_full[rs], 2 * kTile * 128 + 2 * 512 + 2 * kTile * 4);
+        tma_load_2d(r.q, &tm_q, &sm.row_full[rs], 0, q_slab * p.N + it * kTile);
+        tma_load_2d(r.dO, &tm_dO, &sm.row_full[rs], 0, q_slab * p.N + it * kTile);
+        bulk_load_1d(r.sf_q, p.q_sf + sf_tile, 512, &sm.row_full[rs]);
+        bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile, 512, &sm.row_full[rs]);
+        bulk_load_1d(r.lse, p.lse + row0, kTile * 4, &sm.row_full[rs]);
+        bulk_load_1d(r.delta, p.delta + row0, kTile * 4, &sm.row_full[rs]);
+        ++issued_row;
+        ok = mbar_wait(&sm.col_empty[cs], ((n / kColStages) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        KvColStage& c = sm.cst[cs];
+        mbar_arrive_expect_tx(&sm.col_full[cs], (p.dqk + p.dv) * 128 + 2 * 512);
+        tma_load_2d(c.qc, &tm_qc, &sm.col_full[cs], it * kTile, q_slab * p.dqk);
+        tma_load_2d(c.dOc, &tm_dOc, &sm.col_full[cs], it * kTile, q_slab * p.dv);
+        bulk_load_1d(c.sf_qc, p.qc_sf + sf_tile, 512, &sm.col_full[cs]);
+        bulk_load_1d(c.sf_dOc, p.dOc_sf + sf_tile, 512, &sm.col_full[cs]);
+        ++issued_col;
       }
       if (!ok) {
         int dummy = 0;
-        for (int n = max(0, issued - kStages); n < issued; ++n)
-          mbar_wait(&sm.q_full[n % kStages], (n / kStages) & 1, &dummy);
+        for (int n = max(0, issued_row - kRowStages); n < issued_row; ++n)
+          mbar_wait(&sm.row_full[n % kRowStages], (n / kRowStages) & 1, &dummy);
+        for (int n = max(0, issued_col - kColStages); n < issued_col; ++n)
+          mbar_wait(&sm.col_full[n % kColStages], (n / kColStages) & 1, &dummy);
       }
     }
   } else if (warp == 1) {
@@ -184,25 +215,28 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         sf_copy_elect(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
       }
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
-        KvStage& st = sm.st[s];
+        const int n = u >> 1, half = u & 1, s = n % kRowStages, slot = n & 1;
+        KvRowStage& st = sm.rst[s];
         if (half == 0) {
-          ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+          ok = mbar_wait(&sm.row_full[s], (n / kRowStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           sf_copy_elect(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
         }
+        KV_TRACE(0, u, 0);
         if (u > 0) {
           // the team of the previous sub-tile has pulled S and dP into registers
           ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
+        KV_TRACE(0, u, 1);
         const uint64_t desc_q = make_desc_sw128(smem_u32(st.q)) + half * (kSub * 128 / 16);
         for (int kb = 0; kb < nk_qk; ++kb)
           mma_mxf8_ss_elect(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
                       tmem + kColSFK, tmem + kColSFQ + 4 * slot + 2 * half, kb > 0);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
+        KV_TRACE(0, u, 2);
       }
       if (!ok) {
         int dummy = 0;
@@ -219,10 +253,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       sf_copy_elect(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
     }
     for (int u = 0; u < n_sub && ok; ++u) {
-      const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1;
-      KvStage& st = sm.st[s];
+      const int n = u >> 1, half = u & 1, s = n % kRowStages, slot = n & 1;
+      KvRowStage& st = sm.rst[s];
       if (half == 0) {
-        ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+        ok = mbar_wait(&sm.row_full[s], (n / kRowStages) & 1, abort_flag);
         if (!ok) break;
         // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
         const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
@@ -257,17 +291,22 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int n = u >> 1, half = u & 1, s = n % kStages, slot = n & 1, buf = u & 1;
-        KvStage& st = sm.st[s];
+        const int n = u >> 1, half = u & 1, s = n % kColStages, slot = n & 1, buf = u & 1;
+        KvColStage& st = sm.cst[s];
         if (half == 0) {
-          ok = mbar_wait(&sm.q_full[s], (n / kStages) & 1, abort_flag);
+          ok = mbar_wait(&sm.col_full[s], (n / kColStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           sf_copy_elect(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
           sf_copy_elect(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
         }
+        KV_TRACE(1, u, 0);
         ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
+        KV_TRACE(1, u, 1);
+        // both halves of the tile have been through the softmax: its row set (scores operands,
+        // LSE, D) is no longer read
+        if (half == 1 && lane == 0) mbar_arrive(&sm.row_empty[n % kRowStages]);
         tc_fence_after_sync();
         sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
@@ -285,7 +324,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         // stage may be refilled after the second half (the S^T / dP^T MMAs that read it finished
         // before the softmax team could even start on this sub-tile)
         mma_commit_elect(&sm.pds_free[buf]);
-        if (half == 1) mma_commit_elect(&sm.q_empty[s]);
+        KV_TRACE(1, u, 2);
+        if (half == 1) mma_commit_elect(&sm.col_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.done);
       }
       if (!ok) {
@@ -303,10 +343,12 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
     bool ok = true;
     for (int u = team; u < n_sub; u += kTeams) {
-      const int n = u >> 1, half = u & 1, buf = u & 1, s = n % kStages;
+      const int n = u >> 1, half = u & 1, buf = u & 1, s = n % kRowStages;
       const int it = it0 + n % tiles_per_head;
+      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 0);
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
+      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 1);
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];                       // S then P; dP then dS (in place)
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
@@ -314,10 +356,11 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
-      ok = mbar_wait(&sm.lse_ready[s], (n / kStages) & 1, abort_flag);
+      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 2);
+      ok = mbar_wait(&sm.lse_ready[s], (n / kRowStages) & 1, abort_flag);
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
-      const KvStage& st = sm.st[s];
+      const KvRowStage& st = sm.rst[s];
       float amax_p = 0.f, max_s = 0.f, min_s = 0.f;   // |dS| maximum from a running max and min
       const float* s_lse = &st.neg_lse2[col0];
       const float* s_delta = &st.delta[col0];
@@ -373,6 +416,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.pds_full[buf]);
+      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 3);
     }
     // the epilogue is done by team 0 (group 0 stores dV, group 1 stores dK)
     if (team != 0) ok = false;
