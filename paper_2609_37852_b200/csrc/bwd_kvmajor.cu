@@ -361,15 +361,15 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
       const KvRowStage& st = sm.rst[s];
-      float amax_p = 0.f, max_s = 0.f, min_s = 0.f;   // |dS| maximum from a running max and min
+      float amax_p = 0.f, max_s = 0.f;
       const float* s_lse = &st.neg_lse2[col0];
       const float* s_delta = &st.delta[col0];
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
         for (int c4 = 0; c4 < 32; c4 += 4) {
-          const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[c4]);
-          const float4 d4 = *reinterpret_cast<const float4*>(&s_delta[c4]);
+          const float4 l4 = lds_f4(&s_lse[c4]);
+          const float4 d4 = lds_f4(&s_delta[c4]);
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
           const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
@@ -382,8 +382,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             sr[c] = __float_as_uint(pv);
             dpr[c] = __float_as_uint(dsv);
             amax_p = fmaxf(amax_p, pv);
-            max_s = fmaxf(max_s, dsv);
-            min_s = fminf(min_s, dsv);
+            max_s = fmaxf(max_s, fabsf(dsv));
           }
         }
       };
@@ -391,7 +390,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       uint32_t byte_p, byte_s;
       float inv_p, inv_s;
       block_scale(amax_p, byte_p, inv_p);
-      block_scale(fmaxf(max_s, -min_s), byte_s, inv_s);
+      block_scale(max_s, byte_s, inv_s);
       if (u >= 2) {
         // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
         ok = mbar_wait(&sm.pds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
@@ -410,8 +409,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
                               __uint_as_float(dpr[4 * i + 2]) * inv_s, __uint_as_float(dpr[4 * i + 3]) * inv_s);
       tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
       const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
-      sm.sf_p[buf][sf_at] = static_cast<uint8_t>(byte_p);
-      sm.sf_ds[buf][sf_at] = static_cast<uint8_t>(byte_s);
+      sts_u8(&sm.sf_p[buf][sf_at], byte_p);
+      sts_u8(&sm.sf_ds[buf][sf_at], byte_s);
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();

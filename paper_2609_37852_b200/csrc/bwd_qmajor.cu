@@ -335,7 +335,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           tc_fence_after_sync();
         }
         tmem_st8(tmem + kColdS + 32 * buf + lane_addr + 8 * grp, words);
-        sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
+        sts_u8(&sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
         tmem_wait_st();
         fence_proxy_async_smem();
         tc_fence_before_sync();

@@ -258,11 +258,11 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
 #pragma unroll
         for (int c = 0; c < 32; ++c) mx = fmaxf(mx, sv[c]);
       }
-      sm.xch[u & 1][grp][row] = mx;
+      sts_f32(&sm.xch[u & 1][grp][row], mx);
       mbar_arrive(&sm.pair[quad]);                    // the two warps that share these 32 rows
       ok = mbar_wait(&sm.pair[quad], u & 1, abort_flag);
       if (!ok) break;
-      mx = fmaxf(mx, sm.xch[u & 1][grp ^ 1][row]);
+      mx = fmaxf(mx, lds_f32(&sm.xch[u & 1][grp ^ 1][row]));
       // a fully masked sub-tile (second half of the diagonal tile for the first 64 rows) gives -inf:
       // it never raises M and contributes zeros
       const float m_new = ceilf(mx * p.scale_log2);
@@ -315,7 +315,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         tc_fence_after_sync();
       }
       tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
-      sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp] = static_cast<uint8_t>(byte);
+      sts_u8(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
