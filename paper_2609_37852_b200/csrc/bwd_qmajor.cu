@@ -21,6 +21,8 @@
 // release the buffers at once, so the next tile's MMAs overlap the exponentials of this one.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "mxfp8_device.cuh"
 #include "sm100_ptx.cuh"
@@ -50,6 +52,7 @@ constexpr int kSoftmaxThreads = 128 * kGroups;  // 16 warps: 4 TMEM lane quadran
 constexpr int kThreads = 128 + kSoftmaxThreads;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
+constexpr float kLn2 = 0.6931471805599453f;
 
 constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* 2 x 32 */, kColdQ = 320;
 constexpr uint32_t kColSFQ = 448, kColSFdO = 452, kColSFK = 456 /* 2 x 4 */, kColSFV = 464 /* 2 x 4 */,
@@ -288,6 +291,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float lse2 = lse_nat * kLog2e;
     const float lse2_lo = fmaf(lse_nat, kLog2e, -lse2) + lse_nat * kLog2eLo;
     const float D = kDQ ? p.delta_in[grow] : 0.f;
+    const float f_lo = fmaf(-lse2_lo, kLn2, 1.0f);   // 2^-lo to first order (|lo| < 1e-5)
+    const float fD = f_lo * D;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
     bool ok = true;
     for (int t = 0; t < n_tiles; ++t) {
@@ -304,27 +309,33 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free);
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 2);
-      const bool diag = p.causal && (t == qt);
       const int col0 = 32 * grp;                      // column of this thread's first element inside the key tile
       float ds[32];
       float part = 0.f;
+      // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
+      // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
+      // a loop without it
+      auto body = [&](auto diag_tag) {
+        constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -lse2) - lse2_lo;
-        if (diag && (col0 + c > row)) x = -INFINITY;
-        const float pr = ex2_approx(x);
-        const float dp = __uint_as_float(dpr[c]);
-        if (kDQ) {
-          const float d = pr * (dp - D);
-          ds[c] = d;
-          acc0 += d;
-          acc1 += fabsf(d);
-        } else {
-          part = fmaf(pr, dp, part);
+        for (int c = 0; c < 32; ++c) {
+          float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -lse2);
+          if (kDiag && (col0 + c > row)) x = -INFINITY;
+          const float pr = ex2_approx(x);
+          const float dp = __uint_as_float(dpr[c]);
+          if (kDQ) {
+            const float d = pr * fmaf(dp, f_lo, -fD);
+            ds[c] = d;
+            acc0 += d;
+            acc1 += fabsf(d);
+          } else {
+            part = fmaf(pr, dp, part);
+          }
         }
-      }
+      };
+      if (p.causal && t == qt) body(std::true_type{}); else body(std::false_type{});
       if (!kDQ) {
-        acc0 += part;
+        acc0 = fmaf(part, f_lo, acc0);
       } else {
         uint32_t words[8];
         const uint32_t byte = quantize_block32(ds, words);
