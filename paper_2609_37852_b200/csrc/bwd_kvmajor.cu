@@ -119,8 +119,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   extern __shared__ uint8_t smem_raw[];
   KvSmem& sm = *reinterpret_cast<KvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int jt = blockIdx.x;                        // key tile; tile 0 has the most work under the causal mask
-  const int g = blockIdx.y, b = blockIdx.z;
+  // blocks are handed out x-fastest: KV heads vary fastest, key tiles in order, so the heaviest
+  // tiles (the earliest keys under the causal mask) of all heads go first
+  const int jt = blockIdx.y;
+  const int g = blockIdx.x, b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
   const int tiles_n = p.N / kTile;
   const int it0 = p.causal ? jt : 0;                // first query tile that sees these keys
@@ -475,7 +477,7 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   const size_t smem = sizeof(KvSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.N / kTile, s.Hkv, s.B);
+  dim3 grid(s.Hkv, s.N / kTile, s.B);
   kvmajor_kernel<<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));

@@ -107,8 +107,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   constexpr int kStages = kStagesFor<kDQ>;
   QmSmem<kDQ>& sm = *reinterpret_cast<QmSmem<kDQ>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qt = p.causal ? (gridDim.x - 1 - blockIdx.x) : blockIdx.x;
-  const int h = blockIdx.y, b = blockIdx.z;
+  // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
+  // all heads go first, so the light tiles fill the tail of the launch
+  const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
+  const int h = blockIdx.x, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
   const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
@@ -423,7 +425,7 @@ attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t
   const size_t smem = sizeof(QmSmem<kDQ>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<kDQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.N / kTile, s.Hq, s.B);
+  dim3 grid(s.Hq, s.N / kTile, s.B);
   qmajor_kernel<kDQ><<<grid, kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: launch: %s", cudaGetErrorString(e));

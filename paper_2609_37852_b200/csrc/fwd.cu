@@ -90,8 +90,10 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   FwdSmem& sm = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // heavy (late) query tiles first
-  const int qt = p.causal ? (gridDim.x - 1 - blockIdx.x) : blockIdx.x;
-  const int h = blockIdx.y, b = blockIdx.z;
+  // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
+  // all heads go first, so the light tiles fill the tail of the launch
+  const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
+  const int h = blockIdx.x, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
   const int n_sub = 2 * n_tiles;
@@ -380,7 +382,7 @@ attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k,
   const size_t smem = sizeof(FwdSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.N / kTile, s.Hq, s.B);
+  dim3 grid(s.Hq, s.N / kTile, s.B);
   fwd_kernel<<<grid, kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));
