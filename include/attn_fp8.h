@@ -30,8 +30,17 @@
  *   - Changing delta_mode changes only `delta`, dQ and dK -- never O, LSE or dV.
  *
  * Supported shapes: seqlen a multiple of 128 (Nq == Nk, causal means key j <= query i);
- * heads_q a multiple of heads_kv; head dims: (qk, v) in {(64,64), (128,128)} for the
- * attention entry points; the quantiser accepts any d that is a multiple of 32 up to 256.
+ * heads_q a multiple of heads_kv; head dims (qk, v): {(64,64), (128,128)} for every attention
+ * entry point, plus (192,128) and (256,256) where an entry point says so; the quantiser accepts
+ * any d that is a multiple of 32 up to 256.  Anything else returns ATTN_ERR_UNSUPPORTED.
+ *
+ * BF16 mode (attn_params_t.precision = ATTN_PREC_BF16; the paper's BF16 reference point, Section
+ * 2.1): the same kernels with BF16 operands and no block scales.  An attn_qtensor_t then carries
+ *   row_codes = BF16 [B, H, N, d]   (the tensor itself, rounded to BF16)
+ *   col_codes = BF16 [B, H, d, N]   (its transpose)
+ * and both scale pointers are ignored (may be NULL); attn_fp8_prepare_bf16 writes the two copies.
+ * Probabilities and score gradients are rounded to BF16 where the FP8 mode quantises them; the
+ * normaliser, LSE, the row correction and every accumulation stay FP32 exactly as in FP8 mode.
  */
 #ifndef ATTN_FP8_H_
 #define ATTN_FP8_H_
@@ -109,10 +118,19 @@ size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols);
 attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
                                 int32_t d, attn_qtensor_t out, void* stream);
 
+/* Operand preparation for BF16 mode: writes the BF16 rounding of `src` to out.row_codes
+ * ([B, H, N, d]) and its transpose to out.col_codes ([B, H, d, N]); an orientation whose pointer
+ * is NULL is skipped, the scale pointers are ignored.  A caller whose source already is BF16 may
+ * pass the source itself as row_codes of the attention calls and ask only for the transpose.
+ *   N % 128 == 0, d % 32 == 0, 32 <= d <= 256; pointers 16-byte aligned.                      */
+attn_status_t attn_fp8_prepare_bf16(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
+                                    int32_t d, attn_qtensor_t out, void* stream);
+
 /* Forward (paper Appendix "Forward Probability Encoding"): per query row, online softmax of
  * S = scale * Q^ K^^T over key tiles with a running INTEGER power-of-two shift, normaliser l
  * taken from the exponentials BEFORE the FP8 cast, probabilities quantised in-register in
  * blocks of 32 keys, O = (P^ V^) / l.
+ *   head dims: (64,64), (128,128), (192,128), (256,256) in FP8 mode; (64,64), (128,128) in BF16 mode
  *   reads   q.row_*, k.row_*, v.col_*
  *   writes  o_bf16 [B, Hq, N, dv] (BF16), lse [B, Hq, N] (FP32, natural log)                  */
 attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,

@@ -32,7 +32,7 @@ ATTN_SRC_BF16, ATTN_SRC_FP32 = 0, 1
 ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_fwd", "attn_fp8_bwd_delta",
+    "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
 )
@@ -63,6 +63,8 @@ _lib.attn_fp8_scale_bytes.restype = _sz
 _lib.attn_fp8_scale_bytes.argtypes = [ctypes.c_int64] * 4
 _lib.attn_fp8_quantize.restype = _i32
 _lib.attn_fp8_quantize.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _QTensor, _vp]
+_lib.attn_fp8_prepare_bf16.restype = _i32
+_lib.attn_fp8_prepare_bf16.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _QTensor, _vp]
 _lib.attn_fp8_fwd.restype = _i32
 _lib.attn_fp8_fwd.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _vp, _vp, _vp, _sz, _vp]
 _lib.attn_fp8_bwd_delta.restype = _i32
@@ -181,6 +183,29 @@ def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool =
     elif tuple(out.shape) != (B, H, N, d):
         raise ValueError("out was allocated for another shape")
     _check(_lib.attn_fp8_quantize(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
+    return out
+
+
+def attn_fp8_prepare_bf16(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None) -> QTensor:
+    """BF16-mode operands of ``src`` [B, H, N, d]: ``row_codes`` = BF16 [B, H, N, d] (``src`` itself when
+    it already is BF16), ``col_codes`` = BF16 [B, H, d, N]; no scales."""
+    if not src.is_cuda or not src.is_contiguous() or src.dim() != 4:
+        raise ValueError("src must be a contiguous CUDA tensor [B, H, N, d]")
+    if src.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("src must be bfloat16 or float32")
+    dt = ATTN_SRC_BF16 if src.dtype == torch.bfloat16 else ATTN_SRC_FP32
+    B, H, N, d = src.shape
+    out = QTensor(shape=(B, H, N, d))
+    bf = dict(dtype=torch.bfloat16, device=src.device)
+    write_row = want_row and src.dtype != torch.bfloat16
+    if write_row:
+        out.row_codes = torch.empty((B, H, N, d), **bf)
+    if want_col:
+        out.col_codes = torch.empty((B, H, d, N), **bf)
+    if write_row or want_col:
+        _check(_lib.attn_fp8_prepare_bf16(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
+    if want_row and not write_row:
+        out.row_codes = src
     return out
 
 

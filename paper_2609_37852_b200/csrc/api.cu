@@ -60,22 +60,33 @@ static attn_status_t check_device() {
   return ATTN_OK;
 }
 
-static attn_status_t check_params(const attn_params_t* p, AttnShape* s) {
+enum Entry { kEntryFwd = 0, kEntryDelta = 1, kEntryDq = 2, kEntryDkdv = 3 };
+
+// Head-dimension pairs each kernel family is built for, per operand width.
+static bool dims_supported(int entry, int eb, int dqk, int dv) {
+  const bool narrow = (dqk == 64 && dv == 64) || (dqk == 128 && dv == 128);
+  if (narrow) return eb == 1 || entry == kEntryFwd;
+  const bool wide = (dqk == 192 && dv == 128) || (dqk == 256 && dv == 256);
+  if (eb == 1 && wide) return entry == kEntryFwd;
+  return false;
+}
+
+static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entry) {
   if (!p) return fail(ATTN_ERR_INVALID_ARG, "params is NULL");
   if (p->batch <= 0 || p->seqlen <= 0 || p->heads_q <= 0 || p->heads_kv <= 0)
     return fail(ATTN_ERR_INVALID_ARG, "batch, seqlen and head counts must be positive");
   if (p->heads_q % p->heads_kv) return fail(ATTN_ERR_INVALID_ARG, "heads_q must be a multiple of heads_kv");
   if (p->causal != 0 && p->causal != 1) return fail(ATTN_ERR_INVALID_ARG, "causal must be 0 or 1");
   if (!(p->softmax_scale > 0.f)) return fail(ATTN_ERR_INVALID_ARG, "softmax_scale must be positive");
-  if (p->precision != ATTN_PREC_MXFP8)
-    return fail(ATTN_ERR_UNSUPPORTED, "precision %d: only ATTN_PREC_MXFP8 is built", p->precision);
+  if (p->precision != ATTN_PREC_MXFP8 && p->precision != ATTN_PREC_BF16)
+    return fail(ATTN_ERR_INVALID_ARG, "precision %d unknown", p->precision);
   if (p->seqlen % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen must be a multiple of 128");
-  const bool dims_ok = (p->head_dim_qk == 64 && p->head_dim_v == 64) || (p->head_dim_qk == 128 && p->head_dim_v == 128);
-  if (!dims_ok)
-    return fail(ATTN_ERR_UNSUPPORTED, "head dims (%d, %d): supported are (64,64) and (128,128)", p->head_dim_qk,
-                p->head_dim_v);
+  const int eb = p->precision == ATTN_PREC_BF16 ? 2 : 1;
+  if (!dims_supported(entry, eb, p->head_dim_qk, p->head_dim_v))
+    return fail(ATTN_ERR_UNSUPPORTED, "head dims (%d, %d) are not built for this entry point in %s mode",
+                p->head_dim_qk, p->head_dim_v, eb == 1 ? "MXFP8" : "BF16");
   *s = AttnShape{p->batch, p->seqlen, p->heads_q, p->heads_kv, p->head_dim_qk, p->head_dim_v, p->causal,
-                 p->softmax_scale};
+                 p->softmax_scale, eb};
   return ATTN_OK;
 }
 
@@ -84,6 +95,13 @@ static attn_status_t check_ptr(const void* p, const char* name) {
   if (!aligned16(p)) return fail(ATTN_ERR_ALIGNMENT, "%s is not 16-byte aligned", name);
   return ATTN_OK;
 }
+
+// One orientation of an operand: the codes (or BF16 values) always, the scale bytes in FP8 mode.
+#define CHECK_OPERAND(t, orient, fp8)                                                   \
+  do {                                                                                   \
+    CHECK(check_ptr(t.orient##_codes, #t "." #orient "_codes"));                          \
+    if (fp8) CHECK(check_ptr(t.orient##_scales, #t "." #orient "_scales"));               \
+  } while (0)
 
 #define CHECK(x)                        \
   do {                                  \
@@ -134,6 +152,21 @@ attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, i
   return launch_quantize(src, src_dtype, B, H, N, d, out, static_cast<cudaStream_t>(stream));
 }
 
+attn_status_t attn_fp8_prepare_bf16(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
+                                    attn_qtensor_t out, void* stream) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return fail(ATTN_ERR_INVALID_ARG, "sizes must be positive");
+  if (src_dtype != ATTN_SRC_BF16 && src_dtype != ATTN_SRC_FP32)
+    return fail(ATTN_ERR_INVALID_ARG, "src_dtype %d is neither BF16 nor FP32", src_dtype);
+  if (N % 128 || d % 32 || d > 256)
+    return fail(ATTN_ERR_UNSUPPORTED, "prepare_bf16 needs N %% 128 == 0 and d %% 32 == 0, d <= 256 (N=%d d=%d)", N, d);
+  CHECK(check_ptr(src, "src"));
+  if (!out.row_codes && !out.col_codes) return fail(ATTN_ERR_INVALID_ARG, "no output orientation requested");
+  if (out.row_codes) CHECK(check_ptr(out.row_codes, "row_codes"));
+  if (out.col_codes) CHECK(check_ptr(out.col_codes, "col_codes"));
+  CHECK(check_device());
+  return launch_bf16_copies(src, src_dtype, B, H, N, d, out.row_codes, out.col_codes, static_cast<cudaStream_t>(stream));
+}
+
 size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which) {
   (void)p;
   (void)which;
@@ -143,10 +176,9 @@ size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which) {
 attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                            void* o_bf16, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
   AttnShape s;
-  CHECK(check_params(p, &s));
-  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
-  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
-  CHECK(check_ptr(v.col_codes, "v.col_codes")); CHECK(check_ptr(v.col_scales, "v.col_scales"));
+  CHECK(check_params(p, &s, kEntryFwd));
+  const bool fp8 = s.eb == 1;
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, col, fp8);
   CHECK(check_ptr(o_bf16, "o_bf16")); CHECK(check_ptr(lse, "lse"));
   CHECK(check_device());
   int* status = nullptr;
@@ -159,7 +191,8 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
                                  attn_qtensor_t dO, const void* dO_bf16, const void* o_bf16, const float* lse,
                                  float* delta, void* workspace, size_t workspace_bytes, void* stream) {
   AttnShape s;
-  CHECK(check_params(p, &s));
+  CHECK(check_params(p, &s, kEntryDelta));
+  const bool fp8 = s.eb == 1;
   CHECK(check_ptr(delta, "delta"));
   CHECK(check_device());
   int* status = nullptr;
@@ -170,10 +203,7 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
     return launch_stale_delta(s, dO_bf16, o_bf16, delta, st);
   }
   if (p->delta_mode != ATTN_DELTA_MATCHED) return fail(ATTN_ERR_INVALID_ARG, "delta_mode %d unknown", p->delta_mode);
-  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
-  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
-  CHECK(check_ptr(v.row_codes, "v.row_codes")); CHECK(check_ptr(v.row_scales, "v.row_scales"));
-  CHECK(check_ptr(dO.row_codes, "dO.row_codes")); CHECK(check_ptr(dO.row_scales, "dO.row_scales"));
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8); CHECK_OPERAND(dO, row, fp8);
   CHECK(check_ptr(lse, "lse"));
   return launch_bwd_delta(s, q, k, v, dO, lse, delta, status, st);
 }
@@ -183,21 +213,19 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
                               void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
                               size_t workspace_bytes, void* stream, bool want_dq, bool want_dkdv) {
   AttnShape s;
-  CHECK(check_params(p, &s));
-  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
-  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
-  CHECK(check_ptr(v.row_codes, "v.row_codes")); CHECK(check_ptr(v.row_scales, "v.row_scales"));
-  CHECK(check_ptr(dO.row_codes, "dO.row_codes")); CHECK(check_ptr(dO.row_scales, "dO.row_scales"));
+  if (want_dq) CHECK(check_params(p, &s, kEntryDq));
+  if (want_dkdv) CHECK(check_params(p, &s, kEntryDkdv));
+  const bool fp8 = s.eb == 1;
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8); CHECK_OPERAND(dO, row, fp8);
   CHECK(check_ptr(lse, "lse")); CHECK(check_ptr(delta, "delta"));
   if (want_dq) {
-    CHECK(check_ptr(k.col_codes, "k.col_codes")); CHECK(check_ptr(k.col_scales, "k.col_scales"));
+    CHECK_OPERAND(k, col, fp8);
     CHECK(check_ptr(dq_bf16, "dq_bf16"));
     if ((diag_rowsum_ds == nullptr) != (diag_rowsum_abs_ds == nullptr))
       return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
   }
   if (want_dkdv) {
-    CHECK(check_ptr(q.col_codes, "q.col_codes")); CHECK(check_ptr(q.col_scales, "q.col_scales"));
-    CHECK(check_ptr(dO.col_codes, "dO.col_codes")); CHECK(check_ptr(dO.col_scales, "dO.col_scales"));
+    CHECK_OPERAND(q, col, fp8); CHECK_OPERAND(dO, col, fp8);
     CHECK(check_ptr(dk_bf16, "dk_bf16")); CHECK(check_ptr(dv_bf16, "dv_bf16"));
   }
   CHECK(check_device());
@@ -286,10 +314,9 @@ static attn_status_t builtin_scratch_for_current_device(void** out) {
 extern "C" attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k,
                                               attn_qtensor_t v, void* o_bf16, float* lse, void* stream) {
   AttnShape s;
-  CHECK(check_params(p, &s));
-  CHECK(check_ptr(q.row_codes, "q.row_codes")); CHECK(check_ptr(q.row_scales, "q.row_scales"));
-  CHECK(check_ptr(k.row_codes, "k.row_codes")); CHECK(check_ptr(k.row_scales, "k.row_scales"));
-  CHECK(check_ptr(v.col_codes, "v.col_codes")); CHECK(check_ptr(v.col_scales, "v.col_scales"));
+  CHECK(check_params(p, &s, kEntryFwd));
+  const bool fp8 = s.eb == 1;
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, col, fp8);
   CHECK(check_ptr(o_bf16, "o_bf16")); CHECK(check_ptr(lse, "lse"));
   const size_t need = attn_fp8_workspace_bytes(p, ATTN_WS_FWD);
   if (need > kBuiltinScratchBytes)

@@ -24,11 +24,14 @@ attn_status_t encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t 
 struct AttnShape {
   int B, N, Hq, Hkv, dqk, dv, causal;
   float scale;
+  int eb;   // bytes per operand element: 1 = E4M3 codes with E8M0 block scales, 2 = BF16 without scales
 };
 
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).
 attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
                               cudaStream_t stream);
+attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, int N, int d, void* row_out, void* col_out,
+                                 cudaStream_t stream);
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
                          float* lse, int* status, cudaStream_t stream);
 attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,

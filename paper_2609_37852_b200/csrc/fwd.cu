@@ -18,6 +18,12 @@
 // M is only raised when the sub-tile maximum exceeds it by more than kLazyShift (the block scales
 // absorb the difference), so the accumulator in tensor memory is almost never rescaled.
 // Two MMA-issuing warps because one warp issues at most one tcgen05.mma per ~130 cycles.
+//
+// The kernel is a template over the operand width: element bytes (1: E4M3 codes with E8M0 block
+// scales; 2: BF16 without scales, the reference-point mode), 128-byte chunks per row of the
+// Q / K tiles (head dims above 128 bytes per row take two) and 128-row tiles of the V operand
+// (dv = 256 takes two).  A shared-memory stage always holds one 128-byte chunk of the token
+// dimension: 128 keys of codes or 64 keys of BF16.
 #include <cuda_bf16.h>
 
 #include <type_traits>
@@ -41,23 +47,38 @@ constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kL
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
 constexpr int kLazyShift = 8;
 
-// tensor-memory columns (256 allocated)
-constexpr uint32_t kColS = 0;        // scores of the current sub-tile, 64 columns
-constexpr uint32_t kColP = 64;       // probability codes, two buffers of 16 columns
-constexpr uint32_t kColO = 96;       // output accumulator, dv (<= 128) columns
-constexpr uint32_t kColSFQ = 224;    // scale factors: Q (4), K (2 x 4), V (2 x 4), P (2 x 4)
-constexpr uint32_t kColSFK = 228;
-constexpr uint32_t kColSFV = 236;
-constexpr uint32_t kColSFP = 244;
-constexpr uint32_t kTmemCols = 256;
+// Operand geometry and tensor-memory map of one instantiation.
+template <int kEB_, int kCq_, int kRv_>
+struct FwdCfg {
+  static constexpr int kEB = kEB_;                      // bytes per operand element
+  static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row
+  static constexpr int kRv = kRv_;                      // 128-row tiles of the V^T operand (dv / 128, rounded up)
+  static constexpr bool kFp8 = kEB == 1;
+  static constexpr int kTileKeys = kTile / kEB;         // keys per K / V stage
+  static constexpr int kSubPerTile = kTileKeys / kSub;  // 64-key steps per stage
+  static constexpr int kPCols = 16 * kEB;               // columns of one probability buffer (64 keys)
+  static constexpr uint32_t kColS = 0;                  // scores of the current sub-tile, 64 columns
+  static constexpr uint32_t kColP = 64;                 // probability operand, two buffers
+  static constexpr uint32_t kColO = kColP + 2 * kPCols; // output accumulator, dv columns
+  // scale factors (FP8 only): Q (4 per chunk), K (2 slots), V (2 slots x row tiles), P (2 x 4)
+  static constexpr uint32_t kColSFQ = kColO + 128 * kRv;
+  static constexpr uint32_t kColSFK = kColSFQ + 4 * kCq;
+  static constexpr uint32_t kColSFV = kColSFK + 8 * kCq;
+  static constexpr uint32_t kColSFP = kColSFV + 8 * kRv;
+  static constexpr uint32_t kColsUsed = kFp8 ? kColSFP + 8 : kColSFQ;
+  static constexpr uint32_t kTmemCols = kColsUsed <= 256 ? 256 : 512;
+  static constexpr int kCtasPerSm = kTmemCols == 256 ? 2 : 1;
+  static_assert(kColsUsed <= 512, "tensor memory exceeded");
+};
 
+template <class C>
 struct FwdSmem {
-  alignas(1024) uint8_t q[kTile * 128];
-  alignas(1024) uint8_t k[kStages][kTile * 128];
-  alignas(1024) uint8_t v[kStages][kTile * 128];
-  alignas(16) uint8_t sf_q[512];
-  alignas(16) uint8_t sf_k[kStages][512];
-  alignas(16) uint8_t sf_v[kStages][512];
+  alignas(1024) uint8_t q[C::kCq][kTile * 128];
+  alignas(1024) uint8_t k[kStages][C::kCq][C::kTileKeys * 128];
+  alignas(1024) uint8_t v[kStages][C::kRv * kTile * 128];
+  alignas(16) uint8_t sf_q[C::kCq * 512];
+  alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
+  alignas(16) uint8_t sf_v[kStages][C::kRv * 512];
   alignas(16) uint8_t sf_p[2][512];
   alignas(16) float xch[2][2][kTile];       // row maxima (and at the end normaliser shares) of the thread pairs
   uint64_t q_full;
@@ -83,11 +104,16 @@ struct FwdParams {
   float scale_log2;         // softmax_scale * log2(e)
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+template <class C>
+__global__ void __launch_bounds__(kThreads, C::kCtasPerSm)
 fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ uint8_t smem_raw[];
-  FwdSmem& sm = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  FwdSmem<C>& sm = *reinterpret_cast<FwdSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr bool kFp8 = C::kFp8;
+  constexpr int kEB = C::kEB, kCq = C::kCq, kRv = C::kRv, kSubPerTile = C::kSubPerTile;
+  constexpr uint32_t kColS = C::kColS, kColP = C::kColP, kColO = C::kColO, kColSFQ = C::kColSFQ, kColSFK = C::kColSFK,
+                     kColSFV = C::kColSFV, kColSFP = C::kColSFP, kTmemCols = C::kTmemCols, kPCols = C::kPCols;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // heavy (late) query tiles first
   // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
@@ -97,7 +123,9 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
   const int n_sub = 2 * n_tiles;
-  const int nk_qk = p.dqk / 32;                 // K blocks of the score MMA
+  const int n_stage_tiles = n_tiles * kEB;      // K / V stages to stream
+  const int nk_qk = p.dqk * kEB / 32;           // 32-byte K steps of the score MMA
+  const int rv = (p.dv + 127) / 128;            // 128-row tiles of V^T actually present
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
@@ -128,25 +156,32 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     if (lane == 0) {
       prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
       const int q_row = (b * p.Hq + h) * p.N + qt * kTile;
-      mbar_arrive_expect_tx(&sm.q_full, kTile * 128 + 512);
-      tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_row);
-      bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(b * p.Hq + h) * (p.N / kTile) + qt) * 512, 512, &sm.q_full);
+      const int tiles_n = p.N / kTile;
+      mbar_arrive_expect_tx(&sm.q_full, kCq * kTile * 128 + (kFp8 ? kCq * 512 : 0));
+      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[c], &tm_q, &sm.q_full, 128 * c, q_row);
+      if (kFp8)
+        bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(b * p.Hq + h) * tiles_n + qt) * kCq * 512, kCq * 512, &sm.q_full);
       const int kv_slab = b * p.Hkv + g;
       int issued_k = 0, issued_v = 0;
       bool ok = true;
-      for (int t = 0; t < n_tiles && ok; ++t) {
+      for (int t = 0; t < n_stage_tiles && ok; ++t) {
         const int s = t % kStages, u = t / kStages;
         ok = mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
-        tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
-        bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * (p.N / kTile) + t) * 512, 512, &sm.k_full[s]);
+        mbar_arrive_expect_tx(&sm.k_full[s], kCq * C::kTileKeys * 128 + (kFp8 ? kCq * 512 : 0));
+        for (int c = 0; c < kCq; ++c)
+          tma_load_2d(sm.k[s][c], &tm_k, &sm.k_full[s], 128 * c, kv_slab * p.N + t * C::kTileKeys);
+        if (kFp8)
+          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.k_full[s]);
         ++issued_k;
         ok = mbar_wait(&sm.v_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
-        tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * kTile, kv_slab * p.dv);
-        bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * (p.N / kTile) + t) * 512, 512, &sm.v_full[s]);
+        mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + (kFp8 ? rv * 512 : 0));
+        tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
+        if (kFp8)
+          for (int r = 0; r < rv; ++r)
+            bulk_load_1d(sm.sf_v[s] + 512 * r, p.v_sf + ((static_cast<size_t>(kv_slab) * rv + r) * tiles_n + t) * 512, 512,
+                         &sm.v_full[s]);
         ++issued_v;
       }
       if (!ok) {
@@ -161,19 +196,21 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S = Q K^T issuer
     {
-      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
+      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[0]));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok) {
+      if (ok && kFp8) {
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+        for (int c = 0; c < kCq; ++c) sf_copy_elect(tmem + kColSFQ + 4 * c, make_desc_sf(smem_u32(sm.sf_q + 512 * c)));
       }
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1;
-        if (half == 0) {
+        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1;
+        if (sub == 0) {
           ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy_elect(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+          if (kFp8)
+            for (int c = 0; c < kCq; ++c)
+              sf_copy_elect(tmem + kColSFK + 4 * kCq * slot + 4 * c, make_desc_sf(smem_u32(sm.sf_k[s] + 512 * c)));
         }
         if (u > 0) {
           // the softmax threads have pulled the previous scores into registers
@@ -181,12 +218,19 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           if (!ok) break;
           tc_fence_after_sync();
         }
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + half * (kSub * 128 / 16);
-        for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss_elect(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
-                      tmem + kColSFQ, tmem + kColSFK + 4 * slot + 2 * half, kb > 0);
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0])) + sub * (kSub * 128 / 16);
+        for (int kb = 0; kb < nk_qk; ++kb) {
+          const int c = kb >> 2, w = kb & 3;          // chunk and 32-byte step inside it
+          const uint64_t a = desc_q + c * (kTile * 128 / 16) + 2 * w;
+          const uint64_t bdesc = desc_k + c * (C::kTileKeys * 128 / 16) + 2 * w;
+          if (kFp8)
+            mma_mxf8_ss_elect(tmem + kColS, a, bdesc, make_idesc_mxf8(128, kSub, w, w), tmem + kColSFQ + 4 * c,
+                              tmem + kColSFK + 4 * kCq * slot + 4 * c + 2 * sub, kb > 0);
+          else
+            mma_bf16_ss_elect(tmem + kColS, a, bdesc, make_idesc_bf16(128, kSub), kb > 0);
+        }
         mma_commit_elect(&sm.s_full);
-        if (half == 1) mma_commit_elect(&sm.k_empty[s]);
+        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
       }
       if (!ok) {
         int dummy = 0;
@@ -199,24 +243,37 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int t = u >> 1, half = u & 1, s = t % kStages, slot = t & 1, buf = u & 1;
-        if (half == 0) {
+        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1, buf = u & 1;
+        if (sub == 0) {
           ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy_elect(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+          if (kFp8)
+            for (int r = 0; r < rv; ++r)
+              sf_copy_elect(tmem + kColSFV + 4 * kRv * slot + 4 * r, make_desc_sf(smem_u32(sm.sf_v[s] + 512 * r)));
         }
         ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+        if (kFp8) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
-        for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts_elect(tmem + kColO, tmem + kColP + 16 * buf + 8 * kb, desc_v + 2 * (2 * half + kb),
-                      make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
-                      tmem + kColSFV + 4 * slot, (u > 0 || kb > 0));
-        mma_commit_elect(&sm.p_free[buf]);              // codes / scale bytes of this buffer consumed; O updated
-        if (half == 1) mma_commit_elect(&sm.v_empty[s]);
+        // 64 keys = 2 (codes) or 4 (BF16) steps of 32 bytes; the V^T operand is taken 128 rows at a time
+        for (int r = 0; r < rv; ++r) {
+          const int n = min(128, p.dv - 128 * r);
+          for (int kb = 0; kb < 2 * kEB; ++kb) {
+            const int koff = 2 * sub + kb;            // 32-byte step inside the stage's chunk
+            const uint64_t bdesc = desc_v + r * (kTile * 128 / 16) + 2 * koff;
+            if (kFp8)
+              mma_mxf8_ts_elect(tmem + kColO + 128 * r, tmem + kColP + kPCols * buf + 8 * kb, bdesc,
+                                make_idesc_mxf8(128, n, kb, koff), tmem + kColSFP + 4 * buf,
+                                tmem + kColSFV + 4 * kRv * slot + 4 * r, (u > 0 || kb > 0));
+            else
+              mma_bf16_ts_elect(tmem + kColO + 128 * r, tmem + kColP + kPCols * buf + 8 * kb, bdesc,
+                                make_idesc_bf16(128, n), (u > 0 || kb > 0));
+          }
+        }
+        mma_commit_elect(&sm.p_free[buf]);              // operand (and scale bytes) of this buffer consumed; O updated
+        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.o_done);
       }
       if (!ok) {
@@ -303,21 +360,28 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         amax = fmaxf(amax, fmaxf(p0, p1));
       }
       l += bs0 + bs1;
-      uint32_t byte;
-      float inv;
-      block_scale(amax, byte, inv);
-      uint32_t words[8];
+      uint32_t byte = 0;
+      uint32_t words[8 * kEB];
+      if (kFp8) {
+        float inv;
+        block_scale(amax, byte, inv);
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        words[i] = cvt_e4m3x4(sv[4 * i] * inv, sv[4 * i + 1] * inv, sv[4 * i + 2] * inv, sv[4 * i + 3] * inv);
+        for (int i = 0; i < 8; ++i)
+          words[i] = cvt_e4m3x4(sv[4 * i] * inv, sv[4 * i + 1] * inv, sv[4 * i + 2] * inv, sv[4 * i + 3] * inv);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8 * kEB; ++i) words[i] = cvt_bf16x2(sv[(2 * i) & 31], sv[(2 * i + 1) & 31]);
+      }
       if (u >= 2) {
-        // the P V MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+        // the P V MMAs of sub-tile u-2 have consumed this buffer's operand and scale bytes
         ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
-      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
-      sts_u8(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
+#pragma unroll
+      for (int i = 0; i < kEB; ++i)
+        tmem_st8(tmem + kColP + kPCols * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
+      if (kFp8) sts_u8(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
@@ -362,31 +426,48 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
 }
 
-}  // namespace
-
-attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
-                         int* status, cudaStream_t stream) {
+template <class C>
+attn_status_t launch_fwd_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
+                           int* status, cudaStream_t stream) {
   CUtensorMap tm_q, tm_k, tm_v;
   attn_status_t st;
-  st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
+  constexpr int eb = C::kEB;
+  st = encode_tmap_u8_sw128(&tm_q, q.row_codes, static_cast<uint64_t>(s.dqk) * eb, static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, static_cast<uint64_t>(s.B) * s.Hkv * s.N, kTile);
+  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.N,
+                            C::kTileKeys);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
+  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.N) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
   if (st != ATTN_OK) return st;
   FwdParams p;
   p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
   p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale_log2 = s.scale * kLog2e;
-  const size_t smem = sizeof(FwdSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  const size_t smem = sizeof(FwdSmem<C>) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(fwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(s.Hq, s.N / kTile, s.B);
-  fwd_kernel<<<grid, kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
+  fwd_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
+}
+
+}  // namespace
+
+attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
+                         int* status, cudaStream_t stream) {
+  const int cq = (s.dqk * s.eb + 127) / 128, rv = (s.dv + 127) / 128;
+  if (s.eb == 1) {
+    if (cq == 1 && rv == 1) return launch_fwd_t<FwdCfg<1, 1, 1>>(s, q, k, v, o, lse, status, stream);
+    if (cq == 2 && rv == 1) return launch_fwd_t<FwdCfg<1, 2, 1>>(s, q, k, v, o, lse, status, stream);
+    if (cq == 2 && rv == 2) return launch_fwd_t<FwdCfg<1, 2, 2>>(s, q, k, v, o, lse, status, stream);
+  } else {
+    if (cq == 1 && rv == 1) return launch_fwd_t<FwdCfg<2, 1, 1>>(s, q, k, v, o, lse, status, stream);
+    if (cq == 2 && rv == 1) return launch_fwd_t<FwdCfg<2, 2, 1>>(s, q, k, v, o, lse, status, stream);
+  }
+  return fail(ATTN_ERR_UNSUPPORTED, "fwd: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv, s.eb);
 }
 
 }  // namespace attnfp8

@@ -147,7 +147,57 @@ attn_status_t launch_t(const void* src, int B, int H, int N, int d, attn_qtensor
   return ATTN_OK;
 }
 
+// BF16 mode: the operands are the tensors themselves, rounded to BF16, in both orientations.
+// One CTA transposes a tile of 64 tokens x d channels through shared memory.
+constexpr int kCopyTokens = 64;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) bf16_copies_kernel(const T* __restrict__ src, int N, int d,
+                                                               __nv_bfloat16* __restrict__ row_out,
+                                                               __nv_bfloat16* __restrict__ col_out) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(smem);       // [64][d + 2]
+  const int pitch = d + 2;
+  const size_t slab = blockIdx.y;
+  const size_t tok0 = static_cast<size_t>(blockIdx.x) * kCopyTokens;
+  const T* g_src = src + (slab * N + tok0) * d;
+  for (int i = threadIdx.x; i < kCopyTokens * d / 2; i += kThreads) {
+    const int e0 = 2 * i, tok = e0 / d, ch = e0 - tok * d;
+    const __nv_bfloat162 v2 = __floats2bfloat162_rn(to_f32(g_src[e0]), to_f32(g_src[e0 + 1]));
+    *reinterpret_cast<__nv_bfloat162*>(tile + tok * pitch + ch) = v2;
+    if (row_out) *reinterpret_cast<__nv_bfloat162*>(row_out + (slab * N + tok0) * d + e0) = v2;
+  }
+  if (!col_out) return;
+  __syncthreads();
+  for (int i = threadIdx.x; i < d * (kCopyTokens / 2); i += kThreads) {
+    const int c = i / (kCopyTokens / 2), tp = i % (kCopyTokens / 2);
+    __nv_bfloat162 v2;
+    v2.x = tile[(2 * tp) * pitch + c];
+    v2.y = tile[(2 * tp + 1) * pitch + c];
+    *reinterpret_cast<__nv_bfloat162*>(col_out + (slab * d + c) * N + tok0 + 2 * tp) = v2;
+  }
+}
+
+template <typename T>
+attn_status_t launch_copies_t(const void* src, int B, int H, int N, int d, void* row_out, void* col_out,
+                              cudaStream_t stream) {
+  const size_t smem = static_cast<size_t>(kCopyTokens) * (d + 2) * sizeof(__nv_bfloat16);
+  dim3 grid(N / kCopyTokens, B * H);
+  bf16_copies_kernel<T><<<grid, kThreads, smem, stream>>>(static_cast<const T*>(src), N, d,
+                                                         static_cast<__nv_bfloat16*>(row_out),
+                                                         static_cast<__nv_bfloat16*>(col_out));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bf16 copies: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
 }  // namespace
+
+attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, int N, int d, void* row_out, void* col_out,
+                                 cudaStream_t stream) {
+  if (src_dtype == ATTN_SRC_BF16) return launch_copies_t<__nv_bfloat16>(src, B, H, N, d, row_out, col_out, stream);
+  return launch_copies_t<float>(src, B, H, N, d, row_out, col_out, stream);
+}
 
 attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
                               cudaStream_t stream) {

@@ -349,6 +349,38 @@ __device__ __forceinline__ void sf_copy_elect(uint32_t tmem_dst, uint64_t sf_des
       ::"r"(tmem_dst), "l"(sf_desc) : "memory");
 }
 
+// ------------------------------------------------------------------ BF16 MMA (no block scales)
+// Instruction descriptor of a dense kind::f16 MMA: BF16 x BF16 -> FP32, both operands K-major.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 16 BF16 elements (32 bytes) of K per instruction.
+__device__ __forceinline__ void mma_bf16_ss_elect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Same with the A operand read from tensor memory (row m in lane m, two BF16 values per cell).
+__device__ __forceinline__ void mma_bf16_ts_elect(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "elect.sync _|q, 0xffffffff;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // ------------------------------------------------------------------ conversions
 // Two floats -> two E4M3 codes (lo in bits 0..7), round to nearest even, saturating.
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
@@ -365,6 +397,12 @@ __device__ __forceinline__ uint32_t cvt_e4m3x4(float a, float b, float c, float 
       "mov.b32 %0, {lo, hi};\n"
       "}\n"
       : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+  return r;
+}
+// Two floats -> two BF16 values (lo in bits 0..15), round to nearest even.
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
 __device__ __forceinline__ float ex2_approx(float x) {
