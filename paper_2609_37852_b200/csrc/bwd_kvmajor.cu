@@ -18,11 +18,20 @@
 // cannot issue tcgen05.mma fast enough for small tiles); warps 4..19 are two softmax teams that
 // take alternate sub-tiles (within a team, warp % 4 selects the 32 TMEM lanes and the column
 // group w takes query columns 32w..32w+31).
+//
+// The kernel is a template over the operand width (element bytes 1: E4M3 codes with E8M0 block
+// scales, 2: BF16 without scales; 128-byte chunks per operand row) and over which gradients it
+// accumulates.  The column copies are streamed one 128-byte chunk of the query dimension at a
+// time (128 queries of codes, 64 of BF16); the row copies 128 queries at a time in the narrow FP8
+// configuration and 64 otherwise.  When dV and dK together do not fit in tensor memory beside the
+// score tiles (qk head dim above 128), the launcher runs the kernel twice: a pass that rebuilds P
+// and accumulates dV, and a pass that rebuilds P and dS and accumulates dK.
 #include <cuda_bf16.h>
 
 #include <type_traits>
 
 #include "common.cuh"
+#include "mma_issue.cuh"
 #include "mxfp8_device.cuh"
 #include "sm100_ptx.cuh"
 
@@ -45,54 +54,89 @@ using namespace sm100;
 
 constexpr int kTile = 128;
 constexpr int kSub = 64;
-// Per query tile the CTA streams a 'row' set (Q and dO row copies, their scales, LSE, D: read by
-// the S^T / dP^T MMAs and the softmax) and a 'col' set (Q and dO column copies: read by the dV / dK
-// MMAs).  The row set is released early and has three stages, so that a reload never sits between
-// the end of one tile's gradient MMAs and the start of the next tile's scores.
-constexpr int kRowStages = 3;
-constexpr int kColStages = 2;
 constexpr int kTeams = 2;                       // softmax teams; team t takes sub-tiles u with u % kTeams == t
 constexpr int kTeamThreads = 256;               // 8 warps: 4 TMEM lane quadrants x 2 column groups
 constexpr int kThreads = 128 + kTeams * kTeamThreads;
-constexpr int kPrepThreads = 32;                // warp 2 turns LSE into -LSE*log2(e) once per query tile
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kSmemLimit = 232448;              // dynamic shared memory a CTA may ask for
 
-constexpr uint32_t kColS = 0, kColdP = 64, kColP = 128 /* 2 x 16 */, kColdS = 160 /* 2 x 16 */;
-constexpr uint32_t kColdV = 192, kColdK = 320;
-constexpr uint32_t kColSFK = 448, kColSFV = 452, kColSFQ = 456 /* 2 x 4 */, kColSFdO = 464 /* 2 x 4 */,
-                   kColSFP = 472 /* 2 x 4 */, kColSFdS = 480 /* 2 x 4 */, kColSFdOc = 488 /* 2 x 4 */,
-                   kColSFQc = 496 /* 2 x 4 */;
-constexpr uint32_t kTmemCols = 512;
+enum KvMode { kBoth = 0, kDvOnly = 1, kDkOnly = 2 };
 
+// Operand geometry, ring depths and tensor-memory map of one instantiation.
+template <int kEB_, int kCq_, int kCv_, int kMode_>
+struct KvCfg {
+  static constexpr int kEB = kEB_, kCq = kCq_, kCv = kCv_, kMode = kMode_;
+  static constexpr bool kFp8 = kEB == 1;
+  static constexpr bool kHasDv = kMode != kDkOnly;     // accumulates dV (needs P^)
+  static constexpr bool kHasDk = kMode != kDvOnly;     // accumulates dK (needs dP^T, D, dS^)
+  static constexpr int kRq = kCq / kEB > 0 ? (kCq + kEB - 1) / kEB : 1;   // 128-row tiles of the Q^c operand (dqk / 128, rounded up)
+  static constexpr int kRv = (kCv + kEB - 1) / kEB;                       // 128-row tiles of the dO^c operand
+  // Per query tile the CTA streams a 'row' set (Q and dO row copies, their scales, LSE, D: read by
+  // the S^T / dP^T MMAs and the softmax) and a 'col' set (Q and dO column copies: read by the dV /
+  // dK MMAs).  The row set is released early and gets the deeper ring, so that a reload never sits
+  // between the end of one tile's gradient MMAs and the start of the next tile's scores.
+  static constexpr int kRowTok = (kFp8 && kCq == 1 && kCv == 1) ? 128 : 64;   // queries per row stage
+  static constexpr int kColTok = kTile / kEB;                                 // queries per col stage
+  static constexpr int kSubPerRow = kRowTok / kSub, kSubPerCol = kColTok / kSub;
+  static constexpr int kKvBytes = (kCq + (kHasDk ? kCv : 0)) * kTile * 128;
+  static constexpr int kRowBytes = (kCq + (kHasDk ? kCv : 0)) * kRowTok * 128;
+  static constexpr int kColBytes = ((kHasDk ? kRq : 0) + (kHasDv ? kRv : 0)) * kTile * 128;
+  static constexpr int kColStages = 2;
+  static constexpr int kRowRaw = (216 * 1024 - kKvBytes - kColStages * kColBytes) / kRowBytes;
+  static constexpr int kRowStages = kRowRaw < 2 ? 2 : (kRowRaw > 3 ? 3 : kRowRaw);
+  // tensor memory
+  static constexpr int kOpCols = 16 * kEB;             // columns of one P^ / dS^ buffer (64 queries)
+  static constexpr uint32_t kColS = 0;
+  static constexpr uint32_t kColdP = 64;
+  static constexpr uint32_t kColP = kColdP + (kHasDk ? 64 : 0);
+  static constexpr uint32_t kColdS = kColP + (kHasDv ? 2 * kOpCols : 0);
+  static constexpr uint32_t kColdV = kColdS + (kHasDk ? 2 * kOpCols : 0);
+  static constexpr uint32_t kColdK = kColdV + (kHasDv ? 128 * kRv : 0);
+  static constexpr uint32_t kColSFK = kColdK + (kHasDk ? 128 * kRq : 0);
+  static constexpr uint32_t kColSFV = kColSFK + 4 * kCq;
+  static constexpr uint32_t kColSFQ = kColSFV + (kHasDk ? 4 * kCv : 0);        // 2 slots
+  static constexpr uint32_t kColSFdO = kColSFQ + 8 * kCq;                      // 2 slots
+  static constexpr uint32_t kColSFP = kColSFdO + (kHasDk ? 8 * kCv : 0);       // 2 x 4
+  static constexpr uint32_t kColSFdS = kColSFP + (kHasDv ? 8 : 0);             // 2 x 4
+  static constexpr uint32_t kColSFdOc = kColSFdS + (kHasDk ? 8 : 0);           // 2 slots x row tiles
+  static constexpr uint32_t kColSFQc = kColSFdOc + (kHasDv ? 8 * kRv : 0);     // 2 slots x row tiles
+  static constexpr uint32_t kColsUsed = kFp8 ? kColSFQc + (kHasDk ? 8 * kRq : 0) : kColSFK;
+  static constexpr uint32_t kTmemCols = 512;
+  static_assert(kColsUsed <= 512, "tensor memory exceeded");
+};
+
+template <class C>
 struct KvRowStage {
-  alignas(1024) uint8_t q[kTile * 128];       // Q row copy  [128 queries][dqk]
-  alignas(1024) uint8_t dO[kTile * 128];      // dO row copy [128 queries][dv]
-  alignas(16) uint8_t sf_q[512];
-  alignas(16) uint8_t sf_dO[512];
-  alignas(16) float lse[kTile];
-  alignas(16) float delta[kTile];
-  alignas(16) float neg_lse2[kTile];          // -LSE * log2(e), written by the prep warp
+  alignas(1024) uint8_t q[C::kCq][C::kRowTok * 128];                    // Q row copy  [queries][dqk]
+  alignas(1024) uint8_t dO[C::kHasDk ? C::kCv : 1][C::kHasDk ? C::kRowTok * 128 : 16];   // dO row copy [queries][dv]
+  alignas(16) uint8_t sf_q[C::kCq * 512];
+  alignas(16) uint8_t sf_dO[C::kCv * 512];
+  alignas(16) float lse[C::kRowTok];
+  alignas(16) float delta[C::kRowTok];
+  alignas(16) float neg_lse2[C::kRowTok];       // -LSE * log2(e), written by the prep warp
 };
+template <class C>
 struct KvColStage {
-  alignas(1024) uint8_t qc[kTile * 128];      // Q col copy  [dqk][128 queries]
-  alignas(1024) uint8_t dOc[kTile * 128];     // dO col copy [dv][128 queries]
-  alignas(16) uint8_t sf_qc[512];
-  alignas(16) uint8_t sf_dOc[512];
+  alignas(1024) uint8_t qc[C::kHasDk ? C::kRq * kTile * 128 : 16];      // Q col copy  [dqk][queries]
+  alignas(1024) uint8_t dOc[C::kHasDv ? C::kRv * kTile * 128 : 16];     // dO col copy [dv][queries]
+  alignas(16) uint8_t sf_qc[C::kRq * 512];
+  alignas(16) uint8_t sf_dOc[C::kRv * 512];
 };
 
+template <class C>
 struct KvSmem {
-  alignas(1024) uint8_t k[kTile * 128];
-  alignas(1024) uint8_t v[kTile * 128];
-  KvRowStage rst[kRowStages];
-  KvColStage cst[kColStages];
-  alignas(16) uint8_t sf_k[512];
-  alignas(16) uint8_t sf_v[512];
+  alignas(1024) uint8_t k[C::kCq][kTile * 128];
+  alignas(1024) uint8_t v[C::kHasDk ? C::kCv : 1][C::kHasDk ? kTile * 128 : 16];
+  KvRowStage<C> rst[C::kRowStages];
+  KvColStage<C> cst[C::kColStages];
+  alignas(16) uint8_t sf_k[C::kCq * 512];
+  alignas(16) uint8_t sf_v[C::kCv * 512];
   alignas(16) uint8_t sf_p[2][512];
   alignas(16) uint8_t sf_ds[2][512];
   uint64_t kv_full;
-  uint64_t row_full[kRowStages], row_empty[kRowStages];
-  uint64_t col_full[kColStages], col_empty[kColStages];
-  uint64_t lse_ready[kRowStages];
+  uint64_t row_full[C::kRowStages], row_empty[C::kRowStages];
+  uint64_t col_full[C::kColStages], col_empty[C::kColStages];
+  uint64_t lse_ready[C::kRowStages];
   uint64_t sdp_full[kTeams], sdp_free[kTeams];
   uint64_t pds_full[2], pds_free[2];
   uint64_t done;
@@ -112,12 +156,21 @@ struct KvParams {
   float scale, scale_log2;
 };
 
+template <class C>
 __global__ void __launch_bounds__(kThreads, 1)
 kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
                const __grid_constant__ CUtensorMap tm_qc, const __grid_constant__ CUtensorMap tm_dOc) {
   extern __shared__ uint8_t smem_raw[];
-  KvSmem& sm = *reinterpret_cast<KvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr bool kFp8 = C::kFp8, kHasDv = C::kHasDv, kHasDk = C::kHasDk;
+  constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRq, kRv = C::kRv;
+  constexpr int kRowStages = C::kRowStages, kColStages = C::kColStages, kRowTok = C::kRowTok;
+  constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
+  constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
+                     kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
+                     kColSFdO = C::kColSFdO, kColSFP = C::kColSFP, kColSFdS = C::kColSFdS, kColSFdOc = C::kColSFdOc,
+                     kColSFQc = C::kColSFQc, kTmemCols = C::kTmemCols;
+  KvSmem<C>& sm = *reinterpret_cast<KvSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // blocks are handed out x-fastest: KV heads vary fastest, key tiles in order, so the heaviest
   // tiles (the earliest keys under the causal mask) of all heads go first
@@ -129,17 +182,17 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   const int tiles_per_head = tiles_n - it0;
   const int n_qtiles = G * tiles_per_head;          // query tiles this CTA walks
   const int n_sub = 2 * n_qtiles;
-  const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
+  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * kEB / 32;       // 32-byte K steps of S^T and dP^T
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < kRowStages; ++s) {
-      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], 1);      // released once both softmax teams are done with the tile
+      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], 1);      // released once the softmax teams are done with the rows
       mbar_init(&sm.lse_ready[s], 1);                 // one arrival by the prep warp
     }
     for (int s = 0; s < kColStages; ++s) { mbar_init(&sm.col_full[s], 1); mbar_init(&sm.col_empty[s], 1); }
-    for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], 2); mbar_init(&sm.sdp_free[t], kTeamThreads); }
+    for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], kHasDk ? 2 : 1); mbar_init(&sm.sdp_free[t], kTeamThreads); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); }
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     mbar_init(&sm.done, 1);
@@ -155,46 +208,68 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_base;
 
-
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO);
       prefetch_tmap(&tm_qc); prefetch_tmap(&tm_dOc);
       const int kv_slab = b * p.Hkv + g;
-      mbar_arrive_expect_tx(&sm.kv_full, 2 * (kTile * 128 + 512));
-      tma_load_2d(sm.k, &tm_k, &sm.kv_full, 0, kv_slab * p.N + jt * kTile);
-      tma_load_2d(sm.v, &tm_v, &sm.kv_full, 0, kv_slab * p.N + jt * kTile);
-      bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
-      bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * 512, 512, &sm.kv_full);
+      const int n_kv_ops = kCq + (kHasDk ? kCv : 0);
+      mbar_arrive_expect_tx(&sm.kv_full, n_kv_ops * (kTile * 128 + (kFp8 ? 512 : 0)));
+      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[c], &tm_k, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
+      if (kFp8) bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCq * 512, kCq * 512, &sm.kv_full);
+      if (kHasDk) {
+        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[c], &tm_v, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
+        if (kFp8) bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCv * 512, kCv * 512, &sm.kv_full);
+      }
       int issued_row = 0, issued_col = 0;
       bool ok = true;
-      for (int n = 0; n < n_qtiles && ok; ++n) {
-        const int rs = n % kRowStages, cs = n % kColStages;
+      for (int u = 0; u < n_sub && ok; ++u) {
+        const int n = u >> 1, half = u & 1;
         const int h = g * G + n / tiles_per_head, it = it0 + n % tiles_per_head;
         const int q_slab = b * p.Hq + h;
-        const size_t sf_tile = (static_cast<size_t>(q_slab) * tiles_n + it) * 512;
-        const size_t row0 = static_cast<size_t>(q_slab) * p.N + it * kTile;
-        ok = mbar_wait(&sm.row_empty[rs], ((n / kRowStages) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        KvRowStage& r = sm.rst[rs];
-        mbar_arrive_expect_tx(&sm.row_full[rs], 2 * kTile * 128 + 2 * 512 + 2 * kTile * 4);
-        tma_load_2d(r.q, &tm_q, &sm.row_full[rs], 0, q_slab * p.N + it * kTile);
-        tma_load_2d(r.dO, &tm_dO, &sm.row_full[rs], 0, q_slab * p.N + it * kTile);
-        bulk_load_1d(r.sf_q, p.q_sf + sf_tile, 512, &sm.row_full[rs]);
-        bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile, 512, &sm.row_full[rs]);
-        bulk_load_1d(r.lse, p.lse + row0, kTile * 4, &sm.row_full[rs]);
-        bulk_load_1d(r.delta, p.delta + row0, kTile * 4, &sm.row_full[rs]);
-        ++issued_row;
-        ok = mbar_wait(&sm.col_empty[cs], ((n / kColStages) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        KvColStage& c = sm.cst[cs];
-        mbar_arrive_expect_tx(&sm.col_full[cs], (p.dqk + p.dv) * 128 + 2 * 512);
-        tma_load_2d(c.qc, &tm_qc, &sm.col_full[cs], it * kTile, q_slab * p.dqk);
-        tma_load_2d(c.dOc, &tm_dOc, &sm.col_full[cs], it * kTile, q_slab * p.dv);
-        bulk_load_1d(c.sf_qc, p.qc_sf + sf_tile, 512, &sm.col_full[cs]);
-        bulk_load_1d(c.sf_dOc, p.dOc_sf + sf_tile, 512, &sm.col_full[cs]);
-        ++issued_col;
+        const size_t sf_tile = static_cast<size_t>(q_slab) * tiles_n + it;
+        if (u % kSubPerRow == 0) {
+          const int ri = u / kSubPerRow, rs = ri % kRowStages;
+          const int tok0 = it * kTile + (kSubPerRow == 1 ? half * kSub : 0);     // first query of the stage
+          ok = mbar_wait(&sm.row_empty[rs], ((ri / kRowStages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          KvRowStage<C>& r = sm.rst[rs];
+          mbar_arrive_expect_tx(&sm.row_full[rs], n_kv_ops * (kRowTok * 128 + (kFp8 ? 512 : 0)) + (kHasDk ? 2 : 1) * kRowTok * 4);
+          for (int c = 0; c < kCq; ++c) tma_load_2d(r.q[c], &tm_q, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
+          if (kFp8) bulk_load_1d(r.sf_q, p.q_sf + sf_tile * kCq * 512, kCq * 512, &sm.row_full[rs]);
+          bulk_load_1d(r.lse, p.lse + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
+          if (kHasDk) {
+            for (int c = 0; c < kCv; ++c) tma_load_2d(r.dO[c], &tm_dO, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
+            if (kFp8) bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile * kCv * 512, kCv * 512, &sm.row_full[rs]);
+            bulk_load_1d(r.delta, p.delta + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
+          }
+          ++issued_row;
+        }
+        if (u % kSubPerCol == 0) {
+          const int ci = u / kSubPerCol, cs = ci % kColStages;
+          const int x0 = (it * kTile + (kSubPerCol == 1 ? half * kSub : 0)) * kEB;   // byte offset along the query dim
+          ok = mbar_wait(&sm.col_empty[cs], ((ci / kColStages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          KvColStage<C>& c = sm.cst[cs];
+          mbar_arrive_expect_tx(&sm.col_full[cs], (kHasDk ? p.dqk * 128 + (kFp8 ? kRq * 512 : 0) : 0) +
+                                                      (kHasDv ? p.dv * 128 + (kFp8 ? kRv * 512 : 0) : 0));
+          if (kHasDk) {
+            tma_load_2d(c.qc, &tm_qc, &sm.col_full[cs], x0, q_slab * p.dqk);
+            if (kFp8)
+              for (int r = 0; r < kRq; ++r)
+                bulk_load_1d(c.sf_qc + 512 * r, p.qc_sf + ((static_cast<size_t>(q_slab) * kRq + r) * tiles_n + it) * 512, 512,
+                             &sm.col_full[cs]);
+          }
+          if (kHasDv) {
+            tma_load_2d(c.dOc, &tm_dOc, &sm.col_full[cs], x0, q_slab * p.dv);
+            if (kFp8)
+              for (int r = 0; r < kRv; ++r)
+                bulk_load_1d(c.sf_dOc + 512 * r, p.dOc_sf + ((static_cast<size_t>(q_slab) * kRv + r) * tiles_n + it) * 512, 512,
+                             &sm.col_full[cs]);
+          }
+          ++issued_col;
+        }
       }
       if (!ok) {
         int dummy = 0;
@@ -210,20 +285,20 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // products are spread over three issuing warps; orderings that a single issuer would give
     // for free are carried by mbarriers instead.
     {
-      const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k));
+      const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[0]));
       bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-      if (ok) {
+      if (ok && kFp8) {
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFK, make_desc_sf(smem_u32(sm.sf_k)));
+        sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k);
       }
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int n = u >> 1, half = u & 1, s = n % kRowStages, slot = n & 1;
-        KvRowStage& st = sm.rst[s];
-        if (half == 0) {
-          ok = mbar_wait(&sm.row_full[s], (n / kRowStages) & 1, abort_flag);
+        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri & 1, sub_r = u % kSubPerRow;
+        KvRowStage<C>& st = sm.rst[s];
+        if (sub_r == 0) {
+          ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy_elect(tmem + kColSFQ + 4 * slot, make_desc_sf(smem_u32(st.sf_q)));
+          if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * slot, st.sf_q);
         }
         KV_TRACE(0, u, 0);
         if (u > 0) {
@@ -233,10 +308,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           tc_fence_after_sync();
         }
         KV_TRACE(0, u, 1);
-        const uint64_t desc_q = make_desc_sw128(smem_u32(st.q)) + half * (kSub * 128 / 16);
-        for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss_elect(tmem + kColS, desc_k + 2 * kb, desc_q + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
-                      tmem + kColSFK, tmem + kColSFQ + 4 * slot + 2 * half, kb > 0);
+        const uint64_t desc_q = make_desc_sw128(smem_u32(st.q[0])) + sub_r * (kSub * 128 / 16);
+        issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
+            tmem + kColS, desc_k, desc_q, nk_qk, tmem + kColSFK, tmem + kColSFQ + 4 * kCq * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
         KV_TRACE(0, u, 2);
       }
@@ -248,42 +322,43 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ dP^T issuer + LSE preparation
-    const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v));
+    const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[0]));
     bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-    if (ok) {
+    if (ok && kFp8 && kHasDk) {
       tc_fence_after_sync();
-      sf_copy_elect(tmem + kColSFV, make_desc_sf(smem_u32(sm.sf_v)));
+      sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v);
     }
     for (int u = 0; u < n_sub && ok; ++u) {
-      const int n = u >> 1, half = u & 1, s = n % kRowStages, slot = n & 1;
-      KvRowStage& st = sm.rst[s];
-      if (half == 0) {
-        ok = mbar_wait(&sm.row_full[s], (n / kRowStages) & 1, abort_flag);
+      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri & 1, sub_r = u % kSubPerRow;
+      KvRowStage<C>& st = sm.rst[s];
+      if (sub_r == 0) {
+        ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
         if (!ok) break;
         // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
-        const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
-        *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
-            make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
+        if (4 * lane < kRowTok) {
+          const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
+          *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
+              make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
+        }
         mbar_arrive_warp(&sm.lse_ready[s]);
-        {
+        if (kFp8 && kHasDk) {
           tc_fence_after_sync();
-          sf_copy_elect(tmem + kColSFdO + 4 * slot, make_desc_sf(smem_u32(st.sf_dO)));
+          sf_copy_tiles<kCv>(tmem + kColSFdO + 4 * kCv * slot, st.sf_dO);
         }
       }
-      if (u > 0) {
-        ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
-        if (!ok) break;
-      }
-      {
+      if (kHasDk) {
+        if (u > 0) {
+          ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
+          if (!ok) break;
+        }
         tc_fence_after_sync();
-        const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO)) + half * (kSub * 128 / 16);
-        for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss_elect(tmem + kColdP, desc_v + 2 * kb, desc_dO + 2 * kb, make_idesc_mxf8(128, kSub, kb, kb),
-                      tmem + kColSFV, tmem + kColSFdO + 4 * slot + 2 * half, kb > 0);
+        const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO[0])) + sub_r * (kSub * 128 / 16);
+        issue_ss<kFp8, kCv, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
+            tmem + kColdP, desc_v, desc_dO, nk_v, tmem + kColSFV, tmem + kColSFdO + 4 * kCv * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
       }
     }
-    if (!ok) {
+    if (!ok && kHasDk) {
       int dummy = 0;
       mma_commit_elect(&sm.drain[1]);
       mbar_wait(&sm.drain[1], 0, &dummy);
@@ -293,41 +368,41 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int n = u >> 1, half = u & 1, s = n % kColStages, slot = n & 1, buf = u & 1;
-        KvColStage& st = sm.cst[s];
-        if (half == 0) {
-          ok = mbar_wait(&sm.col_full[s], (n / kColStages) & 1, abort_flag);
+        const int buf = u & 1, ci = u / kSubPerCol, s = ci % kColStages, slot = ci & 1, sub_c = u % kSubPerCol;
+        KvColStage<C>& st = sm.cst[s];
+        if (sub_c == 0) {
+          ok = mbar_wait(&sm.col_full[s], (ci / kColStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          sf_copy_elect(tmem + kColSFdOc + 4 * slot, make_desc_sf(smem_u32(st.sf_dOc)));
-          sf_copy_elect(tmem + kColSFQc + 4 * slot, make_desc_sf(smem_u32(st.sf_qc)));
+          if (kFp8) {
+            if (kHasDv) sf_copy_tiles<kRv>(tmem + kColSFdOc + 4 * kRv * slot, st.sf_dOc);
+            if (kHasDk) sf_copy_tiles<kRq>(tmem + kColSFQc + 4 * kRq * slot, st.sf_qc);
+          }
         }
         KV_TRACE(1, u, 0);
         ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
         KV_TRACE(1, u, 1);
-        // both halves of the tile have been through the softmax: its row set (scores operands,
+        // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
-        if (half == 1 && lane == 0) mbar_arrive(&sm.row_empty[n % kRowStages]);
+        if (u % kSubPerRow == kSubPerRow - 1 && lane == 0) mbar_arrive(&sm.row_empty[(u / kSubPerRow) % kRowStages]);
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
-        sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
-        const uint64_t desc_dOc = make_desc_sw128(smem_u32(st.dOc));
-        const uint64_t desc_qc = make_desc_sw128(smem_u32(st.qc));
-        for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts_elect(tmem + kColdV, tmem + kColP + 16 * buf + 8 * kb, desc_dOc + 2 * (2 * half + kb),
-                      make_idesc_mxf8(128, p.dv, kb, 2 * half + kb), tmem + kColSFP + 4 * buf,
-                      tmem + kColSFdOc + 4 * slot, (u > 0 || kb > 0));
-        for (int kb = 0; kb < 2; ++kb)
-          mma_mxf8_ts_elect(tmem + kColdK, tmem + kColdS + 16 * buf + 8 * kb, desc_qc + 2 * (2 * half + kb),
-                      make_idesc_mxf8(128, p.dqk, kb, 2 * half + kb), tmem + kColSFdS + 4 * buf,
-                      tmem + kColSFQc + 4 * slot, (u > 0 || kb > 0));
-        // codes and scale bytes of this buffer may be overwritten once these MMAs have run; the
-        // stage may be refilled after the second half (the S^T / dP^T MMAs that read it finished
-        // before the softmax team could even start on this sub-tile)
+        if (kFp8) {
+          if (kHasDv) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
+          if (kHasDk) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        }
+        // 64 queries = 2 (codes) or 4 (BF16) steps of 32 bytes; the B operands are taken 128 rows at a time
+        if (kHasDv)
+          issue_ts<kFp8, kEB, kRv>(tmem + kColdV, tmem + kColP + kOpCols * buf, make_desc_sw128(smem_u32(st.dOc)), p.dv,
+                                   sub_c, tmem + kColSFP + 4 * buf, tmem + kColSFdOc + 4 * kRv * slot, u > 0);
+        if (kHasDk)
+          issue_ts<kFp8, kEB, kRq>(tmem + kColdK, tmem + kColdS + kOpCols * buf, make_desc_sw128(smem_u32(st.qc)), p.dqk,
+                                   sub_c, tmem + kColSFdS + 4 * buf, tmem + kColSFQc + 4 * kRq * slot, u > 0);
+        // operands and scale bytes of this buffer may be overwritten once these MMAs have run; the
+        // col stage may be refilled after its last sub-tile
         mma_commit_elect(&sm.pds_free[buf]);
         KV_TRACE(1, u, 2);
-        if (half == 1) mma_commit_elect(&sm.col_empty[s]);
+        if (sub_c == kSubPerCol - 1) mma_commit_elect(&sm.col_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.done);
       }
       if (!ok) {
@@ -345,7 +420,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
     bool ok = true;
     for (int u = team; u < n_sub; u += kTeams) {
-      const int n = u >> 1, half = u & 1, buf = u & 1, s = n % kRowStages;
+      const int n = u >> 1, half = u & 1, buf = u & 1, ri = u / kSubPerRow, s = ri % kRowStages;
       const int it = it0 + n % tiles_per_head;
       if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 0);
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
@@ -354,24 +429,26 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];                       // S then P; dP then dS (in place)
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
-      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
+      if (kHasDk) tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
       if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 2);
-      ok = mbar_wait(&sm.lse_ready[s], (n / kRowStages) & 1, abort_flag);
+      ok = mbar_wait(&sm.lse_ready[s], (ri / kRowStages) & 1, abort_flag);
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
-      const KvRowStage& st = sm.rst[s];
+      const int st0 = (u % kSubPerRow) * kSub + 32 * grp;   // the same inside the row stage
+      const KvRowStage<C>& st = sm.rst[s];
       float amax_p = 0.f, max_s = 0.f;
-      const float* s_lse = &st.neg_lse2[col0];
-      const float* s_delta = &st.delta[col0];
+      const float* s_lse = &st.neg_lse2[st0];
+      const float* s_delta = &st.delta[st0];
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
         for (int c4 = 0; c4 < 32; c4 += 4) {
           const float4 l4 = lds_f4(&s_lse[c4]);
-          const float4 d4 = lds_f4(&s_delta[c4]);
+          float4 d4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (kHasDk) d4 = lds_f4(&s_delta[c4]);
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
           const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
@@ -380,39 +457,63 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, lv[e]);
             if (kDiag && (row > col0 + c)) x = -INFINITY;      // key after the query
             const float pv = ex2_approx(x);
-            const float dsv = pv * (__uint_as_float(dpr[c]) - dv4[e]);
             sr[c] = __float_as_uint(pv);
-            dpr[c] = __float_as_uint(dsv);
             amax_p = fmaxf(amax_p, pv);
-            max_s = fmaxf(max_s, fabsf(dsv));
+            if (kHasDk) {
+              const float dsv = pv * (__uint_as_float(dpr[c]) - dv4[e]);
+              dpr[c] = __float_as_uint(dsv);
+              max_s = fmaxf(max_s, fabsf(dsv));
+            }
           }
         }
       };
       if (p.causal && it == jt) body(std::true_type{}); else body(std::false_type{});
-      uint32_t byte_p, byte_s;
-      float inv_p, inv_s;
-      block_scale(amax_p, byte_p, inv_p);
-      block_scale(max_s, byte_s, inv_s);
+      uint32_t byte_p = 0, byte_s = 0;
+      float inv_p = 1.f, inv_s = 1.f;
+      if (kFp8) {
+        if (kHasDv) block_scale(amax_p, byte_p, inv_p);
+        if (kHasDk) block_scale(max_s, byte_s, inv_s);
+      }
       if (u >= 2) {
-        // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's codes and scale bytes
+        // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's operands and scale bytes
         ok = mbar_wait(&sm.pds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
-      uint32_t words[8];
+      uint32_t words[8 * kEB];
+      if (kHasDv) {
+        if (kFp8) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        words[i] = cvt_e4m3x4(__uint_as_float(sr[4 * i]) * inv_p, __uint_as_float(sr[4 * i + 1]) * inv_p,
-                              __uint_as_float(sr[4 * i + 2]) * inv_p, __uint_as_float(sr[4 * i + 3]) * inv_p);
-      tmem_st8(tmem + kColP + 16 * buf + lane_addr + 8 * grp, words);
+          for (int i = 0; i < 8; ++i)
+            words[i] = cvt_e4m3x4(__uint_as_float(sr[4 * i]) * inv_p, __uint_as_float(sr[4 * i + 1]) * inv_p,
+                                  __uint_as_float(sr[4 * i + 2]) * inv_p, __uint_as_float(sr[4 * i + 3]) * inv_p);
+        } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        words[i] = cvt_e4m3x4(__uint_as_float(dpr[4 * i]) * inv_s, __uint_as_float(dpr[4 * i + 1]) * inv_s,
-                              __uint_as_float(dpr[4 * i + 2]) * inv_s, __uint_as_float(dpr[4 * i + 3]) * inv_s);
-      tmem_st8(tmem + kColdS + 16 * buf + lane_addr + 8 * grp, words);
-      const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
-      sts_u8(&sm.sf_p[buf][sf_at], byte_p);
-      sts_u8(&sm.sf_ds[buf][sf_at], byte_s);
+          for (int i = 0; i < 8 * kEB; ++i)
+            words[i] = cvt_bf16x2(__uint_as_float(sr[(2 * i) & 31]), __uint_as_float(sr[(2 * i + 1) & 31]));
+        }
+#pragma unroll
+        for (int i = 0; i < kEB; ++i) tmem_st8(tmem + kColP + kOpCols * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
+      }
+      if (kHasDk) {
+        if (kFp8) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            words[i] = cvt_e4m3x4(__uint_as_float(dpr[4 * i]) * inv_s, __uint_as_float(dpr[4 * i + 1]) * inv_s,
+                                  __uint_as_float(dpr[4 * i + 2]) * inv_s, __uint_as_float(dpr[4 * i + 3]) * inv_s);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8 * kEB; ++i)
+            words[i] = cvt_bf16x2(__uint_as_float(dpr[(2 * i) & 31]), __uint_as_float(dpr[(2 * i + 1) & 31]));
+        }
+#pragma unroll
+        for (int i = 0; i < kEB; ++i) tmem_st8(tmem + kColdS + kOpCols * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
+      }
+      if (kFp8) {
+        const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
+        if (kHasDv) sts_u8(&sm.sf_p[buf][sf_at], byte_p);
+        if (kHasDk) sts_u8(&sm.sf_ds[buf][sf_at], byte_s);
+      }
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
@@ -421,11 +522,11 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     }
     // the epilogue is done by team 0 (group 0 stores dV, group 1 stores dK)
     if (team != 0) ok = false;
+    if (grp == 0 ? !kHasDv : !kHasDk) ok = false;
     if (ok) ok = mbar_wait(&sm.done, 0, abort_flag);
     if (ok) {
       tc_fence_after_sync();
       const size_t grow = static_cast<size_t>(b * p.Hkv + g) * p.N + jt * kTile + row;
-      // group 0 stores dV, group 1 stores dK (scaled)
       const uint32_t col = grp == 0 ? kColdV : kColdK;
       const int width = grp == 0 ? p.dv : p.dqk;
       const float mul = grp == 0 ? 1.f : p.scale;
@@ -453,20 +554,21 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
 }
 
-}  // namespace
-
-attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
-                              const float* lse, const float* delta, void* dk, void* dv, int* status,
-                              cudaStream_t stream) {
+template <class C>
+attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                               const float* lse, const float* delta, void* dk, void* dv, int* status,
+                               cudaStream_t stream) {
+  static_assert(sizeof(KvSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc;
   attn_status_t st;
+  const uint64_t eb = C::kEB;
   const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
-  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, kv_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv, kv_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, q_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv, q_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, s.dqk)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_dOc, dO.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hq * s.dv, s.dv)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * eb, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, s.dqk)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dOc, dO.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dv, s.dv)) != ATTN_OK) return st;
   KvParams p;
   p.k_sf = k.row_scales; p.v_sf = v.row_scales; p.q_sf = q.row_scales; p.dO_sf = dO.row_scales;
   p.qc_sf = q.col_scales; p.dOc_sf = dO.col_scales;
@@ -474,14 +576,41 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.dk = static_cast<__nv_bfloat16*>(dk); p.dv_out = static_cast<__nv_bfloat16*>(dv); p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
-  const size_t smem = sizeof(KvSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  const size_t smem = sizeof(KvSmem<C>) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(s.Hkv, s.N / kTile, s.B);
-  kvmajor_kernel<<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
+  kvmajor_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
+}
+
+}  // namespace
+
+attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                              const float* lse, const float* delta, void* dk, void* dv, int* status,
+                              cudaStream_t stream) {
+  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.eb + 127) / 128;
+  if (s.eb == 1 && cq == 1 && cv == 1)
+    return launch_kvmajor_t<KvCfg<1, 1, 1, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  if (s.eb == 2 && cq == 1 && cv == 1)
+    return launch_kvmajor_t<KvCfg<2, 1, 1, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  if (s.eb == 2 && cq == 2 && cv == 2)
+    return launch_kvmajor_t<KvCfg<2, 2, 2, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  // qk head dim above 128: dV and dK do not fit in tensor memory together; one pass each
+  if (s.eb == 1 && cq == 2 && cv == 1) {
+    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 1, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (st != ATTN_OK) return st;
+    return launch_kvmajor_t<KvCfg<1, 2, 1, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  }
+  if (s.eb == 1 && cq == 2 && cv == 2) {
+    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (st != ATTN_OK) return st;
+    return launch_kvmajor_t<KvCfg<1, 2, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  }
+  return fail(ATTN_ERR_UNSUPPORTED, "bwd kv-major: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv,
+              s.eb);
 }
 
 }  // namespace attnfp8

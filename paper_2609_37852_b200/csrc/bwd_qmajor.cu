@@ -19,11 +19,18 @@
 // spread over three warps); warps 4..19 softmax: warp % 4 selects the 32 TMEM lanes (query rows),
 // (warp - 4) / 4 the 32-key column group.  The softmax threads pull S and dP into registers and
 // release the buffers at once, so the next tile's MMAs overlap the exponentials of this one.
+//
+// The kernel is a template over the operand width: element bytes (1: E4M3 codes with E8M0 block
+// scales, 2: BF16 without scales) and the number of 128-byte chunks per operand row.  A key step
+// always spans one 128-byte chunk of the token dimension (128 keys of codes, 64 keys of BF16).
+// When the qk head dim exceeds 128 the dQ accumulator no longer fits beside S and dP in tensor
+// memory; the dQ columns are then split in tiles of 128 over CTAs that each repeat the S / dP work.
 #include <cuda_bf16.h>
 
 #include <type_traits>
 
 #include "common.cuh"
+#include "mma_issue.cuh"
 #include "mxfp8_device.cuh"
 #include "sm100_ptx.cuh"
 
@@ -45,38 +52,62 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
-// K/V ring depth: deep enough to cover the L2 -> shared-memory latency of a tile (what fits)
-template <bool kDQ> constexpr int kStagesFor = kDQ ? 3 : 4;
-constexpr int kGroups = 4;                      // 32-key column groups of a tile
-constexpr int kSoftmaxThreads = 128 * kGroups;  // 16 warps: 4 TMEM lane quadrants x 4 column groups
-constexpr int kThreads = 128 + kSoftmaxThreads;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLog2eLo = 1.92596299e-8f;          // log2(e) minus its FP32 rounding
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kSmemLimit = 232448;                  // dynamic shared memory a CTA may ask for
 
-constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* 2 x 32 */, kColdQ = 320;
-constexpr uint32_t kColSFQ = 448, kColSFdO = 452, kColSFK = 456 /* 2 x 4 */, kColSFV = 464 /* 2 x 4 */,
-                   kColSFdS = 472 /* 2 x 4 */, kColSFKc = 480 /* 2 x 4 */;
-constexpr uint32_t kTmemCols = 512;
+// Operand geometry, ring depths and tensor-memory map of one instantiation.
+template <bool kDQ_, int kEB_, int kCq_, int kCv_>
+struct QmCfg {
+  static constexpr bool kDQ = kDQ_;
+  static constexpr int kEB = kEB_;                      // bytes per operand element
+  static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row
+  static constexpr int kCv = kCv_;                      // 128-byte chunks per dO / V row
+  static constexpr bool kFp8 = kEB == 1;
+  static constexpr int kStep = kTile / kEB;             // keys per step
+  static constexpr int kGroups = kStep / 32;            // 32-key column groups of a step
+  static constexpr int kSoftmaxThreads = 128 * kGroups; // 4 TMEM lane quadrants x column groups
+  static constexpr int kThreads = 128 + kSoftmaxThreads;
+  // K/V ring depth: deep enough to cover the L2 -> shared-memory latency of a tile (what fits);
+  // the K^T ring of the dQ product falls back to one stage when two do not fit
+  static constexpr int kFixedBytes = (kCq + kCv) * kTile * 128;
+  static constexpr int kKvBytes = (kCq + kCv) * kStep * 128;
+  static constexpr int kKcBytes = kDQ ? kTile * 128 : 0;
+  static constexpr int kRaw = (224 * 1024 - kFixedBytes - kKcBytes) / (kKvBytes + kKcBytes);
+  static constexpr int kStages = kRaw < 2 ? 2 : (kRaw > 4 ? 4 : kRaw);
+  static constexpr int kKcStages = !kDQ ? 1 : (kRaw < 2 ? 1 : kStages);
+  // tensor memory
+  static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* 2 x 32 */, kColdQ = 2 * kStep + 64;
+  static constexpr uint32_t kColSFQ = kColdQ + 128;
+  static constexpr uint32_t kColSFdO = kColSFQ + 4 * kCq;
+  static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv;    // 2 slots
+  static constexpr uint32_t kColSFV = kColSFK + 8 * kCq;     // 2 slots
+  static constexpr uint32_t kColSFdS = kColSFV + 8 * kCv;    // 2 x 4
+  static constexpr uint32_t kColSFKc = kColSFdS + 8;         // 2 x 4
+  static constexpr uint32_t kColsUsed = kFp8 ? kColSFKc + 8 : kColSFQ;
+  static constexpr uint32_t kTmemCols = 512;
+  static_assert(kColsUsed <= 512, "tensor memory exceeded");
+};
 
-template <bool kDQ>
+template <class C>
 struct QmSmem {
-  static constexpr int kStages = kStagesFor<kDQ>;
-  alignas(1024) uint8_t q[kTile * 128];
-  alignas(1024) uint8_t dO[kTile * 128];
-  alignas(1024) uint8_t k[kStages][kTile * 128];
-  alignas(1024) uint8_t v[kStages][kTile * 128];
-  alignas(1024) uint8_t kc[kDQ ? kStages : 1][kTile * 128];
-  alignas(16) uint8_t sf_q[512];
-  alignas(16) uint8_t sf_dO[512];
-  alignas(16) uint8_t sf_k[kStages][512];
-  alignas(16) uint8_t sf_v[kStages][512];
-  alignas(16) uint8_t sf_kc[kStages][512];
+  static constexpr int kStages = C::kStages;
+  alignas(1024) uint8_t q[C::kCq][kTile * 128];
+  alignas(1024) uint8_t dO[C::kCv][kTile * 128];
+  alignas(1024) uint8_t k[kStages][C::kCq][C::kStep * 128];
+  alignas(1024) uint8_t v[kStages][C::kCv][C::kStep * 128];
+  alignas(1024) uint8_t kc[C::kKcStages][kTile * 128];
+  alignas(16) uint8_t sf_q[C::kCq * 512];
+  alignas(16) uint8_t sf_dO[C::kCv * 512];
+  alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
+  alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
+  alignas(16) uint8_t sf_kc[C::kKcStages][512];
   alignas(16) uint8_t sf_ds[2][512];
-  alignas(16) float red[kGroups][2][kTile];      // partial row sums of every column group
+  alignas(16) float red[C::kGroups][2][kTile];   // partial row sums of every column group
   uint64_t q_full;
   uint64_t kv_full[kStages], kv_empty[kStages];
-  uint64_t kc_full[kStages], kc_empty[kStages];
+  uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
   uint64_t sdp_full, sdp_free;
   uint64_t ds_full[2], ds_free[2];
   uint64_t dq_done;
@@ -98,30 +129,38 @@ struct QmParams {
   float scale, scale_log2;
 };
 
-template <bool kDQ>
-__global__ void __launch_bounds__(kThreads, 1)
+template <class C>
+__global__ void __launch_bounds__(C::kThreads, 1)
 qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
               const __grid_constant__ CUtensorMap tm_kc) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int kStages = kStagesFor<kDQ>;
-  QmSmem<kDQ>& sm = *reinterpret_cast<QmSmem<kDQ>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8;
+  constexpr int kStages = C::kStages, kKcStages = C::kKcStages, kEB = C::kEB, kCq = C::kCq, kCv = C::kCv;
+  constexpr int kStep = C::kStep, kGroups = C::kGroups, kSoftmaxThreads = C::kSoftmaxThreads;
+  constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColdS = C::kColdS, kColdQ = C::kColdQ, kColSFQ = C::kColSFQ,
+                     kColSFdO = C::kColSFdO, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFdS = C::kColSFdS,
+                     kColSFKc = C::kColSFKc, kTmemCols = C::kTmemCols;
+  QmSmem<C>& sm = *reinterpret_cast<QmSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
   // all heads go first, so the light tiles fill the tail of the launch
   const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
-  const int h = blockIdx.x, b = blockIdx.z;
+  // dQ column tiles (128 wide) of one head sit next to each other in the grid
+  const int rq = kDQ ? (p.dqk + 127) / 128 : 1;
+  const int h = blockIdx.x / rq, r_tile = blockIdx.x % rq, b = blockIdx.z;
+  const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
   const int g = h / (p.Hq / p.Hkv);
-  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
-  const int nk_qk = p.dqk / 32, nk_v = p.dv / 32;
+  const int n_tiles = (p.causal ? qt + 1 : p.N / kTile) * kEB;      // key steps
+  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * kEB / 32;       // 32-byte K steps of the two products
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 2);   // released by the S and the dP issuer
-      mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1);
     }
+    for (int s = 0; s < kKcStages; ++s) { mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1); }
     mbar_init(&sm.sdp_full, 2); mbar_init(&sm.sdp_free, kSoftmaxThreads);
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kSoftmaxThreads); mbar_init(&sm.ds_free[i], 1); }
     mbar_init(&sm.dq_done, 1);
@@ -145,11 +184,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       if (kDQ) prefetch_tmap(&tm_kc);
       const int q_slab = b * p.Hq + h, kv_slab = b * p.Hkv + g;
       const int tiles_n = p.N / kTile;
-      mbar_arrive_expect_tx(&sm.q_full, 2 * (kTile * 128 + 512));
-      tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_slab * p.N + qt * kTile);
-      tma_load_2d(sm.dO, &tm_dO, &sm.q_full, 0, q_slab * p.N + qt * kTile);
-      bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * 512, 512, &sm.q_full);
-      bulk_load_1d(sm.sf_dO, p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * 512, 512, &sm.q_full);
+      mbar_arrive_expect_tx(&sm.q_full, (kCq + kCv) * (kTile * 128 + (kFp8 ? 512 : 0)));
+      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[c], &tm_q, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
+      for (int c = 0; c < kCv; ++c) tma_load_2d(sm.dO[c], &tm_dO, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
+      if (kFp8) {
+        bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCq * 512, kCq * 512, &sm.q_full);
+        bulk_load_1d(sm.sf_dO, p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCv * 512, kCv * 512, &sm.q_full);
+      }
       int issued_kv = 0, issued_kc = 0;
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
@@ -157,18 +198,23 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
         QM_TRACE(0, t, 0);
-        mbar_arrive_expect_tx(&sm.kv_full[s], 2 * (kTile * 128 + 512));
-        tma_load_2d(sm.k[s], &tm_k, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
-        tma_load_2d(sm.v[s], &tm_v, &sm.kv_full[s], 0, kv_slab * p.N + t * kTile);
-        bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kv_full[s]);
-        bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kv_full[s]);
+        mbar_arrive_expect_tx(&sm.kv_full[s], (kCq + kCv) * (kStep * 128 + (kFp8 ? 512 : 0)));
+        for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
+        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
+        if (kFp8) {
+          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
+          bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
+        }
         ++issued_kv;
         if (kDQ) {
-          ok = mbar_wait(&sm.kc_empty[s], (u & 1) ^ 1, abort_flag);
+          const int sc = t % kKcStages;
+          ok = mbar_wait(&sm.kc_empty[sc], ((t / kKcStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(&sm.kc_full[s], p.dqk * 128 + 512);
-          tma_load_2d(sm.kc[s], &tm_kc, &sm.kc_full[s], t * kTile, kv_slab * p.dqk);
-          bulk_load_1d(sm.sf_kc[s], p.kc_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.kc_full[s]);
+          mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
+          tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * r_tile);
+          if (kFp8)
+            bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + r_tile) * tiles_n + t) * 512, 512,
+                         &sm.kc_full[sc]);
           ++issued_kc;
         }
       }
@@ -176,18 +222,18 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         int dummy = 0;
         for (int t = max(0, issued_kv - kStages); t < issued_kv; ++t)
           mbar_wait(&sm.kv_full[t % kStages], (t / kStages) & 1, &dummy);
-        for (int t = max(0, issued_kc - kStages); t < issued_kc; ++t)
-          mbar_wait(&sm.kc_full[t % kStages], (t / kStages) & 1, &dummy);
+        for (int t = max(0, issued_kc - kKcStages); t < issued_kc; ++t)
+          mbar_wait(&sm.kc_full[t % kKcStages], (t / kKcStages) & 1, &dummy);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S issuer
     {
-      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
+      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[0]));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok) {
+      if (ok && kFp8) {
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFQ, make_desc_sf(smem_u32(sm.sf_q)));
+        sf_copy_tiles<kCq>(tmem + kColSFQ, sm.sf_q);
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kStages, slot = t & 1;
@@ -195,7 +241,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (!ok) break;
         QM_TRACE(1, t, 0);
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFK + 4 * slot, make_desc_sf(smem_u32(sm.sf_k[s])));
+        if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
         QM_TRACE(1, t, 1);
         if (t > 0) {
           // the softmax threads have pulled the previous S and dP into registers
@@ -204,10 +250,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           tc_fence_after_sync();
         }
         QM_TRACE(1, t, 2);
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s]));
-        for (int kb = 0; kb < nk_qk; ++kb)
-          mma_mxf8_ss_elect(tmem + kColS, desc_q + 2 * kb, desc_k + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
-                      tmem + kColSFQ, tmem + kColSFK + 4 * slot, kb > 0);
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
+        issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, tmem + kColSFQ,
+                                                                        tmem + kColSFK + 4 * kCq * slot);
         mma_commit_elect(&sm.sdp_full);
         mma_commit_elect(&sm.kv_empty[s]);
         QM_TRACE(1, t, 3);
@@ -221,27 +266,26 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   } else if (warp == 2) {
     // ------------------------------------------------------------------ dP issuer
     {
-      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO));
+      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO[0]));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok) {
+      if (ok && kFp8) {
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFdO, make_desc_sf(smem_u32(sm.sf_dO)));
+        sf_copy_tiles<kCv>(tmem + kColSFdO, sm.sf_dO);
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kStages, slot = t & 1;
         ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFV + 4 * slot, make_desc_sf(smem_u32(sm.sf_v[s])));
+        if (kFp8) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
         if (t > 0) {
           ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
-        for (int kb = 0; kb < nk_v; ++kb)
-          mma_mxf8_ss_elect(tmem + kColdP, desc_dO + 2 * kb, desc_v + 2 * kb, make_idesc_mxf8(128, kTile, kb, kb),
-                      tmem + kColSFdO, tmem + kColSFV + 4 * slot, kb > 0);
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
+        issue_ss<kFp8, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, tmem + kColSFdO,
+                                                                        tmem + kColSFV + 4 * kCv * slot);
         mma_commit_elect(&sm.sdp_full);
         mma_commit_elect(&sm.kv_empty[s]);
       }
@@ -256,21 +300,27 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     if (kDQ) {
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % kStages, slot = t & 1, buf = t & 1;
-        ok = mbar_wait(&sm.kc_full[s], (t / kStages) & 1, abort_flag);
+        const int s = t % kKcStages, slot = t & 1, buf = t & 1;
+        ok = mbar_wait(&sm.kc_full[s], (t / kKcStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+        if (kFp8) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
         ok = mbar_wait(&sm.ds_full[buf], (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+        if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
-        for (int kb = 0; kb < 4; ++kb)
-          mma_mxf8_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
-                      make_idesc_mxf8(128, p.dqk, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
-                      (t > 0 || kb > 0));
-        mma_commit_elect(&sm.ds_free[buf]);            // codes and scale bytes of this buffer may be overwritten
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          if (kFp8)
+            mma_mxf8_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+                              make_idesc_mxf8(128, n_dq, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
+                              (t > 0 || kb > 0));
+          else
+            mma_bf16_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+                              make_idesc_bf16(128, n_dq), (t > 0 || kb > 0));
+        }
+        mma_commit_elect(&sm.ds_free[buf]);            // operand and scale bytes of this buffer may be overwritten
         mma_commit_elect(&sm.kc_empty[s]);
         if (t == n_tiles - 1) mma_commit_elect(&sm.dq_done);
       }
@@ -311,7 +361,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free);
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 2);
-      const int col0 = 32 * grp;                      // column of this thread's first element inside the key tile
+      // column, inside the query tile's own key range, of this thread's first element (negative
+      // before the diagonal tile)
+      const int col0 = t * kStep - qt * kTile + 32 * grp;
       float ds[32];
       float part = 0.f;
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
@@ -335,20 +387,27 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           }
         }
       };
-      if (p.causal && t == qt) body(std::true_type{}); else body(std::false_type{});
+      if (p.causal && t * kStep >= qt * kTile) body(std::true_type{}); else body(std::false_type{});
       if (!kDQ) {
         acc0 = fmaf(part, f_lo, acc0);
       } else {
-        uint32_t words[8];
-        const uint32_t byte = quantize_block32(ds, words);
+        uint32_t words[8 * kEB];
+        uint32_t byte = 0;
+        if (kFp8) {
+          byte = quantize_block32(ds, words);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8 * kEB; ++i) words[i] = cvt_bf16x2(ds[(2 * i) & 31], ds[(2 * i + 1) & 31]);
+        }
         if (t >= 2) {
-          // the dQ MMAs of tile t-2 have consumed this buffer's codes and scale bytes
+          // the dQ MMAs of tile t-2 have consumed this buffer's operand and scale bytes
           ok = mbar_wait(&sm.ds_free[buf], ((t - 2) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        tmem_st8(tmem + kColdS + 32 * buf + lane_addr + 8 * grp, words);
-        sts_u8(&sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
+#pragma unroll
+        for (int i = 0; i < kEB; ++i) tmem_st8(tmem + kColdS + 32 * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
+        if (kFp8) sts_u8(&sm.sf_ds[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
         tmem_wait_st();
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -364,7 +423,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       for (int i = 0; i < kGroups; ++i) { acc0 += sm.red[i][0][row]; acc1 += sm.red[i][1][row]; }
       if (!kDQ) {
         p.delta_out[grow] = acc0;
-      } else if (p.rowsum) {
+      } else if (p.rowsum && r_tile == 0) {
         p.rowsum[grow] = acc0;
         p.rowabs[grow] = acc1;
       }
@@ -373,8 +432,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       ok = mbar_wait(&sm.dq_done, 0, abort_flag);
       if (ok) {
         tc_fence_after_sync();
-        __nv_bfloat16* out_row = p.dq + grow * p.dqk;
-        for (int c0 = grp * 32; c0 < p.dqk; c0 += 32 * kGroups) {
+        __nv_bfloat16* out_row = p.dq + grow * p.dqk + 128 * r_tile;
+        for (int c0 = grp * 32; c0 < n_dq; c0 += 32 * kGroups) {
           uint32_t r[32];
           tmem_ld32(tmem + kColdQ + lane_addr + c0, r);
           tmem_wait_ld();
@@ -398,19 +457,23 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
 }
 
-template <bool kDQ>
-attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
-                            const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
-                            float* rowabs, int* status, cudaStream_t stream) {
+template <class C>
+attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                              const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
+                              float* rowabs, int* status, cudaStream_t stream) {
+  constexpr bool kDQ = C::kDQ;
+  static_assert(sizeof(QmSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
   attn_status_t st;
+  const uint64_t eb = C::kEB;
   const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
-  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk, q_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv, q_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk, kv_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * eb, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, C::kStep)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * eb, kv_rows, C::kStep)) != ATTN_OK) return st;
   if (kDQ) {
-    if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.N, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk, s.dqk)) != ATTN_OK)
+    if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
+                                   s.dqk < 128 ? s.dqk : 128)) != ATTN_OK)
       return st;
   } else {
     tm_kc = tm_k;
@@ -422,14 +485,34 @@ attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t
   p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
-  const size_t smem = sizeof(QmSmem<kDQ>) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<kDQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  const size_t smem = sizeof(QmSmem<C>) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.Hq, s.N / kTile, s.B);
-  qmajor_kernel<kDQ><<<grid, kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
+  const int rq = kDQ ? (s.dqk + 127) / 128 : 1;
+  dim3 grid(s.Hq * rq, s.N / kTile, s.B);
+  qmajor_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
+}
+
+template <bool kDQ>
+attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
+                            const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
+                            float* rowabs, int* status, cudaStream_t stream) {
+  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.eb + 127) / 128;
+#define ATTN_QM_CASE(EB, CQ, CV)                                                                              \
+  if (s.eb == EB && cq == CQ && cv == CV)                                                                     \
+    return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
+                                                  status, stream);
+  ATTN_QM_CASE(1, 1, 1)
+  ATTN_QM_CASE(1, 2, 1)
+  ATTN_QM_CASE(1, 2, 2)
+  ATTN_QM_CASE(2, 1, 1)
+  ATTN_QM_CASE(2, 2, 2)
+#undef ATTN_QM_CASE
+  return fail(ATTN_ERR_UNSUPPORTED, "bwd q-major: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv,
+              s.eb);
 }
 
 // Stale delta: D_i = sum_c dO_ic O_ic from the BF16 tensors (paper Section 3.2).  One warp per row.

@@ -29,6 +29,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "mma_issue.cuh"
 #include "mxfp8_device.cuh"
 #include "sm100_ptx.cuh"
 
@@ -125,7 +126,6 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   const int n_sub = 2 * n_tiles;
   const int n_stage_tiles = n_tiles * kEB;      // K / V stages to stream
   const int nk_qk = p.dqk * kEB / 32;           // 32-byte K steps of the score MMA
-  const int rv = (p.dv + 127) / 128;            // 128-row tiles of V^T actually present
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
@@ -176,11 +176,11 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         ++issued_k;
         ok = mbar_wait(&sm.v_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + (kFp8 ? rv * 512 : 0));
+        mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + (kFp8 ? kRv * 512 : 0));
         tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
         if (kFp8)
-          for (int r = 0; r < rv; ++r)
-            bulk_load_1d(sm.sf_v[s] + 512 * r, p.v_sf + ((static_cast<size_t>(kv_slab) * rv + r) * tiles_n + t) * 512, 512,
+          for (int r = 0; r < kRv; ++r)
+            bulk_load_1d(sm.sf_v[s] + 512 * r, p.v_sf + ((static_cast<size_t>(kv_slab) * kRv + r) * tiles_n + t) * 512, 512,
                          &sm.v_full[s]);
         ++issued_v;
       }
@@ -200,7 +200,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
       if (ok && kFp8) {
         tc_fence_after_sync();
-        for (int c = 0; c < kCq; ++c) sf_copy_elect(tmem + kColSFQ + 4 * c, make_desc_sf(smem_u32(sm.sf_q + 512 * c)));
+        sf_copy_tiles<kCq>(tmem + kColSFQ, sm.sf_q);
       }
       for (int u = 0; u < n_sub && ok; ++u) {
         const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1;
@@ -208,9 +208,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8)
-            for (int c = 0; c < kCq; ++c)
-              sf_copy_elect(tmem + kColSFK + 4 * kCq * slot + 4 * c, make_desc_sf(smem_u32(sm.sf_k[s] + 512 * c)));
+          if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
         }
         if (u > 0) {
           // the softmax threads have pulled the previous scores into registers
@@ -219,16 +217,8 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tc_fence_after_sync();
         }
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0])) + sub * (kSub * 128 / 16);
-        for (int kb = 0; kb < nk_qk; ++kb) {
-          const int c = kb >> 2, w = kb & 3;          // chunk and 32-byte step inside it
-          const uint64_t a = desc_q + c * (kTile * 128 / 16) + 2 * w;
-          const uint64_t bdesc = desc_k + c * (C::kTileKeys * 128 / 16) + 2 * w;
-          if (kFp8)
-            mma_mxf8_ss_elect(tmem + kColS, a, bdesc, make_idesc_mxf8(128, kSub, w, w), tmem + kColSFQ + 4 * c,
-                              tmem + kColSFK + 4 * kCq * slot + 4 * c + 2 * sub, kb > 0);
-          else
-            mma_bf16_ss_elect(tmem + kColS, a, bdesc, make_idesc_bf16(128, kSub), kb > 0);
-        }
+        issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, C::kTileKeys * 128 / 16>(
+            tmem + kColS, desc_q, desc_k, nk_qk, tmem + kColSFQ, tmem + kColSFK + 4 * kCq * slot + 2 * sub);
         mma_commit_elect(&sm.s_full);
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
       }
@@ -248,30 +238,15 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8)
-            for (int r = 0; r < rv; ++r)
-              sf_copy_elect(tmem + kColSFV + 4 * kRv * slot + 4 * r, make_desc_sf(smem_u32(sm.sf_v[s] + 512 * r)));
+          if (kFp8) sf_copy_tiles<kRv>(tmem + kColSFV + 4 * kRv * slot, sm.sf_v[s]);
         }
         ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
         if (kFp8) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
         // 64 keys = 2 (codes) or 4 (BF16) steps of 32 bytes; the V^T operand is taken 128 rows at a time
-        for (int r = 0; r < rv; ++r) {
-          const int n = min(128, p.dv - 128 * r);
-          for (int kb = 0; kb < 2 * kEB; ++kb) {
-            const int koff = 2 * sub + kb;            // 32-byte step inside the stage's chunk
-            const uint64_t bdesc = desc_v + r * (kTile * 128 / 16) + 2 * koff;
-            if (kFp8)
-              mma_mxf8_ts_elect(tmem + kColO + 128 * r, tmem + kColP + kPCols * buf + 8 * kb, bdesc,
-                                make_idesc_mxf8(128, n, kb, koff), tmem + kColSFP + 4 * buf,
-                                tmem + kColSFV + 4 * kRv * slot + 4 * r, (u > 0 || kb > 0));
-            else
-              mma_bf16_ts_elect(tmem + kColO + 128 * r, tmem + kColP + kPCols * buf + 8 * kb, bdesc,
-                                make_idesc_bf16(128, n), (u > 0 || kb > 0));
-          }
-        }
+        issue_ts<kFp8, kEB, kRv>(tmem + kColO, tmem + kColP + kPCols * buf, make_desc_sw128(smem_u32(sm.v[s])), p.dv, sub,
+                                 tmem + kColSFP + 4 * buf, tmem + kColSFV + 4 * kRv * slot, u > 0);
         mma_commit_elect(&sm.p_free[buf]);              // operand (and scale bytes) of this buffer consumed; O updated
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.o_done);

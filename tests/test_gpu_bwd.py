@@ -13,11 +13,13 @@ TOL_GRAD = 5e-3     # relative Frobenius error on dQ, dK, dV
 TOL_DELTA = 1e-4    # relative Frobenius error on the row correction (FP32 sums of identical operands)
 
 
-def run_all(w, q, k, v, dO, delta_mode=0, diagnostics=True):
+def run_all(w, q, k, v, dO, delta_mode=0, diagnostics=True, bf16=False):
     from paper_2609_37852_b200 import binding
     params = binding.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
-                                w.softmax_scale, delta_mode=delta_mode)
-    qq, kq, vq, dOq = (binding.attn_fp8_quantize(x.cuda()) for x in (q, k, v, dO))
+                                w.softmax_scale, delta_mode=delta_mode,
+                                precision=binding.ATTN_PREC_BF16 if bf16 else binding.ATTN_PREC_MXFP8)
+    prep = binding.attn_fp8_prepare_bf16 if bf16 else binding.attn_fp8_quantize
+    qq, kq, vq, dOq = (prep(x.cuda()) for x in (q, k, v, dO))
     o, lse, ws = binding.attn_fp8_fwd(params, qq, kq, vq)
     binding.attn_fp8_read_status(ws)
     dO_bf = dO.cuda().to(torch.bfloat16)
@@ -81,6 +83,51 @@ def test_matched_backward_matches_oracle(name, kw):
     assert np.median(r_pre) <= 1e-5
     if w.recipe in ("iid", "qknorm"):
         assert np.mean(r_pre <= 1e-5) > 0.999
+
+
+def _check_backward(w, q, k, v, dO, got, prec):
+    qn, kn, vn, dOn = (to_np(x) for x in (q, k, v, dO))
+    lse = to_np(got["lse"])
+    D_or = A.emu_delta(qn, kn, vn, dOn, lse, w.softmax_scale, w.causal, prec=prec)
+    assert rel_fro(to_np(got["delta"]), D_or) <= TOL_DELTA
+    delta = to_np(got["delta"])
+    dQ, dK, dV, rs, ra = A.emu_backward(qn, kn, vn, dOn, lse, delta, w.softmax_scale, w.causal, prec=prec)
+    assert rel_fro(to_np(got["dq"]), dQ) <= TOL_GRAD
+    assert rel_fro(to_np(got["dk"]), dK) <= TOL_GRAD
+    assert rel_fro(to_np(got["dv"]), dV) <= TOL_GRAD
+    assert rel_fro(to_np(got["ra"]), ra) <= 1e-3
+    g_rs, g_ra = to_np(got["rs"]), to_np(got["ra"])
+    live = g_ra[..., 64:] > 0
+    r_pre = np.abs(g_rs[..., 64:][live]) / g_ra[..., 64:][live]
+    print(f"\n[{w.name} {prec}] r_pre median {np.median(r_pre):.3e} max {r_pre.max():.3e}")
+    assert np.median(r_pre) <= 1e-5
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=640)),                  # qk 192 / v 128
+    ("gqa8k_d256", dict(heads_q=4, heads_kv=2, seqlen=640)),             # 256 / 256
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=384, causal=False)),
+])
+def test_backward_wide_heads_matches_oracle(name, kw):
+    """Head dims above 128: dQ columns split over CTAs, dV and dK in separate key-major passes."""
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    q, k, v, dO = workloads.make_inputs(w)
+    got = run_all(w, q, k, v, dO)
+    _check_backward(w, q, k, v, dO, got, "mxfp8")
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", {}),
+    ("tiny", dict(causal=True, seqlen=384)),
+    ("gqa4k", dict(batch=2, heads_q=4, heads_kv=2, seqlen=640)),
+    ("gqa8k_outlier", dict(heads_q=4, heads_kv=1, seqlen=768)),
+])
+def test_backward_bf16_mode_matches_oracle(name, kw):
+    """BF16 mode against the oracle's BF16-operand path."""
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    q, k, v, dO = workloads.make_inputs(w)
+    got = run_all(w, q, k, v, dO, bf16=True)
+    _check_backward(w, q, k, v, dO, got, "bf16")
 
 
 def test_stale_mode_changes_only_delta_dq_dk():
