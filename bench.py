@@ -37,8 +37,9 @@ FP8_OVER_BF16 = 2.0                 # nominal dense FP8 : BF16 tensor ratio on B
 # the ncu captures summarised under profiles/; None where no capture has been taken.
 NCU_TRAFFIC_BYTES = {"quantize": 92.1e6, "fwd": 70.3e6, "bwd_delta": 90.6e6, "bwd_dq": 128.5e6, "bwd_dkdv": 320.9e6}
 
-# executed matmul products per kernel (each 2*d FLOPs per unmasked (i, j) pair and query head)
-PRODUCTS = {"fwd": 2, "bwd_delta": 2, "bwd_dq": 3, "bwd_dkdv": 4}
+# executed matmul products per kernel as (contractions or outputs of width dqk, of width dv): each is
+# 2*width FLOPs per unmasked (i, j) pair and query head
+PRODUCTS = {"fwd": (1, 1), "bwd_delta": (1, 1), "bwd_dq": (2, 1), "bwd_dkdv": (2, 2)}
 
 
 def _measured_peaks():
@@ -104,7 +105,7 @@ class ClockSampler:
         return out
 
 
-def oracle_step(w, sample_tokens, q, k, v, dO):
+def oracle_step(w, sample_tokens, q, k, v, dO, prec="mxfp8"):
     """One pass of the oracle (forward, matched correction, gradient pass) on the causal prefix of
     ``sample_tokens`` tokens of one KV group.  Returns credited FLOPs."""
     import numpy as np
@@ -112,9 +113,9 @@ def oracle_step(w, sample_tokens, q, k, v, dO):
     G = w.heads_q // w.heads_kv
     qs, ks, vs, dOs = (x[:1, :hh, :sample_tokens].float().numpy().astype(np.float64)
                        for x, hh in ((q, G), (k, 1), (v, 1), (dO, G)))
-    O, LSE = A.emu_forward(qs, ks, vs, w.softmax_scale, w.causal)
-    D = A.emu_delta(qs, ks, vs, dOs, LSE, w.softmax_scale, w.causal)
-    A.emu_backward(qs, ks, vs, dOs, LSE, D, w.softmax_scale, w.causal)
+    O, LSE = A.emu_forward(qs, ks, vs, w.softmax_scale, w.causal, prec=prec)
+    D = A.emu_delta(qs, ks, vs, dOs, LSE, w.softmax_scale, w.causal, prec=prec)
+    A.emu_backward(qs, ks, vs, dOs, LSE, D, w.softmax_scale, w.causal, prec=prec)
     sub = w.scaled(batch=1, heads_q=G, heads_kv=1, seqlen=sample_tokens)
     return sum(sub.credited_flops())
 
@@ -138,11 +139,11 @@ def run_reference(args, w):
     small = w.scaled(heads_q=w.heads_q // w.heads_kv, heads_kv=1, seqlen=sample_tokens)
     q, k, v, dO = workloads.make_inputs(small)
     for _ in range(args.warmup):
-        oracle_step(w, sample_tokens, q, k, v, dO)
+        oracle_step(w, sample_tokens, q, k, v, dO, args.precision)
     t0 = time.perf_counter()
     flops = 0
     for _ in range(args.steps):
-        flops += oracle_step(w, sample_tokens, q, k, v, dO)
+        flops += oracle_step(w, sample_tokens, q, k, v, dO, args.precision)
     dt = time.perf_counter() - t0
     value = flops / dt / 1e12
     sample = (f"causal prefix of {sample_tokens} tokens of one KV group ({small.heads_q} query heads) of {w.name}, "
@@ -166,6 +167,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD)
+    ap.add_argument("--precision", default="mxfp8", choices=["mxfp8", "bf16"],
+                    help="bf16: the same kernels with BF16 operands and no block scales (reference point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -198,15 +201,18 @@ def main():
         torch.cuda.synchronize()
 
     warmup = max(args.warmup, 3)
+    bf16_mode = args.precision == "bf16"
     params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
-                          w.softmax_scale)
+                          w.softmax_scale, precision=B.ATTN_PREC_BF16 if bf16_mode else B.ATTN_PREC_MXFP8)
+    # operand preparation: block-scaling quantiser, or (BF16 mode) the transposed BF16 copies
+    prepare = B.attn_fp8_prepare_bf16 if bf16_mode else B.attn_fp8_quantize
     host = [x.pin_memory() for x in workloads.make_inputs(w)]
     q, k, v, dO = (x.to(dev, non_blocking=True) for x in host)
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
 
     # pre-allocated operands, outputs and workspaces (device memory is PyTorch's job; the path is the library's)
-    qq, kq, vq, dOq = (B.attn_fp8_quantize(x) for x in (q, k, v, dO))
+    qq, kq, vq, dOq = (prepare(x) for x in (q, k, v, dO))
     bf = dict(dtype=torch.bfloat16, device=dev)
     o = torch.empty((w.batch, w.heads_q, w.seqlen, w.head_dim_v), **bf)
     lse = torch.empty((w.batch, w.heads_q, w.seqlen), dtype=torch.float32, device=dev)
@@ -223,8 +229,8 @@ def main():
             if events is not None:
                 events[i].record(stream)
         mark(0)
-        B.attn_fp8_quantize(q, out=qq); B.attn_fp8_quantize(k, out=kq)
-        B.attn_fp8_quantize(v, out=vq); B.attn_fp8_quantize(dO, out=dOq)
+        prepare(q, out=qq); prepare(k, out=kq)
+        prepare(v, out=vq); prepare(dO, out=dOq)
         mark(1)
         B.attn_fp8_fwd(params, qq, kq, vq, o=o, lse=lse, workspace=ws)
         mark(2)
@@ -235,7 +241,8 @@ def main():
         B.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, dk=dk, dv=dv, workspace=ws)
         mark(5)
 
-    kernels_per_step = 8            # 4 quantiser launches + fwd + delta + dQ + dK/dV
+    # 4 quantiser launches + fwd + delta + dQ + dK/dV (two key-major passes when the qk head dim exceeds 128)
+    kernels_per_step = 8 + (1 if (not bf16_mode and w.head_dim_qk > 128) else 0)
 
     # ---- device-resident timing -------------------------------------------------------------
     for _ in range(warmup):
@@ -286,8 +293,8 @@ def main():
                 stream.wait_event(out_done[i - n_slots])             # outputs of that step already on the host
             qi, ki, vi, dOi = in_dev[slot]
             oo, ll, dqo, dko, dvo = out_dev[slot]
-            B.attn_fp8_quantize(qi, out=qq); B.attn_fp8_quantize(ki, out=kq)
-            B.attn_fp8_quantize(vi, out=vq); B.attn_fp8_quantize(dOi, out=dOq)
+            prepare(qi, out=qq); prepare(ki, out=kq)
+            prepare(vi, out=vq); prepare(dOi, out=dOq)
             B.attn_fp8_fwd(params, qq, kq, vq, o=oo, lse=ll, workspace=ws)
             B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, ll, delta=delta, workspace=ws)
             B.attn_fp8_bwd(params, qq, kq, vq, dOq, ll, delta, dq=dqo, dk=dko, dv=dvo, workspace=ws)
@@ -327,26 +334,32 @@ def main():
     attn_stages = {n: stage_ms[n] for n in PRODUCTS}
     dominant = max(attn_stages, key=attn_stages.get)
     c = 1 if w.causal else 2
-    pair_flops = c * w.batch * w.heads_q * w.seqlen * w.seqlen * w.head_dim_qk     # 2*d flops x N^2/2 pairs per head
-    kernel_flops = PRODUCTS[dominant] * pair_flops
+    pairs2 = c * w.batch * w.heads_q * w.seqlen * w.seqlen                          # 2 x (N^2 / 2) pairs per head
+    n_qk, n_v = PRODUCTS[dominant]
+    kernel_flops = pairs2 * (n_qk * w.head_dim_qk + n_v * w.head_dim_v)
     achieved = kernel_flops / (stage_ms[dominant] * 1e-3) / 1e12
-    peak = peaks["bf16_sustained"] * FP8_OVER_BF16
+    ratio = 1.0 if bf16_mode else FP8_OVER_BF16
+    peak = peaks["bf16_sustained"] * ratio
     roofline = {
         "kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
         "frac": achieved / peak,
-        "peak_source": f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x {FP8_OVER_BF16} (nominal fp8:bf16)",
-        "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+        "peak_source": (f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s"
+                        + ("" if bf16_mode else f" x {FP8_OVER_BF16} (nominal fp8:bf16)")),
+        "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (w.name == WORKLOAD and not bf16_mode) else None,
     }
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "fp8_e4m3", "data": "synthetic",
+        "dtype": "bf16" if bf16_mode else "fp8_e4m3", "data": "synthetic",
         "config": {"workload": w.name, "batch": w.batch, "heads_q": w.heads_q, "heads_kv": w.heads_kv,
-                   "seqlen": w.seqlen, "head_dim": w.head_dim_qk, "causal": w.causal, "delta_mode": "matched",
+                   "seqlen": w.seqlen, "head_dim": w.head_dim_qk, "head_dim_v": w.head_dim_v, "causal": w.causal,
+                   "delta_mode": "matched", "precision": args.precision,
                    "l2": "working set per step (>500 MB) exceeds the 126 MB L2", "parallelism": f"replicas x{world}",
-                   "step": "quantize(Q,K,V,dO) + fwd + matched delta + dQ + dK/dV"},
+                   "step": ("transposed BF16 copies of Q,K,V,dO" if bf16_mode else "quantize(Q,K,V,dO)")
+                           + " + fwd + matched delta + dQ + dK/dV"},
         "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
+        "pct_of_nominal_peak_of_dtype": 100.0 * value / world / (NOMINAL_FP8_TFLOPS / (FP8_OVER_BF16 if bf16_mode else 1.0)),
         "stage_ms": stage_ms,
         "attn_only_tflops": credited / ((sum(attn_stages.values())) * 1e-3) / 1e12,
         "fwd_tflops": fwd_flops / (stage_ms["fwd"] * 1e-3) / 1e12,
@@ -363,7 +376,7 @@ def main():
         small = w.scaled(heads_q=w.heads_q // w.heads_kv, heads_kv=1, seqlen=sample_tokens)
         sq, sk, sv, sdO = workloads.make_inputs(small)
         t0 = time.perf_counter()
-        flops = oracle_step(w, sample_tokens, sq, sk, sv, sdO)
+        flops = oracle_step(w, sample_tokens, sq, sk, sv, sdO, args.precision)
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = {
             "value": flops / dt / 1e12, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "seconds": dt,

@@ -186,25 +186,33 @@ def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool =
     return out
 
 
-def attn_fp8_prepare_bf16(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None) -> QTensor:
+def attn_fp8_prepare_bf16(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None,
+                          out: Optional[QTensor] = None) -> QTensor:
     """BF16-mode operands of ``src`` [B, H, N, d]: ``row_codes`` = BF16 [B, H, N, d] (``src`` itself when
-    it already is BF16), ``col_codes`` = BF16 [B, H, d, N]; no scales."""
+    it already is BF16), ``col_codes`` = BF16 [B, H, d, N]; no scales.  ``out`` reuses the buffers of an
+    earlier call of the same shape."""
     if not src.is_cuda or not src.is_contiguous() or src.dim() != 4:
         raise ValueError("src must be a contiguous CUDA tensor [B, H, N, d]")
     if src.dtype not in (torch.bfloat16, torch.float32):
         raise ValueError("src must be bfloat16 or float32")
     dt = ATTN_SRC_BF16 if src.dtype == torch.bfloat16 else ATTN_SRC_FP32
     B, H, N, d = src.shape
-    out = QTensor(shape=(B, H, N, d))
-    bf = dict(dtype=torch.bfloat16, device=src.device)
-    write_row = want_row and src.dtype != torch.bfloat16
-    if write_row:
-        out.row_codes = torch.empty((B, H, N, d), **bf)
-    if want_col:
-        out.col_codes = torch.empty((B, H, d, N), **bf)
-    if write_row or want_col:
-        _check(_lib.attn_fp8_prepare_bf16(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
-    if want_row and not write_row:
+    alias_row = src.dtype == torch.bfloat16      # the row operand is the source itself
+    if out is None:
+        out = QTensor(shape=(B, H, N, d))
+        bf = dict(dtype=torch.bfloat16, device=src.device)
+        if want_row and not alias_row:
+            out.row_codes = torch.empty((B, H, N, d), **bf)
+        if want_col:
+            out.col_codes = torch.empty((B, H, d, N), **bf)
+    elif tuple(out.shape) != (B, H, N, d):
+        raise ValueError("out was allocated for another shape")
+    row_buf = None if alias_row else out.row_codes
+    if row_buf is not None or out.col_codes is not None:
+        c = _QTensor(None if row_buf is None else row_buf.data_ptr(), None,
+                     None if out.col_codes is None else out.col_codes.data_ptr(), None)
+        _check(_lib.attn_fp8_prepare_bf16(_ptr(src), dt, B, H, N, d, c, _stream(stream)))
+    if alias_row and (want_row or out.row_codes is not None):
         out.row_codes = src
     return out
 

@@ -17,12 +17,13 @@ from tests.util import rel_fro, to_np
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, tensors):
+def _run(w, tensors, prec="mxfp8"):
     from paper_2609_37852_b200 import binding as B
     params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
-                          w.softmax_scale)
+                          w.softmax_scale, precision=B.ATTN_PREC_BF16 if prec == "bf16" else B.ATTN_PREC_MXFP8)
     dev = [x.cuda() for x in tensors]
-    qq, kq, vq, dOq = (B.attn_fp8_quantize(x) for x in dev)
+    prep = B.attn_fp8_prepare_bf16 if prec == "bf16" else B.attn_fp8_quantize
+    qq, kq, vq, dOq = (prep(x) for x in dev)
     o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
     delta, ws = B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
     dq, dk, dv, rs, ra, ws = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, diagnostics=True, workspace=ws)
@@ -30,7 +31,7 @@ def _run(w, tensors):
     return dict(o=o, lse=lse, delta=delta, dq=dq, dk=dk, dv=dv, rs=rs, ra=ra)
 
 
-def _check_sampled(w, tensors, got, heads, rows, col_groups, seed):
+def _check_sampled(w, tensors, got, heads, rows, col_groups, seed, prec="mxfp8"):
     """``heads``: (batch, query head) pairs to sample; ``rows`` query rows per head; ``col_groups``
     number of 32-key groups per sampled KV head."""
     q, k, v, dO = tensors
@@ -43,31 +44,31 @@ def _check_sampled(w, tensors, got, heads, rows, col_groups, seed):
         qh, dOh = to_np(q[b:b + 1, h:h + 1]), to_np(dO[b:b + 1, h:h + 1])
         kh, vh = to_np(k[b:b + 1, g:g + 1]), to_np(v[b:b + 1, g:g + 1])
         r = np.unique(np.concatenate([[0, 1, 63, 64, 127, 128, N - 1], rng.integers(0, N, rows)]))
-        O_or, LSE_or = A.emu_forward(qh, kh, vh, w.softmax_scale, w.causal, rows=r)
+        O_or, LSE_or = A.emu_forward(qh, kh, vh, w.softmax_scale, w.causal, rows=r, prec=prec)
         assert rel_fro(to_np(got["o"][b, h])[r], O_or[0, 0]) <= 2e-3
         lse_gpu = to_np(got["lse"][b, h])
         assert rel_fro(lse_gpu[r], LSE_or[0, 0]) <= 2e-3
         assert np.abs(lse_gpu[r] - LSE_or[0, 0]).max() <= 2e-4 * max(1.0, np.abs(LSE_or).max())
         lse_full = lse_gpu[None, None]
-        D_or = A.emu_delta(qh, kh, vh, dOh, lse_full, w.softmax_scale, w.causal, rows=r)
+        D_or = A.emu_delta(qh, kh, vh, dOh, lse_full, w.softmax_scale, w.causal, rows=r, prec=prec)
         d_gpu = to_np(got["delta"][b, h])
         assert rel_fro(d_gpu[r], D_or[0, 0]) <= 1e-4
-        dq_or, rs_or, ra_or = A.emu_backward_rows(qh, kh, vh, dOh, lse_gpu, d_gpu, w.softmax_scale, w.causal, 0, 0, r)
+        dq_or, rs_or, ra_or = A.emu_backward_rows(qh, kh, vh, dOh, lse_gpu, d_gpu, w.softmax_scale, w.causal, 0, 0, r,
+                                                  prec=prec)
         assert rel_fro(to_np(got["dq"][b, h])[r], dq_or) <= 5e-3
         g_rs, g_ra = to_np(got["rs"][b, h])[r], to_np(got["ra"][b, h])[r]
         assert rel_fro(g_ra, ra_or) <= 1e-3
         # zero-row-sum invariant, same form as in the small-size test: 1e-5 of sum|dS| plus
         # |D| |1 - sum P| with |1 - sum P| <= one ulp of the FP32-stored LSE + 2^-20
-        from oracle import mxfp8
-        P = A._probabilities(mxfp8.fake_quant(qh[0, 0]), mxfp8.fake_quant(kh[0, 0]), lse_gpu, w.softmax_scale,
+        P = A._probabilities(A._fq(qh[0, 0], -1, prec), A._fq(kh[0, 0], -1, prec), lse_gpu, w.softmax_scale,
                              w.causal, r, np.arange(N))
-        dust = (P * np.abs(mxfp8.fake_quant(dOh[0, 0])[r] @ mxfp8.fake_quant(vh[0, 0]).T)).sum(-1)
+        dust = (P * np.abs(A._fq(dOh[0, 0], -1, prec)[r] @ A._fq(vh[0, 0], -1, prec).T)).sum(-1)
         ulp = np.spacing(np.abs(lse_gpu[r]).astype(np.float32)).astype(np.float64)
         assert np.all(np.abs(g_rs) <= 1e-5 * g_ra + (ulp + 2.0 ** -20) * dust)
         live = (g_ra > 0) & (r >= 64)
         r_pre = np.abs(g_rs[live]) / g_ra[live]
         print(f"\n[{w.name} b{b} h{h}] sampled r_pre median {np.median(r_pre):.2e} max {r_pre.max():.2e}")
-        if w.recipe in ("iid", "qknorm"):
+        if w.recipe in ("iid", "qknorm", "plain"):
             assert np.median(r_pre) <= 1e-5
     # dK / dV: all query heads of the sampled KV heads, a few 32-key groups each
     for (b, g) in sorted({(b, h // G) for (b, h) in heads}):
@@ -77,7 +78,7 @@ def _check_sampled(w, tensors, got, heads, rows, col_groups, seed):
         lse_g, d_g = to_np(got["lse"][b, hs]), to_np(got["delta"][b, hs])
         starts = np.unique(np.concatenate([[0, N - 32], 32 * rng.integers(0, N // 32, col_groups)]))
         cols = np.concatenate([np.arange(s, s + 32) for s in starts])
-        dk_or, dv_or = A.emu_backward_cols(qg, kg, vg, dOg, lse_g, d_g, w.softmax_scale, w.causal, 0, 0, cols)
+        dk_or, dv_or = A.emu_backward_cols(qg, kg, vg, dOg, lse_g, d_g, w.softmax_scale, w.causal, 0, 0, cols, prec=prec)
         assert rel_fro(to_np(got["dk"][b, g])[cols], dk_or) <= 5e-3
         assert rel_fro(to_np(got["dv"][b, g])[cols], dv_or) <= 5e-3
 
@@ -105,3 +106,27 @@ def test_long_context_sampled():
     tensors = workloads.make_inputs(w)
     got = _run(w, tensors)
     _check_sampled(w, tensors, got, heads=[(0, 5)], rows=32, col_groups=2, seed=3)
+
+
+def test_mla_full_size_sampled():
+    """mla8k: B=1, 16/16 heads, N=8192, qk head dim 192, v head dim 128."""
+    w = workloads.WORKLOADS["mla8k"]
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors)
+    _check_sampled(w, tensors, got, heads=[(0, 3), (0, 15)], rows=32, col_groups=2, seed=4)
+
+
+def test_d256_full_size_sampled():
+    """gqa8k_d256: B=1, 8/2 heads, N=8192, head dim 256."""
+    w = workloads.WORKLOADS["gqa8k_d256"]
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors)
+    _check_sampled(w, tensors, got, heads=[(0, 1), (0, 7)], rows=32, col_groups=2, seed=5)
+
+
+def test_bench_workload_bf16_mode_sampled():
+    """gqa8k_outlier in BF16 mode (the reference-point configuration bench.py --precision bf16 times)."""
+    w = workloads.WORKLOADS["gqa8k_outlier"]
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors, prec="bf16")
+    _check_sampled(w, tensors, got, heads=[(0, 6), (0, 31)], rows=32, col_groups=2, seed=6, prec="bf16")
