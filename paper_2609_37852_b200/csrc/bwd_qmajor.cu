@@ -369,8 +369,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
       // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
       // a loop without it
-      auto body = [&](auto diag_tag) {
+      auto body = [&](auto diag_tag, auto stats_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
+        constexpr bool kStats = decltype(stats_tag)::value;      // pre-cast row statistics requested
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -lse2);
@@ -380,14 +381,21 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           if (kDQ) {
             const float d = pr * fmaf(dp, f_lo, -fD);
             ds[c] = d;
-            acc0 += d;
-            acc1 += fabsf(d);
+            if (kStats) {
+              acc0 += d;
+              acc1 += fabsf(d);
+            }
           } else {
             part = fmaf(pr, dp, part);
           }
         }
       };
-      if (p.causal && t * kStep >= qt * kTile) body(std::true_type{}); else body(std::false_type{});
+      const bool diag = p.causal && t * kStep >= qt * kTile;
+      if (kDQ && p.rowsum != nullptr) {
+        if (diag) body(std::true_type{}, std::true_type{}); else body(std::false_type{}, std::true_type{});
+      } else {
+        if (diag) body(std::true_type{}, std::false_type{}); else body(std::false_type{}, std::false_type{});
+      }
       if (!kDQ) {
         acc0 = fmaf(part, f_lo, acc0);
       } else {

@@ -292,6 +292,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
 #pragma unroll
         for (int c = 0; c < 32; ++c) mx = fmaxf(mx, sv[c]);
       }
+      const float mx_own = mx;                        // maximum of this thread's 32 keys (one quantisation block)
       sts_f32(&sm.xch[u & 1][grp][row], mx);
       mbar_arrive(&sm.pair[quad]);                    // the two warps that share these 32 rows
       ok = mbar_wait(&sm.pair[quad], u & 1, abort_flag);
@@ -323,29 +324,39 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         }
       }
       const float neg_m = -M;
-      float bs0 = 0.f, bs1 = 0.f, amax = 0.f;          // two short chains for the block sum
-#pragma unroll
-      for (int c = 0; c < 32; c += 2) {
-        const float p0 = ex2_approx(fmaf(sv[c], p.scale_log2, neg_m));
-        const float p1 = ex2_approx(fmaf(sv[c + 1], p.scale_log2, neg_m));
-        sv[c] = p0;
-        sv[c + 1] = p1;
-        bs0 += p0;
-        bs1 += p1;
-        amax = fmaxf(amax, fmaxf(p0, p1));
-      }
-      l += bs0 + bs1;
       uint32_t byte = 0;
       uint32_t words[8 * kEB];
       if (kFp8) {
+        // The block's scale 2^e follows from its largest exponential, which is the exponential of
+        // the thread's own score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the
+        // value the E4M3 cast wants, and the block sum is put back on the common scale by one
+        // exact multiplication.
         float inv;
-        block_scale(amax, byte, inv);
+        block_scale(ex2_approx(fmaf(mx_own, p.scale_log2, neg_m)), byte, inv);
+        const float neg_me = neg_m - static_cast<float>(static_cast<int>(byte) - 127);
+        float bs0 = 0.f, bs1 = 0.f;                    // two short chains for the block sum
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          words[i] = cvt_e4m3x4(sv[4 * i] * inv, sv[4 * i + 1] * inv, sv[4 * i + 2] * inv, sv[4 * i + 3] * inv);
+        for (int i = 0; i < 8; ++i) {
+          const float t0 = ex2_approx(fmaf(sv[4 * i], p.scale_log2, neg_me));
+          const float t1 = ex2_approx(fmaf(sv[4 * i + 1], p.scale_log2, neg_me));
+          const float t2 = ex2_approx(fmaf(sv[4 * i + 2], p.scale_log2, neg_me));
+          const float t3 = ex2_approx(fmaf(sv[4 * i + 3], p.scale_log2, neg_me));
+          bs0 += t0 + t2;
+          bs1 += t1 + t3;
+          words[i] = cvt_e4m3x4(t0, t1, t2, t3);
+        }
+        l = fmaf(bs0 + bs1, __uint_as_float(byte << 23), l);      // 2^e (0 for an all-masked block, whose sum is 0)
       } else {
+        float bs0 = 0.f, bs1 = 0.f;
 #pragma unroll
-        for (int i = 0; i < 8 * kEB; ++i) words[i] = cvt_bf16x2(sv[(2 * i) & 31], sv[(2 * i + 1) & 31]);
+        for (int c = 0; c < 32; c += 2) {
+          const float p0 = ex2_approx(fmaf(sv[c], p.scale_log2, neg_m));
+          const float p1 = ex2_approx(fmaf(sv[c + 1], p.scale_log2, neg_m));
+          bs0 += p0;
+          bs1 += p1;
+          words[c >> 1] = cvt_bf16x2(p0, p1);
+        }
+        l += bs0 + bs1;
       }
       if (u >= 2) {
         // the P V MMAs of sub-tile u-2 have consumed this buffer's operand and scale bytes
