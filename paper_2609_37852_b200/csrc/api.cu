@@ -267,6 +267,8 @@ attn_status_t attn_fp8_read_status(const void* workspace, void* stream) {
   cudaError_t e = cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "read_status: %s", cudaGetErrorString(e));
+  if (host == ATTN_ERR_ALIGNMENT)
+    return fail(ATTN_ERR_ALIGNMENT, "a kernel found its dynamic shared memory not 1024-byte aligned and did not run");
   if (host != 0) return fail(ATTN_ERR_TIMEOUT, "a bounded device-side wait expired (status word %d)", host);
   return ATTN_OK;
 }

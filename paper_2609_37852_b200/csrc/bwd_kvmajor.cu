@@ -161,7 +161,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
                const __grid_constant__ CUtensorMap tm_qc, const __grid_constant__ CUtensorMap tm_dOc) {
-  extern __shared__ uint8_t smem_raw[];
+  // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
+  // shared state space of every access derived from it (checked below)
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   constexpr bool kFp8 = C::kFp8, kHasDv = C::kHasDv, kHasDk = C::kHasDk;
   constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRq, kRv = C::kRv;
   constexpr int kRowStages = C::kRowStages, kColStages = C::kColStages, kRowTok = C::kRowTok;
@@ -170,7 +172,11 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
                      kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
                      kColSFdO = C::kColSFdO, kColSFP = C::kColSFP, kColSFdS = C::kColSFdS, kColSFdOc = C::kColSFdOc,
                      kColSFQc = C::kColSFQc, kTmemCols = C::kTmemCols;
-  KvSmem<C>& sm = *reinterpret_cast<KvSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  KvSmem<C>& sm = *reinterpret_cast<KvSmem<C>*>(smem_raw);
+  if (smem_u32(smem_raw) & 1023u) {               // never expected: report instead of computing garbage
+    if (threadIdx.x == 0) atomicExch(p.status, static_cast<int>(ATTN_ERR_ALIGNMENT));
+    return;
+  }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // blocks are handed out x-fastest: KV heads vary fastest, key tiles in order, so the heaviest
   // tiles (the earliest keys under the causal mask) of all heads go first
@@ -419,9 +425,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     const int row = quad * 32 + lane;                 // key inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
     bool ok = true;
+    int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
+    static_assert(kTeams == 2, "a team advances by one query tile per iteration");
     for (int u = team; u < n_sub; u += kTeams) {
-      const int n = u >> 1, half = u & 1, buf = u & 1, ri = u / kSubPerRow, s = ri % kRowStages;
-      const int it = it0 + n % tiles_per_head;
+      const int half = u & 1, buf = u & 1, ri = u / kSubPerRow, s = ri % kRowStages;
       if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 0);
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
@@ -471,8 +478,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       uint32_t byte_p = 0, byte_s = 0;
       float inv_p = 1.f, inv_s = 1.f;
       if (kFp8) {
-        if (kHasDv) block_scale(amax_p, byte_p, inv_p);
-        if (kHasDk) block_scale(max_s, byte_s, inv_s);
+        if (kHasDv) block_scale_finite(amax_p, byte_p, inv_p);
+        if (kHasDk) block_scale_finite(max_s, byte_s, inv_s);
       }
       if (u >= 2) {
         // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's operands and scale bytes
@@ -519,6 +526,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tc_fence_before_sync();
       mbar_arrive(&sm.pds_full[buf]);
       if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 3);
+      it = (it + 1 == tiles_n) ? it0 : it + 1;        // next tile of this head, or the first tile of the next head
     }
     // the epilogue is done by team 0 (group 0 stores dV, group 1 stores dK)
     if (team != 0) ok = false;

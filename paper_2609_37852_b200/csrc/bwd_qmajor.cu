@@ -134,14 +134,20 @@ __global__ void __launch_bounds__(C::kThreads, 1)
 qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_dO,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
               const __grid_constant__ CUtensorMap tm_kc) {
-  extern __shared__ uint8_t smem_raw[];
+  // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
+  // shared state space of every access derived from it (checked below)
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8;
   constexpr int kStages = C::kStages, kKcStages = C::kKcStages, kEB = C::kEB, kCq = C::kCq, kCv = C::kCv;
   constexpr int kStep = C::kStep, kGroups = C::kGroups, kSoftmaxThreads = C::kSoftmaxThreads;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColdS = C::kColdS, kColdQ = C::kColdQ, kColSFQ = C::kColSFQ,
                      kColSFdO = C::kColSFdO, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFdS = C::kColSFdS,
                      kColSFKc = C::kColSFKc, kTmemCols = C::kTmemCols;
-  QmSmem<C>& sm = *reinterpret_cast<QmSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  QmSmem<C>& sm = *reinterpret_cast<QmSmem<C>*>(smem_raw);
+  if (smem_u32(smem_raw) & 1023u) {               // never expected: report instead of computing garbage
+    if (threadIdx.x == 0) atomicExch(p.status, static_cast<int>(ATTN_ERR_ALIGNMENT));
+    return;
+  }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
   // all heads go first, so the light tiles fill the tail of the launch

@@ -34,6 +34,18 @@
 #include "sm100_ptx.cuh"
 
 namespace attnfp8 {
+
+#ifdef ATTN_TRACE
+// Debug build only: clock stamps of one CTA (roles x steps x events), read back by the host.
+__device__ long long g_fw_trace[4][256][8];
+#define FW_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_fw_trace[role][step][ev] = clock64(); } while (0)
+extern "C" int attn_fp8_debug_fw_trace(long long* host_out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_fw_trace, sizeof(g_fw_trace)));
+}
+#else
+#define FW_TRACE(role, step, ev) do { } while (0)
+#endif
+
 namespace {
 
 using namespace sm100;
@@ -41,16 +53,18 @@ using namespace sm100;
 constexpr int kTile = 128;          // query rows per CTA; keys per K / V tile in shared memory
 constexpr int kSub = 64;            // keys per softmax step
 constexpr int kStages = 2;          // K ring and V ring depth
-constexpr int kThreads = 384;
-constexpr int kSoftmaxThreads = 256;      // two threads per query row
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
 constexpr int kLazyShift = 8;
 
 // Operand geometry and tensor-memory map of one instantiation.
-template <int kEB_, int kCq_, int kRv_>
+template <int kEB_, int kCq_, int kRv_, int kSplit_ = 2>
 struct FwdCfg {
+  static constexpr int kSplit = kSplit_;                // softmax threads per query row (1 or 2)
+  static constexpr int kBpt = 2 / kSplit;               // 32-key quantisation blocks per thread and step
+  static constexpr int kSoftmaxThreads = 128 * kSplit;
+  static constexpr int kThreads = 128 + kSoftmaxThreads;
   static constexpr int kEB = kEB_;                      // bytes per operand element
   static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row
   static constexpr int kRv = kRv_;                      // 128-row tiles of the V^T operand (dv / 128, rounded up)
@@ -106,13 +120,20 @@ struct FwdParams {
 };
 
 template <class C>
-__global__ void __launch_bounds__(kThreads, C::kCtasPerSm)
+__global__ void __launch_bounds__(C::kThreads, C::kCtasPerSm)
 fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v) {
-  extern __shared__ uint8_t smem_raw[];
-  FwdSmem<C>& sm = *reinterpret_cast<FwdSmem<C>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
+  // shared state space of every access derived from it (checked below)
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  FwdSmem<C>& sm = *reinterpret_cast<FwdSmem<C>*>(smem_raw);
+  if (smem_u32(smem_raw) & 1023u) {               // never expected: report instead of computing garbage
+    if (threadIdx.x == 0) atomicExch(p.status, static_cast<int>(ATTN_ERR_ALIGNMENT));
+    return;
+  }
   constexpr bool kFp8 = C::kFp8;
   constexpr int kEB = C::kEB, kCq = C::kCq, kRv = C::kRv, kSubPerTile = C::kSubPerTile;
+  constexpr int kSplit = C::kSplit, kBpt = C::kBpt, kSoftmaxThreads = C::kSoftmaxThreads;
   constexpr uint32_t kColS = C::kColS, kColP = C::kColP, kColO = C::kColO, kColSFQ = C::kColSFQ, kColSFK = C::kColSFK,
                      kColSFV = C::kColSFV, kColSFP = C::kColSFP, kTmemCols = C::kTmemCols, kPCols = C::kPCols;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -210,16 +231,19 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
         }
+        FW_TRACE(0, u, 0);
         if (u > 0) {
           // the softmax threads have pulled the previous scores into registers
           ok = mbar_wait(&sm.s_free, (u - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
+        FW_TRACE(0, u, 1);
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0])) + sub * (kSub * 128 / 16);
         issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, C::kTileKeys * 128 / 16>(
             tmem + kColS, desc_q, desc_k, nk_qk, tmem + kColSFQ, tmem + kColSFK + 4 * kCq * slot + 2 * sub);
         mma_commit_elect(&sm.s_full);
+        FW_TRACE(0, u, 2);
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
       }
       if (!ok) {
@@ -240,14 +264,17 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kRv>(tmem + kColSFV + 4 * kRv * slot, sm.sf_v[s]);
         }
+        FW_TRACE(1, u, 0);
         ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
+        FW_TRACE(1, u, 1);
         tc_fence_after_sync();
         if (kFp8) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         // 64 keys = 2 (codes) or 4 (BF16) steps of 32 bytes; the V^T operand is taken 128 rows at a time
         issue_ts<kFp8, kEB, kRv>(tmem + kColO, tmem + kColP + kPCols * buf, make_desc_sw128(smem_u32(sm.v[s])), p.dv, sub,
                                  tmem + kColSFP + 4 * buf, tmem + kColSFV + 4 * kRv * slot, u > 0);
         mma_commit_elect(&sm.p_free[buf]);              // operand (and scale bytes) of this buffer consumed; O updated
+        FW_TRACE(1, u, 2);
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.o_done);
       }
@@ -259,50 +286,73 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax
-    // Two threads per query row: column group `grp` owns keys 32*grp .. 32*grp+31 of the sub-tile
-    // (one quantisation block).  The pair lives in two warps with the same TMEM lane quadrant and
-    // exchanges its block maxima through shared memory, so that both use the same shift M.
-    const int grp = (warp - 4) >> 2;
+    // kSplit threads per query row.  With two, column group `grp` owns keys 32*grp .. 32*grp+31 of
+    // the sub-tile (one quantisation block); the pair lives in two warps with the same TMEM lane
+    // quadrant and exchanges its block maxima through shared memory, so that both use the same
+    // shift M.  With one, the thread owns both blocks and nothing is exchanged (measured slower on
+    // B200: four softmax warps per CTA hide less latency than the exchange costs).
+    const int grp = kSplit == 2 ? (warp - 4) >> 2 : 0;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                 // row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    const int blk0 = grp * kBpt;                      // first 32-key block of this thread inside a sub-tile
     float M = -INFINITY;                              // integer-valued running shift (log2 units)
     float l = 0.f;                                    // this thread's share of the normaliser
     bool ok = true;
     for (int u = 0; u < n_sub; ++u) {
       const int t = u >> 1, half = u & 1, buf = u & 1;
+#define SM_TRACE(ev) do { if (lane == 0 && (warp == 4 || warp == 8)) FW_TRACE(warp == 4 ? 2 : 3, u, ev); } while (0)
+      SM_TRACE(0);
       ok = mbar_wait(&sm.s_full, u & 1, abort_flag);
       if (!ok) break;
+      SM_TRACE(1);
       tc_fence_after_sync();
-      float sv[32];
-      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, reinterpret_cast<uint32_t*>(sv));
+      float sv[32 * kBpt];
+#pragma unroll
+      for (int bk = 0; bk < kBpt; ++bk)
+        tmem_ld32(tmem + kColS + lane_addr + 32 * (blk0 + bk), reinterpret_cast<uint32_t*>(sv + 32 * bk));
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.s_free);
-      // maximum of the raw accumulators (the scale is positive), masked on the diagonal tile
-      float mx = -INFINITY;
+      SM_TRACE(2);
+      // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
+      float mxb[kBpt];
       if (p.causal && t == qt) {
-        const int col0 = half * kSub + 32 * grp;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          if (col0 + c > row) sv[c] = -INFINITY;
-          mx = fmaxf(mx, sv[c]);
+        for (int bk = 0; bk < kBpt; ++bk) {
+          const int col0 = half * kSub + 32 * (blk0 + bk);
+          float m = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            if (col0 + c > row) sv[32 * bk + c] = -INFINITY;
+            m = fmaxf(m, sv[32 * bk + c]);
+          }
+          mxb[bk] = m;
         }
       } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, sv[c]);
+        for (int bk = 0; bk < kBpt; ++bk) {
+          float m = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) m = fmaxf(m, sv[32 * bk + c]);
+          mxb[bk] = m;
+        }
       }
-      const float mx_own = mx;                        // maximum of this thread's 32 keys (one quantisation block)
-      sts_f32(&sm.xch[u & 1][grp][row], mx);
-      mbar_arrive(&sm.pair[quad]);                    // the two warps that share these 32 rows
-      ok = mbar_wait(&sm.pair[quad], u & 1, abort_flag);
-      if (!ok) break;
-      mx = fmaxf(mx, lds_f32(&sm.xch[u & 1][grp ^ 1][row]));
+      float mx = mxb[0];
+      if (kBpt == 2) mx = fmaxf(mx, mxb[kBpt - 1]);
+      if (kSplit == 2) {
+        sts_f32(&sm.xch[u & 1][grp][row], mx);
+        mbar_arrive(&sm.pair[quad]);                  // the two warps that share these 32 rows
+        ok = mbar_wait(&sm.pair[quad], u & 1, abort_flag);
+        if (!ok) break;
+        mx = fmaxf(mx, lds_f32(&sm.xch[u & 1][grp ^ 1][row]));
+      }
+      SM_TRACE(3);
       // a fully masked sub-tile (second half of the diagonal tile for the first 64 rows) gives -inf:
       // it never raises M and contributes zeros
       const float m_new = ceilf(mx * p.scale_log2);
       const bool raise = m_new > M + static_cast<float>(kLazyShift);   // true on the first sub-tile
-      if (__any_sync(0xffffffffu, raise)) {             // same rows, same decision in both warps of the pair
+      if (__any_sync(0xffffffffu, raise)) {             // same rows, same decision in both warps of a pair
         const float factor = raise ? exp2f(M - m_new) : 1.f;            // exact power of two (0 at the start)
         if (raise) { l *= factor; M = m_new; }
         if (u > 0) {
@@ -310,9 +360,9 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           ok = mbar_wait(&sm.p_free[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          // rare path; each thread of the pair rescales its half of the output columns
-          const int half_cols = p.dv / 2;
-          for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 8) {
+          // rare path; each thread of a row rescales its share of the output columns
+          const int my_cols = p.dv / kSplit;
+          for (int c0 = grp * my_cols; c0 < (grp + 1) * my_cols; c0 += 8) {
             uint32_t r[8];
             tmem_ld8(tmem + kColO + lane_addr + c0, r);
             tmem_wait_ld();
@@ -324,57 +374,68 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         }
       }
       const float neg_m = -M;
-      uint32_t byte = 0;
-      uint32_t words[8 * kEB];
-      if (kFp8) {
-        // The block's scale 2^e follows from its largest exponential, which is the exponential of
-        // the thread's own score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the
-        // value the E4M3 cast wants, and the block sum is put back on the common scale by one
-        // exact multiplication.
-        float inv;
-        block_scale(ex2_approx(fmaf(mx_own, p.scale_log2, neg_m)), byte, inv);
-        const float neg_me = neg_m - static_cast<float>(static_cast<int>(byte) - 127);
-        float bs0 = 0.f, bs1 = 0.f;                    // two short chains for the block sum
+      uint32_t bytes[kBpt];
+      uint32_t words[kBpt][8 * kEB];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float t0 = ex2_approx(fmaf(sv[4 * i], p.scale_log2, neg_me));
-          const float t1 = ex2_approx(fmaf(sv[4 * i + 1], p.scale_log2, neg_me));
-          const float t2 = ex2_approx(fmaf(sv[4 * i + 2], p.scale_log2, neg_me));
-          const float t3 = ex2_approx(fmaf(sv[4 * i + 3], p.scale_log2, neg_me));
-          bs0 += t0 + t2;
-          bs1 += t1 + t3;
-          words[i] = cvt_e4m3x4(t0, t1, t2, t3);
-        }
-        l = fmaf(bs0 + bs1, __uint_as_float(byte << 23), l);      // 2^e (0 for an all-masked block, whose sum is 0)
-      } else {
-        float bs0 = 0.f, bs1 = 0.f;
+      for (int bk = 0; bk < kBpt; ++bk) {
+        const float* x = sv + 32 * bk;
+        bytes[bk] = 0;
+        if (kFp8) {
+          // The block's scale 2^e follows from its largest exponential, which is the exponential of
+          // the block's score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the
+          // value the E4M3 cast wants, and the block sum is put back on the common scale by one
+          // exact multiplication.
+          float inv;
+          block_scale_finite(ex2_approx(fmaf(mxb[bk], p.scale_log2, neg_m)), bytes[bk], inv);
+          const float neg_me = neg_m - static_cast<float>(static_cast<int>(bytes[bk]) - 127);
+          float bs0 = 0.f, bs1 = 0.f;                  // two short chains for the block sum
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float p0 = ex2_approx(fmaf(sv[c], p.scale_log2, neg_m));
-          const float p1 = ex2_approx(fmaf(sv[c + 1], p.scale_log2, neg_m));
-          bs0 += p0;
-          bs1 += p1;
-          words[c >> 1] = cvt_bf16x2(p0, p1);
+          for (int i = 0; i < 8; ++i) {
+            const float t0 = ex2_approx(fmaf(x[4 * i], p.scale_log2, neg_me));
+            const float t1 = ex2_approx(fmaf(x[4 * i + 1], p.scale_log2, neg_me));
+            const float t2 = ex2_approx(fmaf(x[4 * i + 2], p.scale_log2, neg_me));
+            const float t3 = ex2_approx(fmaf(x[4 * i + 3], p.scale_log2, neg_me));
+            bs0 += t0 + t2;
+            bs1 += t1 + t3;
+            words[bk][i] = cvt_e4m3x4(t0, t1, t2, t3);
+          }
+          l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
+        } else {
+          float bs0 = 0.f, bs1 = 0.f;
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, neg_m));
+            const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, neg_m));
+            bs0 += p0;
+            bs1 += p1;
+            words[bk][c >> 1] = cvt_bf16x2(p0, p1);
+          }
+          l += bs0 + bs1;
         }
-        l += bs0 + bs1;
       }
+      SM_TRACE(4);
       if (u >= 2) {
         // the P V MMAs of sub-tile u-2 have consumed this buffer's operand and scale bytes
         ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
+      SM_TRACE(5);
 #pragma unroll
-      for (int i = 0; i < kEB; ++i)
-        tmem_st8(tmem + kColP + kPCols * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
-      if (kFp8) sts_u8(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + grp], byte);
+      for (int bk = 0; bk < kBpt; ++bk) {
+#pragma unroll
+        for (int i = 0; i < kEB; ++i)
+          tmem_st8(tmem + kColP + kPCols * buf + lane_addr + 8 * kEB * (blk0 + bk) + 8 * i, words[bk] + 8 * i);
+        if (kFp8) sts_u8(&sm.sf_p[buf][(row & 31) * 16 + (row >> 5) * 4 + blk0 + bk], bytes[bk]);
+      }
       tmem_wait_st();
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.p_full[buf]);
+      SM_TRACE(6);
     }
-    // total normaliser of the row = sum of the pair's shares
-    if (ok) {
+    // total normaliser of the row = sum of the shares of its threads
+    if (ok && kSplit == 2) {
       sm.xch[0][grp][row] = l;
       mbar_arrive(&sm.pair[quad]);
       ok = mbar_wait(&sm.pair[quad], n_sub & 1, abort_flag);
@@ -386,8 +447,8 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       const float inv_l = 1.f / l;
       const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
       __nv_bfloat16* o_row = p.o + grow * p.dv;
-      const int half_cols = p.dv / 2;                 // each thread of the pair stores half of the row
-      for (int c0 = grp * half_cols; c0 < (grp + 1) * half_cols; c0 += 32) {
+      const int my_cols = p.dv / kSplit;              // each thread of a row stores its share of the row
+      for (int c0 = grp * my_cols; c0 < (grp + 1) * my_cols; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem + kColO + lane_addr + c0, r);
         tmem_wait_ld();
@@ -434,7 +495,7 @@ attn_status_t launch_fwd_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t 
   cudaError_t e = cudaFuncSetAttribute(fwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(s.Hq, s.N / kTile, s.B);
-  fwd_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
+  fwd_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;

@@ -29,6 +29,16 @@ __device__ __forceinline__ void block_scale(float amax, uint32_t& byte, float& i
   inv = ib > 0 ? __uint_as_float(static_cast<uint32_t>(ib) << 23) : __uint_as_float(0x00400000u);
 }
 
+// The same rule for a maximum known to be finite and non-negative (probabilities, score
+// gradients), in five integer operations: adding 0x1FFFFF to the bit pattern carries into the
+// exponent field exactly when the mantissa exceeds 1.75.  Maxima below 2^-119 (biased exponent
+// under 8, zero included) give byte 0, as block_scale does.
+__device__ __forceinline__ void block_scale_finite(float amax, uint32_t& byte, float& inv) {
+  const int eb = max(static_cast<int>((__float_as_uint(amax) + 0x1FFFFFu) >> 23) - 8, 0);
+  byte = static_cast<uint32_t>(eb);
+  inv = __uint_as_float(static_cast<uint32_t>(254 - eb) << 23);
+}
+
 // Quantise 32 values held in registers: codes packed four per word (element 0 in the low byte)
 // and the block's scale byte.
 __device__ __forceinline__ uint32_t quantize_block32(const float* x, uint32_t* words) {
@@ -37,7 +47,7 @@ __device__ __forceinline__ uint32_t quantize_block32(const float* x, uint32_t* w
   for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(x[i]));
   uint32_t byte;
   float inv;
-  block_scale(amax, byte, inv);
+  block_scale_finite(amax, byte, inv);
 #pragma unroll
   for (int i = 0; i < 8; ++i)
     words[i] = sm100::cvt_e4m3x4(x[4 * i] * inv, x[4 * i + 1] * inv, x[4 * i + 2] * inv, x[4 * i + 3] * inv);
