@@ -180,6 +180,9 @@ def emu_delta(q, k, v, dO, lse, scale, causal, prec="mxfp8", mode="matched", o=N
     matched: D_i = sum_j P_ij dP^_ij with dP^ = dO^ V^^T from the row-blocked
              copies of dO and V (contraction over the value channels) -- Eq. 4.
     stale:   D_i = sum_k dO_ik O_ik from the BF16 dO and the saved BF16 O.
+    consistent: the saved-output shortcut with dO replaced by the operand the backward matmuls
+             consume, D_i = sum_k dO^_ik O_ik (paper Section 3.3, "consistent dO", Eq.
+             delta_consistent_do_residual); dO^ is the row-blocked copy, the one dP^ uses.
     Stored FP32 unless ``exact_stats``."""
     B, Hq, N, _ = q.shape
     G = Hq // k.shape[1]
@@ -191,6 +194,8 @@ def emu_delta(q, k, v, dO, lse, scale, causal, prec="mxfp8", mode="matched", o=N
             g = h // G
             if mode == "stale":
                 d = (mxfp8.round_bf16(dO[b, h])[rows] * np.asarray(o[b, h], np.float64)[rows]).sum(-1)
+            elif mode == "consistent":
+                d = (_fq(dO[b, h], -1, prec)[rows] * np.asarray(o[b, h], np.float64)[rows]).sum(-1)
             elif mode == "matched":
                 P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec),
                                    lse[b, h], scale, causal, rows, allc)

@@ -346,6 +346,36 @@ def test_stale_delta_residual_and_decomposition():
     assert np.nanmedian(r_s) > 1e-4
 
 
+def test_consistent_dO_residual_identity_and_ordering():
+    """Consistent dO (Section 3.3): with dO^ in the saved-output shortcut the gradient-quantisation
+    term of the stale residual disappears; what is left is the probability-quantisation term of
+    Eq. delta_consistent_do_residual, plus (this build's number format) the term of the two V
+    copies and the BF16 storage of O.  Median residuals order stale > consistent > matched."""
+    q, k, v, dO, scale, causal = _setup_fp8(seed=21)
+    O, LSE, fwd = A.emu_forward(q, k, v, scale, causal, exact_stats=True, return_internals=True)
+    Dm = A.emu_delta(q, k, v, dO, LSE, scale, causal, exact_stats=True)
+    Ds = A.emu_delta(q, k, v, dO, LSE, scale, causal, mode="stale", o=O, exact_stats=True)
+    Dc = A.emu_delta(q, k, v, dO, LSE, scale, causal, mode="consistent", o=O, exact_stats=True)
+    _, _, _, rsm, ram = A.emu_backward(q, k, v, dO, LSE, Dm, scale, causal)
+    _, _, _, rss, ras = A.emu_backward(q, k, v, dO, LSE, Ds, scale, causal)
+    _, _, _, rsc, rac, t = A.emu_backward(q, k, v, dO, LSE, Dc, scale, causal, return_internals=True)
+    G = q.shape[1] // k.shape[1]
+    for (b, h), tt in t.items():
+        g = h // G
+        assert np.abs(rsc[b, h] - (Dm[b, h] - Dc[b, h])).max() < 1e-12
+        P = tt["P"]
+        Phat = fwd[(b, h)]["Ph"] / fwd[(b, h)]["l"][:, None]
+        Vr, Vc = mxfp8.fake_quant(v[b, g], -1), mxfp8.fake_quant(v[b, g], 0)
+        dOr = mxfp8.fake_quant(dO[b, h], -1)
+        O_unrounded = Phat @ Vc
+        term_p = (dOr * ((P - Phat) @ Vr)).sum(-1)           # the paper's remaining term
+        term_v = (dOr * (Phat @ (Vr - Vc))).sum(-1)          # two V copies (1x32 blocks per contraction dim)
+        term_store = (dOr * (O_unrounded - O[b, h])).sum(-1)   # BF16 storage of the saved output
+        assert np.abs(rsc[b, h] - (term_p + term_v + term_store)).max() < 1e-12
+    med = lambda rs, ra: np.nanmedian(A.residual_ratio(rs, ra)[..., 64:])
+    assert med(rss, ras) > med(rsc, rac) > 100 * med(rsm, ram)
+
+
 def test_subset_functions_agree_with_full_pass():
     q, k, v, dO, scale, causal = _setup_fp8(seed=14)
     O, LSE = A.emu_forward(q, k, v, scale, causal)
