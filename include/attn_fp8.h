@@ -64,7 +64,7 @@ typedef enum {
 } attn_status_t;
 
 typedef enum { ATTN_PREC_MXFP8 = 0, ATTN_PREC_BF16 = 1 } attn_precision_t;
-typedef enum { ATTN_DELTA_MATCHED = 0, ATTN_DELTA_STALE = 1 } attn_delta_mode_t;
+typedef enum { ATTN_DELTA_MATCHED = 0, ATTN_DELTA_STALE = 1, ATTN_DELTA_CONSISTENT_DO = 2 } attn_delta_mode_t;
 typedef enum { ATTN_SRC_BF16 = 0, ATTN_SRC_FP32 = 1 } attn_src_dtype_t;
 typedef enum { ATTN_WS_FWD = 0, ATTN_WS_BWD_DELTA = 1, ATTN_WS_BWD = 2 } attn_ws_kind_t;
 
@@ -143,6 +143,10 @@ attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtenso
  *            reads q.row_*, k.row_*, v.row_*, dO.row_*, lse.  dO_bf16 / o_bf16 are ignored.
  *   STALE:   delta_i = sum_c dO_ic O_ic from BF16 dO and the saved BF16 O (both [B,Hq,N,dv]).
  *            reads dO_bf16, o_bf16 only.
+ *   CONSISTENT_DO (paper Section 3.3, Eq. delta_consistent_do_residual; an ablation): the same
+ *            shortcut with dO replaced by the operand the backward matmuls consume,
+ *            delta_i = sum_c dO^_ic O_ic, dO^ = the dequantised row copy of dO.
+ *            reads dO.row_*, o_bf16.
  *   writes  delta [B, Hq, N] (FP32)                                                           */
 attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                  attn_qtensor_t dO, const void* dO_bf16, const void* o_bf16,

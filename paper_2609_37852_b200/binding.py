@@ -27,7 +27,7 @@ ATTN_OK = 0
 STATUS_NAMES = {0: "ATTN_OK", 1: "ATTN_ERR_INVALID_ARG", 2: "ATTN_ERR_UNSUPPORTED", 3: "ATTN_ERR_ALIGNMENT",
                 4: "ATTN_ERR_WORKSPACE", 5: "ATTN_ERR_ARCH", 6: "ATTN_ERR_CUDA", 7: "ATTN_ERR_TIMEOUT"}
 ATTN_PREC_MXFP8, ATTN_PREC_BF16 = 0, 1
-ATTN_DELTA_MATCHED, ATTN_DELTA_STALE = 0, 1
+ATTN_DELTA_MATCHED, ATTN_DELTA_STALE, ATTN_DELTA_CONSISTENT_DO = 0, 1, 2
 ATTN_SRC_BF16, ATTN_SRC_FP32 = 0, 1
 ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 

@@ -201,6 +201,15 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
     CHECK(check_ptr(dO_bf16, "dO_bf16")); CHECK(check_ptr(o_bf16, "o_bf16"));
     return launch_stale_delta(s, dO_bf16, o_bf16, delta, st);
   }
+  if (p->delta_mode == ATTN_DELTA_CONSISTENT_DO) {
+    CHECK(check_ptr(o_bf16, "o_bf16"));
+    if (!fp8) {                                       // BF16 operands: dO^ is the BF16 dO itself
+      CHECK(check_ptr(dO.row_codes, "dO.row_codes"));
+      return launch_stale_delta(s, dO.row_codes, o_bf16, delta, st);
+    }
+    CHECK_OPERAND(dO, row, fp8);
+    return launch_consistent_delta(s, dO, o_bf16, delta, st);
+  }
   if (p->delta_mode != ATTN_DELTA_MATCHED) return fail(ATTN_ERR_INVALID_ARG, "delta_mode %d unknown", p->delta_mode);
   CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8); CHECK_OPERAND(dO, row, fp8);
   CHECK(check_ptr(lse, "lse"));

@@ -26,6 +26,7 @@
 // When the qk head dim exceeds 128 the dQ accumulator no longer fits beside S and dP in tensor
 // memory; the dQ columns are then split in tiles of 128 over CTAs that each repeat the S / dP work.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <type_traits>
 
@@ -547,7 +548,56 @@ __global__ void stale_delta_kernel(const __nv_bfloat16* __restrict__ dO, const _
   if (lane == 0) delta[row] = acc;
 }
 
+// Consistent dO (paper Section 3.3): the saved-output shortcut with dO replaced by the FP8 operand
+// the backward matmuls consume, D_i = sum_c dO^_ic O_ic with dO^ = code * 2^(byte - 127) from the
+// row-blocked copy.  One warp per row, four codes per lane and step.
+__global__ void consistent_delta_kernel(const uint8_t* __restrict__ dO_codes, const uint8_t* __restrict__ dO_scales,
+                                        const __nv_bfloat16* __restrict__ o, float* __restrict__ delta, size_t rows,
+                                        int N, int dv) {
+  const size_t row = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const size_t slab = row / N;
+  const int r = static_cast<int>(row % N);
+  const int n_ct = (dv / 32 + 3) / 4;                 // 512-byte scale tiles per 128-row tile
+  const uint8_t* sf = dO_scales + (slab * (N / 128) + r / 128) * n_ct * 512 + sf_tile_offset(r & 127, 0);
+  float acc = 0.f;
+  for (int c = lane * 4; c < dv; c += 128) {
+    const uint32_t codes = *reinterpret_cast<const uint32_t*>(dO_codes + row * dv + c);
+    const int blk = c >> 5;
+    const float sc = __uint_as_float(static_cast<uint32_t>(sf[(blk >> 2) * 512 + (blk & 3)]) << 23);   // 2^(byte-127); 0 for byte 0
+    const uint2 ov = *reinterpret_cast<const uint2*>(o + row * dv + c);
+    const __nv_bfloat162 o01 = *reinterpret_cast<const __nv_bfloat162*>(&ov.x);
+    const __nv_bfloat162 o23 = *reinterpret_cast<const __nv_bfloat162*>(&ov.y);
+    uint32_t h01, h23;                                 // E4M3 -> FP16 is exact
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"(static_cast<uint16_t>(codes & 0xFFFF)));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"(static_cast<uint16_t>(codes >> 16)));
+    const float2 d01 = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+    const float2 d23 = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+    float part = d01.x * __bfloat162float(o01.x);
+    part = fmaf(d01.y, __bfloat162float(o01.y), part);
+    part = fmaf(d23.x, __bfloat162float(o23.x), part);
+    part = fmaf(d23.y, __bfloat162float(o23.y), part);
+    acc = fmaf(part, sc, acc);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) delta[row] = acc;
+}
+
 }  // namespace
+
+attn_status_t launch_consistent_delta(const AttnShape& s, attn_qtensor_t dO, const void* o_bf16, float* delta,
+                                      cudaStream_t stream) {
+  const size_t rows = static_cast<size_t>(s.B) * s.Hq * s.N;
+  const int threads = 256;
+  const size_t blocks = (rows * 32 + threads - 1) / threads;
+  consistent_delta_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+      dO.row_codes, dO.row_scales, static_cast<const __nv_bfloat16*>(o_bf16), delta, rows, s.N, s.dv);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "consistent delta: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
 
 attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream) {

@@ -38,6 +38,8 @@ attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtenso
                                attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream);
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,
                                  cudaStream_t stream);
+attn_status_t launch_consistent_delta(const AttnShape& s, attn_qtensor_t dO, const void* o_bf16, float* delta,
+                                      cudaStream_t stream);
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                             attn_qtensor_t dO, const float* lse, const float* delta, void* dq, float* rowsum,
                             float* rowabs, int* status, cudaStream_t stream);

@@ -150,6 +150,24 @@ def test_stale_mode_changes_only_delta_dq_dk():
     assert rel_fro(to_np(s["rs"]), rs) <= 1e-2
 
 
+def test_consistent_dO_mode():
+    """Consistent dO: the saved-output shortcut with the FP8 dO operand; residual between stale and matched."""
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
+    q, k, v, dO = workloads.make_inputs(w)
+    m = run_all(w, q, k, v, dO, delta_mode=0)
+    s = run_all(w, q, k, v, dO, delta_mode=1)
+    c = run_all(w, q, k, v, dO, delta_mode=2)
+    assert torch.equal(m["o"], c["o"]) and torch.equal(m["lse"], c["lse"]) and torch.equal(m["dv"], c["dv"])
+    qn, kn, vn, dOn = (to_np(x) for x in (q, k, v, dO))
+    D_c = A.emu_delta(qn, kn, vn, dOn, to_np(c["lse"]), w.softmax_scale, w.causal, mode="consistent", o=to_np(c["o"]))
+    assert rel_fro(to_np(c["delta"]), D_c) <= 1e-5
+    dQ, dK, dV, rs, ra = A.emu_backward(qn, kn, vn, dOn, to_np(c["lse"]), to_np(c["delta"]), w.softmax_scale, w.causal)
+    assert rel_fro(to_np(c["dq"]), dQ) <= TOL_GRAD and rel_fro(to_np(c["dk"]), dK) <= TOL_GRAD
+    med = lambda d: np.nanmedian((np.abs(to_np(d["rs"])) / to_np(d["ra"]))[..., 64:])
+    print(f"\nmedian r_pre: stale {med(s):.3e} consistent {med(c):.3e} matched {med(m):.3e}")
+    assert med(s) > med(c) > 100 * med(m)
+
+
 def test_backward_is_reproducible():
     w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
     q, k, v, dO = workloads.make_inputs(w)
