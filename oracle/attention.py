@@ -98,7 +98,9 @@ def ref_backward(q, k, v, dO, scale, causal, return_internals=False):
             dK[b, g] += scale * (dS.T @ Q)
             D[b, h] = delta
             if return_internals:
-                internals[(b, h)] = dict(P=P, dP=dP, dS=dS)
+                # dS_q / dS_k: the cast score gradients the dQ / dK matmuls consume (blocks of 32
+                # keys per row / of 32 query rows per key)
+                internals[(b, h)] = dict(P=P, dP=dP, dS=dS, dS_q=_fq(dS, -1, prec), dS_k=_fq(dS, 0, prec))
     if return_internals:
         return dQ, dK, dV, D, internals
     return dQ, dK, dV, D
@@ -243,7 +245,9 @@ def emu_backward(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", round_out
             dK[b, g] += scale * (_fq(dS, 0, prec).T @ _fq(q[b, h], 0, prec))
             dQ[b, h] = scale * (_fq(dS, -1, prec) @ _fq(k[b, g], 0, prec))
             if return_internals:
-                internals[(b, h)] = dict(P=P, dP=dP, dS=dS)
+                # dS_q / dS_k: the cast score gradients the dQ / dK matmuls consume (blocks of 32
+                # keys per row / of 32 query rows per key)
+                internals[(b, h)] = dict(P=P, dP=dP, dS=dS, dS_q=_fq(dS, -1, prec), dS_k=_fq(dS, 0, prec))
     if round_out and prec != "none":
         dQ, dK, dV = (mxfp8.round_bf16(x) for x in (dQ, dK, dV))
     out = (dQ, dK, dV, rowsum, rowabs)
@@ -281,6 +285,41 @@ def emu_backward_cols(q, k, v, dO, lse, delta, scale, causal, b, g, cols, prec="
         dv += _fq(P, 0, prec).T @ _fq(dO[b, h], 0, prec)
         dk += scale * (_fq(dS, 0, prec).T @ _fq(q[b, h], 0, prec))
     return mxfp8.round_bf16(dk), mxfp8.round_bf16(dv)
+
+
+def postcast_row_sums(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", rows=None, b=0, h=0):
+    """Row sums of the CAST score gradient the dQ matmul consumes, dS'_ij (dS quantised in blocks of
+    32 keys per row): sum_j dS'_ij and sum_j |dS'_ij| for one head (paper Appendix "dS Quantization
+    Residuals", Eq. app_ds_quantization_residuals).  ``lse`` and ``delta`` are that head's [N] vectors."""
+    N = q.shape[2]
+    g = h // (q.shape[1] // k.shape[1])
+    rows = np.arange(N) if rows is None else np.asarray(rows)
+    allc = np.arange(N)
+    P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec), lse, scale, causal, rows, allc)
+    dP = _fq(dO[b, h], -1, prec)[rows] @ _fq(v[b, g], -1, prec).T
+    dS = P * (dP - np.asarray(delta, np.float64)[rows][:, None])
+    dSq = _fq(dS, -1, prec)
+    return dSq.sum(axis=-1), np.abs(dSq).sum(axis=-1)
+
+
+def postcast_residuals(rowsum_pre, rowabs_pre, rowsum_post, rowabs_post):
+    """r_post = |sum dS'| / sum|dS|, r_post_own = |sum dS'| / sum|dS'| and the signed casting offset
+    kappa = (sum dS' - sum dS) / sum|dS| (Eq. app_ds_quantization_residuals, app_ds_signed_increment);
+    NaN where the denominator is zero."""
+    with np.errstate(divide="ignore", invalid="ignore"):
+        r_post = np.where(rowabs_pre > 0, np.abs(rowsum_post) / rowabs_pre, np.nan)
+        r_own = np.where(rowabs_post > 0, np.abs(rowsum_post) / rowabs_post, np.nan)
+        kappa = np.where(rowabs_pre > 0, (rowsum_post - rowsum_pre) / rowabs_pre, np.nan)
+    return r_post, r_own, kappa
+
+
+def key_common_mode(dK):
+    """c_K = || sum_j dK_j ||_2 / ( sum_j ||dK_j||_2^2 )^(1/2) per (batch, KV head) for dK [B,Hkv,N,d]
+    (Eq. app_ds_key_gradient_sum)."""
+    dK = np.asarray(dK, np.float64)
+    num = np.linalg.norm(dK.sum(axis=2), axis=-1)
+    den = np.sqrt((dK ** 2).sum(axis=(2, 3)))
+    return num / den
 
 
 def residual_ratio(rowsum, rowabs):

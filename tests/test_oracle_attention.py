@@ -376,6 +376,39 @@ def test_consistent_dO_residual_identity_and_ordering():
     assert med(rss, ras) > med(rsc, rac) > 100 * med(rsm, ram)
 
 
+def test_postcast_statistics_and_key_common_mode():
+    """Post-cast row sums (Appendix "dS Quantization Residuals"): equal to the pre-cast ones when the
+    cast is the identity; bounded by the E4M3 half-ulp otherwise; and the key-gradient sum identity
+    of Eq. app_ds_gqa_key_sum, which ties sum_j dK_j to the row sums of the cast operand."""
+    q, k, v, dO, scale, causal = _setup_fp8(seed=22)
+    O, LSE = A.emu_forward(q, k, v, scale, causal, exact_stats=True)
+    D = A.emu_delta(q, k, v, dO, LSE, scale, causal, exact_stats=True)
+    dQ, dK, dV, rs, ra, t = A.emu_backward(q, k, v, dO, LSE, D, scale, causal, round_out=False, return_internals=True)
+    G = q.shape[1] // k.shape[1]
+    for (b, h), tt in t.items():
+        ps, pa = A.postcast_row_sums(q, k, v, dO, LSE[b, h], D[b, h], scale, causal, b=b, h=h)
+        assert np.array_equal(ps, tt["dS_q"].sum(-1)) and np.array_equal(pa, np.abs(tt["dS_q"]).sum(-1))
+        # round to nearest with 3 mantissa bits: every element moves by at most 2^-4 of the block maximum
+        assert np.all(np.abs(ps - rs[b, h]) <= 2.0 ** -4 * ra[b, h] + 1e-300)
+        r_post, r_own, kappa = A.postcast_residuals(rs[b, h], ra[b, h], ps, pa)
+        live = ra[b, h] > 0
+        assert np.all(np.abs(kappa[live]) <= 2.0 ** -4)
+        assert np.nanmedian(r_post[64:]) > 10 * np.nanmedian(A.residual_ratio(rs[b, h], ra[b, h])[64:])
+        # identity cast: nothing changes
+        ps0, pa0 = A.postcast_row_sums(q, k, v, dO, LSE[b, h], D[b, h], scale, causal, prec="none", b=b, h=h)
+        _, _, _, rs0, ra0 = A.emu_backward(q, k, v, dO, LSE, D, scale, causal, prec="none")
+        assert np.allclose(ps0, rs0[b, h], atol=1e-15) and np.allclose(pa0, ra0[b, h], rtol=1e-13)
+    # key-gradient sum: sum_j dK_{g,j} = scale * sum_{h in g} sum_i Q^c_{h,i} * (sum_j dS^i_{h,ij})
+    for b in range(q.shape[0]):
+        for g in range(k.shape[1]):
+            want = np.zeros(q.shape[-1])
+            for h in range(g * G, (g + 1) * G):
+                want += scale * (mxfp8.fake_quant(q[b, h], 0) * t[(b, h)]["dS_k"].sum(-1)[:, None]).sum(0)
+            assert np.abs(dK[b, g].sum(0) - want).max() <= 1e-12 * max(1.0, np.abs(want).max())
+    cK = A.key_common_mode(dK)
+    assert cK.shape == dK.shape[:2] and np.all((cK >= 0) & (cK <= np.sqrt(dK.shape[2]) + 1e-9))
+
+
 def test_subset_functions_agree_with_full_pass():
     q, k, v, dO, scale, causal = _setup_fp8(seed=14)
     O, LSE = A.emu_forward(q, k, v, scale, causal)
