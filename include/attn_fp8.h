@@ -184,6 +184,19 @@ attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_q
                                 void* dk_bf16, void* dv_bf16,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* attn_fp8_bwd_dq with the post-cast probe of the paper's Appendix "dS Quantization Residuals"
+ * (Eq. app_ds_quantization_residuals): besides the pre-cast sums it writes, per query row,
+ *   diag_post_rowsum_ds      sum_j dS'_ij     dS' = the cast score gradient the dQ matmul consumes
+ *   diag_post_rowsum_abs_ds  sum_j |dS'_ij|   (code * 2^(scale byte - 127); the BF16 value in BF16 mode)
+ * both [B, Hq, N] FP32.  From the four outputs a caller forms r_pre, r_post, r_post,own and the
+ * signed casting offset kappa.  All four diagnostic pointers are required; dQ is identical to
+ * attn_fp8_bwd_dq's.                                                                          */
+attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                       attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                                       float* diag_rowsum_ds, float* diag_rowsum_abs_ds,
+                                       float* diag_post_rowsum_ds, float* diag_post_rowsum_abs_ds,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* Forward without a workspace argument (the paper has no counterpart; this is a packaging variant
  * of attn_fp8_fwd and computes exactly the same O and LSE).
  *

@@ -98,9 +98,7 @@ def ref_backward(q, k, v, dO, scale, causal, return_internals=False):
             dK[b, g] += scale * (dS.T @ Q)
             D[b, h] = delta
             if return_internals:
-                # dS_q / dS_k: the cast score gradients the dQ / dK matmuls consume (blocks of 32
-                # keys per row / of 32 query rows per key)
-                internals[(b, h)] = dict(P=P, dP=dP, dS=dS, dS_q=_fq(dS, -1, prec), dS_k=_fq(dS, 0, prec))
+                internals[(b, h)] = dict(P=P, dP=dP, dS=dS)
     if return_internals:
         return dQ, dK, dV, D, internals
     return dQ, dK, dV, D

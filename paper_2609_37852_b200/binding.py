@@ -33,7 +33,7 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
-    "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
+    "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
 )
 
@@ -304,6 +304,28 @@ def attn_fp8_bwd_dq(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: 
                                 _ptr(delta), _ptr(dq), _ptr(rs), _ptr(ra), _ptr(workspace), workspace.numel(),
                                 _stream(stream)))
     return dq, rs, ra, workspace
+
+
+_lib.attn_fp8_bwd_dq_postcast.restype = _i32
+_lib.attn_fp8_bwd_dq_postcast.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp,
+                                          _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+
+
+def attn_fp8_bwd_dq_postcast(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dq=None,
+                             workspace=None, stream=None):
+    """dQ plus the pre- and post-cast row statistics of dS.  Returns
+    (dQ, rowsum_dS, rowsum_abs_dS, rowsum_dS_cast, rowsum_abs_dS_cast, workspace)."""
+    dev = lse.device
+    B, N = params.batch, params.seqlen
+    if dq is None:
+        dq = torch.empty((B, params.heads_q, N, params.head_dim_qk), dtype=torch.bfloat16, device=dev)
+    stats = [torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev) for _ in range(4)]
+    workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd_dq_postcast(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),
+                                         _ptr(lse), _ptr(delta), _ptr(dq), *(_ptr(t) for t in stats), _ptr(workspace),
+                                         workspace.numel(), _stream(stream)))
+    return (dq, *stats, workspace)
 
 
 def attn_fp8_bwd_dkdv(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dk=None,

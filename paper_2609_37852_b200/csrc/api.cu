@@ -219,7 +219,8 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
 static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                               attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
                               void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
-                              size_t workspace_bytes, void* stream, bool want_dq, bool want_dkdv) {
+                              size_t workspace_bytes, void* stream, bool want_dq, bool want_dkdv,
+                              float* post_rowsum = nullptr, float* post_rowabs = nullptr) {
   AttnShape s;
   if (want_dq) CHECK(check_params(p, &s, kEntryDq));
   if (want_dkdv) CHECK(check_params(p, &s, kEntryDkdv));
@@ -231,6 +232,8 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
     CHECK(check_ptr(dq_bf16, "dq_bf16"));
     if ((diag_rowsum_ds == nullptr) != (diag_rowsum_abs_ds == nullptr))
       return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
+    if ((post_rowsum == nullptr) != (post_rowabs == nullptr) || (post_rowsum && !diag_rowsum_ds))
+      return fail(ATTN_ERR_INVALID_ARG, "the post-cast outputs come as a pair and need the pre-cast pair as well");
   }
   if (want_dkdv) {
     CHECK_OPERAND(q, col, fp8); CHECK_OPERAND(dO, col, fp8);
@@ -241,7 +244,8 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD), st, &status));
   if (want_dq)
-    CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, status, st));
+    CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, post_rowsum, post_rowabs,
+                        status, st));
   if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));
   return ATTN_OK;
 }
@@ -260,6 +264,17 @@ attn_status_t attn_fp8_bwd_dq(const attn_params_t* p, attn_qtensor_t q, attn_qte
                               size_t workspace_bytes, void* stream) {
   return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, nullptr, nullptr, diag_rowsum_ds, diag_rowsum_abs_ds,
                   workspace, workspace_bytes, stream, true, false);
+}
+
+attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                       attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                                       float* diag_rowsum_ds, float* diag_rowsum_abs_ds, float* diag_post_rowsum_ds,
+                                       float* diag_post_rowsum_abs_ds, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  if (!diag_post_rowsum_ds || !diag_post_rowsum_abs_ds || !diag_rowsum_ds || !diag_rowsum_abs_ds)
+    return fail(ATTN_ERR_INVALID_ARG, "attn_fp8_bwd_dq_postcast needs all four diagnostic outputs");
+  return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, nullptr, nullptr, diag_rowsum_ds, diag_rowsum_abs_ds,
+                  workspace, workspace_bytes, stream, true, false, diag_post_rowsum_ds, diag_post_rowsum_abs_ds);
 }
 
 attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,

@@ -105,7 +105,7 @@ struct QmSmem {
   alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
   alignas(16) uint8_t sf_kc[C::kKcStages][512];
   alignas(16) uint8_t sf_ds[2][512];
-  alignas(16) float red[C::kGroups][2][kTile];   // partial row sums of every column group
+  alignas(16) float red[C::kGroups][4][kTile];   // partial row sums of every column group
   uint64_t q_full;
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
@@ -125,6 +125,8 @@ struct QmParams {
   __nv_bfloat16* dq;
   float* rowsum;
   float* rowabs;
+  float* post_rowsum;       // optional: row sums of the CAST score gradient (the dQ operand) and of its magnitude
+  float* post_rowabs;
   int* status;
   int N, Hq, Hkv, dqk, dv, causal;
   float scale, scale_log2;
@@ -353,6 +355,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float f_lo = fmaf(-lse2_lo, kLn2, 1.0f);   // 2^-lo to first order (|lo| < 1e-5)
     const float fD = f_lo * D;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
+    // kDQ, on request: sum dS', sum |dS'| of the cast values, kept in shared memory so that the
+    // common path carries no extra registers
+    const bool want_post = kDQ && p.post_rowsum != nullptr;
+    if (want_post) {
+      sm.red[grp][2][row] = 0.f;
+      sm.red[grp][3][row] = 0.f;
+    }
     bool ok = true;
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
@@ -414,6 +423,34 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
 #pragma unroll
           for (int i = 0; i < 8 * kEB; ++i) words[i] = cvt_bf16x2(ds[(2 * i) & 31], ds[(2 * i + 1) & 31]);
         }
+        if (__builtin_expect(want_post, 0)) {
+          // decode what the tensor cores will read: code * 2^(byte - 127), or the BF16 value
+          float ps = 0.f, pa = 0.f;
+          if (kFp8) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              uint32_t h01, h23;                       // E4M3 -> FP16 is exact
+              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"(static_cast<uint16_t>(words[i] & 0xFFFF)));
+              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"(static_cast<uint16_t>(words[i] >> 16)));
+              const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+              const float2 bq = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+              ps += (a.x + a.y) + (bq.x + bq.y);
+              pa += (fabsf(a.x) + fabsf(a.y)) + (fabsf(bq.x) + fabsf(bq.y));
+            }
+            const float sc = __uint_as_float(byte << 23);     // 2^(byte - 127); an all-zero block has byte 0 and sums 0
+            ps *= sc;
+            pa *= sc;
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8 * kEB; ++i) {
+              const float lo = __uint_as_float(words[i] << 16), hi = __uint_as_float(words[i] & 0xFFFF0000u);
+              ps += lo + hi;
+              pa += fabsf(lo) + fabsf(hi);
+            }
+          }
+          sm.red[grp][2][row] += ps;
+          sm.red[grp][3][row] += pa;
+        }
         if (t >= 2) {
           // the dQ MMAs of tile t-2 have consumed this buffer's operand and scale bytes
           ok = mbar_wait(&sm.ds_free[buf], ((t - 2) >> 1) & 1, abort_flag);
@@ -441,6 +478,12 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       } else if (p.rowsum && r_tile == 0) {
         p.rowsum[grow] = acc0;
         p.rowabs[grow] = acc1;
+        if (p.post_rowsum) {
+          float post0 = 0.f, post1 = 0.f;
+          for (int i = 0; i < kGroups; ++i) { post0 += sm.red[i][2][row]; post1 += sm.red[i][3][row]; }
+          p.post_rowsum[grow] = post0;
+          p.post_rowabs[grow] = post1;
+        }
       }
     }
     if (kDQ && ok) {
@@ -475,7 +518,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
 template <class C>
 attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                               const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
-                              float* rowabs, int* status, cudaStream_t stream) {
+                              float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
   constexpr bool kDQ = C::kDQ;
   static_assert(sizeof(QmSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
@@ -497,7 +540,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.q_sf = q.row_scales; p.dO_sf = dO.row_scales; p.k_sf = k.row_scales; p.v_sf = v.row_scales;
   p.kc_sf = kDQ ? k.col_scales : nullptr;
   p.lse = lse; p.delta_in = delta_in; p.delta_out = delta_out;
-  p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.status = status;
+  p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   const size_t smem = sizeof(QmSmem<C>) + 1024;
@@ -514,12 +557,12 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
 template <bool kDQ>
 attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
-                            float* rowabs, int* status, cudaStream_t stream) {
+                            float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
   const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.eb + 127) / 128;
 #define ATTN_QM_CASE(EB, CQ, CV)                                                                              \
   if (s.eb == EB && cq == CQ && cv == CV)                                                                     \
     return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
-                                                  status, stream);
+                                                  post_rowsum, post_rowabs, status, stream);
   ATTN_QM_CASE(1, 1, 1)
   ATTN_QM_CASE(1, 2, 1)
   ATTN_QM_CASE(1, 2, 2)
@@ -601,13 +644,13 @@ attn_status_t launch_consistent_delta(const AttnShape& s, attn_qtensor_t dO, con
 
 attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream) {
-  return launch_qmajor<false>(s, q, k, v, dO, lse, nullptr, delta, nullptr, nullptr, nullptr, status, stream);
+  return launch_qmajor<false>(s, q, k, v, dO, lse, nullptr, delta, nullptr, nullptr, nullptr, nullptr, nullptr, status, stream);
 }
 
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
-                            const float* lse, const float* delta, void* dq, float* rowsum, float* rowabs, int* status,
-                            cudaStream_t stream) {
-  return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, status, stream);
+                            const float* lse, const float* delta, void* dq, float* rowsum, float* rowabs,
+                            float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
+  return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, post_rowsum, post_rowabs, status, stream);
 }
 
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,

@@ -168,6 +168,39 @@ def test_consistent_dO_mode():
     assert med(s) > med(c) > 100 * med(m)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_postcast_statistics(bf16):
+    """Post-cast probe: row sums of the cast score gradient the dQ matmul consumes."""
+    from paper_2609_37852_b200 import binding
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
+    q, k, v, dO = workloads.make_inputs(w)
+    prec = "bf16" if bf16 else "mxfp8"
+    params = binding.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                                w.softmax_scale, precision=binding.ATTN_PREC_BF16 if bf16 else binding.ATTN_PREC_MXFP8)
+    prep = binding.attn_fp8_prepare_bf16 if bf16 else binding.attn_fp8_quantize
+    qq, kq, vq, dOq = (prep(x.cuda()) for x in (q, k, v, dO))
+    o, lse, ws = binding.attn_fp8_fwd(params, qq, kq, vq)
+    delta, ws = binding.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
+    dq0, rs0, ra0, ws = binding.attn_fp8_bwd_dq(params, qq, kq, vq, dOq, lse, delta, diagnostics=True, workspace=ws)
+    dq, rs, ra, ps, pa, ws = binding.attn_fp8_bwd_dq_postcast(params, qq, kq, vq, dOq, lse, delta, workspace=ws)
+    binding.attn_fp8_read_status(ws)
+    assert torch.equal(dq, dq0) and torch.equal(rs, rs0) and torch.equal(ra, ra0)
+    qn, kn, vn, dOn = (to_np(x) for x in (q, k, v, dO))
+    for h in range(w.heads_q):
+        ps_or, pa_or = A.postcast_row_sums(qn, kn, vn, dOn, to_np(lse[0, h]), to_np(delta[0, h]), w.softmax_scale,
+                                           w.causal, prec=prec, b=0, h=h)
+        assert rel_fro(to_np(pa[0, h]), pa_or) <= 1e-3
+        # a code that rounds the other way moves a row sum by one E4M3 step of one element
+        assert np.abs(to_np(ps[0, h]) - ps_or).max() <= 2e-2 * np.abs(pa_or).max()
+        assert rel_fro(to_np(ps[0, h]), ps_or) <= (0.2 if bf16 else 5e-2)
+    r_post, r_own, kappa = A.postcast_residuals(to_np(rs), to_np(ra), to_np(ps), to_np(pa))
+    r_pre = A.residual_ratio(to_np(rs), to_np(ra))
+    print(f"\n[{prec}] median r_pre {np.nanmedian(r_pre[..., 64:]):.2e} r_post {np.nanmedian(r_post[..., 64:]):.2e} "
+          f"r_post_own {np.nanmedian(r_own[..., 64:]):.2e} mean kappa {np.nanmean(kappa[..., 64:]):.2e}")
+    assert np.nanmedian(r_post[..., 64:]) > 10 * np.nanmedian(r_pre[..., 64:])
+    assert np.nanmax(np.abs(kappa)) <= 2.0 ** -4
+
+
 def test_backward_is_reproducible():
     w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
     q, k, v, dO = workloads.make_inputs(w)
