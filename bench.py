@@ -371,6 +371,24 @@ def main():
         "roofline": roofline,
     }
 
+    # ---- row-sum residual of dS (the metric's second half), from one untimed instrumented pass -------
+    if rank == 0:
+        _, rs, ra, ps, pa, _ = B.attn_fp8_bwd_dq_postcast(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
+        B.attn_fp8_read_status(ws)
+        rs, ra, ps = (t[..., 64:].double().flatten() for t in (rs, ra, ps))          # rows i >= 64, as in the paper
+        live = ra > 0
+        r_pre = (rs[live].abs() / ra[live])
+        r_post = (ps[live].abs() / ra[live])
+        kappa = ((ps[live] - rs[live]) / ra[live])
+        dkf = dk.double()
+        c_k = (dkf.sum(dim=2).norm(dim=-1) / dkf.pow(2).sum(dim=(2, 3)).sqrt()).flatten()
+        line["rowsum_ds_residual"] = {
+            "rows": "query rows i >= 64 with a non-zero sum_j |dS_ij|", "delta_mode": "matched",
+            "r_pre_median": float(r_pre.median()), "r_pre_p99": float(r_pre.quantile(0.99)) if r_pre.numel() < 16_000_000 else None,
+            "r_post_median": float(r_post.median()), "kappa_mean": float(kappa.mean()),
+            "key_common_mode_median": float(c_k.median()),
+        }
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_tokens = 2048
         small = w.scaled(heads_q=w.heads_q // w.heads_kv, heads_kv=1, seqlen=sample_tokens)
