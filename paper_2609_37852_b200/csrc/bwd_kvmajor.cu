@@ -449,6 +449,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       float amax_p = 0.f, max_s = 0.f;
       const float* s_lse = &st.neg_lse2[st0];
       const float* s_delta = &st.delta[st0];
+      // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
+      // bound by instruction issue, not by a pipe
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), minus1 = make_float2(-1.f, -1.f);
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
@@ -456,20 +459,26 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           const float4 l4 = lds_f4(&s_lse[c4]);
           float4 d4 = make_float4(0.f, 0.f, 0.f, 0.f);
           if (kHasDk) d4 = lds_f4(&s_delta[c4]);
-          const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
-          const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
+          for (int e = 0; e < 4; e += 2) {
             const int c = c4 + e;
-            float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, lv[e]);
-            if (kDiag && (row > col0 + c)) x = -INFINITY;      // key after the query
-            const float pv = ex2_approx(x);
-            sr[c] = __float_as_uint(pv);
-            amax_p = fmaxf(amax_p, pv);
+            const float2 lv2 = e == 0 ? make_float2(l4.x, l4.y) : make_float2(l4.z, l4.w);
+            float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, lv2);
+            if (kDiag) {                                      // key after the query
+              if (row > col0 + c) x2.x = -INFINITY;
+              if (row > col0 + c + 1) x2.y = -INFINITY;
+            }
+            const float2 p2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
+            sr[c] = __float_as_uint(p2.x);
+            sr[c + 1] = __float_as_uint(p2.y);
+            amax_p = fmaxf(amax_p, fmaxf(p2.x, p2.y));
             if (kHasDk) {
-              const float dsv = pv * (__uint_as_float(dpr[c]) - dv4[e]);
-              dpr[c] = __float_as_uint(dsv);
-              max_s = fmaxf(max_s, fabsf(dsv));
+              const float2 dv2 = e == 0 ? make_float2(d4.x, d4.y) : make_float2(d4.z, d4.w);
+              const float2 t2 = __ffma2_rn(dv2, minus1, make_float2(__uint_as_float(dpr[c]), __uint_as_float(dpr[c + 1])));
+              const float2 ds2 = __fmul2_rn(p2, t2);          // dS = P (dP - D)
+              dpr[c] = __float_as_uint(ds2.x);
+              dpr[c + 1] = __float_as_uint(ds2.y);
+              max_s = fmaxf(max_s, fmaxf(fabsf(ds2.x), fabsf(ds2.y)));
             }
           }
         }
@@ -490,10 +499,13 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       uint32_t words[8 * kEB];
       if (kHasDv) {
         if (kFp8) {
+          const float2 inv2 = make_float2(inv_p, inv_p);
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            words[i] = cvt_e4m3x4(__uint_as_float(sr[4 * i]) * inv_p, __uint_as_float(sr[4 * i + 1]) * inv_p,
-                                  __uint_as_float(sr[4 * i + 2]) * inv_p, __uint_as_float(sr[4 * i + 3]) * inv_p);
+          for (int i = 0; i < 8; ++i) {
+            const float2 a = __fmul2_rn(make_float2(__uint_as_float(sr[4 * i]), __uint_as_float(sr[4 * i + 1])), inv2);
+            const float2 bq = __fmul2_rn(make_float2(__uint_as_float(sr[4 * i + 2]), __uint_as_float(sr[4 * i + 3])), inv2);
+            words[i] = cvt_e4m3x4(a.x, a.y, bq.x, bq.y);
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 8 * kEB; ++i)
@@ -504,10 +516,13 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       }
       if (kHasDk) {
         if (kFp8) {
+          const float2 inv2 = make_float2(inv_s, inv_s);
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            words[i] = cvt_e4m3x4(__uint_as_float(dpr[4 * i]) * inv_s, __uint_as_float(dpr[4 * i + 1]) * inv_s,
-                                  __uint_as_float(dpr[4 * i + 2]) * inv_s, __uint_as_float(dpr[4 * i + 3]) * inv_s);
+          for (int i = 0; i < 8; ++i) {
+            const float2 a = __fmul2_rn(make_float2(__uint_as_float(dpr[4 * i]), __uint_as_float(dpr[4 * i + 1])), inv2);
+            const float2 bq = __fmul2_rn(make_float2(__uint_as_float(dpr[4 * i + 2]), __uint_as_float(dpr[4 * i + 3])), inv2);
+            words[i] = cvt_e4m3x4(a.x, a.y, bq.x, bq.y);
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 8 * kEB; ++i)

@@ -381,28 +381,35 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // before the diagonal tile)
       const int col0 = t * kStep - qt * kTile + 32 * grp;
       float ds[32];
-      float part = 0.f;
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
       // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
       // a loop without it
+      // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nl2 = make_float2(-lse2, -lse2);
+      const float2 fl2 = make_float2(f_lo, f_lo), nfd2 = make_float2(-fD, -fD);
+      float2 part2 = make_float2(0.f, 0.f);
       auto body = [&](auto diag_tag, auto stats_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
         constexpr bool kStats = decltype(stats_tag)::value;      // pre-cast row statistics requested
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          float x = fmaf(__uint_as_float(sr[c]), p.scale_log2, -lse2);
-          if (kDiag && (col0 + c > row)) x = -INFINITY;
-          const float pr = ex2_approx(x);
-          const float dp = __uint_as_float(dpr[c]);
+        for (int c = 0; c < 32; c += 2) {
+          float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nl2);
+          if (kDiag) {
+            if (col0 + c > row) x2.x = -INFINITY;
+            if (col0 + c + 1 > row) x2.y = -INFINITY;
+          }
+          const float2 pr2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
+          const float2 dp2 = make_float2(__uint_as_float(dpr[c]), __uint_as_float(dpr[c + 1]));
           if (kDQ) {
-            const float d = pr * fmaf(dp, f_lo, -fD);
-            ds[c] = d;
+            const float2 d2 = __fmul2_rn(pr2, __ffma2_rn(dp2, fl2, nfd2));
+            ds[c] = d2.x;
+            ds[c + 1] = d2.y;
             if (kStats) {
-              acc0 += d;
-              acc1 += fabsf(d);
+              acc0 += d2.x + d2.y;
+              acc1 += fabsf(d2.x) + fabsf(d2.y);
             }
           } else {
-            part = fmaf(pr, dp, part);
+            part2 = __ffma2_rn(pr2, dp2, part2);
           }
         }
       };
@@ -413,7 +420,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (diag) body(std::true_type{}, std::false_type{}); else body(std::false_type{}, std::false_type{});
       }
       if (!kDQ) {
-        acc0 = fmaf(part, f_lo, acc0);
+        acc0 = fmaf(part2.x + part2.y, f_lo, acc0);
       } else {
         uint32_t words[8 * kEB];
         uint32_t byte = 0;

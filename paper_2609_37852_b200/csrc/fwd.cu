@@ -388,17 +388,19 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           float inv;
           block_scale_finite(ex2_approx(fmaf(mxb[bk], p.scale_log2, neg_m)), bytes[bk], inv);
           const float neg_me = neg_m - static_cast<float>(static_cast<int>(bytes[bk]) - 127);
-          float bs0 = 0.f, bs1 = 0.f;                  // two short chains for the block sum
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nme2 = make_float2(neg_me, neg_me);
+          float2 bs01 = make_float2(0.f, 0.f), bs23 = make_float2(0.f, 0.f);   // two chains of pairs for the block sum
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float t0 = ex2_approx(fmaf(x[4 * i], p.scale_log2, neg_me));
-            const float t1 = ex2_approx(fmaf(x[4 * i + 1], p.scale_log2, neg_me));
-            const float t2 = ex2_approx(fmaf(x[4 * i + 2], p.scale_log2, neg_me));
-            const float t3 = ex2_approx(fmaf(x[4 * i + 3], p.scale_log2, neg_me));
-            bs0 += t0 + t2;
-            bs1 += t1 + t3;
-            words[bk][i] = cvt_e4m3x4(t0, t1, t2, t3);
+            const float2 a = __ffma2_rn(make_float2(x[4 * i], x[4 * i + 1]), sc2, nme2);
+            const float2 c = __ffma2_rn(make_float2(x[4 * i + 2], x[4 * i + 3]), sc2, nme2);
+            const float2 t01 = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+            const float2 t23 = make_float2(ex2_approx(c.x), ex2_approx(c.y));
+            bs01 = __fadd2_rn(bs01, t01);
+            bs23 = __fadd2_rn(bs23, t23);
+            words[bk][i] = cvt_e4m3x4(t01.x, t01.y, t23.x, t23.y);
           }
+          const float bs0 = bs01.x + bs01.y, bs1 = bs23.x + bs23.y;
           l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
         } else {
           float bs0 = 0.f, bs1 = 0.f;

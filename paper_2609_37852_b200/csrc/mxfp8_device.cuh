@@ -48,9 +48,13 @@ __device__ __forceinline__ uint32_t quantize_block32(const float* x, uint32_t* w
   uint32_t byte;
   float inv;
   block_scale_finite(amax, byte, inv);
+  const float2 inv2 = make_float2(inv, inv);
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-    words[i] = sm100::cvt_e4m3x4(x[4 * i] * inv, x[4 * i + 1] * inv, x[4 * i + 2] * inv, x[4 * i + 3] * inv);
+  for (int i = 0; i < 8; ++i) {
+    const float2 a = __fmul2_rn(make_float2(x[4 * i], x[4 * i + 1]), inv2);
+    const float2 b = __fmul2_rn(make_float2(x[4 * i + 2], x[4 * i + 3]), inv2);
+    words[i] = sm100::cvt_e4m3x4(a.x, a.y, b.x, b.y);
+  }
   return byte;
 }
 
