@@ -1,0 +1,142 @@
+"""Edge cases of the CUDA path: smallest shapes, head-group extremes, batches, argument errors on the device."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as A
+from oracle import mxfp8
+from paper_2609_37852_b200 import workloads
+from tests.util import rel_fro, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_pass(w, tensors, bf16=False):
+    from paper_2609_37852_b200 import binding as B
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                          w.softmax_scale, precision=B.ATTN_PREC_BF16 if bf16 else B.ATTN_PREC_MXFP8)
+    prep = B.attn_fp8_prepare_bf16 if bf16 else B.attn_fp8_quantize
+    qq, kq, vq, dOq = (prep(x.cuda()) for x in tensors)
+    o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
+    delta, ws = B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
+    dq, dk, dv, rs, ra, ws = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, diagnostics=True, workspace=ws)
+    B.attn_fp8_read_status(ws)
+    return dict(o=o, lse=lse, delta=delta, dq=dq, dk=dk, dv=dv, rs=rs, ra=ra)
+
+
+def _check(w, tensors, got, prec="mxfp8"):
+    qn, kn, vn, dOn = (to_np(x) for x in tensors)
+    O, LSE = A.emu_forward(qn, kn, vn, w.softmax_scale, w.causal, prec=prec)
+    assert rel_fro(to_np(got["o"]), O) <= 2e-3
+    assert rel_fro(to_np(got["lse"]), LSE) <= 2e-3
+    lse, delta = to_np(got["lse"]), to_np(got["delta"])
+    D = A.emu_delta(qn, kn, vn, dOn, lse, w.softmax_scale, w.causal, prec=prec)
+    assert rel_fro(delta, D) <= 1e-4
+    dQ, dK, dV, rs, ra = A.emu_backward(qn, kn, vn, dOn, lse, delta, w.softmax_scale, w.causal, prec=prec)
+    assert rel_fro(to_np(got["dq"]), dQ) <= 5e-3
+    assert rel_fro(to_np(got["dk"]), dK) <= 5e-3
+    assert rel_fro(to_np(got["dv"]), dV) <= 5e-3
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", dict(seqlen=128)),                                         # one tile, non-causal, d = 64
+    ("tiny", dict(seqlen=128, causal=True)),                            # one (diagonal) tile
+    ("gqa4k", dict(batch=1, heads_q=1, heads_kv=1, seqlen=128)),        # one tile, d = 128
+    ("gqa4k", dict(batch=1, heads_q=2, heads_kv=2, seqlen=256, causal=False)),   # non-causal at d = 128, one head per group
+    ("gqa4k", dict(batch=3, heads_q=8, heads_kv=1, seqlen=256)),        # batch of 3, one KV head for eight query heads
+    ("gqa8k_outlier", dict(batch=2, heads_q=2, heads_kv=1, seqlen=384)),
+])
+def test_small_and_extreme_shapes(name, kw):
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    tensors = workloads.make_inputs(w)
+    _check(w, tensors, _full_pass(w, tensors))
+
+
+def test_first_row_sees_one_key():
+    """Causal row 0 attends to key 0 only: P = 1 up to the rounding of LSE, so dS_0 and dQ_0 vanish
+    (to FP32 rounding level), and O_0 is V^c_0 times the ratio of the cast probability to the exact one."""
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=2, heads_kv=1, seqlen=256)
+    tensors = workloads.make_inputs(w)
+    got = _full_pass(w, tensors)
+    qn, kn, vn = (to_np(x) for x in tensors[:3])
+    O0, _ = A.emu_forward(qn, kn, vn, w.softmax_scale, w.causal, rows=[0])
+    assert np.abs(to_np(got["o"][0, :, 0]) - O0[0, :, 0]).max() <= 2.0 ** -7 * np.abs(O0).max()
+    v_c = mxfp8.fake_quant(vn[0, 0], 0)                                 # blocks along tokens
+    ratio = to_np(got["o"][0, 0, 0]) / np.where(v_c[0] == 0, 1.0, v_c[0])
+    assert np.all(np.abs(ratio[v_c[0] != 0] - 1.0) <= 2.0 ** -4 + 2.0 ** -7)      # one E4M3 half-ulp and the BF16 store
+    assert float(got["dq"][0, :, 0].float().abs().max()) <= 1e-5 * float(got["dq"].float().abs().max())
+    assert float(got["rs"][0, :, 0].abs().max()) <= 1e-6 * float(got["ra"].abs().max())
+
+
+def test_zero_output_gradient_gives_zero_gradients():
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=2, heads_kv=1, seqlen=256)
+    q, k, v, dO = workloads.make_inputs(w)
+    got = _full_pass(w, (q, k, v, torch.zeros_like(dO)))
+    for key in ("delta", "dq", "dk", "dv", "rs", "ra"):
+        assert float(got[key].float().abs().max()) == 0.0, key
+
+
+def test_argument_errors_on_the_device():
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=2, heads_kv=1, seqlen=256)
+    q, k, v, dO = (x.cuda() for x in workloads.make_inputs(w))
+    qq, kq, vq = (B.attn_fp8_quantize(x) for x in (q, k, v))
+    ok = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, 128, 128, True, w.softmax_scale)
+    # workspace too small
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_fwd(ok, qq, kq, vq, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
+    # missing orientation: the forward needs the column copy of V
+    v_rows_only = B.attn_fp8_quantize(v, want_col=False)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_fwd(ok, qq, kq, v_rows_only)
+    assert e.value.status == 1 and "v.col_codes" in str(e.value)
+    # unsupported head dims, unknown precision, unknown delta mode
+    for bad, status in ((B.AttnParams(1, 256, 2, 1, 96, 96, True, 0.1), 2),
+                        (B.AttnParams(1, 256, 2, 1, 128, 128, True, 0.1, precision=7), 1),
+                        (B.AttnParams(1, 200, 2, 1, 128, 128, True, 0.1), 2)):
+        with pytest.raises(B.AttnFp8Error) as e:
+            B.attn_fp8_fwd(bad, qq, kq, vq)
+        assert e.value.status == status
+    o, lse, ws = B.attn_fp8_fwd(ok, qq, kq, vq)
+    dOq = B.attn_fp8_quantize(dO)
+    bad_mode = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, 128, 128, True, w.softmax_scale, delta_mode=9)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_bwd_delta(bad_mode, qq, kq, vq, dOq, lse)
+    assert e.value.status == 1
+    # misaligned output pointer
+    o_mis = torch.empty(o.numel() + 8, dtype=torch.bfloat16, device="cuda")[1:1 + o.numel()].view_as(o)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_fwd(ok, qq, kq, vq, o=o_mis)
+    assert e.value.status == 3
+    # the context is still usable
+    o2, lse2, ws = B.attn_fp8_fwd(ok, qq, kq, vq)
+    B.attn_fp8_read_status(ws)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_prepare_bf16_is_an_exact_rounding_and_transpose(dtype):
+    from paper_2609_37852_b200 import binding as B
+    g = torch.Generator().manual_seed(5)
+    x = torch.randn((2, 3, 256, 128), generator=g).to(dtype).cuda()
+    t = B.attn_fp8_prepare_bf16(x)
+    want = x.to(torch.bfloat16)
+    assert torch.equal(t.row_codes, want)
+    assert torch.equal(t.col_codes, want.transpose(2, 3).contiguous())
+
+
+@pytest.mark.parametrize("d", [192, 256])
+def test_quantize_wide_heads_bit_exact(d):
+    """Two 512-byte scale tiles per 128-row tile in both orientations."""
+    from paper_2609_37852_b200 import binding as B
+    g = torch.Generator().manual_seed(d)
+    x = (torch.randn((1, 2, 256, d), generator=g) * torch.exp2(torch.randint(-6, 6, (1, 2, 256, 1), generator=g).float())
+         ).to(torch.bfloat16)
+    t = B.attn_fp8_quantize(x.cuda())
+    xn = to_np(x)
+    for axis, codes, scales, rows, cols in ((-1, t.row_codes, t.row_scales, 256, d), (-2, t.col_codes, t.col_scales, d, 256)):
+        c_or, e_or = mxfp8.quantize(xn if axis == -1 else np.swapaxes(xn, -1, -2), axis=-1)
+        assert np.array_equal(codes.cpu().numpy(), c_or)
+        got_e = B.unpack_scales(scales, 1, 2, rows, cols).cpu().numpy()
+        assert np.array_equal(got_e, e_or)
