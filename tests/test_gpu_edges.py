@@ -76,6 +76,40 @@ def test_zero_output_gradient_gives_zero_gradients():
         assert float(got[key].float().abs().max()) == 0.0, key
 
 
+@pytest.mark.parametrize("name,kw,bf16", [
+    ("gqa4k", dict(batch=2, heads_q=4, heads_kv=2, seqlen=384), False),
+    ("gqa4k", dict(batch=1, heads_q=2, heads_kv=1, seqlen=256), True),
+    ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=256), False),
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=256), False),
+])
+def test_every_output_element_is_written(name, kw, bf16):
+    """Outputs pre-filled with NaN: a region no CTA writes would survive the call."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    tensors = [x.cuda() for x in workloads.make_inputs(w)]
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                          w.softmax_scale, precision=B.ATTN_PREC_BF16 if bf16 else B.ATTN_PREC_MXFP8)
+    prep = B.attn_fp8_prepare_bf16 if bf16 else B.attn_fp8_quantize
+    qq, kq, vq, dOq = (prep(x) for x in tensors)
+    nan = lambda shape, dt: torch.full(shape, float("nan"), dtype=dt, device="cuda")
+    Bn, Hq, Hkv, N = w.batch, w.heads_q, w.heads_kv, w.seqlen
+    o, lse = nan((Bn, Hq, N, w.head_dim_v), torch.bfloat16), nan((Bn, Hq, N), torch.float32)
+    _, _, ws = B.attn_fp8_fwd(params, qq, kq, vq, o=o, lse=lse)
+    delta = nan((Bn, Hq, N), torch.float32)
+    B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, delta=delta, workspace=ws)
+    dq, dk, dv = (nan((Bn, h, N, d), torch.bfloat16) for h, d in ((Hq, w.head_dim_qk), (Hkv, w.head_dim_qk), (Hkv, w.head_dim_v)))
+    stats = [nan((Bn, Hq, N), torch.float32) for _ in range(4)]
+    B.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, dk=dk, dv=dv, workspace=ws)
+    c = params.c_struct()
+    import ctypes
+    B._check(B._lib.attn_fp8_bwd_dq_postcast(ctypes.byref(c), qq.c_struct(), kq.c_struct(), vq.c_struct(), dOq.c_struct(),
+                                             B._ptr(lse), B._ptr(delta), B._ptr(dq), *(B._ptr(t) for t in stats),
+                                             B._ptr(ws), ws.numel(), B._stream(None)))
+    B.attn_fp8_read_status(ws)
+    for nm, t in dict(o=o, lse=lse, delta=delta, dq=dq, dk=dk, dv=dv, rs=stats[0], ra=stats[1], ps=stats[2], pa=stats[3]).items():
+        assert not torch.isnan(t.float()).any(), nm
+
+
 def test_argument_errors_on_the_device():
     from paper_2609_37852_b200 import binding as B
     w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=2, heads_kv=1, seqlen=256)
