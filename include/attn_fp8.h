@@ -118,6 +118,22 @@ size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols);
 attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
                                 int32_t d, attn_qtensor_t out, void* stream);
 
+/* The quantiser with the paper's operand producer fused in front (Appendix "Operands, Scaling, and
+ * Accumulation"), for callers that hold q / k BEFORE rotary embedding, scale folding or key centering:
+ *   1. rotary embedding, if rope_cos / rope_sin (FP32 [N, d/2], device) are given: channel c < d/2 is
+ *      paired with c + d/2;  r1 = fma(x1, cos, -fl32(x2 sin)),  r2 = fma(x2, cos, fl32(x1 sin)) in FP32,
+ *      rotated channels rounded to BF16;
+ *   2. key centering, if `mean` (FP32 [B, H, d], device) is given: the mean over the N tokens of the
+ *      values of step 1, per (batch, head, channel), is WRITTEN to `mean` (exact sum, correctly rounded
+ *      quotient) and subtracted in FP32; needs a BF16 source;
+ *   3. multiplication by `scale` in FP32 when scale != 1 (tau = d^-1/2 folded into Q: the attention
+ *      calls then take softmax_scale = 1);
+ *   4. attn_fp8_quantize of the result.
+ * Bitwise reproducible.  Other arguments and errors as attn_fp8_quantize.                       */
+attn_status_t attn_fp8_quantize_fused(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
+                                      int32_t d, const float* rope_cos, const float* rope_sin, float scale,
+                                      float* mean, attn_qtensor_t out, void* stream);
+
 /* Operand preparation for BF16 mode: writes the BF16 rounding of `src` to out.row_codes
  * ([B, H, N, d]) and its transpose to out.col_codes ([B, H, d, N]); an orientation whose pointer
  * is NULL is skipped, the scale pointers are ignored.  A caller whose source already is BF16 may

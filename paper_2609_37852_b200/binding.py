@@ -32,7 +32,7 @@ ATTN_SRC_BF16, ATTN_SRC_FP32 = 0, 1
 ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
+    "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
 )
@@ -184,6 +184,38 @@ def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool =
         raise ValueError("out was allocated for another shape")
     _check(_lib.attn_fp8_quantize(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
     return out
+
+
+_lib.attn_fp8_quantize_fused.restype = _i32
+_lib.attn_fp8_quantize_fused.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, ctypes.c_float, _vp, _QTensor, _vp]
+
+
+def attn_fp8_quantize_fused(src: torch.Tensor, rope_cos: Optional[torch.Tensor] = None,
+                            rope_sin: Optional[torch.Tensor] = None, scale: float = 1.0, center: bool = False,
+                            want_row: bool = True, want_col: bool = True, stream=None):
+    """Quantiser with the producer fused in front: optional rotary embedding (FP32 tables [N, d/2]),
+    optional key centering, optional FP32 scale.  Returns (QTensor, mean [B, H, d] fp32 or None)."""
+    if not src.is_cuda or not src.is_contiguous() or src.dim() != 4:
+        raise ValueError("src must be a contiguous CUDA tensor [B, H, N, d]")
+    if src.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("src must be bfloat16 or float32")
+    dt = ATTN_SRC_BF16 if src.dtype == torch.bfloat16 else ATTN_SRC_FP32
+    B, H, N, d = src.shape
+    out = QTensor(shape=(B, H, N, d))
+    u8 = dict(dtype=torch.uint8, device=src.device)
+    if want_row:
+        out.row_codes = torch.empty((B, H, N, d), **u8)
+        out.row_scales = torch.empty(attn_fp8_scale_bytes(B, H, N, d), **u8)
+    if want_col:
+        out.col_codes = torch.empty((B, H, d, N), **u8)
+        out.col_scales = torch.empty(attn_fp8_scale_bytes(B, H, d, N), **u8)
+    mean = torch.empty((B, H, d), dtype=torch.float32, device=src.device) if center else None
+    for t in (rope_cos, rope_sin):
+        if t is not None and (t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != (N, d // 2)):
+            raise ValueError("rotary tables must be contiguous float32 [N, d/2]")
+    _check(_lib.attn_fp8_quantize_fused(_ptr(src), dt, B, H, N, d, _ptr(rope_cos), _ptr(rope_sin), float(scale),
+                                        _ptr(mean), out.c_struct(), _stream(stream)))
+    return out, mean
 
 
 def attn_fp8_prepare_bf16(src: torch.Tensor, want_row: bool = True, want_col: bool = True, stream=None,

@@ -151,6 +151,33 @@ attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, i
   return launch_quantize(src, src_dtype, B, H, N, d, out, static_cast<cudaStream_t>(stream));
 }
 
+attn_status_t attn_fp8_quantize_fused(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
+                                      const float* rope_cos, const float* rope_sin, float scale, float* mean,
+                                      attn_qtensor_t out, void* stream) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return fail(ATTN_ERR_INVALID_ARG, "sizes must be positive");
+  if (src_dtype != ATTN_SRC_BF16 && src_dtype != ATTN_SRC_FP32)
+    return fail(ATTN_ERR_INVALID_ARG, "src_dtype %d is neither BF16 nor FP32", src_dtype);
+  if (N % 128 || d % 32 || d > 256)
+    return fail(ATTN_ERR_UNSUPPORTED, "quantize needs N %% 128 == 0 and d %% 32 == 0, d <= 256 (N=%d d=%d)", N, d);
+  if ((rope_cos == nullptr) != (rope_sin == nullptr))
+    return fail(ATTN_ERR_INVALID_ARG, "rope_cos and rope_sin must be given together");
+  if (!(scale > 0.f) || !(scale < 3.0e38f)) return fail(ATTN_ERR_INVALID_ARG, "scale must be positive and finite");
+  if (mean != nullptr && src_dtype != ATTN_SRC_BF16)
+    return fail(ATTN_ERR_UNSUPPORTED, "key centering needs a BF16 source (the mean is an exact sum of BF16 terms)");
+  CHECK(check_ptr(src, "src"));
+  if (rope_cos) { CHECK(check_ptr(rope_cos, "rope_cos")); CHECK(check_ptr(rope_sin, "rope_sin")); }
+  if (mean) CHECK(check_ptr(mean, "mean"));
+  if (!out.row_codes && !out.col_codes) return fail(ATTN_ERR_INVALID_ARG, "no output orientation requested");
+  if ((out.row_codes == nullptr) != (out.row_scales == nullptr) ||
+      (out.col_codes == nullptr) != (out.col_scales == nullptr))
+    return fail(ATTN_ERR_INVALID_ARG, "codes and scales of an orientation must be given together");
+  if (out.row_codes) { CHECK(check_ptr(out.row_codes, "row_codes")); CHECK(check_ptr(out.row_scales, "row_scales")); }
+  if (out.col_codes) { CHECK(check_ptr(out.col_codes, "col_codes")); CHECK(check_ptr(out.col_scales, "col_scales")); }
+  CHECK(check_device());
+  return launch_quantize_fused(src, src_dtype, B, H, N, d, rope_cos, rope_sin, scale, mean, out,
+                               static_cast<cudaStream_t>(stream));
+}
+
 attn_status_t attn_fp8_prepare_bf16(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
                                     attn_qtensor_t out, void* stream) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return fail(ATTN_ERR_INVALID_ARG, "sizes must be positive");

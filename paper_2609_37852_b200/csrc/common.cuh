@@ -30,6 +30,9 @@ struct AttnShape {
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).
 attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
                               cudaStream_t stream);
+attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H, int N, int d, const float* cos,
+                                    const float* sin, float scale, float* mean, attn_qtensor_t out,
+                                    cudaStream_t stream);
 attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, int N, int d, void* row_out, void* col_out,
                                  cudaStream_t stream);
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,

@@ -8,6 +8,8 @@
 // copy are staged in shared memory so that they leave as full 128-byte rows.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "mxfp8_device.cuh"
 #include "sm100_ptx.cuh"
@@ -21,18 +23,38 @@ constexpr int kThreads = 256;
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ __forceinline__ float to_f32(float x) { return x; }
 
-template <typename T>
+// Producer steps fused in front of the quantiser (paper Appendix "Operands, Scaling, and
+// Accumulation"): rotary embedding in FP32 with the rotated channels rounded to BF16, subtraction
+// of the FP32 token mean (key centering), FP32 multiplication by a scale (tau folded into Q).
+struct Producer {
+  const float* cos;     // [N, d/2] or nullptr
+  const float* sin;
+  const float* mean;    // [B*H, d] or nullptr
+  float scale;
+  int use_scale;
+};
+
+// One rotated channel: x*cos -+ partner*sin with one rounding for the product and a fused
+// multiply-add, then BF16 (the order the oracle writes out).
+__device__ __forceinline__ float rotate_bf16(float x, float partner, float c, float s, bool upper) {
+  const float t = __fmul_rn(partner, s);
+  const float r = __fmaf_rn(x, c, upper ? t : -t);
+  return __bfloat162float(__float2bfloat16_rn(r));
+}
+
+template <typename T, bool kFused>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict__ src, int N, int d,
                                                             uint8_t* __restrict__ row_codes,
                                                             uint8_t* __restrict__ row_scales,
                                                             uint8_t* __restrict__ col_codes,
-                                                            uint8_t* __restrict__ col_scales) {
+                                                            uint8_t* __restrict__ col_scales, const Producer prod) {
   extern __shared__ __align__(16) uint8_t smem[];
-  const int pitch = d + 16 / static_cast<int>(sizeof(T)) * 1;       // elements; +16 bytes per row
-  T* tile = reinterpret_cast<T*>(smem);
+  using TT = typename std::conditional<kFused, float, T>::type;     // what the parked tile holds
+  const int pitch = d + 16 / static_cast<int>(sizeof(TT)) * 1;      // elements; +16 bytes per row
+  TT* tile = reinterpret_cast<TT*>(smem);
   const int n_ct = (d / 32 + 3) / 4;                                 // row-copy scale tiles of this CTA
   const int n_rt = (d + 127) / 128;                                  // col-copy scale tiles of this CTA
-  uint8_t* s_row_sf = smem + static_cast<size_t>(kTokens) * pitch * sizeof(T);
+  uint8_t* s_row_sf = smem + static_cast<size_t>(kTokens) * pitch * sizeof(TT);
   uint8_t* s_col_sf = s_row_sf + n_ct * 512;
   uint8_t* s_col_codes = s_col_sf + n_rt * 512;                      // [d][128 + 16]
   constexpr int kColPitch = kTokens + 16;
@@ -60,14 +82,38 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict_
       const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&raw);
 #pragma unroll
       for (int i = 0; i < 8; ++i) x[i] = to_f32(h[i]);
-      if (want_col) *reinterpret_cast<uint4*>(tile + tok * pitch + ch) = raw;
+      if (!kFused && want_col) *reinterpret_cast<uint4*>(tile + tok * pitch + ch) = raw;
     } else {
       const float4 a = *reinterpret_cast<const float4*>(g_src + e0);
       const float4 b = *reinterpret_cast<const float4*>(g_src + e0 + 4);
       x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-      if (want_col) {
+      if (!kFused && want_col) {
         *reinterpret_cast<float4*>(tile + tok * pitch + ch) = a;
         *reinterpret_cast<float4*>(tile + tok * pitch + ch + 4) = b;
+      }
+    }
+    if constexpr (kFused) {
+      if (prod.cos != nullptr) {
+        const int half = d >> 1;
+        const bool upper = ch >= half;
+        const int pc = upper ? ch - half : ch;                       // pair index; 8 consecutive pairs per thread
+        const T* g_partner = g_src + e0 + (upper ? -half : half);
+        const size_t tab = (tok0 + tok) * half + pc;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          x[i] = rotate_bf16(x[i], to_f32(g_partner[i]), prod.cos[tab + i], prod.sin[tab + i], upper);
+      }
+      if (prod.mean != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = __fsub_rn(x[i], prod.mean[slab * d + ch + i]);
+      }
+      if (prod.use_scale) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(x[i], prod.scale);
+      }
+      if (want_col) {
+        *reinterpret_cast<float4*>(tile + tok * pitch + ch) = make_float4(x[0], x[1], x[2], x[3]);
+        *reinterpret_cast<float4*>(tile + tok * pitch + ch + 4) = make_float4(x[4], x[5], x[6], x[7]);
       }
     }
     if (want_row) {
@@ -130,21 +176,63 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict_
   }
 }
 
-template <typename T>
-attn_status_t launch_t(const void* src, int B, int H, int N, int d, attn_qtensor_t out, cudaStream_t stream) {
-  const int pitch = d + 16 / static_cast<int>(sizeof(T));
+template <typename T, bool kFused>
+attn_status_t launch_t(const void* src, int B, int H, int N, int d, attn_qtensor_t out, const Producer& prod,
+                       cudaStream_t stream) {
+  const int tile_elem = kFused ? 4 : static_cast<int>(sizeof(T));
+  const int pitch = d + 16 / tile_elem;
   const int n_ct = (d / 32 + 3) / 4, n_rt = (d + 127) / 128;
-  const size_t smem = static_cast<size_t>(kTokens) * pitch * sizeof(T) + (n_ct + n_rt) * 512 +
+  const size_t smem = static_cast<size_t>(kTokens) * pitch * tile_elem + (n_ct + n_rt) * 512 +
                       static_cast<size_t>(d) * (kTokens + 16);
-  cudaError_t e = cudaFuncSetAttribute(quantize_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(quantize_kernel<T, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(N / kTokens, B * H);
-  quantize_kernel<T><<<grid, kThreads, smem, stream>>>(static_cast<const T*>(src), N, d, out.row_codes,
-                                                      out.row_scales, out.col_codes, out.col_scales);
+  quantize_kernel<T, kFused><<<grid, kThreads, smem, stream>>>(static_cast<const T*>(src), N, d, out.row_codes,
+                                                              out.row_scales, out.col_codes, out.col_scales, prod);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
+}
+
+// FP32 mean over tokens of the (rotated, BF16-rounded) tensor, per (batch, head, channel).  The
+// terms are BF16 values, so a double-precision sum is exact whatever its order, and the result is
+// the correctly rounded quotient: bitwise reproducible.  One CTA per (batch, head).
+constexpr int kMeanThreads = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(kMeanThreads) token_mean_kernel(const T* __restrict__ src, int N, int d,
+                                                                  const float* __restrict__ cos,
+                                                                  const float* __restrict__ sin,
+                                                                  float* __restrict__ mean) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  double* part = reinterpret_cast<double*>(smem);                   // [phases][d]
+  const int half = d >> 1;
+  const int phases = kMeanThreads / half;
+  const int pc = threadIdx.x % half, ph = threadIdx.x / half;
+  const size_t slab = blockIdx.x;
+  const T* g = src + slab * N * d;
+  double a1 = 0.0, a2 = 0.0;
+  if (ph < phases) {
+    for (int n = ph; n < N; n += phases) {
+      float x1 = to_f32(g[static_cast<size_t>(n) * d + pc]), x2 = to_f32(g[static_cast<size_t>(n) * d + half + pc]);
+      if (cos != nullptr) {
+        const float c = cos[static_cast<size_t>(n) * half + pc], s = sin[static_cast<size_t>(n) * half + pc];
+        const float r1 = rotate_bf16(x1, x2, c, s, false), r2 = rotate_bf16(x2, x1, c, s, true);
+        x1 = r1; x2 = r2;
+      }
+      a1 += static_cast<double>(x1);
+      a2 += static_cast<double>(x2);
+    }
+    part[ph * d + pc] = a1;
+    part[ph * d + half + pc] = a2;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += kMeanThreads) {
+    double sum = 0.0;
+    for (int i = 0; i < phases; ++i) sum += part[i * d + c];
+    mean[slab * d + c] = static_cast<float>(sum / static_cast<double>(N));
+  }
 }
 
 // BF16 mode: the operands are the tensors themselves, rounded to BF16, in both orientations.
@@ -201,8 +289,26 @@ attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, i
 
 attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
                               cudaStream_t stream) {
-  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16>(src, B, H, N, d, out, stream);
-  return launch_t<float>(src, B, H, N, d, out, stream);
+  const Producer none{nullptr, nullptr, nullptr, 1.f, 0};
+  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16, false>(src, B, H, N, d, out, none, stream);
+  return launch_t<float, false>(src, B, H, N, d, out, none, stream);
+}
+
+attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H, int N, int d, const float* cos,
+                                    const float* sin, float scale, float* mean, attn_qtensor_t out,
+                                    cudaStream_t stream) {
+  if (mean != nullptr) {
+    const size_t smem = static_cast<size_t>(kMeanThreads / (d / 2)) * d * sizeof(double);
+    if (src_dtype == ATTN_SRC_BF16)
+      token_mean_kernel<__nv_bfloat16><<<B * H, kMeanThreads, smem, stream>>>(static_cast<const __nv_bfloat16*>(src), N, d, cos, sin, mean);
+    else
+      token_mean_kernel<float><<<B * H, kMeanThreads, smem, stream>>>(static_cast<const float*>(src), N, d, cos, sin, mean);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "token mean: launch: %s", cudaGetErrorString(e));
+  }
+  const Producer prod{cos, sin, mean, scale, scale != 1.f ? 1 : 0};
+  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16, true>(src, B, H, N, d, out, prod, stream);
+  return launch_t<float, true>(src, B, H, N, d, out, prod, stream);
 }
 
 }  // namespace attnfp8
