@@ -174,7 +174,7 @@ def _probabilities(q_row, k_row, lse, scale, causal, rows, cols):
 
 
 def emu_delta(q, k, v, dO, lse, scale, causal, prec="mxfp8", mode="matched", o=None,
-              exact_stats=False, rows=None):
+              exact_stats=False, rows=None, dp_prec=None):
     """Row correction D [B,Hq,R].
 
     matched: D_i = sum_j P_ij dP^_ij with dP^ = dO^ V^^T from the row-blocked
@@ -199,7 +199,7 @@ def emu_delta(q, k, v, dO, lse, scale, causal, prec="mxfp8", mode="matched", o=N
             elif mode == "matched":
                 P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec),
                                    lse[b, h], scale, causal, rows, allc)
-                dP = _fq(dO[b, h], -1, prec)[rows] @ _fq(v[b, g], -1, prec).T
+                dP = _fq(dO[b, h], -1, dp_prec or prec)[rows] @ _fq(v[b, g], -1, dp_prec or prec).T
                 d = (P * dP).sum(axis=-1)
             else:
                 raise ValueError(mode)
@@ -208,7 +208,7 @@ def emu_delta(q, k, v, dO, lse, scale, causal, prec="mxfp8", mode="matched", o=N
 
 
 def emu_backward(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", round_out=True,
-                 return_internals=False):
+                 return_internals=False, dp_prec=None):
     """Gradient pass given the saved LSE [B,Hq,N] and a row correction delta [B,Hq,N].
 
     Per head: S, P as in ``_probabilities``; dP^ = dO^r V^r^T (row-blocked
@@ -218,6 +218,9 @@ def emu_backward(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", round_out
       dQ    = scale dS^j K^c     dS^j: dS quantised in blocks of 32 keys per row
     with ^c the copies of dO, Q, K blocked along tokens.  dK, dV are summed over
     the query heads of the group before rounding; all three are stored BF16.
+
+    ``dp_prec`` overrides the operand precision of dP^ = dO V^T alone (the paper's protected-dP
+    ablation, Appendix "Protected dP": dP from BF16 operands, the other products unchanged).
 
     Also returns the pre-cast row statistics sum_j dS_ij and sum_j |dS_ij|."""
     B, Hq, N, _ = q.shape
@@ -235,7 +238,7 @@ def emu_backward(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", round_out
             g = h // G
             P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec),
                                lse[b, h], scale, causal, allr, allr)
-            dP = _fq(dO[b, h], -1, prec) @ _fq(v[b, g], -1, prec).T
+            dP = _fq(dO[b, h], -1, dp_prec or prec) @ _fq(v[b, g], -1, dp_prec or prec).T
             dS = P * (dP - np.asarray(delta[b, h], np.float64)[:, None])
             rowsum[b, h] = dS.sum(axis=-1)
             rowabs[b, h] = np.abs(dS).sum(axis=-1)
@@ -252,7 +255,7 @@ def emu_backward(q, k, v, dO, lse, delta, scale, causal, prec="mxfp8", round_out
     return out + (internals,) if return_internals else out
 
 
-def emu_backward_rows(q, k, v, dO, lse, delta, scale, causal, b, h, rows, prec="mxfp8"):
+def emu_backward_rows(q, k, v, dO, lse, delta, scale, causal, b, h, rows, prec="mxfp8", dp_prec=None):
     """dQ rows and pre-cast row statistics of one head for some query rows
     (every query row of dQ is independent of the others).  ``lse`` and
     ``delta`` are that head's full [N] vectors."""
@@ -261,13 +264,13 @@ def emu_backward_rows(q, k, v, dO, lse, delta, scale, causal, b, h, rows, prec="
     rows = np.asarray(rows)
     allc = np.arange(N)
     P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec), lse, scale, causal, rows, allc)
-    dP = _fq(dO[b, h], -1, prec)[rows] @ _fq(v[b, g], -1, prec).T
+    dP = _fq(dO[b, h], -1, dp_prec or prec)[rows] @ _fq(v[b, g], -1, dp_prec or prec).T
     dS = P * (dP - np.asarray(delta, np.float64)[rows][:, None])
     dq = scale * (_fq(dS, -1, prec) @ _fq(k[b, g], 0, prec))
     return mxfp8.round_bf16(dq), dS.sum(-1), np.abs(dS).sum(-1)
 
 
-def emu_backward_cols(q, k, v, dO, lse, delta, scale, causal, b, g, cols, prec="mxfp8"):
+def emu_backward_cols(q, k, v, dO, lse, delta, scale, causal, b, g, cols, prec="mxfp8", dp_prec=None):
     """dK and dV rows of one KV head for some keys (every key column of dS is
     independent of the others).  ``lse`` and ``delta`` are [Hq, N] for batch b."""
     N = q.shape[2]
@@ -278,7 +281,7 @@ def emu_backward_cols(q, k, v, dO, lse, delta, scale, causal, b, g, cols, prec="
     dv = np.zeros((len(cols), v.shape[-1]))
     for h in range(g * G, (g + 1) * G):
         P = _probabilities(_fq(q[b, h], -1, prec), _fq(k[b, g], -1, prec), lse[h], scale, causal, allr, cols)
-        dP = _fq(dO[b, h], -1, prec) @ _fq(v[b, g], -1, prec)[cols].T
+        dP = _fq(dO[b, h], -1, dp_prec or prec) @ _fq(v[b, g], -1, dp_prec or prec)[cols].T
         dS = P * (dP - np.asarray(delta[h], np.float64)[:, None])
         dv += _fq(P, 0, prec).T @ _fq(dO[b, h], 0, prec)
         dk += scale * (_fq(dS, 0, prec).T @ _fq(q[b, h], 0, prec))

@@ -409,6 +409,37 @@ def test_postcast_statistics_and_key_common_mode():
     assert cK.shape == dK.shape[:2] and np.all((cK >= 0) & (cK <= np.sqrt(dK.shape[2]) + 1e-9))
 
 
+def test_protected_dP_variant():
+    """Protected dP (Appendix "Protected dP"): dP from BF16 operands, everything else FP8.  The matched
+    correction built from that dP still zeroes the row sums (Eq. 5 only needs P normalised and one dP);
+    with the stale correction the residual is the saved-output mismatch seen through BF16 dO and V."""
+    q, k, v, dO, scale, causal = _setup_fp8(seed=23)
+    O, LSE, fwd = A.emu_forward(q, k, v, scale, causal, exact_stats=True, return_internals=True)
+    Dm = A.emu_delta(q, k, v, dO, LSE, scale, causal, exact_stats=True, dp_prec="bf16")
+    Ds = A.emu_delta(q, k, v, dO, LSE, scale, causal, mode="stale", o=O, exact_stats=True)
+    _, _, dVm, rsm, ram = A.emu_backward(q, k, v, dO, LSE, Dm, scale, causal, dp_prec="bf16")
+    dQs, dKs, dVs, rss, ras, t = A.emu_backward(q, k, v, dO, LSE, Ds, scale, causal, dp_prec="bf16", return_internals=True)
+    assert np.nanmedian(A.residual_ratio(rsm, ram)[..., 64:]) < 1e-12
+    assert np.array_equal(dVm, dVs)                     # dV does not see dP
+    _, _, dV8, _, _ = A.emu_backward(q, k, v, dO, LSE, Ds, scale, causal)
+    assert np.array_equal(dVs, dV8)
+    G = q.shape[1] // k.shape[1]
+    for (b, h), tt in t.items():
+        g = h // G
+        assert np.abs(rss[b, h] - (Dm[b, h] - Ds[b, h])).max() < 1e-12
+        dOb, Vb = mxfp8.round_bf16(dO[b, h]), mxfp8.round_bf16(v[b, g])
+        assert np.array_equal(tt["dP"], dOb @ Vb.T)     # BF16 inputs: the rounding is the identity here
+        Phat = fwd[(b, h)]["Ph"] / fwd[(b, h)]["l"][:, None]
+        Vc = mxfp8.fake_quant(v[b, g], 0)
+        want = (dOb * ((tt["P"] - Phat) @ Vb)).sum(-1) + (dOb * (Phat @ (Vb - Vc))).sum(-1) \
+            + (dOb * (Phat @ Vc - O[b, h])).sum(-1)
+        assert np.abs(rss[b, h] - want).max() < 1e-12
+    # dK / dQ differ from the all-FP8 gradients only through dP
+    dQ8, dK8, _, _, _ = A.emu_backward(q, k, v, dO, LSE, Ds, scale, causal)
+    assert not np.array_equal(dQs, dQ8)
+    assert np.linalg.norm(dQs - dQ8) / np.linalg.norm(dQ8) < 0.2
+
+
 def test_subset_functions_agree_with_full_pass():
     q, k, v, dO, scale, causal = _setup_fp8(seed=14)
     O, LSE = A.emu_forward(q, k, v, scale, causal)
