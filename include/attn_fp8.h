@@ -41,6 +41,14 @@
  * and both scale pointers are ignored (may be NULL); attn_fp8_prepare_bf16 writes the two copies.
  * Probabilities and score gradients are rounded to BF16 where the FP8 mode quantises them; the
  * normaliser, LSE, the row correction and every accumulation stay FP32 exactly as in FP8 mode.
+ *
+ * Protected dP (precision = ATTN_PREC_MXFP8_PROTECTED_DP; the paper's ablation of that name,
+ * Appendix "Protected dP"): FP8 mode in which dP = dO V^T alone is computed from BF16 operands.
+ * The backward entry points (bwd_delta, bwd, bwd_dq, bwd_dkdv) then take
+ *   dO.row_codes = BF16 [B, Hq, N, dv]  and  v.row_codes = BF16 [B, Hkv, N, dv]
+ * (row scales ignored); every other operand, the column copies of dO and V included, stays FP8.
+ * The forward treats this precision as ATTN_PREC_MXFP8.  Head dims (64,64) and (128,128).  The
+ * paper pairs it with the stale correction; any delta_mode is accepted.
  */
 #ifndef ATTN_FP8_H_
 #define ATTN_FP8_H_
@@ -63,7 +71,7 @@ typedef enum {
   ATTN_ERR_TIMEOUT = 7        /* a bounded device-side wait expired (reported by read_status)   */
 } attn_status_t;
 
-typedef enum { ATTN_PREC_MXFP8 = 0, ATTN_PREC_BF16 = 1 } attn_precision_t;
+typedef enum { ATTN_PREC_MXFP8 = 0, ATTN_PREC_BF16 = 1, ATTN_PREC_MXFP8_PROTECTED_DP = 2 } attn_precision_t;
 typedef enum { ATTN_DELTA_MATCHED = 0, ATTN_DELTA_STALE = 1, ATTN_DELTA_CONSISTENT_DO = 2 } attn_delta_mode_t;
 typedef enum { ATTN_SRC_BF16 = 0, ATTN_SRC_FP32 = 1 } attn_src_dtype_t;
 typedef enum { ATTN_WS_FWD = 0, ATTN_WS_BWD_DELTA = 1, ATTN_WS_BWD = 2 } attn_ws_kind_t;

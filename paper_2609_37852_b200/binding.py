@@ -26,7 +26,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 ATTN_OK = 0
 STATUS_NAMES = {0: "ATTN_OK", 1: "ATTN_ERR_INVALID_ARG", 2: "ATTN_ERR_UNSUPPORTED", 3: "ATTN_ERR_ALIGNMENT",
                 4: "ATTN_ERR_WORKSPACE", 5: "ATTN_ERR_ARCH", 6: "ATTN_ERR_CUDA", 7: "ATTN_ERR_TIMEOUT"}
-ATTN_PREC_MXFP8, ATTN_PREC_BF16 = 0, 1
+ATTN_PREC_MXFP8, ATTN_PREC_BF16, ATTN_PREC_MXFP8_PROTECTED_DP = 0, 1, 2
 ATTN_DELTA_MATCHED, ATTN_DELTA_STALE, ATTN_DELTA_CONSISTENT_DO = 0, 1, 2
 ATTN_SRC_BF16, ATTN_SRC_FP32 = 0, 1
 ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
@@ -136,6 +136,14 @@ class QTensor:
     def c_struct(self) -> _QTensor:
         return _QTensor(*(None if t is None else t.data_ptr()
                           for t in (self.row_codes, self.row_scales, self.col_codes, self.col_scales)))
+
+
+def protect_dp_operand(qt: QTensor, src_bf16: torch.Tensor) -> QTensor:
+    """Operand of the protected-dP precision: ``qt`` with its row copy replaced by the BF16 tensor
+    itself (dO or V); the column copy stays FP8."""
+    if src_bf16.dtype != torch.bfloat16 or not src_bf16.is_contiguous() or tuple(src_bf16.shape) != tuple(qt.shape):
+        raise ValueError("src_bf16 must be a contiguous bfloat16 tensor of the operand's shape")
+    return QTensor(shape=qt.shape, row_codes=src_bf16, row_scales=None, col_codes=qt.col_codes, col_scales=qt.col_scales)
 
 
 def attn_fp8_scale_offset(row: int, block: int, n_blocks: int) -> int:

@@ -77,15 +77,19 @@ static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entr
   if (p->heads_q % p->heads_kv) return fail(ATTN_ERR_INVALID_ARG, "heads_q must be a multiple of heads_kv");
   if (p->causal != 0 && p->causal != 1) return fail(ATTN_ERR_INVALID_ARG, "causal must be 0 or 1");
   if (!(p->softmax_scale > 0.f)) return fail(ATTN_ERR_INVALID_ARG, "softmax_scale must be positive");
-  if (p->precision != ATTN_PREC_MXFP8 && p->precision != ATTN_PREC_BF16)
+  if (p->precision != ATTN_PREC_MXFP8 && p->precision != ATTN_PREC_BF16 && p->precision != ATTN_PREC_MXFP8_PROTECTED_DP)
     return fail(ATTN_ERR_INVALID_ARG, "precision %d unknown", p->precision);
   if (p->seqlen % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen must be a multiple of 128");
   const int eb = p->precision == ATTN_PREC_BF16 ? 2 : 1;
   if (!dims_supported(entry, eb, p->head_dim_qk, p->head_dim_v))
     return fail(ATTN_ERR_UNSUPPORTED, "head dims (%d, %d) are not built for this entry point in %s mode",
                 p->head_dim_qk, p->head_dim_v, eb == 1 ? "MXFP8" : "BF16");
+  // protected dP: the row copies of dO and V (the operands of dP alone) are BF16; the forward never sees them
+  const bool protect = p->precision == ATTN_PREC_MXFP8_PROTECTED_DP && entry != kEntryFwd;
+  if (protect && !((p->head_dim_qk == 64 && p->head_dim_v == 64) || (p->head_dim_qk == 128 && p->head_dim_v == 128)))
+    return fail(ATTN_ERR_UNSUPPORTED, "protected dP is built for head dims (64,64) and (128,128)");
   *s = AttnShape{p->batch, p->seqlen, p->heads_q, p->heads_kv, p->head_dim_qk, p->head_dim_v, p->causal,
-                 p->softmax_scale, eb};
+                 p->softmax_scale, eb, protect ? 2 : eb};
   return ATTN_OK;
 }
 
@@ -230,7 +234,7 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
   }
   if (p->delta_mode == ATTN_DELTA_CONSISTENT_DO) {
     CHECK(check_ptr(o_bf16, "o_bf16"));
-    if (!fp8) {                                       // BF16 operands: dO^ is the BF16 dO itself
+    if (s.ebv == 2) {                                 // BF16 row copy of dO: dO^ is the BF16 dO itself
       CHECK(check_ptr(dO.row_codes, "dO.row_codes"));
       return launch_stale_delta(s, dO.row_codes, o_bf16, delta, st);
     }
@@ -238,7 +242,8 @@ attn_status_t attn_fp8_bwd_delta(const attn_params_t* p, attn_qtensor_t q, attn_
     return launch_consistent_delta(s, dO, o_bf16, delta, st);
   }
   if (p->delta_mode != ATTN_DELTA_MATCHED) return fail(ATTN_ERR_INVALID_ARG, "delta_mode %d unknown", p->delta_mode);
-  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8); CHECK_OPERAND(dO, row, fp8);
+  const bool fp8v = s.ebv == 1;
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8v); CHECK_OPERAND(dO, row, fp8v);
   CHECK(check_ptr(lse, "lse"));
   return launch_bwd_delta(s, q, k, v, dO, lse, delta, status, st);
 }
@@ -251,8 +256,8 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
   AttnShape s;
   if (want_dq) CHECK(check_params(p, &s, kEntryDq));
   if (want_dkdv) CHECK(check_params(p, &s, kEntryDkdv));
-  const bool fp8 = s.eb == 1;
-  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8); CHECK_OPERAND(dO, row, fp8);
+  const bool fp8 = s.eb == 1, fp8v = s.ebv == 1;
+  CHECK_OPERAND(q, row, fp8); CHECK_OPERAND(k, row, fp8); CHECK_OPERAND(v, row, fp8v); CHECK_OPERAND(dO, row, fp8v);
   CHECK(check_ptr(lse, "lse")); CHECK(check_ptr(delta, "delta"));
   if (want_dq) {
     CHECK_OPERAND(k, col, fp8);

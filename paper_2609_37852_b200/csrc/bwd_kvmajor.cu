@@ -63,14 +63,17 @@ constexpr int kSmemLimit = 232448;              // dynamic shared memory a CTA m
 enum KvMode { kBoth = 0, kDvOnly = 1, kDkOnly = 2 };
 
 // Operand geometry, ring depths and tensor-memory map of one instantiation.
-template <int kEB_, int kCq_, int kCv_, int kMode_>
+template <int kEB_, int kCq_, int kCv_, int kMode_, int kEBv_ = kEB_>
 struct KvCfg {
   static constexpr int kEB = kEB_, kCq = kCq_, kCv = kCv_, kMode = kMode_;
+  static constexpr int kEBv = kEBv_;                   // bytes per element of the V / dO row operands (dP^T only):
+                                                       // 2 with kEB == 1 is the protected-dP ablation
   static constexpr bool kFp8 = kEB == 1;
+  static constexpr bool kFp8v = kEBv == 1;
   static constexpr bool kHasDv = kMode != kDkOnly;     // accumulates dV (needs P^)
   static constexpr bool kHasDk = kMode != kDvOnly;     // accumulates dK (needs dP^T, D, dS^)
   static constexpr int kRq = kCq / kEB > 0 ? (kCq + kEB - 1) / kEB : 1;   // 128-row tiles of the Q^c operand (dqk / 128, rounded up)
-  static constexpr int kRv = (kCv + kEB - 1) / kEB;                       // 128-row tiles of the dO^c operand
+  static constexpr int kRv = (kCv + kEBv - 1) / kEBv;                     // 128-row tiles of the dO^c operand
   // Per query tile the CTA streams a 'row' set (Q and dO row copies, their scales, LSE, D: read by
   // the S^T / dP^T MMAs and the softmax) and a 'col' set (Q and dO column copies: read by the dV /
   // dK MMAs).  The row set is released early and gets the deeper ring, so that a reload never sits
@@ -94,9 +97,9 @@ struct KvCfg {
   static constexpr uint32_t kColdK = kColdV + (kHasDv ? 128 * kRv : 0);
   static constexpr uint32_t kColSFK = kColdK + (kHasDk ? 128 * kRq : 0);
   static constexpr uint32_t kColSFV = kColSFK + 4 * kCq;
-  static constexpr uint32_t kColSFQ = kColSFV + (kHasDk ? 4 * kCv : 0);        // 2 slots
+  static constexpr uint32_t kColSFQ = kColSFV + (kHasDk && kFp8v ? 4 * kCv : 0);   // 2 slots
   static constexpr uint32_t kColSFdO = kColSFQ + 8 * kCq;                      // 2 slots
-  static constexpr uint32_t kColSFP = kColSFdO + (kHasDk ? 8 * kCv : 0);       // 2 x 4
+  static constexpr uint32_t kColSFP = kColSFdO + (kHasDk && kFp8v ? 8 * kCv : 0);  // 2 x 4
   static constexpr uint32_t kColSFdS = kColSFP + (kHasDv ? 8 : 0);             // 2 x 4
   static constexpr uint32_t kColSFdOc = kColSFdS + (kHasDk ? 8 : 0);           // 2 slots x row tiles
   static constexpr uint32_t kColSFQc = kColSFdOc + (kHasDv ? 8 * kRv : 0);     // 2 slots x row tiles
@@ -164,7 +167,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
   // shared state space of every access derived from it (checked below)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  constexpr bool kFp8 = C::kFp8, kHasDv = C::kHasDv, kHasDk = C::kHasDk;
+  constexpr bool kFp8 = C::kFp8, kFp8v = C::kFp8v, kHasDv = C::kHasDv, kHasDk = C::kHasDk;
   constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRq, kRv = C::kRv;
   constexpr int kRowStages = C::kRowStages, kColStages = C::kColStages, kRowTok = C::kRowTok;
   constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
@@ -188,7 +191,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   const int tiles_per_head = tiles_n - it0;
   const int n_qtiles = G * tiles_per_head;          // query tiles this CTA walks
   const int n_sub = 2 * n_qtiles;
-  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * kEB / 32;       // 32-byte K steps of S^T and dP^T
+  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * C::kEBv / 32;   // 32-byte K steps of S^T and dP^T
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
@@ -220,13 +223,13 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO);
       prefetch_tmap(&tm_qc); prefetch_tmap(&tm_dOc);
       const int kv_slab = b * p.Hkv + g;
-      const int n_kv_ops = kCq + (kHasDk ? kCv : 0);
-      mbar_arrive_expect_tx(&sm.kv_full, n_kv_ops * (kTile * 128 + (kFp8 ? 512 : 0)));
+      mbar_arrive_expect_tx(&sm.kv_full, kCq * (kTile * 128 + (kFp8 ? 512 : 0)) +
+                                             (kHasDk ? kCv * (kTile * 128 + (kFp8v ? 512 : 0)) : 0));
       for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[c], &tm_k, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
       if (kFp8) bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCq * 512, kCq * 512, &sm.kv_full);
       if (kHasDk) {
         for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[c], &tm_v, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
-        if (kFp8) bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCv * 512, kCv * 512, &sm.kv_full);
+        if (kFp8v) bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCv * 512, kCv * 512, &sm.kv_full);
       }
       int issued_row = 0, issued_col = 0;
       bool ok = true;
@@ -241,13 +244,15 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           ok = mbar_wait(&sm.row_empty[rs], ((ri / kRowStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
           KvRowStage<C>& r = sm.rst[rs];
-          mbar_arrive_expect_tx(&sm.row_full[rs], n_kv_ops * (kRowTok * 128 + (kFp8 ? 512 : 0)) + (kHasDk ? 2 : 1) * kRowTok * 4);
+          mbar_arrive_expect_tx(&sm.row_full[rs], kCq * (kRowTok * 128 + (kFp8 ? 512 : 0)) +
+                                                      (kHasDk ? kCv * (kRowTok * 128 + (kFp8v ? 512 : 0)) : 0) +
+                                                      (kHasDk ? 2 : 1) * kRowTok * 4);
           for (int c = 0; c < kCq; ++c) tma_load_2d(r.q[c], &tm_q, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
           if (kFp8) bulk_load_1d(r.sf_q, p.q_sf + sf_tile * kCq * 512, kCq * 512, &sm.row_full[rs]);
           bulk_load_1d(r.lse, p.lse + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
           if (kHasDk) {
             for (int c = 0; c < kCv; ++c) tma_load_2d(r.dO[c], &tm_dO, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
-            if (kFp8) bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile * kCv * 512, kCv * 512, &sm.row_full[rs]);
+            if (kFp8v) bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile * kCv * 512, kCv * 512, &sm.row_full[rs]);
             bulk_load_1d(r.delta, p.delta + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
           }
           ++issued_row;
@@ -330,7 +335,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // ------------------------------------------------------------------ dP^T issuer + LSE preparation
     const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[0]));
     bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-    if (ok && kFp8 && kHasDk) {
+    if (ok && kFp8v && kHasDk) {
       tc_fence_after_sync();
       sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v);
     }
@@ -347,7 +352,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
               make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
         }
         mbar_arrive_warp(&sm.lse_ready[s]);
-        if (kFp8 && kHasDk) {
+        if (kFp8v && kHasDk) {
           tc_fence_after_sync();
           sf_copy_tiles<kCv>(tmem + kColSFdO + 4 * kCv * slot, st.sf_dO);
         }
@@ -359,7 +364,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         }
         tc_fence_after_sync();
         const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO[0])) + sub_r * (kSub * 128 / 16);
-        issue_ss<kFp8, kCv, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
+        issue_ss<kFp8v, kCv, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColdP, desc_v, desc_dO, nk_v, tmem + kColSFV, tmem + kColSFdO + 4 * kCv * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
       }
@@ -584,12 +589,12 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   static_assert(sizeof(KvSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc;
   attn_status_t st;
-  const uint64_t eb = C::kEB;
+  const uint64_t eb = C::kEB, ebv = C::kEBv;
   const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
   if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * eb, kv_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * ebv, q_rows, C::kRowTok)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, s.dqk)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_dOc, dO.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dv, s.dv)) != ATTN_OK) return st;
   KvParams p;
@@ -614,7 +619,14 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
 attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                               const float* lse, const float* delta, void* dk, void* dv, int* status,
                               cudaStream_t stream) {
-  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.eb + 127) / 128;
+  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.ebv + 127) / 128;
+  if (s.eb == 1 && s.ebv == 2) {                     // protected dP: BF16 row copies of V and dO
+    if (cq == 1 && cv == 1)
+      return launch_kvmajor_t<KvCfg<1, 1, 1, kBoth, 2>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (cq == 1 && cv == 2)
+      return launch_kvmajor_t<KvCfg<1, 1, 2, kBoth, 2>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    return fail(ATTN_ERR_UNSUPPORTED, "bwd kv-major: protected dP is built for head dims (64,64) and (128,128)");
+  }
   if (s.eb == 1 && cq == 1 && cv == 1)
     return launch_kvmajor_t<KvCfg<1, 1, 1, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   if (s.eb == 2 && cq == 1 && cv == 1)

@@ -59,13 +59,16 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kSmemLimit = 232448;                  // dynamic shared memory a CTA may ask for
 
 // Operand geometry, ring depths and tensor-memory map of one instantiation.
-template <bool kDQ_, int kEB_, int kCq_, int kCv_>
+template <bool kDQ_, int kEB_, int kCq_, int kCv_, int kEBv_ = kEB_>
 struct QmCfg {
   static constexpr bool kDQ = kDQ_;
   static constexpr int kEB = kEB_;                      // bytes per operand element
   static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row
   static constexpr int kCv = kCv_;                      // 128-byte chunks per dO / V row
+  static constexpr int kEBv = kEBv_;                    // bytes per element of the dO / V row operands (dP only):
+                                                        // 2 with kEB == 1 is the protected-dP ablation
   static constexpr bool kFp8 = kEB == 1;
+  static constexpr bool kFp8v = kEBv == 1;
   static constexpr int kStep = kTile / kEB;             // keys per step
   static constexpr int kGroups = kStep / 32;            // 32-key column groups of a step
   static constexpr int kSoftmaxThreads = 128 * kGroups; // 4 TMEM lane quadrants x column groups
@@ -140,7 +143,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
   // shared state space of every access derived from it (checked below)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8;
+  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8, kFp8v = C::kFp8v;
   constexpr int kStages = C::kStages, kKcStages = C::kKcStages, kEB = C::kEB, kCq = C::kCq, kCv = C::kCv;
   constexpr int kStep = C::kStep, kGroups = C::kGroups, kSoftmaxThreads = C::kSoftmaxThreads;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColdS = C::kColdS, kColdQ = C::kColdQ, kColSFQ = C::kColSFQ,
@@ -161,7 +164,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
   const int g = h / (p.Hq / p.Hkv);
   const int n_tiles = (p.causal ? qt + 1 : p.N / kTile) * kEB;      // key steps
-  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * kEB / 32;       // 32-byte K steps of the two products
+  const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * C::kEBv / 32;       // 32-byte K steps of the two products
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
@@ -193,13 +196,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       if (kDQ) prefetch_tmap(&tm_kc);
       const int q_slab = b * p.Hq + h, kv_slab = b * p.Hkv + g;
       const int tiles_n = p.N / kTile;
-      mbar_arrive_expect_tx(&sm.q_full, (kCq + kCv) * (kTile * 128 + (kFp8 ? 512 : 0)));
+      mbar_arrive_expect_tx(&sm.q_full, kCq * (kTile * 128 + (kFp8 ? 512 : 0)) + kCv * (kTile * 128 + (kFp8v ? 512 : 0)));
       for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[c], &tm_q, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
       for (int c = 0; c < kCv; ++c) tma_load_2d(sm.dO[c], &tm_dO, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
-      if (kFp8) {
+      if (kFp8)
         bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCq * 512, kCq * 512, &sm.q_full);
+      if (kFp8v)
         bulk_load_1d(sm.sf_dO, p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCv * 512, kCv * 512, &sm.q_full);
-      }
       int issued_kv = 0, issued_kc = 0;
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
@@ -207,13 +210,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
         QM_TRACE(0, t, 0);
-        mbar_arrive_expect_tx(&sm.kv_full[s], (kCq + kCv) * (kStep * 128 + (kFp8 ? 512 : 0)));
+        mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
         for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
         for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
-        if (kFp8) {
+        if (kFp8)
           bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
+        if (kFp8v)
           bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
-        }
         ++issued_kv;
         if (kDQ) {
           const int sc = t % kKcStages;
@@ -277,7 +280,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     {
       const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO[0]));
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok && kFp8) {
+      if (ok && kFp8v) {
         tc_fence_after_sync();
         sf_copy_tiles<kCv>(tmem + kColSFdO, sm.sf_dO);
       }
@@ -286,14 +289,14 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        if (kFp8) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
+        if (kFp8v) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
         if (t > 0) {
           ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
         const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
-        issue_ss<kFp8, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, tmem + kColSFdO,
+        issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, tmem + kColSFdO,
                                                                         tmem + kColSFV + 4 * kCv * slot);
         mma_commit_elect(&sm.sdp_full);
         mma_commit_elect(&sm.kv_empty[s]);
@@ -530,12 +533,12 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   static_assert(sizeof(QmSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
   attn_status_t st;
-  const uint64_t eb = C::kEB;
+  const uint64_t eb = C::kEB, ebv = C::kEBv;
   const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
   if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, kTile)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * eb, q_rows, kTile)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * ebv, q_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, C::kStep)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * eb, kv_rows, C::kStep)) != ATTN_OK) return st;
+  if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, C::kStep)) != ATTN_OK) return st;
   if (kDQ) {
     if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
                                    s.dqk < 128 ? s.dqk : 128)) != ATTN_OK)
@@ -565,16 +568,18 @@ template <bool kDQ>
 attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
                             float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
-  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.eb + 127) / 128;
-#define ATTN_QM_CASE(EB, CQ, CV)                                                                              \
-  if (s.eb == EB && cq == CQ && cv == CV)                                                                     \
-    return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
-                                                  post_rowsum, post_rowabs, status, stream);
-  ATTN_QM_CASE(1, 1, 1)
-  ATTN_QM_CASE(1, 2, 1)
-  ATTN_QM_CASE(1, 2, 2)
-  ATTN_QM_CASE(2, 1, 1)
-  ATTN_QM_CASE(2, 2, 2)
+  const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.ebv + 127) / 128;
+#define ATTN_QM_CASE(EB, CQ, CV, EBV)                                                                         \
+  if (s.eb == EB && s.ebv == EBV && cq == CQ && cv == CV)                                                     \
+    return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV, EBV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
+                                                       post_rowsum, post_rowabs, status, stream);
+  ATTN_QM_CASE(1, 1, 1, 1)
+  ATTN_QM_CASE(1, 2, 1, 1)
+  ATTN_QM_CASE(1, 2, 2, 1)
+  ATTN_QM_CASE(2, 1, 1, 2)
+  ATTN_QM_CASE(2, 2, 2, 2)
+  ATTN_QM_CASE(1, 1, 1, 2)   // protected dP, d = 64
+  ATTN_QM_CASE(1, 1, 2, 2)   // protected dP, d = 128
 #undef ATTN_QM_CASE
   return fail(ATTN_ERR_UNSUPPORTED, "bwd q-major: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv,
               s.eb);

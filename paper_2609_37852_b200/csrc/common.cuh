@@ -25,6 +25,7 @@ struct AttnShape {
   int B, N, Hq, Hkv, dqk, dv, causal;
   float scale;
   int eb;   // bytes per operand element: 1 = E4M3 codes with E8M0 block scales, 2 = BF16 without scales
+  int ebv;  // the same for the row copies of dO and V, the operands of dP alone (2 with eb == 1: protected dP)
 };
 
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).

@@ -201,6 +201,48 @@ def test_postcast_statistics(bf16):
     assert np.nanmax(np.abs(kappa)) <= 2.0 ** -4
 
 
+@pytest.mark.parametrize("name,kw,delta_mode", [
+    ("gqa4k", dict(batch=1, heads_q=4, heads_kv=2, seqlen=640), 1),      # the paper's pairing: stale correction
+    ("gqa4k", dict(batch=1, heads_q=4, heads_kv=2, seqlen=384), 0),      # matched correction from the protected dP
+    ("tiny", dict(causal=True, seqlen=384), 1),                          # d = 64
+])
+def test_protected_dP_precision(name, kw, delta_mode):
+    """dP = dO V^T from BF16 operands, the other products FP8 (paper Appendix "Protected dP")."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    q, k, v, dO = workloads.make_inputs(w)
+    base = dict(batch=w.batch, seqlen=w.seqlen, heads_q=w.heads_q, heads_kv=w.heads_kv, head_dim_qk=w.head_dim_qk,
+                head_dim_v=w.head_dim_v, causal=w.causal, softmax_scale=w.softmax_scale, delta_mode=delta_mode)
+    p8 = B.AttnParams(**base)
+    pp = B.AttnParams(precision=B.ATTN_PREC_MXFP8_PROTECTED_DP, **base)
+    qq, kq, vq, dOq = (B.attn_fp8_quantize(x.cuda()) for x in (q, k, v, dO))
+    v_bf, dO_bf = v.cuda().to(torch.bfloat16), dO.cuda().to(torch.bfloat16)
+    vp, dOp = B.protect_dp_operand(vq, v_bf), B.protect_dp_operand(dOq, dO_bf)
+    o, lse, ws = B.attn_fp8_fwd(pp, qq, kq, vq)
+    o8, lse8, _ = B.attn_fp8_fwd(p8, qq, kq, vq)
+    assert torch.equal(o, o8) and torch.equal(lse, lse8)                 # the forward does not know about it
+    delta, ws = B.attn_fp8_bwd_delta(pp, qq, kq, vp, dOp, lse, dO_bf16=dO_bf, o_bf16=o, workspace=ws)
+    dq, dk, dv, rs, ra, ws = B.attn_fp8_bwd(pp, qq, kq, vp, dOp, lse, delta, diagnostics=True, workspace=ws)
+    B.attn_fp8_read_status(ws)
+    qn, kn, vn, dOn = (to_np(x) for x in (q, k, v, dO))
+    lse_n, delta_n = to_np(lse), to_np(delta)
+    if delta_mode == 0:
+        D = A.emu_delta(qn, kn, vn, dOn, lse_n, w.softmax_scale, w.causal, dp_prec="bf16")
+        assert rel_fro(delta_n, D) <= TOL_DELTA
+    dQ, dK, dV, rs_or, ra_or = A.emu_backward(qn, kn, vn, dOn, lse_n, delta_n, w.softmax_scale, w.causal, dp_prec="bf16")
+    assert rel_fro(to_np(dq), dQ) <= TOL_GRAD and rel_fro(to_np(dk), dK) <= TOL_GRAD and rel_fro(to_np(dv), dV) <= TOL_GRAD
+    assert rel_fro(to_np(ra), ra_or) <= 1e-3
+    r_pre = A.residual_ratio(to_np(rs), to_np(ra))[..., 64:]
+    if delta_mode == 0:
+        assert np.nanmedian(r_pre) <= 1e-5
+    else:
+        assert np.nanmedian(r_pre) > 1e-5                                # the stale residual remains
+        assert rel_fro(to_np(rs), rs_or) <= 1e-2
+    # it differs from the all-FP8 gradient pass only through dP
+    dq8, dk8, dv8, _, _, _ = B.attn_fp8_bwd(p8, qq, kq, vq, dOq, lse, delta)
+    assert torch.equal(dv, dv8) and not torch.equal(dq, dq8)
+
+
 def test_backward_is_reproducible():
     w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
     q, k, v, dO = workloads.make_inputs(w)
