@@ -256,6 +256,13 @@ size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which);
  * call are then undefined).  This is the one call that synchronises.                          */
 attn_status_t attn_fp8_read_status(const void* workspace, void* stream);
 
+/* Self-test of the device-side time-out report: enqueues a one-CTA kernel that waits, with a limit
+ * of about 2 ms, on a barrier nothing completes, gives up and sets the status word of `workspace`
+ * (>= attn_fp8_workspace_bytes) exactly as an attention kernel whose wait expired would.  A later
+ * attn_fp8_read_status(workspace) therefore returns ATTN_ERR_TIMEOUT; the context stays usable.
+ * For tests of the error path: nothing faults, traps or hangs.                                 */
+attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes, void* stream);
+
 /* Message for the last non-OK return on this host thread (static storage; never NULL).        */
 const char* attn_fp8_last_error(void);
 

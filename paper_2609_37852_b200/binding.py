@@ -34,7 +34,7 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
-    "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error",
+    "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
 )
 
 
@@ -267,6 +267,15 @@ def _workspace(params, which, workspace, device):
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=device)
     return workspace
+
+
+_lib.attn_fp8_selftest_timeout.restype = _i32
+_lib.attn_fp8_selftest_timeout.argtypes = [_vp, _sz, _vp]
+
+
+def attn_fp8_selftest_timeout(workspace: torch.Tensor, stream=None) -> None:
+    """Enqueues the bounded-wait self-test: the next attn_fp8_read_status(workspace) raises ATTN_ERR_TIMEOUT."""
+    _check(_lib.attn_fp8_selftest_timeout(_ptr(workspace), workspace.numel(), _stream(stream)))
 
 
 def attn_fp8_read_status(workspace: torch.Tensor, stream=None) -> None:

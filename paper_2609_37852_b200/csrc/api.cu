@@ -5,6 +5,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace attnfp8 {
 
@@ -388,4 +389,36 @@ extern "C" attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtens
   // the array keeps whatever the previous call left: clear the part that must start at zero
   CHECK(prepare_workspace(scratch, kBuiltinScratchBytes, need, st, &status));
   return launch_fwd(s, q, k, v, o_bf16, lse, status, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded-wait machinery: one CTA waits on a barrier that nothing completes, with
+// a limit of a few milliseconds, gives up, and reports through the workspace status word exactly as
+// the attention kernels do.  The context stays usable; nothing traps.
+namespace attnfp8 {
+__global__ void wait_selftest_kernel(int* status, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    sm100::mbar_init(&bar, 1);
+    abort_flag = 0;
+    sm100::fence_mbar_init();
+  }
+  __syncthreads();
+  // each thread polls in short bursts so that the limit is looked at every few microseconds
+  const bool ok = sm100::mbar_wait_limited(&bar, 0, &abort_flag, limit_cycles, 4);
+  __syncthreads();
+  if (threadIdx.x == 0 && (abort_flag || !ok)) atomicExch(status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+}  // namespace attnfp8
+
+extern "C" attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes, void* stream) {
+  CHECK(check_device());
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
+  wait_selftest_kernel<<<1, 64, 0, st>>>(status, 4000000LL);     // ~2 ms of SM cycles
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "selftest: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
 }

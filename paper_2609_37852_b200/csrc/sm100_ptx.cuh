@@ -93,16 +93,20 @@ __device__ __forceinline__ uint32_t mbar_poll(uint64_t* bar, uint32_t parity, ui
       : "memory");
   return ok;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit_cycles, uint32_t polls_per_check) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!mbar_poll(bar, parity, kPollsPerCheck)) {
-    if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+  while (!mbar_poll(bar, parity, polls_per_check)) {
+    if (*abort_flag || clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
       return false;
     }
   }
   return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limited(bar, parity, abort_flag, kWaitLimitCycles, kPollsPerCheck);
 }
 
 // 16-byte load from shared memory (the address space is stated, so no generic load is emitted).

@@ -174,3 +174,25 @@ def test_quantize_wide_heads_bit_exact(d):
         assert np.array_equal(codes.cpu().numpy(), c_or)
         got_e = B.unpack_scales(scales, 1, 2, rows, cols).cpu().numpy()
         assert np.array_equal(got_e, e_or)
+
+
+def test_expired_wait_is_reported_and_the_context_survives():
+    """A bounded device-side wait that runs out (a barrier nothing completes, ~2 ms limit) sets the
+    workspace status word; read_status reports ATTN_ERR_TIMEOUT; later calls work as before."""
+    import time
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=2, heads_kv=1, seqlen=256)
+    q, k, v, dO = (x.cuda() for x in workloads.make_inputs(w))
+    qq, kq, vq = (B.attn_fp8_quantize(x) for x in (q, k, v))
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, 128, 128, True, w.softmax_scale)
+    o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
+    B.attn_fp8_read_status(ws)
+    t0 = time.perf_counter()
+    B.attn_fp8_selftest_timeout(ws)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_read_status(ws)
+    assert e.value.status == 7
+    assert time.perf_counter() - t0 < 1.0                              # it gave up within its limit
+    o2, lse2, ws = B.attn_fp8_fwd(params, qq, kq, vq, workspace=ws)    # the call clears the status word
+    B.attn_fp8_read_status(ws)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
