@@ -12,18 +12,12 @@ namespace attnfp8 {
 // exceeds 1.75).  Returns the stored byte e + 127 (0 for an all-zero block) and the exact
 // multiplier 2^-e.
 __device__ __forceinline__ void block_scale(float amax, uint32_t& byte, float& inv) {
+  // adding 0x1FFFFF to the bit pattern carries into the exponent field exactly when the mantissa
+  // exceeds 1.75; biased exponents below 8 (zero and subnormal maxima included) clamp to byte 0;
+  // a non-finite maximum takes the largest scale
   const uint32_t bits = __float_as_uint(amax);
-  const int E = static_cast<int>((bits >> 23) & 0xFF);
-  const uint32_t mant = bits & 0x7FFFFF;
-  int eb;
-  if (E == 0) {
-    eb = 0;                                    // zero (or subnormal) block
-  } else if (E == 255) {
-    eb = 254;                                  // non-finite maximum
-  } else {
-    eb = E - 8 + (mant > 0x600000 ? 1 : 0);
-    eb = eb < 0 ? 0 : (eb > 254 ? 254 : eb);
-  }
+  int eb = max(static_cast<int>((bits + 0x1FFFFFu) >> 23) - 8, 0);
+  eb = bits >= 0x7F800000u ? 254 : eb;
   byte = static_cast<uint32_t>(eb);
   const int ib = 254 - eb;                     // biased exponent of 2^-e
   inv = ib > 0 ? __uint_as_float(static_cast<uint32_t>(ib) << 23) : __uint_as_float(0x00400000u);
