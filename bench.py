@@ -266,8 +266,9 @@ def main():
 
     # ---- end to end through the library with host buffers --------------------------------------
     # Host buffers in, host buffers out, every step: copies run on their own streams and overlap the
-    # kernels of the neighbouring steps (two slots of device inputs / outputs), as a user pipeline would.
-    n_slots = 2
+    # kernels of the neighbouring steps (three slots of device inputs / outputs), as a user pipeline would.
+    # The first upload and the last download are inside the timed region and overlap nothing.
+    n_slots = 3
     in_dev = [[torch.empty_like(x) for x in (q, k, v, dO)] for _ in range(n_slots)]
     out_dev = [[torch.empty_like(x) for x in (o, lse, dq, dk, dv)] for _ in range(n_slots)]
     outs_host = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)] for _ in range(n_slots)]
@@ -308,7 +309,7 @@ def main():
         torch.cuda.synchronize()
         return first.elapsed_time(last)
 
-    e2e_steps = 0 if args.no_e2e else max(4, min(args.steps, 16))
+    e2e_steps = 0 if args.no_e2e else max(4, args.steps)
     e2e_ms = 1e-9
     if e2e_steps:
         e2e_run(3)
