@@ -72,6 +72,9 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict_
 
   // ---- pass 1: rows.  8 elements per thread per step, 4 lanes per block of 32 channels.
   const int steps = kTokens * d / (8 * kThreads);
+  // unrolled so that the loads of several steps are in flight together (a CTA is short-lived:
+  // the latency of its own loads is most of its life)
+#pragma unroll 8
   for (int s = 0; s < steps; ++s) {
     const int ci = s * kThreads + tid;
     const int e0 = ci * 8;
