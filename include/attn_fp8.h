@@ -30,9 +30,10 @@
  *   - Changing delta_mode changes only `delta`, dQ and dK -- never O, LSE or dV.
  *
  * Supported shapes: seqlen a multiple of 128 (Nq == Nk, causal means key j <= query i);
- * heads_q a multiple of heads_kv; head dims (qk, v): {(64,64), (128,128)} for every attention
- * entry point, plus (192,128) and (256,256) where an entry point says so; the quantiser accepts
- * any d that is a multiple of 32 up to 256.  Anything else returns ATTN_ERR_UNSUPPORTED.
+ * heads_q a multiple of heads_kv; head dims (qk, v): (64,64), (128,128), (192,128), (256,256) for
+ * every attention entry point in FP8 mode, (64,64) and (128,128) in BF16 mode and with protected dP;
+ * the quantiser accepts any d that is a multiple of 32 up to 256.  Anything else returns
+ * ATTN_ERR_UNSUPPORTED.
  *
  * BF16 mode (attn_params_t.precision = ATTN_PREC_BF16; the paper's BF16 reference point, Section
  * 2.1): the same kernels with BF16 operands and no block scales.  An attn_qtensor_t then carries
@@ -154,7 +155,6 @@ attn_status_t attn_fp8_prepare_bf16(const void* src, int32_t src_dtype, int32_t 
  * S = scale * Q^ K^^T over key tiles with a running INTEGER power-of-two shift, normaliser l
  * taken from the exponentials BEFORE the FP8 cast, probabilities quantised in-register in
  * blocks of 32 keys, O = (P^ V^) / l.
- *   head dims: (64,64), (128,128), (192,128), (256,256) in FP8 mode; (64,64), (128,128) in BF16 mode
  *   reads   q.row_*, k.row_*, v.col_*
  *   writes  o_bf16 [B, Hq, N, dv] (BF16), lse [B, Hq, N] (FP32, natural log)                  */
 attn_status_t attn_fp8_fwd(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
