@@ -28,7 +28,7 @@ class Workload:
     head_dim_v: int
     causal: bool
     dtype: str            # "bf16" or "fp32": source dtype of Q, K, V, dO
-    recipe: str           # "iid", "qknorm", "outlier_rope", "plain", "student_t"
+    recipe: str           # "iid", "qknorm", "outlier_rope", "outlier_rope_aligned" (stress), "plain", "student_t"
     dO_std: float
 
     @property
@@ -81,6 +81,19 @@ def _rope_half_split(x: torch.Tensor, base: float = 10000.0) -> torch.Tensor:
     return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1)
 
 
+def _aligned_outlier_gain(w: Workload, heads: int, d: int) -> torch.Tensor:
+    """Stress variant of the outlier recipe: a query head shares the four outlier channels of its
+    KV head (scores then have a standard deviation of ~70 and rows are nearly one-hot)."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(SEED_BASE + 100 * w.index + 50)
+    per_kv = [torch.randperm(d, generator=g)[:4] for _ in range(w.heads_kv)]
+    gain = torch.ones(heads, d)
+    group = heads // w.heads_kv
+    for h in range(heads):
+        gain[h, per_kv[h // group]] = 20.0
+    return gain
+
+
 def _condition_qk(w: Workload, x: torch.Tensor, g: torch.Generator) -> torch.Tensor:
     if w.recipe == "qknorm":
         return x / torch.sqrt(x.pow(2).mean(dim=-1, keepdim=True) + 1e-6)
@@ -90,6 +103,8 @@ def _condition_qk(w: Workload, x: torch.Tensor, g: torch.Generator) -> torch.Ten
         for h in range(heads):
             gain[h, torch.randperm(d, generator=g)[:4]] = 20.0
         return _rope_half_split(x * gain[None, :, None, :])
+    if w.recipe == "outlier_rope_aligned":
+        return _rope_half_split(x * _aligned_outlier_gain(w, x.shape[1], x.shape[-1])[None, :, None, :])
     if w.recipe == "student_t":
         heads, d = x.shape[1], x.shape[-1]
         z = torch.randn(heads, d, generator=g)
