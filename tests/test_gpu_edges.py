@@ -67,14 +67,21 @@ def test_nearly_one_hot_rows_stress():
     assert torch.isfinite(got["o"].float()).all() and torch.isfinite(got["lse"]).all()
     lse, delta = to_np(got["lse"]), to_np(got["delta"])
     assert rel_fro(delta, A.emu_delta(qn, kn, vn, dOn, lse, w.softmax_scale, w.causal)) <= 1e-4
-    # On a nearly one-hot row dS = P (dP - D) is a difference of nearly equal numbers: the FP32
-    # probabilities of the kernel (ex2.approx, 2^-22) and the float64 ones of the oracle then differ
-    # by percents of what is left of dS, whatever the operand precision.  The bound is therefore
-    # loose here; dV, which does not go through that difference, keeps the usual one.
+    # Nearly every row is one-hot to ~1e-5 and has a vanishing dS, so a head's whole gradient sits in
+    # a handful of rows and elements; where the largest of them lies on an E4M3 rounding tie (here
+    # one does, 5e-7 away), the float64 oracle and the FP32 kernel round it to neighbouring codes and
+    # that single step is percents of dQ.  dQ is therefore bounded loosely as a whole and by the usual
+    # tolerance once the single worst row of each head is set aside.
     dQ, dK, dV, _, _ = A.emu_backward(qn, kn, vn, dOn, lse, delta, w.softmax_scale, w.causal)
     errs = {n: rel_fro(to_np(got[n]), r) for n, r in (("dq", dQ), ("dk", dK), ("dv", dV))}
+    dq_gpu = to_np(got["dq"])
+    row_err = np.linalg.norm(dq_gpu - dQ, axis=-1)                      # [B, Hq, N]
+    keep = np.ones_like(row_err, dtype=bool)
+    np.put_along_axis(keep, row_err.argmax(axis=-1)[..., None], False, axis=-1)
+    errs["dq_without_worst_row"] = float(np.linalg.norm((dq_gpu - dQ)[keep]) / np.linalg.norm(dQ[keep]))
     print("\nstress errors", errs)
-    assert errs["dv"] <= 5e-3 and errs["dq"] <= 2e-2 and errs["dk"] <= 1e-2
+    assert errs["dv"] <= 5e-3 and errs["dk"] <= 5e-3
+    assert errs["dq"] <= 2e-2 and errs["dq_without_worst_row"] <= 5e-3
 
 
 def test_first_row_sees_one_key():
