@@ -276,10 +276,12 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
   int* status = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD), st, &status));
+  // Key-major kernel first: its CTAs are few and long, so its last wave leaves SMs idle, which
+  // the many short CTAs of the query-major kernel, launched behind it, fill.
+  if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));
   if (want_dq)
     CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, post_rowsum, post_rowabs,
-                        status, st));
-  if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));
+                        status, st, /*behind_dkdv=*/want_dkdv));
   return ATTN_OK;
 }
 

@@ -215,6 +215,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  // the query-major kernel of the same call may be queued behind this grid: let its CTAs take the
+  // SMs that this grid's last wave leaves idle (nothing it does depends on this grid's output)
+  griddep_launch_dependents();
   const uint32_t tmem = sm.tmem_base;
 
   if (warp == 0) {

@@ -132,6 +132,7 @@ struct QmParams {
   float* post_rowabs;
   int* status;
   int N, Hq, Hkv, dqk, dv, causal;
+  int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
   float scale, scale_log2;
 };
 
@@ -523,12 +524,18 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+  // This grid may have started while the grid ahead of it was draining.  One CTA, the last in
+  // launch order, stays until that grid has completed, so that the completion of this grid
+  // implies the completion of both for whatever follows in the stream.
+  if (p.tail_wait && tid == 0 && blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1 && blockIdx.z == gridDim.z - 1)
+    griddep_wait();
 }
 
 template <class C>
 attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                               const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
-                              float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
+                              float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
+                              bool behind_dkdv) {
   constexpr bool kDQ = C::kDQ;
   static_assert(sizeof(QmSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
@@ -553,12 +560,26 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
+  p.tail_wait = behind_dkdv ? 1 : 0;
   const size_t smem = sizeof(QmSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   const int rq = kDQ ? (s.dqk + 127) / 128 : 1;
   dim3 grid(s.Hq * rq, s.N / kTile, s.B);
-  qmajor_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
+  if (behind_dkdv) {
+    // the key-major kernel ahead in the stream reads what this one reads and writes other buffers:
+    // this grid may take the SMs that kernel's last wave leaves idle
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, qmajor_kernel<C>, p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
+    if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: launch: %s", cudaGetErrorString(e));
+  } else {
+    qmajor_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_dO, tm_k, tm_v, tm_kc);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
@@ -567,12 +588,13 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
 template <bool kDQ>
 attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
-                            float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
+                            float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
+                            bool behind_dkdv = false) {
   const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.ebv + 127) / 128;
 #define ATTN_QM_CASE(EB, CQ, CV, EBV)                                                                         \
   if (s.eb == EB && s.ebv == EBV && cq == CQ && cv == CV)                                                     \
     return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV, EBV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
-                                                       post_rowsum, post_rowabs, status, stream);
+                                                       post_rowsum, post_rowabs, status, stream, behind_dkdv);
   ATTN_QM_CASE(1, 1, 1, 1)
   ATTN_QM_CASE(1, 2, 1, 1)
   ATTN_QM_CASE(1, 2, 2, 1)
@@ -661,8 +683,9 @@ attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtenso
 
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta, void* dq, float* rowsum, float* rowabs,
-                            float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream) {
-  return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, post_rowsum, post_rowabs, status, stream);
+                            float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream, bool behind_dkdv) {
+  return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, post_rowsum, post_rowabs, status, stream,
+                             behind_dkdv);
 }
 
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,

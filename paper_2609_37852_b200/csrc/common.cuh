@@ -46,7 +46,8 @@ attn_status_t launch_consistent_delta(const AttnShape& s, attn_qtensor_t dO, con
                                       cudaStream_t stream);
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                             attn_qtensor_t dO, const float* lse, const float* delta, void* dq, float* rowsum,
-                            float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream);
+                            float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
+                            bool behind_dkdv = false);
 attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                               attn_qtensor_t dO, const float* lse, const float* delta, void* dk, void* dv,
                               int* status, cudaStream_t stream);

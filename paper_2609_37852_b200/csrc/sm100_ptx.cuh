@@ -182,6 +182,12 @@ __device__ __forceinline__ void tmem_alloc(uint32_t* smem_holder, uint32_t ncols
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                ::"r"(smem_u32(smem_holder)), "r"(ncols) : "memory");
 }
+// Programmatic dependent launch.  launch_dependents: once every CTA of this grid has executed it
+// (or exited), a grid launched behind it with programmatic stream serialisation may begin to
+// occupy SMs that this grid no longer fills.  wait: returns once the grids this one was made
+// dependent on have completed and their writes are visible (at once when there are none).
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tmem_relinquish() {
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
