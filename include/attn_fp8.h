@@ -127,6 +127,31 @@ size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols);
 attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
                                 int32_t d, attn_qtensor_t out, void* stream);
 
+/* One tensor of a batched quantiser call: the arguments of attn_fp8_quantize.                   */
+typedef struct {
+  const void* src;
+  int32_t src_dtype;
+  int32_t B, H, N, d;
+  attn_qtensor_t out;
+} attn_quantize_job_t;
+
+#define ATTN_QUANTIZE_MAX_JOBS 8
+#define ATTN_STATUS_WORKSPACE_BYTES 256   /* workspace that carries only the device status word */
+
+/* attn_fp8_quantize of up to ATTN_QUANTIZE_MAX_JOBS tensors (the four operands of a step) in ONE
+ * launch: a persistent grid walks the 128-token tiles of all tensors and keeps the next tile in
+ * flight (bulk asynchronous copies into a shared-memory ring) while it quantises the current one.
+ * Outputs are bit-identical to those of attn_fp8_quantize on each tensor.
+ *   jobs       host array; every job as attn_fp8_quantize documents; all jobs share one src_dtype
+ *              (ATTN_ERR_INVALID_ARG otherwise); outputs of different jobs must not overlap
+ *   workspace  device, >= ATTN_STATUS_WORKSPACE_BYTES, 16-byte aligned: its status word reports a
+ *              copy that never completed (attn_fp8_read_status -> ATTN_ERR_TIMEOUT), as for the
+ *              attention entry points; a workspace of those calls may be passed
+ * Shapes whose two-tile ring does not fit in shared memory (FP32 source with d = 256) are
+ * processed by one attn_fp8_quantize launch per job instead.                                     */
+attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n_jobs, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
 /* The quantiser with the paper's operand producer fused in front (Appendix "Operands, Scaling, and
  * Accumulation"), for callers that hold q / k BEFORE rotary embedding, scale folding or key centering:
  *   1. rotary embedding, if rope_cos / rope_sin (FP32 [N, d/2], device) are given: channel c < d/2 is

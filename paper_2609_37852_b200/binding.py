@@ -34,7 +34,7 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
-    "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
+    "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
 )
 
 
@@ -192,6 +192,53 @@ def attn_fp8_quantize(src: torch.Tensor, want_row: bool = True, want_col: bool =
         raise ValueError("out was allocated for another shape")
     _check(_lib.attn_fp8_quantize(_ptr(src), dt, B, H, N, d, out.c_struct(), _stream(stream)))
     return out
+
+
+class _QuantizeJob(ctypes.Structure):
+    _fields_ = [("src", _vp), ("src_dtype", _i32), ("B", _i32), ("H", _i32), ("N", _i32), ("d", _i32),
+                ("out", _QTensor)]
+
+
+ATTN_QUANTIZE_MAX_JOBS = 8
+ATTN_STATUS_WORKSPACE_BYTES = 256
+_lib.attn_fp8_quantize_batch.restype = _i32
+_lib.attn_fp8_quantize_batch.argtypes = [ctypes.POINTER(_QuantizeJob), _i32, _vp, _sz, _vp]
+
+
+def attn_fp8_quantize_batch(srcs, outs=None, want=None, workspace=None, stream=None):
+    """attn_fp8_quantize of several tensors (each [B, H, N, d], one dtype) in one launch.
+    ``outs``: QTensors of earlier calls to reuse; ``want``: per tensor (want_row, want_col) when
+    ``outs`` is None.  Returns (list of QTensor, workspace)."""
+    srcs = list(srcs)
+    if outs is None:
+        want = want or [(True, True)] * len(srcs)
+        outs = []
+        for x, (wr, wc) in zip(srcs, want):
+            B, H, N, d = x.shape
+            q = QTensor(shape=(B, H, N, d))
+            u8 = dict(dtype=torch.uint8, device=x.device)
+            if wr:
+                q.row_codes = torch.empty((B, H, N, d), **u8)
+                q.row_scales = torch.empty(attn_fp8_scale_bytes(B, H, N, d), **u8)
+            if wc:
+                q.col_codes = torch.empty((B, H, d, N), **u8)
+                q.col_scales = torch.empty(attn_fp8_scale_bytes(B, H, d, N), **u8)
+            outs.append(q)
+    jobs = (_QuantizeJob * len(srcs))()
+    for j, (x, q) in enumerate(zip(srcs, outs)):
+        if not x.is_cuda or not x.is_contiguous() or x.dim() != 4:
+            raise ValueError("every source must be a contiguous CUDA tensor [B, H, N, d]")
+        if x.dtype not in (torch.bfloat16, torch.float32):
+            raise ValueError("sources must be bfloat16 or float32")
+        if tuple(q.shape) != tuple(x.shape):
+            raise ValueError("an output was allocated for another shape")
+        B, H, N, d = x.shape
+        jobs[j] = _QuantizeJob(_ptr(x), ATTN_SRC_BF16 if x.dtype == torch.bfloat16 else ATTN_SRC_FP32, B, H, N, d,
+                               q.c_struct())
+    if workspace is None:
+        workspace = torch.empty(ATTN_STATUS_WORKSPACE_BYTES, dtype=torch.uint8, device=srcs[0].device)
+    _check(_lib.attn_fp8_quantize_batch(jobs, len(srcs), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return list(outs), workspace
 
 
 _lib.attn_fp8_quantize_fused.restype = _i32

@@ -138,8 +138,8 @@ size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols) {
   return static_cast<size_t>(B * H) * scale_tiles_per_slab(rows, cols) * 512;
 }
 
-attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
-                                attn_qtensor_t out, void* stream) {
+static attn_status_t check_quantize_args(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
+                                         const attn_qtensor_t& out) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return fail(ATTN_ERR_INVALID_ARG, "sizes must be positive");
   if (src_dtype != ATTN_SRC_BF16 && src_dtype != ATTN_SRC_FP32)
     return fail(ATTN_ERR_INVALID_ARG, "src_dtype %d is neither BF16 nor FP32", src_dtype);
@@ -152,8 +152,43 @@ attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, i
     return fail(ATTN_ERR_INVALID_ARG, "codes and scales of an orientation must be given together");
   if (out.row_codes) { CHECK(check_ptr(out.row_codes, "row_codes")); CHECK(check_ptr(out.row_scales, "row_scales")); }
   if (out.col_codes) { CHECK(check_ptr(out.col_codes, "col_codes")); CHECK(check_ptr(out.col_scales, "col_scales")); }
+  return ATTN_OK;
+}
+
+attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
+                                attn_qtensor_t out, void* stream) {
+  CHECK(check_quantize_args(src, src_dtype, B, H, N, d, out));
   CHECK(check_device());
   return launch_quantize(src, src_dtype, B, H, N, d, out, static_cast<cudaStream_t>(stream));
+}
+
+attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n_jobs, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  if (!jobs) return fail(ATTN_ERR_INVALID_ARG, "jobs is NULL");
+  if (n_jobs < 1 || n_jobs > ATTN_QUANTIZE_MAX_JOBS)
+    return fail(ATTN_ERR_INVALID_ARG, "n_jobs must be 1..%d (got %d)", ATTN_QUANTIZE_MAX_JOBS, n_jobs);
+  int d_max = 0;
+  long long tiles = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const attn_quantize_job_t& q = jobs[j];
+    CHECK(check_quantize_args(q.src, q.src_dtype, q.B, q.H, q.N, q.d, q.out));
+    if (q.src_dtype != jobs[0].src_dtype) return fail(ATTN_ERR_INVALID_ARG, "all jobs of a batch must share one src_dtype");
+    d_max = q.d > d_max ? q.d : d_max;
+    tiles += static_cast<long long>(q.B) * q.H * (q.N / 128);
+  }
+  if (tiles > 0x7fffffffLL) return fail(ATTN_ERR_UNSUPPORTED, "batch of %lld tiles exceeds the 2^31 - 1 a launch indexes", tiles);
+  CHECK(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* status = nullptr;
+  CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
+  if (!quantize_batch_fits(jobs[0].src_dtype, d_max)) {
+    for (int j = 0; j < n_jobs; ++j) {
+      const attn_quantize_job_t& q = jobs[j];
+      CHECK(launch_quantize(q.src, q.src_dtype, q.B, q.H, q.N, q.d, q.out, st));
+    }
+    return ATTN_OK;
+  }
+  return launch_quantize_batch(jobs, n_jobs, status, st);
 }
 
 attn_status_t attn_fp8_quantize_fused(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,

@@ -13,7 +13,7 @@ namespace attnfp8 {
 attn_status_t fail(attn_status_t code, const char* fmt, ...);
 
 // Bytes at the head of every workspace reserved for the device status word.
-constexpr size_t kWorkspaceHeaderBytes = 256;
+constexpr size_t kWorkspaceHeaderBytes = ATTN_STATUS_WORKSPACE_BYTES;
 
 // cuTensorMapEncodeTiled fetched through the runtime (no link-time dependency on libcuda).
 // Encodes a 2-D uint8 tensor [rows, row_bytes] (row pitch == row_bytes) with a
@@ -34,6 +34,8 @@ attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int 
 attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H, int N, int d, const float* cos,
                                     const float* sin, float scale, float* mean, attn_qtensor_t out,
                                     cudaStream_t stream);
+attn_status_t launch_quantize_batch(const attn_quantize_job_t* jobs, int n_jobs, int* status, cudaStream_t stream);
+bool quantize_batch_fits(int src_dtype, int d_max);   // the two-tile ring fits in shared memory
 attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, int N, int d, void* row_out, void* col_out,
                                  cudaStream_t stream);
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,

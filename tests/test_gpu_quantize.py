@@ -65,3 +65,70 @@ def test_quantize_single_orientation_and_errors():
     with pytest.raises(binding.AttnFp8Error) as e:
         binding.attn_fp8_quantize(torch.randn(1, 1, 100, 64, device="cuda"))
     assert e.value.status == 2
+
+
+def _same(a, b):
+    for f in ("row_codes", "row_scales", "col_codes", "col_scales"):
+        x, y = getattr(a, f), getattr(b, f)
+        assert (x is None) == (y is None), f
+        if x is not None:
+            assert torch.equal(x, y), f
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("gqa8k_outlier", dict(heads_q=8, heads_kv=2, seqlen=1024)),        # d = 128, more tiles than resident CTAs
+    ("tiny", dict(seqlen=256)),                                          # FP32 source, d = 64, two tiles per tensor
+    ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=384)),                  # head dims 192 and 128 in one launch
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=256)),             # d = 256
+])
+def test_quantize_batch_is_bit_identical_to_single_calls(name, kw):
+    """The persistent multi-tensor launch against the oracle (through the single-tensor check) and
+    against attn_fp8_quantize on each tensor, orientations as the attention calls need them."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    srcs = [x.cuda() for x in workloads.make_inputs(w)]
+    want = [(True, True), (True, True), (True, True), (True, True)]
+    outs, ws = B.attn_fp8_quantize_batch(srcs, want=want)
+    B.attn_fp8_read_status(ws)
+    for x, q in zip(srcs, outs):
+        _same(q, B.attn_fp8_quantize(x))
+    # against the oracle directly, first tensor
+    xn = to_np(srcs[0]); Bn, H, N, d = srcs[0].shape
+    rc, rs = mxfp8.quantize(xn, axis=-1)
+    assert np.array_equal(outs[0].row_codes.cpu().numpy(), rc)
+    assert np.array_equal(B.unpack_scales(outs[0].row_scales, Bn, H, N, d).cpu().numpy(), rs)
+    # single orientations, outputs prefilled: only what was asked for is written, and all of it
+    want = [(True, False), (False, True), (True, True), (False, True)]
+    outs2, _ = B.attn_fp8_quantize_batch(srcs, want=want, workspace=ws)
+    for q in outs2:
+        for f in ("row_codes", "row_scales", "col_codes", "col_scales"):
+            if getattr(q, f) is not None:
+                getattr(q, f).fill_(0xAB)
+    outs2, _ = B.attn_fp8_quantize_batch(srcs, outs=outs2, workspace=ws)
+    B.attn_fp8_read_status(ws)
+    for (wr, wc), q, full in zip(want, outs2, outs):
+        assert (q.row_codes is not None) == wr and (q.col_codes is not None) == wc
+        if wr:
+            assert torch.equal(q.row_codes, full.row_codes) and torch.equal(q.row_scales, full.row_scales)
+        if wc:
+            assert torch.equal(q.col_codes, full.col_codes) and torch.equal(q.col_scales, full.col_scales)
+
+
+def test_quantize_batch_fallback_and_errors():
+    from paper_2609_37852_b200 import binding as B
+    g = torch.Generator().manual_seed(5)
+    # FP32 source with d = 256: the two-tile ring does not fit, one launch per tensor instead
+    xs = [torch.randn((1, 2, 256, 256), generator=g).cuda(), torch.randn((1, 1, 128, 256), generator=g).cuda()]
+    outs, ws = B.attn_fp8_quantize_batch(xs)
+    B.attn_fp8_read_status(ws)
+    for x, q in zip(xs, outs):
+        _same(q, B.attn_fp8_quantize(x))
+    with pytest.raises(B.AttnFp8Error) as e:                               # mixed source dtypes
+        B.attn_fp8_quantize_batch([xs[0], xs[1].to(torch.bfloat16)])
+    assert e.value.status == 1
+    with pytest.raises(B.AttnFp8Error) as e:                               # too many tensors
+        B.attn_fp8_quantize_batch([xs[1]] * 9)
+    assert e.value.status == 1
+    with pytest.raises(B.AttnFp8Error) as e:                               # status workspace too small
+        B.attn_fp8_quantize_batch([xs[1]], workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
