@@ -57,8 +57,11 @@ class Case:
         B.attn_fp8_read_status(self.ws)
 
     def prep(self):
-        for x, t in zip(self.src, (self.q, self.k, self.v, self.dO)):
-            self.prepare(x, out=t)
+        if self.prec == "bf16":
+            for x, t in zip(self.src, (self.q, self.k, self.v, self.dO)):
+                self.prepare(x, out=t)
+        else:                                            # the four operands in one quantiser launch
+            B.attn_fp8_quantize_batch(self.src, outs=(self.q, self.k, self.v, self.dO), workspace=self.ws)
 
     def fwd(self):
         B.attn_fp8_fwd(self.params, self.q, self.k, self.v, o=self.o, lse=self.lse, workspace=self.ws)
