@@ -22,8 +22,10 @@ def _run(w, tensors, prec="mxfp8"):
     params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
                           w.softmax_scale, precision=B.ATTN_PREC_BF16 if prec == "bf16" else B.ATTN_PREC_MXFP8)
     dev = [x.cuda() for x in tensors]
-    prep = B.attn_fp8_prepare_bf16 if prec == "bf16" else B.attn_fp8_quantize
-    qq, kq, vq, dOq = (prep(x) for x in dev)
+    if prec == "bf16":
+        qq, kq, vq, dOq = (B.attn_fp8_prepare_bf16(x) for x in dev)
+    else:                                     # as bench.py does: the four operands in one quantiser launch
+        (qq, kq, vq, dOq), _ = B.attn_fp8_quantize_batch(dev)
     o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
     delta, ws = B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
     dq, dk, dv, rs, ra, ws = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, diagnostics=True, workspace=ws)

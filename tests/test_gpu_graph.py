@@ -1,7 +1,7 @@
 """The whole path under CUDA-graph capture.
 
 Every entry point only enqueues work on the caller's stream (the one synchronising call is
-attn_fp8_read_status), so a step -- quantiser, forward, row correction, gradient pass -- can be
+attn_fp8_read_status), so a step -- batched quantiser, forward, row correction, gradient pass -- can be
 captured once and replayed.  The test captures a step into a graph, replays it on two different
 inputs written into the captured buffers and requires every output to be bit-identical to an
 eager step on the same input.  The gradient pass launches its query-major kernel behind the
@@ -17,8 +17,7 @@ pytestmark = pytest.mark.gpu
 
 def _step(B, params, src, bufs):
     """One step into preallocated buffers (no allocation, no synchronisation)."""
-    for x, t in zip(src, bufs["operands"]):
-        B.attn_fp8_quantize(x, out=t)
+    B.attn_fp8_quantize_batch(src, outs=bufs["operands"], workspace=bufs["ws"])
     qq, kq, vq, dOq = bufs["operands"]
     B.attn_fp8_fwd(params, qq, kq, vq, o=bufs["o"], lse=bufs["lse"], workspace=bufs["ws"])
     B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, bufs["lse"], delta=bufs["delta"], workspace=bufs["ws"])
