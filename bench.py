@@ -220,7 +220,7 @@ def main():
     dq = torch.empty((w.batch, w.heads_q, w.seqlen, w.head_dim_qk), **bf)
     dk = torch.empty((w.batch, w.heads_kv, w.seqlen, w.head_dim_qk), **bf)
     dv = torch.empty((w.batch, w.heads_kv, w.seqlen, w.head_dim_v), **bf)
-    ws = torch.empty(max(B.attn_fp8_workspace_bytes(params, i) for i in range(3)), dtype=torch.uint8, device=dev)
+    ws = B.new_workspace(max(B.attn_fp8_workspace_bytes(params, i) for i in range(3)), dev)
 
     def prepare_all(srcs):
         """Q, K, V, dO -> the operand buffers: one batched quantiser launch, or the four BF16 copies."""

@@ -24,6 +24,8 @@
  *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*) and returns;
  *     it never synchronises and never reads device memory from the host, except
  *     attn_fp8_read_status, which says so.
+ *   - Calls that take a `workspace` report device-side failures through its sticky status word
+ *     (see attn_fp8_workspace_bytes): initialise a workspace once, read the status when needed.
  *   - Errors are return codes; nothing aborts or traps.  Arguments are validated before any
  *     launch.  attn_fp8_last_error() gives a thread-local message for the last failure.
  *   - Results of quantize, fwd, bwd_delta and bwd are bitwise reproducible run to run.
@@ -261,10 +263,9 @@ attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q,
  *     rejected with ATTN_ERR_WORKSPACE and a message naming both sizes.
  *   - The first call on each device looks up the array's device address (a one-time runtime query
  *     made with that device current); make that first call outside of any stream capture.
- *   - All calls on a device share the one array, and it keeps the previous call's contents; the
- *     call clears the part that has to start at zero.  Two calls whose kernels overlap on the GPU
- *     (different streams, no ordering between them) race on it: order them, or use attn_fp8_fwd
- *     with separate workspaces.
+ *   - All calls on a device share the one array, and it keeps what earlier calls left; its
+ *     status word is only ever set by a kernel that gave up, so nothing has to be cleared between
+ *     calls and overlapping calls (different streams) do not disturb one another.
  *   - The device status word lands in the built-in array and is not reported by
  *     attn_fp8_read_status; callers that want the time-out report use attn_fp8_fwd.
  * Arguments, layouts and error codes are otherwise those of attn_fp8_fwd.                       */
@@ -272,14 +273,24 @@ attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, att
                                    void* o_bf16, float* lse, void* stream);
 
 /* Bytes of workspace the given entry point needs for `p` (attn_ws_kind_t).  The workspace is
- * scratch: contents are undefined between calls, the library clears what it needs.  Its first
- * word is the device-side status that attn_fp8_read_status returns.                           */
+ * scratch owned by the caller; one workspace may serve all entry points of a stream.  Its first
+ * word is the device-side status word.  The status is STICKY: kernels only ever set it (a bounded
+ * wait that gave up, a launch that found its shared memory misaligned), no entry point clears it,
+ * so one attn_fp8_read_status at the end of a chain of calls reports a failure of any of them.
+ * A workspace must be initialised once before its first use (attn_fp8_workspace_init, or any other
+ * way of zeroing its first ATTN_STATUS_WORKSPACE_BYTES bytes): an uninitialised status word reads
+ * as an error.                                                                                 */
 size_t attn_fp8_workspace_bytes(const attn_params_t* p, int32_t which);
 
+/* Enqueues the clearing of the status header of `workspace` (>= ATTN_STATUS_WORKSPACE_BYTES,
+ * 16-byte aligned) on `stream`.  Once per workspace, before its first use.                     */
+attn_status_t attn_fp8_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
 /* Waits for `stream`, copies the status word of `workspace` to the host and returns it:
- * ATTN_OK, or ATTN_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs of that
- * call are then undefined).  This is the one call that synchronises.                          */
-attn_status_t attn_fp8_read_status(const void* workspace, void* stream);
+ * ATTN_OK, or ATTN_ERR_TIMEOUT / ATTN_ERR_ALIGNMENT if a kernel of any call since the last read (or
+ * the initialisation) gave up (outputs of those calls are then undefined).  A non-OK status is
+ * cleared by the read.  This is the one call that synchronises.                               */
+attn_status_t attn_fp8_read_status(void* workspace, void* stream);
 
 /* Self-test of the device-side time-out report: enqueues a one-CTA kernel that waits, with a limit
  * of about 2 ms, on a barrier nothing completes, gives up and sets the status word of `workspace`

@@ -34,7 +34,7 @@ ATTN_WS_FWD, ATTN_WS_BWD_DELTA, ATTN_WS_BWD = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
-    "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
+    "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_workspace_init", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
 )
 
 
@@ -236,7 +236,7 @@ def attn_fp8_quantize_batch(srcs, outs=None, want=None, workspace=None, stream=N
         jobs[j] = _QuantizeJob(_ptr(x), ATTN_SRC_BF16 if x.dtype == torch.bfloat16 else ATTN_SRC_FP32, B, H, N, d,
                                q.c_struct())
     if workspace is None:
-        workspace = torch.empty(ATTN_STATUS_WORKSPACE_BYTES, dtype=torch.uint8, device=srcs[0].device)
+        workspace = new_workspace(ATTN_STATUS_WORKSPACE_BYTES, srcs[0].device)
     _check(_lib.attn_fp8_quantize_batch(jobs, len(srcs), _ptr(workspace), workspace.numel(), _stream(stream)))
     return list(outs), workspace
 
@@ -309,10 +309,25 @@ def attn_fp8_workspace_bytes(params: AttnParams, which: int) -> int:
     return int(_lib.attn_fp8_workspace_bytes(ctypes.byref(c), which))
 
 
+_lib.attn_fp8_workspace_init.restype = _i32
+_lib.attn_fp8_workspace_init.argtypes = [_vp, _sz, _vp]
+
+
+def attn_fp8_workspace_init(workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    """Clears the status header of a caller-made workspace (once, before its first use)."""
+    _check(_lib.attn_fp8_workspace_init(_ptr(workspace), workspace.numel(), _stream(stream)))
+    return workspace
+
+
+def new_workspace(nbytes: int, device, stream=None) -> torch.Tensor:
+    """A workspace of ``nbytes`` (at least the status header) with its status word cleared."""
+    ws = torch.empty(max(int(nbytes), ATTN_STATUS_WORKSPACE_BYTES), dtype=torch.uint8, device=device)
+    return attn_fp8_workspace_init(ws, stream)
+
+
 def _workspace(params, which, workspace, device):
-    need = attn_fp8_workspace_bytes(params, which)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+        workspace = new_workspace(attn_fp8_workspace_bytes(params, which), device)
     return workspace
 
 

@@ -113,11 +113,11 @@ static attn_status_t check_ptr(const void* p, const char* name) {
     if (st_ != ATTN_OK) return st_;     \
   } while (0)
 
-static attn_status_t prepare_workspace(void* ws, size_t ws_bytes, size_t need, cudaStream_t stream, int** status) {
+// The status word is sticky: kernels only ever set it, attn_fp8_workspace_init and
+// attn_fp8_read_status clear it.  Nothing is enqueued here.
+static attn_status_t prepare_workspace(void* ws, size_t ws_bytes, size_t need, cudaStream_t, int** status) {
   if (!ws || ws_bytes < need) return fail(ATTN_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
   if (!aligned16(ws)) return fail(ATTN_ERR_ALIGNMENT, "workspace is not 16-byte aligned");
-  cudaError_t e = cudaMemsetAsync(ws, 0, kWorkspaceHeaderBytes, stream);
-  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "cudaMemsetAsync(workspace): %s", cudaGetErrorString(e));
   *status = static_cast<int*>(ws);
   return ATTN_OK;
 }
@@ -354,12 +354,25 @@ attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_q
                   workspace_bytes, stream, false, true);
 }
 
-attn_status_t attn_fp8_read_status(const void* workspace, void* stream) {
+attn_status_t attn_fp8_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace || workspace_bytes < kWorkspaceHeaderBytes)
+    return fail(ATTN_ERR_WORKSPACE, "workspace of at least %zu bytes needed, %zu given", kWorkspaceHeaderBytes, workspace_bytes);
+  if (!aligned16(workspace)) return fail(ATTN_ERR_ALIGNMENT, "workspace is not 16-byte aligned");
+  cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "workspace_init: cudaMemsetAsync: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+attn_status_t attn_fp8_read_status(void* workspace, void* stream) {
   if (!workspace) return fail(ATTN_ERR_INVALID_ARG, "workspace is NULL");
   int host = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess && host != 0) {          // reported once: clear it for the calls that follow
+    e = cudaMemsetAsync(workspace, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  }
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "read_status: %s", cudaGetErrorString(e));
   if (host == ATTN_ERR_ALIGNMENT)
     return fail(ATTN_ERR_ALIGNMENT, "a kernel found its dynamic shared memory not 1024-byte aligned and did not run");
@@ -423,7 +436,7 @@ extern "C" attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtens
   CHECK(builtin_scratch_for_current_device(&scratch));
   int* status = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the array keeps whatever the previous call left: clear the part that must start at zero
+  // the array keeps whatever earlier calls left; its status word is only ever set, so nothing needs clearing
   CHECK(prepare_workspace(scratch, kBuiltinScratchBytes, need, st, &status));
   return launch_fwd(s, q, k, v, o_bf16, lse, status, st);
 }

@@ -225,6 +225,19 @@ def test_expired_wait_is_reported_and_the_context_survives():
         B.attn_fp8_read_status(ws)
     assert e.value.status == 7
     assert time.perf_counter() - t0 < 1.0                              # it gave up within its limit
-    o2, lse2, ws = B.attn_fp8_fwd(params, qq, kq, vq, workspace=ws)    # the call clears the status word
+    B.attn_fp8_read_status(ws)                                         # reported once: the read cleared it
+    # the status is sticky across calls: a failure is still reported after later, healthy calls
+    B.attn_fp8_selftest_timeout(ws)
+    o2, lse2, ws = B.attn_fp8_fwd(params, qq, kq, vq, workspace=ws)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_read_status(ws)
+    assert e.value.status == 7
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)               # the forward itself was healthy
+    o3, lse3, ws = B.attn_fp8_fwd(params, qq, kq, vq, workspace=ws)
     B.attn_fp8_read_status(ws)
-    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+    assert torch.equal(o, o3) and torch.equal(lse, lse3)
+    # a workspace the caller made has to be initialised once: garbage in the status word reads as an error
+    raw = torch.full((B.attn_fp8_workspace_bytes(params, 0),), 0xFF, dtype=torch.uint8, device="cuda")
+    B.attn_fp8_workspace_init(raw)
+    B.attn_fp8_fwd(params, qq, kq, vq, workspace=raw)
+    B.attn_fp8_read_status(raw)

@@ -29,7 +29,7 @@ def _buffers(B, params, src):
     operands = [B.attn_fp8_quantize(x) for x in src]
     qq, kq, vq, dOq = operands
     o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
-    ws = torch.empty(max(B.attn_fp8_workspace_bytes(params, i) for i in range(3)), dtype=torch.uint8, device="cuda")
+    ws = B.new_workspace(max(B.attn_fp8_workspace_bytes(params, i) for i in range(3)), "cuda")
     delta, _ = B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
     dq, dk, dv, _, _, _ = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, workspace=ws)
     return dict(operands=operands, o=o, lse=lse, ws=ws, delta=delta, dq=dq, dk=dk, dv=dv)
