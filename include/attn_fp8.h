@@ -125,7 +125,9 @@ size_t attn_fp8_scale_bytes(int64_t B, int64_t H, int64_t rows, int64_t cols);
  *   out        the orientations whose pointers are non-NULL are written (codes AND scales of an
  *              orientation must both be given); all 16-byte aligned
  *   N % 128 == 0, d % 32 == 0, 32 <= d <= 256.
- * Non-finite inputs do not trap: NaN encodes as 0x7F, +-Inf saturates to +-448.               */
+ * Non-finite inputs do not trap: NaN encodes as 0x7F, +-Inf saturates to +-448.
+ * The first call on each device looks up the address of the library's built-in scratch (a
+ * one-time runtime query): make that first call outside of any stream capture.                */
 attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N,
                                 int32_t d, attn_qtensor_t out, void* stream);
 
@@ -149,8 +151,8 @@ typedef struct {
  *   workspace  device, >= ATTN_STATUS_WORKSPACE_BYTES, 16-byte aligned: its status word reports a
  *              copy that never completed (attn_fp8_read_status -> ATTN_ERR_TIMEOUT), as for the
  *              attention entry points; a workspace of those calls may be passed
- * Shapes whose two-tile ring does not fit in shared memory (FP32 source with d = 256) are
- * processed by one attn_fp8_quantize launch per job instead.                                     */
+ * attn_fp8_quantize is this call with one job (its status word lands in the library's built-in
+ * scratch, which attn_fp8_read_status does not reach).                                           */
 attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n_jobs, void* workspace,
                                       size_t workspace_bytes, void* stream);
 

@@ -122,6 +122,8 @@ static attn_status_t prepare_workspace(void* ws, size_t ws_bytes, size_t need, c
   return ATTN_OK;
 }
 
+static attn_status_t builtin_scratch_for_current_device(void** out);   // defined with the built-in scratch, below
+
 }  // namespace attnfp8
 
 using namespace attnfp8;
@@ -158,8 +160,15 @@ static attn_status_t check_quantize_args(const void* src, int32_t src_dtype, int
 attn_status_t attn_fp8_quantize(const void* src, int32_t src_dtype, int32_t B, int32_t H, int32_t N, int32_t d,
                                 attn_qtensor_t out, void* stream) {
   CHECK(check_quantize_args(src, src_dtype, B, H, N, d, out));
+  if (static_cast<long long>(B) * H * (N / 128) > 0x7fffffffLL)
+    return fail(ATTN_ERR_UNSUPPORTED, "tensor of more than 2^31 - 1 tiles of 128 tokens");
   CHECK(check_device());
-  return launch_quantize(src, src_dtype, B, H, N, d, out, static_cast<cudaStream_t>(stream));
+  // a batch of one; this entry point has no workspace argument, so the status word of its kernel
+  // (a bulk copy that never completed) lands in the library's built-in scratch
+  void* scratch = nullptr;
+  CHECK(builtin_scratch_for_current_device(&scratch));
+  const attn_quantize_job_t job = {src, src_dtype, B, H, N, d, out};
+  return launch_quantize_batch(&job, 1, static_cast<int*>(scratch), static_cast<cudaStream_t>(stream));
 }
 
 attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n_jobs, void* workspace,
@@ -167,13 +176,11 @@ attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n
   if (!jobs) return fail(ATTN_ERR_INVALID_ARG, "jobs is NULL");
   if (n_jobs < 1 || n_jobs > ATTN_QUANTIZE_MAX_JOBS)
     return fail(ATTN_ERR_INVALID_ARG, "n_jobs must be 1..%d (got %d)", ATTN_QUANTIZE_MAX_JOBS, n_jobs);
-  int d_max = 0;
   long long tiles = 0;
   for (int j = 0; j < n_jobs; ++j) {
     const attn_quantize_job_t& q = jobs[j];
     CHECK(check_quantize_args(q.src, q.src_dtype, q.B, q.H, q.N, q.d, q.out));
     if (q.src_dtype != jobs[0].src_dtype) return fail(ATTN_ERR_INVALID_ARG, "all jobs of a batch must share one src_dtype");
-    d_max = q.d > d_max ? q.d : d_max;
     tiles += static_cast<long long>(q.B) * q.H * (q.N / 128);
   }
   if (tiles > 0x7fffffffLL) return fail(ATTN_ERR_UNSUPPORTED, "batch of %lld tiles exceeds the 2^31 - 1 a launch indexes", tiles);
@@ -181,13 +188,6 @@ attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* status = nullptr;
   CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
-  if (!quantize_batch_fits(jobs[0].src_dtype, d_max)) {
-    for (int j = 0; j < n_jobs; ++j) {
-      const attn_quantize_job_t& q = jobs[j];
-      CHECK(launch_quantize(q.src, q.src_dtype, q.B, q.H, q.N, q.d, q.out, st));
-    }
-    return ATTN_OK;
-  }
   return launch_quantize_batch(jobs, n_jobs, status, st);
 }
 

@@ -29,13 +29,10 @@ struct AttnShape {
 };
 
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).
-attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
-                              cudaStream_t stream);
 attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H, int N, int d, const float* cos,
                                     const float* sin, float scale, float* mean, attn_qtensor_t out,
                                     cudaStream_t stream);
 attn_status_t launch_quantize_batch(const attn_quantize_job_t* jobs, int n_jobs, int* status, cudaStream_t stream);
-bool quantize_batch_fits(int src_dtype, int d_max);   // the two-tile ring fits in shared memory
 attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, int N, int d, void* row_out, void* col_out,
                                  cudaStream_t stream);
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,

@@ -1,11 +1,13 @@
-// Block-scaling quantiser: E4M3 codes with one E8M0 scale per 32 consecutive elements, written
-// in both orientations (blocks along channels; blocks along tokens, stored transposed).
+// The quantiser with the operand producer fused in front (rotary embedding, key centering, scale
+// folding), the token-mean kernel it needs, and the operand copies of BF16 mode.  The plain
+// quantiser (no producer steps) lives in quantize_batch.cu.
 //
 // One CTA owns a tile of 128 tokens x d channels of one (batch, head) slab, so it owns whole
 // 512-byte scale tiles of both orientations.  Pass 1 reads the tile from HBM once with 16-byte
-// coalesced loads, quantises along channels (4 lanes share a block of 32) and parks the source
-// tile in shared memory; pass 2 walks the parked tile along tokens.  Codes of the transposed
-// copy are staged in shared memory so that they leave as full 128-byte rows.
+// coalesced loads, applies the producer steps in FP32, quantises along channels (4 lanes share a
+// block of 32) and parks the FP32 values in shared memory; pass 2 walks the parked tile along
+// tokens.  Codes of the transposed copy are staged in shared memory so that they leave as full
+// 128-byte rows.
 #include <cuda_bf16.h>
 
 #include <type_traits>
@@ -42,14 +44,14 @@ __device__ __forceinline__ float rotate_bf16(float x, float partner, float c, fl
   return __bfloat162float(__float2bfloat16_rn(r));
 }
 
-template <typename T, bool kFused>
-__global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict__ src, int N, int d,
+template <typename T>
+__global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const T* __restrict__ src, int N, int d,
                                                             uint8_t* __restrict__ row_codes,
                                                             uint8_t* __restrict__ row_scales,
                                                             uint8_t* __restrict__ col_codes,
                                                             uint8_t* __restrict__ col_scales, const Producer prod) {
   extern __shared__ __align__(16) uint8_t smem[];
-  using TT = typename std::conditional<kFused, float, T>::type;     // what the parked tile holds
+  using TT = float;                                                  // what the parked tile holds
   const int pitch = d + 16 / static_cast<int>(sizeof(TT)) * 1;      // elements; +16 bytes per row
   TT* tile = reinterpret_cast<TT*>(smem);
   const int n_ct = (d / 32 + 3) / 4;                                 // row-copy scale tiles of this CTA
@@ -85,17 +87,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict_
       const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&raw);
 #pragma unroll
       for (int i = 0; i < 8; ++i) x[i] = to_f32(h[i]);
-      if (!kFused && want_col) *reinterpret_cast<uint4*>(tile + tok * pitch + ch) = raw;
     } else {
       const float4 a = *reinterpret_cast<const float4*>(g_src + e0);
       const float4 b = *reinterpret_cast<const float4*>(g_src + e0 + 4);
       x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-      if (!kFused && want_col) {
-        *reinterpret_cast<float4*>(tile + tok * pitch + ch) = a;
-        *reinterpret_cast<float4*>(tile + tok * pitch + ch + 4) = b;
-      }
     }
-    if constexpr (kFused) {
+    {
       if (prod.cos != nullptr) {
         const int half = d >> 1;
         const bool upper = ch >= half;
@@ -179,19 +176,19 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const T* __restrict_
   }
 }
 
-template <typename T, bool kFused>
+template <typename T>
 attn_status_t launch_t(const void* src, int B, int H, int N, int d, attn_qtensor_t out, const Producer& prod,
                        cudaStream_t stream) {
-  const int tile_elem = kFused ? 4 : static_cast<int>(sizeof(T));
+  const int tile_elem = 4;                                           // the parked tile is FP32
   const int pitch = d + 16 / tile_elem;
   const int n_ct = (d / 32 + 3) / 4, n_rt = (d + 127) / 128;
   const size_t smem = static_cast<size_t>(kTokens) * pitch * tile_elem + (n_ct + n_rt) * 512 +
                       static_cast<size_t>(d) * (kTokens + 16);
-  cudaError_t e = cudaFuncSetAttribute(quantize_kernel<T, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(quantize_fused_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(N / kTokens, B * H);
-  quantize_kernel<T, kFused><<<grid, kThreads, smem, stream>>>(static_cast<const T*>(src), N, d, out.row_codes,
+  quantize_fused_kernel<T><<<grid, kThreads, smem, stream>>>(static_cast<const T*>(src), N, d, out.row_codes,
                                                               out.row_scales, out.col_codes, out.col_scales, prod);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: launch: %s", cudaGetErrorString(e));
@@ -290,13 +287,6 @@ attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, i
   return launch_copies_t<float>(src, B, H, N, d, row_out, col_out, stream);
 }
 
-attn_status_t launch_quantize(const void* src, int src_dtype, int B, int H, int N, int d, attn_qtensor_t out,
-                              cudaStream_t stream) {
-  const Producer none{nullptr, nullptr, nullptr, 1.f, 0};
-  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16, false>(src, B, H, N, d, out, none, stream);
-  return launch_t<float, false>(src, B, H, N, d, out, none, stream);
-}
-
 attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H, int N, int d, const float* cos,
                                     const float* sin, float scale, float* mean, attn_qtensor_t out,
                                     cudaStream_t stream) {
@@ -310,8 +300,8 @@ attn_status_t launch_quantize_fused(const void* src, int src_dtype, int B, int H
     if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "token mean: launch: %s", cudaGetErrorString(e));
   }
   const Producer prod{cos, sin, mean, scale, scale != 1.f ? 1 : 0};
-  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16, true>(src, B, H, N, d, out, prod, stream);
-  return launch_t<float, true>(src, B, H, N, d, out, prod, stream);
+  if (src_dtype == ATTN_SRC_BF16) return launch_t<__nv_bfloat16>(src, B, H, N, d, out, prod, stream);
+  return launch_t<float>(src, B, H, N, d, out, prod, stream);
 }
 
 }  // namespace attnfp8

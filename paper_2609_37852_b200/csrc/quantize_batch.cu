@@ -1,10 +1,10 @@
-// Block-scaling quantiser for several tensors in one launch (the four operands of a step: Q, K,
-// V, dO).  Same arithmetic and the same output layout as quantize.cu, bit for bit; what differs
-// is how the data moves.
+// Block-scaling quantiser: E4M3 codes with one E8M0 scale per 32 consecutive elements, written
+// in both orientations (blocks along channels; blocks along tokens, stored transposed), for one
+// tensor or for several in one launch (the four operands of a step: Q, K, V, dO).
 //
 // The tiles (128 tokens x d channels, contiguous in the source) of all tensors form one list.  A
-// persistent grid of two CTAs per SM walks it; each CTA keeps a ring of two source tiles in shared
-// memory, filled by bulk asynchronous copies (one instruction per tile, completion counted on an
+// persistent grid (two CTAs per SM at d = 128) walks it; each CTA keeps a ring of two source tiles
+// in shared memory (one where two do not fit), filled by bulk asynchronous copies (one instruction per tile, completion counted on an
 // mbarrier), so that the next tile is in flight while the current one is quantised: the short
 // tails and ramps of four separate launches disappear and every SM always has loads outstanding.
 // Pass 1 walks the tile along channels (row copy), pass 2 along tokens (column copy, staged in
@@ -22,7 +22,7 @@ using namespace sm100;
 
 constexpr int kTokens = 128;
 constexpr int kThreads = 256;
-constexpr int kRing = 2;
+constexpr int kMaxRing = 2;
 constexpr int kColPitch = kTokens + 16;
 
 struct BatchJob {
@@ -37,6 +37,7 @@ struct BatchParams {
   int n_jobs;
   int total_tiles;
   int d_max;
+  int ring;              // source tiles a CTA keeps in shared memory (1 or 2)
   int* status;
 };
 
@@ -165,12 +166,13 @@ __global__ void __launch_bounds__(kThreads, 2) quantize_batch_kernel(const __gri
   extern __shared__ __align__(128) uint8_t smem[];
   const int tile_bytes_max = kTokens * p.d_max * static_cast<int>(sizeof(T));
   auto ring = [&](int slot) { return reinterpret_cast<T*>(smem + slot * tile_bytes_max); };
+  const int n_ring = p.ring;
   const int n_ct_max = (p.d_max / 32 + 3) / 4, n_rt_max = (p.d_max + 127) / 128;
-  uint8_t* s_row_sf = smem + kRing * tile_bytes_max;
+  uint8_t* s_row_sf = smem + n_ring * tile_bytes_max;
   uint8_t* s_col_sf = s_row_sf + n_ct_max * 512;
   uint8_t* s_col_codes = s_col_sf + n_rt_max * 512;                  // [d][128 + 16]
   uint64_t* full = reinterpret_cast<uint64_t*>(s_col_codes + p.d_max * kColPitch);
-  int* abort_flag = reinterpret_cast<int*>(full + kRing);
+  int* abort_flag = reinterpret_cast<int*>(full + kMaxRing);
 
   const int tid = threadIdx.x;
   const int my_tiles = (p.total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
@@ -189,15 +191,15 @@ __global__ void __launch_bounds__(kThreads, 2) quantize_batch_kernel(const __gri
     locate(static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x), j, local);
     const uint32_t bytes = static_cast<uint32_t>(kTokens * p.job[j].d * sizeof(T));
     const uint8_t* g = static_cast<const uint8_t*>(p.job[j].src) + static_cast<size_t>(local) * bytes;
-    mbar_arrive_expect_tx(&full[i % kRing], bytes);
-    bulk_load_1d(ring(i % kRing), g, bytes, &full[i % kRing]);
+    mbar_arrive_expect_tx(&full[i % n_ring], bytes);
+    bulk_load_1d(ring(i % n_ring), g, bytes, &full[i % n_ring]);
   };
 
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s < n_ring; ++s) mbar_init(&full[s], 1);
     *abort_flag = 0;
     fence_mbar_init();
-    for (int i = 0; i < kRing && i < my_tiles; ++i) issue(i);
+    for (int i = 0; i < n_ring && i < my_tiles; ++i) issue(i);
   }
   __syncthreads();
 
@@ -212,11 +214,11 @@ __global__ void __launch_bounds__(kThreads, 2) quantize_batch_kernel(const __gri
     const size_t tok0 = static_cast<size_t>(tok_tile) * kTokens;
     const int n_ct = (d / 32 + 3) / 4, n_rt = (d + 127) / 128;
     const bool want_row = job.row_codes != nullptr, want_col = job.col_codes != nullptr;
-    const T* tile = ring(i % kRing);
+    const T* tile = ring(i % n_ring);
 
     for (int w = tid; w < (n_ct_max + n_rt_max) * 512 / 4; w += kThreads) reinterpret_cast<uint32_t*>(s_row_sf)[w] = 0;
     // bounded wait: a copy that never lands ends the CTA with the time-out status, not a hang
-    const bool landed = mbar_wait(&full[i % kRing], (i / kRing) & 1, abort_flag);
+    const bool landed = mbar_wait(&full[i % n_ring], (i / n_ring) & 1, abort_flag);
     if (__syncthreads_or(!landed)) break;        // all threads take the same way out
 
     switch (d) {                      // compile-time head dims: no integer division, constant strides
@@ -228,9 +230,9 @@ __global__ void __launch_bounds__(kThreads, 2) quantize_batch_kernel(const __gri
     }
     __syncthreads();
     // the source tile is consumed: refill its slot while the staged outputs leave
-    if (tid == 0 && i + kRing < my_tiles) {
+    if (tid == 0 && i + n_ring < my_tiles) {
       fence_proxy_async_smem();
-      issue(i + kRing);
+      issue(i + n_ring);
     }
     if (want_row) {
       uint8_t* g = job.row_scales + (slab * tiles_per_slab + tok_tile) * n_ct * 512;
@@ -254,35 +256,39 @@ __global__ void __launch_bounds__(kThreads, 2) quantize_batch_kernel(const __gri
   if (tid == 0 && *abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
 }
 
+static size_t batch_smem_bytes(size_t elem, int d_max, int ring) {
+  const int n_ct = (d_max / 32 + 3) / 4, n_rt = (d_max + 127) / 128;
+  return ring * static_cast<size_t>(kTokens) * d_max * elem + (n_ct + n_rt) * 512 +
+         static_cast<size_t>(d_max) * kColPitch + 64;
+}
+
 template <typename T>
-attn_status_t launch_batch_t(const BatchParams& p, cudaStream_t stream) {
-  const size_t tile_bytes = static_cast<size_t>(kTokens) * p.d_max * sizeof(T);
-  const int n_ct = (p.d_max / 32 + 3) / 4, n_rt = (p.d_max + 127) / 128;
-  const size_t smem = kRing * tile_bytes + (n_ct + n_rt) * 512 + static_cast<size_t>(p.d_max) * kColPitch + 64;
+attn_status_t launch_batch_t(BatchParams& p, cudaStream_t stream) {
+  // two CTAs per SM come first (each covers the other's stalls), the deeper ring second: measured
+  // at d = 192 one tile x two CTAs 0.078 ms against two tiles x one CTA 0.098 ms
+  const size_t half_sm = 113 * 1024, whole_sm = 227 * 1024;
+  if (batch_smem_bytes(sizeof(T), p.d_max, kMaxRing) <= half_sm) p.ring = kMaxRing;
+  else if (batch_smem_bytes(sizeof(T), p.d_max, 1) <= half_sm) p.ring = 1;
+  else p.ring = batch_smem_bytes(sizeof(T), p.d_max, kMaxRing) <= whole_sm ? kMaxRing : 1;
+  const size_t smem = batch_smem_bytes(sizeof(T), p.d_max, p.ring);
   cudaError_t e = cudaFuncSetAttribute(quantize_batch_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
-  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize_batch: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   int dev = 0, sms = 0, per_sm = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_batch_kernel<T>, kThreads, smem);
   if (e != cudaSuccess || per_sm < 1 || sms < 1)
-    return fail(ATTN_ERR_CUDA, "quantize_batch: occupancy query: %s", cudaGetErrorString(e));
+    return fail(ATTN_ERR_CUDA, "quantize: occupancy query: %s", cudaGetErrorString(e));
   const int resident = sms * per_sm;
   const int grid = p.total_tiles < resident ? p.total_tiles : resident;
   quantize_batch_kernel<T><<<grid, kThreads, smem, stream>>>(p);
   e = cudaGetLastError();
-  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize_batch: launch: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "quantize: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
 }
 
 }  // namespace
-
-bool quantize_batch_fits(int src_dtype, int d_max) {
-  const size_t elem = src_dtype == ATTN_SRC_BF16 ? 2 : 4;
-  const size_t smem = kRing * kTokens * d_max * elem + 2 * 512 * 2 + static_cast<size_t>(d_max) * kColPitch + 64;
-  return smem <= 227 * 1024;
-}
 
 attn_status_t launch_quantize_batch(const attn_quantize_job_t* jobs, int n_jobs, int* status, cudaStream_t stream) {
   BatchParams p = {};

@@ -114,10 +114,10 @@ def test_quantize_batch_is_bit_identical_to_single_calls(name, kw):
             assert torch.equal(q.col_codes, full.col_codes) and torch.equal(q.col_scales, full.col_scales)
 
 
-def test_quantize_batch_fallback_and_errors():
+def test_quantize_batch_single_tile_ring_and_errors():
     from paper_2609_37852_b200 import binding as B
     g = torch.Generator().manual_seed(5)
-    # FP32 source with d = 256: the two-tile ring does not fit, one launch per tensor instead
+    # FP32 source with d = 256: two source tiles do not fit in shared memory, the ring holds one
     xs = [torch.randn((1, 2, 256, 256), generator=g).cuda(), torch.randn((1, 1, 128, 256), generator=g).cuda()]
     outs, ws = B.attn_fp8_quantize_batch(xs)
     B.attn_fp8_read_status(ws)
