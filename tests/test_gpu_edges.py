@@ -52,6 +52,25 @@ def test_small_and_extreme_shapes(name, kw):
     _check(w, tensors, _full_pass(w, tensors))
 
 
+@pytest.mark.parametrize("name,kw,bf16", [
+    ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=384, causal=False), False),        # wide heads without the causal mask
+    ("mla8k", dict(heads_q=4, heads_kv=1, seqlen=256, causal=False), False),
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=384, causal=False), False),
+    ("gqa8k_d256", dict(batch=2, heads_q=4, heads_kv=2, seqlen=256), False),         # d = 256 with a batch
+    ("gqa4k", dict(batch=1, heads_q=4, heads_kv=2, seqlen=384, causal=False), True),  # BF16 mode, non-causal
+    ("tiny", dict(seqlen=384, heads_q=3, heads_kv=3, batch=2), False),               # odd head count, d = 64, FP32 source
+    ("tiny", dict(seqlen=384, heads_q=6, heads_kv=2, causal=True), True),            # BF16 mode at d = 64, groups of 3
+    ("long64k", dict(heads_q=2, heads_kv=1, seqlen=1152), False),                    # heavy-tailed channel gains, 9 tiles
+    ("gqa8k_outlier", dict(batch=3, heads_q=16, heads_kv=1, seqlen=256), False),     # 16 query heads on one KV head
+])
+def test_shape_and_mode_combinations(name, kw, bf16):
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    tensors = workloads.make_inputs(w)
+    if bf16 and w.dtype != "bf16":
+        tensors = tuple(x.to(torch.bfloat16) for x in tensors)
+    _check(w, tensors, _full_pass(w, tensors, bf16=bf16), prec="bf16" if bf16 else "mxfp8")
+
+
 def test_nearly_one_hot_rows_stress():
     """Outlier channels shared by a query head and its KV head: scores with a standard deviation of
     ~70, rows nearly one-hot, the running shift raised (and the output accumulator rescaled) often."""
