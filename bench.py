@@ -230,9 +230,10 @@ def main():
         else:
             B.attn_fp8_quantize_batch(srcs, outs=(qq, kq, vq, dOq), workspace=ws)
 
-    stage_names = ("quantize", "fwd", "bwd_delta", "bwd_dq", "bwd_dkdv")
 
-    def step(events=None):
+    def step(events=None, split=False):
+        """One pass of the path.  ``events``: recorded at the stage boundaries.  ``split``: the two
+        kernels of the gradient pass run once more as separate calls, for their own durations."""
         def mark(i):
             if events is not None:
                 events[i].record(stream)
@@ -243,15 +244,15 @@ def main():
         mark(2)
         B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, delta=delta, workspace=ws)
         mark(3)
-        if events is None:
-            # the gradient pass as a user calls it: one call, the dQ kernel launched behind the dK/dV
-            # kernel so that it fills that kernel's last wave
-            B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, dq=dq, dk=dk, dv=dv, workspace=ws)
-        else:
+        # the gradient pass as a user calls it: one call, the dQ kernel launched behind the dK/dV kernel
+        # so that it fills that kernel's last wave
+        B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, dq=dq, dk=dk, dv=dv, workspace=ws)
+        mark(4)
+        if split:                                   # once more as two serialised calls, an event around each
             B.attn_fp8_bwd_dq(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
-            mark(4)
-            B.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, dk=dk, dv=dv, workspace=ws)
             mark(5)
+            B.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, dk=dk, dv=dv, workspace=ws)
+            mark(6)
 
     # one batched quantiser launch (BF16 mode: four operand-preparation launches) + fwd + delta + dQ + dK/dV
     # (two key-major passes when the qk head dim exceeds 128)
@@ -262,26 +263,26 @@ def main():
         step()
     B.attn_fp8_read_status(ws)
     sampler = ClockSampler(local_rank)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
     barrier()
     sampler.start()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for i in range(args.steps):
-        step()
+        step()                                      # no event inside a step: each one costs a few microseconds
     t_end.record(stream)
     barrier()
     clocks = sampler.stop()
     B.attn_fp8_read_status(ws)
     total_ms = t_start.elapsed_time(t_end)
-    # per-stage breakdown: the same steps once more with an event between the stages (and the two
-    # halves of the gradient pass as separate calls, which serialises them)
+    # per-stage breakdown: the same steps once more with an event at every stage boundary, followed by
+    # the two kernels of the gradient pass as separate (serialised) calls
     for i in range(args.steps):
-        step(events[i])
+        step(events[i], split=True)
     torch.cuda.synchronize()
     B.attn_fp8_read_status(ws)
-    stage_ms = {n: statistics.mean(events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps))
-                for j, n in enumerate(stage_names)}
+    stage_ms = {n: statistics.mean(ev[j].elapsed_time(ev[j + 1]) for ev in events)
+                for j, n in enumerate(("quantize", "fwd", "bwd_delta", "bwd", "bwd_dq", "bwd_dkdv"))}
 
     # ---- end to end through the library with host buffers --------------------------------------
     # Host buffers in, host buffers out, every step: copies run on their own streams and overlap the
@@ -381,9 +382,10 @@ def main():
         "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
         "pct_of_nominal_peak_of_dtype": 100.0 * value / world / (NOMINAL_FP8_TFLOPS / (FP8_OVER_BF16 if bf16_mode else 1.0)),
         "stage_ms": stage_ms,
-        "stage_timing": "a second loop of the same steps with an event between stages; dQ and dK/dV as separate "
-                        "calls there (serialised), one overlapped call in the timed region",
-        # the timed step without the operand preparation (the paper's accounting), and without the forward
+        "stage_timing": "a second loop of the same steps with an event at every stage boundary (the timed region has "
+                        "none: an event costs a few microseconds); bwd = the overlapped gradient call, bwd_dq and "
+                        "bwd_dkdv = its two kernels as separate, serialised calls",
+        # the timed step less the operand preparation (the paper's accounting), and less the forward
         "attn_only_tflops": credited / ((step_ms - stage_ms["quantize"]) * 1e-3) / 1e12,
         "fwd_tflops": fwd_flops / (stage_ms["fwd"] * 1e-3) / 1e12,
         "bwd_tflops": bwd_flops / ((step_ms - stage_ms["quantize"] - stage_ms["fwd"]) * 1e-3) / 1e12,
