@@ -86,3 +86,26 @@ def test_validation_errors_without_touching_a_gpu(lib_path):
     p = binding.AttnParams(1, 128, 4, 2, 96, 96, True, 0.1).c_struct()
     st = binding._lib.attn_fp8_fwd(ctypes.byref(p), q, q, q, None, None, None, 0, None)
     assert st == 2
+
+
+def test_batched_quantiser_and_workspace_validation_without_a_gpu(lib_path):
+    """Argument checks of attn_fp8_quantize_batch and attn_fp8_workspace_init run before any device call."""
+    from paper_2609_37852_b200 import binding
+    lib = binding._lib
+    fake = ctypes.c_void_p(4096)                                   # aligned, never dereferenced on these paths
+    out = binding._QTensor(fake, fake, fake, fake)
+    ok = binding._QuantizeJob(fake, binding.ATTN_SRC_BF16, 1, 1, 128, 128, out)
+    jobs = (binding._QuantizeJob * 2)(ok, ok)
+    assert lib.attn_fp8_quantize_batch(None, 1, fake, 256, None) == 1
+    assert lib.attn_fp8_quantize_batch(jobs, 0, fake, 256, None) == 1
+    assert lib.attn_fp8_quantize_batch(jobs, binding.ATTN_QUANTIZE_MAX_JOBS + 1, fake, 256, None) == 1
+    jobs[1] = binding._QuantizeJob(fake, binding.ATTN_SRC_FP32, 1, 1, 128, 128, out)
+    assert lib.attn_fp8_quantize_batch(jobs, 2, fake, 256, None) == 1 and "src_dtype" in binding.attn_fp8_last_error()
+    jobs[1] = binding._QuantizeJob(fake, binding.ATTN_SRC_BF16, 1, 1, 192, 128, out)      # N not a multiple of 128
+    assert lib.attn_fp8_quantize_batch(jobs, 2, fake, 256, None) == 2
+    jobs[1] = binding._QuantizeJob(fake, binding.ATTN_SRC_BF16, 1, 1, 128, 128, binding._QTensor(fake, None, None, None))
+    assert lib.attn_fp8_quantize_batch(jobs, 2, fake, 256, None) == 1      # codes without their scales
+    assert lib.attn_fp8_workspace_init(None, 256, None) == 4
+    assert lib.attn_fp8_workspace_init(fake, 16, None) == 4
+    assert lib.attn_fp8_workspace_init(ctypes.c_void_p(4100), 256, None) == 3
+    assert lib.attn_fp8_read_status(None, None) == 1
