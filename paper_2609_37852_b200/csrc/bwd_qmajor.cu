@@ -69,23 +69,33 @@ struct QmCfg {
                                                         // 2 with kEB == 1 is the protected-dP ablation
   static constexpr bool kFp8 = kEB == 1;
   static constexpr bool kFp8v = kEBv == 1;
+  // The delta kernel is persistent: one CTA per SM walks a list of query tiles, with the Q / dO
+  // tiles double-buffered and the K / V ring, the score buffers and their barriers running on
+  // across tile boundaries, so that set-up, pipeline fill and drain are paid once per CTA instead
+  // of once per query tile.  The dQ kernel keeps one query tile per CTA (its accumulator has to
+  // leave tensor memory between tiles, and launched behind the key-major kernel its CTAs start at
+  // different times, which a static tile list cannot balance).
   static constexpr int kStep = kTile / kEB;             // keys per step
+  // (where two Q / dO tiles and two K / V stages do not fit in shared memory, the delta kernel is
+  // not persistent either)
+  static constexpr bool kPersist = !kDQ && 2 * (kCq + kCv) * (kTile + kStep) * 128 <= 224 * 1024;
+  static constexpr int kQBufs = kPersist ? 2 : 1;       // Q / dO tile buffers (and scale-factor slots)
   static constexpr int kGroups = kStep / 32;            // 32-key column groups of a step
   static constexpr int kSoftmaxThreads = 128 * kGroups; // 4 TMEM lane quadrants x column groups
   static constexpr int kThreads = 128 + kSoftmaxThreads;
   // K/V ring depth: deep enough to cover the L2 -> shared-memory latency of a tile (what fits);
   // the K^T ring of the dQ product falls back to one stage when two do not fit
-  static constexpr int kFixedBytes = (kCq + kCv) * kTile * 128;
+  static constexpr int kFixedBytes = kQBufs * (kCq + kCv) * kTile * 128;
   static constexpr int kKvBytes = (kCq + kCv) * kStep * 128;
   static constexpr int kKcBytes = kDQ ? kTile * 128 : 0;
-  static constexpr int kRaw = (224 * 1024 - kFixedBytes - kKcBytes) / (kKvBytes + kKcBytes);
+  static constexpr int kRaw = ((kPersist ? 216 : 224) * 1024 - kFixedBytes - kKcBytes) / (kKvBytes + kKcBytes);
   static constexpr int kStages = kRaw < 2 ? 2 : (kRaw > 4 ? 4 : kRaw);
   static constexpr int kKcStages = !kDQ ? 1 : (kRaw < 2 ? 1 : kStages);
   // tensor memory
   static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* 2 x 32 */, kColdQ = 2 * kStep + 64;
-  static constexpr uint32_t kColSFQ = kColdQ + 128;
-  static constexpr uint32_t kColSFdO = kColSFQ + 4 * kCq;
-  static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv;    // 2 slots
+  static constexpr uint32_t kColSFQ = kDQ ? kColdQ + 128 : 2 * kStep;   // kQBufs slots (no dS^ / dQ columns without dQ)
+  static constexpr uint32_t kColSFdO = kColSFQ + 4 * kCq * kQBufs;   // kQBufs slots
+  static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv * kQBufs;   // 2 slots
   static constexpr uint32_t kColSFV = kColSFK + 8 * kCq;     // 2 slots
   static constexpr uint32_t kColSFdS = kColSFV + 8 * kCv;    // 2 x 4
   static constexpr uint32_t kColSFKc = kColSFdS + 8;         // 2 x 4
@@ -97,19 +107,19 @@ struct QmCfg {
 template <class C>
 struct QmSmem {
   static constexpr int kStages = C::kStages;
-  alignas(1024) uint8_t q[C::kCq][kTile * 128];
-  alignas(1024) uint8_t dO[C::kCv][kTile * 128];
+  alignas(1024) uint8_t q[C::kQBufs][C::kCq][kTile * 128];
+  alignas(1024) uint8_t dO[C::kQBufs][C::kCv][kTile * 128];
   alignas(1024) uint8_t k[kStages][C::kCq][C::kStep * 128];
   alignas(1024) uint8_t v[kStages][C::kCv][C::kStep * 128];
   alignas(1024) uint8_t kc[C::kKcStages][kTile * 128];
-  alignas(16) uint8_t sf_q[C::kCq * 512];
-  alignas(16) uint8_t sf_dO[C::kCv * 512];
+  alignas(16) uint8_t sf_q[C::kQBufs][C::kCq * 512];
+  alignas(16) uint8_t sf_dO[C::kQBufs][C::kCv * 512];
   alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
   alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
   alignas(16) uint8_t sf_kc[C::kKcStages][512];
   alignas(16) uint8_t sf_ds[2][512];
   alignas(16) float red[C::kGroups][4][kTile];   // partial row sums of every column group
-  uint64_t q_full;
+  uint64_t q_full[C::kQBufs], q_empty[C::kQBufs];
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
   uint64_t sdp_full, sdp_free;
@@ -132,6 +142,7 @@ struct QmParams {
   float* post_rowabs;
   int* status;
   int N, Hq, Hkv, dqk, dv, causal;
+  int gx, gy, gz;           // the (head x column tile, query tile, batch) grid the work items are numbered in
   int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
   float scale, scale_log2;
 };
@@ -144,7 +155,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
   // shared state space of every access derived from it (checked below)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8, kFp8v = C::kFp8v;
+  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8, kFp8v = C::kFp8v, kPersist = C::kPersist;
   constexpr int kStages = C::kStages, kKcStages = C::kKcStages, kEB = C::kEB, kCq = C::kCq, kCv = C::kCv;
   constexpr int kStep = C::kStep, kGroups = C::kGroups, kSoftmaxThreads = C::kSoftmaxThreads;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColdS = C::kColdS, kColdQ = C::kColdQ, kColSFQ = C::kColSFQ,
@@ -156,20 +167,41 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     return;
   }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
-  // all heads go first, so the light tiles fill the tail of the launch
-  const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
-  // dQ column tiles (128 wide) of one head sit next to each other in the grid
-  const int rq = kDQ ? (p.dqk + 127) / 128 : 1;
-  const int h = blockIdx.x / rq, r_tile = blockIdx.x % rq, b = blockIdx.z;
-  const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
-  const int g = h / (p.Hq / p.Hkv);
-  const int n_tiles = (p.causal ? qt + 1 : p.N / kTile) * kEB;      // key steps
+  // Work items are numbered x-fastest over the grid (gx, gy, gz): heads vary fastest and the heaviest
+  // (latest) query tiles of all heads come first, so the light tiles fill the tail.  Without
+  // persistence a CTA is its own item.  A persistent CTA takes the items c, 2n-1-c, 2n+c, ... (n CTAs,
+  // c its index): alternate rounds run backwards, so that no CTA collects the heavier item of every
+  // round.
+  const int rq = kDQ ? (p.dqk + 127) / 128 : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
+  const int total_items = p.gx * p.gy * p.gz;
+  const int n_cta = static_cast<int>(gridDim.x);
+  const int n_items = !kPersist ? 1
+                                : total_items / n_cta + ((((total_items / n_cta) & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x)
+                                                                                        : static_cast<int>(blockIdx.x)) <
+                                                             total_items % n_cta
+                                                         ? 1 : 0);
+  struct Item { int qt, h, r_tile, b, g, n_tiles; };
+  auto item_at = [&](int i) {
+    int x, y, z;
+    if (kPersist) {
+      const int pos = (i & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
+      const int l = i * n_cta + pos;
+      x = l % p.gx; y = (l / p.gx) % p.gy; z = l / (p.gx * p.gy);
+    } else {
+      x = blockIdx.x; y = blockIdx.y; z = blockIdx.z;
+    }
+    Item it;
+    it.qt = p.causal ? (p.gy - 1 - y) : y;
+    it.h = x / rq; it.r_tile = x % rq; it.b = z;
+    it.g = it.h / (p.Hq / p.Hkv);
+    it.n_tiles = (p.causal ? it.qt + 1 : p.N / kTile) * kEB;       // key steps
+    return it;
+  };
   const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * C::kEBv / 32;       // 32-byte K steps of the two products
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
-    mbar_init(&sm.q_full, 1);
+    for (int i = 0; i < C::kQBufs; ++i) { mbar_init(&sm.q_full[i], 1); mbar_init(&sm.q_empty[i], 2); }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 2);   // released by the S and the dP issuer
     }
@@ -195,41 +227,53 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     if (lane == 0) {
       prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
       if (kDQ) prefetch_tmap(&tm_kc);
-      const int q_slab = b * p.Hq + h, kv_slab = b * p.Hkv + g;
       const int tiles_n = p.N / kTile;
-      mbar_arrive_expect_tx(&sm.q_full, kCq * (kTile * 128 + (kFp8 ? 512 : 0)) + kCv * (kTile * 128 + (kFp8v ? 512 : 0)));
-      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[c], &tm_q, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
-      for (int c = 0; c < kCv; ++c) tma_load_2d(sm.dO[c], &tm_dO, &sm.q_full, 128 * c, q_slab * p.N + qt * kTile);
-      if (kFp8)
-        bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCq * 512, kCq * 512, &sm.q_full);
-      if (kFp8v)
-        bulk_load_1d(sm.sf_dO, p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + qt) * kCv * 512, kCv * 512, &sm.q_full);
       int issued_kv = 0, issued_kc = 0;
       bool ok = true;
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % kStages, u = t / kStages;
-        ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        QM_TRACE(0, t, 0);
-        mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
-        for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
-        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
-        if (kFp8)
-          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
-        if (kFp8v)
-          bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
-        ++issued_kv;
-        if (kDQ) {
-          const int sc = t % kKcStages;
-          ok = mbar_wait(&sm.kc_empty[sc], ((t / kKcStages) & 1) ^ 1, abort_flag);
+      int T = 0;                                      // key steps of the items before this one
+      for (int i = 0; i < n_items && ok; ++i) {
+        const Item it = item_at(i);
+        const int q_slab = it.b * p.Hq + it.h, kv_slab = it.b * p.Hkv + it.g;
+        const int qb = i % C::kQBufs;
+        if (i >= C::kQBufs) {
+          // both issuers have finished with the item that used this Q / dO buffer
+          ok = mbar_wait(&sm.q_empty[qb], ((i / C::kQBufs) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
-          tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * r_tile);
-          if (kFp8)
-            bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + r_tile) * tiles_n + t) * 512, 512,
-                         &sm.kc_full[sc]);
-          ++issued_kc;
         }
+        mbar_arrive_expect_tx(&sm.q_full[qb], kCq * (kTile * 128 + (kFp8 ? 512 : 0)) + kCv * (kTile * 128 + (kFp8v ? 512 : 0)));
+        for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[qb][c], &tm_q, &sm.q_full[qb], 128 * c, q_slab * p.N + it.qt * kTile);
+        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.dO[qb][c], &tm_dO, &sm.q_full[qb], 128 * c, q_slab * p.N + it.qt * kTile);
+        if (kFp8)
+          bulk_load_1d(sm.sf_q[qb], p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + it.qt) * kCq * 512, kCq * 512, &sm.q_full[qb]);
+        if (kFp8v)
+          bulk_load_1d(sm.sf_dO[qb], p.dO_sf + (static_cast<size_t>(q_slab) * tiles_n + it.qt) * kCv * 512, kCv * 512, &sm.q_full[qb]);
+        for (int t = 0; t < it.n_tiles && ok; ++t) {
+          const int gt = T + t;                       // step index over all items of this CTA: the rings run on
+          const int s = gt % kStages, u = gt / kStages;
+          ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          QM_TRACE(0, t, 0);
+          mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
+          for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
+          for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
+          if (kFp8)
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
+          if (kFp8v)
+            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
+          ++issued_kv;
+          if (kDQ) {
+            const int sc = t % kKcStages;
+            ok = mbar_wait(&sm.kc_empty[sc], ((t / kKcStages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
+            tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * it.r_tile);
+            if (kFp8)
+              bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + it.r_tile) * tiles_n + t) * 512, 512,
+                           &sm.kc_full[sc]);
+            ++issued_kc;
+          }
+        }
+        T += it.n_tiles;
       }
       if (!ok) {
         int dummy = 0;
@@ -242,33 +286,44 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ S issuer
     {
-      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[0]));
-      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok && kFp8) {
-        tc_fence_after_sync();
-        sf_copy_tiles<kCq>(tmem + kColSFQ, sm.sf_q);
-      }
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % kStages, slot = t & 1;
-        ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+      bool ok = true;
+      int T = 0;
+      for (int i = 0; i < n_items && ok; ++i) {
+        const Item it = item_at(i);
+        const int qb = i % C::kQBufs;
+        const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[qb][0]));
+        const uint32_t t_sfq = tmem + kColSFQ + 4 * kCq * qb;
+        ok = mbar_wait(&sm.q_full[qb], (i / C::kQBufs) & 1, abort_flag);
         if (!ok) break;
-        QM_TRACE(1, t, 0);
-        tc_fence_after_sync();
-        if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
-        QM_TRACE(1, t, 1);
-        if (t > 0) {
-          // the softmax threads have pulled the previous S and dP into registers
-          ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
-          if (!ok) break;
+        if (kFp8) {
           tc_fence_after_sync();
+          sf_copy_tiles<kCq>(t_sfq, sm.sf_q[qb]);
         }
-        QM_TRACE(1, t, 2);
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
-        issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, tmem + kColSFQ,
-                                                                        tmem + kColSFK + 4 * kCq * slot);
-        mma_commit_elect(&sm.sdp_full);
-        mma_commit_elect(&sm.kv_empty[s]);
-        QM_TRACE(1, t, 3);
+        for (int t = 0; t < it.n_tiles && ok; ++t) {
+          const int gt = T + t;
+          const int s = gt % kStages, slot = gt & 1;
+          ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
+          if (!ok) break;
+          QM_TRACE(1, t, 0);
+          tc_fence_after_sync();
+          if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
+          QM_TRACE(1, t, 1);
+          if (gt > 0) {
+            // the softmax threads have pulled the previous S and dP into registers
+            ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+          QM_TRACE(1, t, 2);
+          const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
+          issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, t_sfq,
+                                                                          tmem + kColSFK + 4 * kCq * slot);
+          mma_commit_elect(&sm.sdp_full);
+          mma_commit_elect(&sm.kv_empty[s]);
+          QM_TRACE(1, t, 3);
+        }
+        if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's Q tile has been read
+        T += it.n_tiles;
       }
       if (!ok) {
         int dummy = 0;
@@ -279,28 +334,39 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   } else if (warp == 2) {
     // ------------------------------------------------------------------ dP issuer
     {
-      const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO[0]));
-      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok && kFp8v) {
-        tc_fence_after_sync();
-        sf_copy_tiles<kCv>(tmem + kColSFdO, sm.sf_dO);
-      }
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % kStages, slot = t & 1;
-        ok = mbar_wait(&sm.kv_full[s], (t / kStages) & 1, abort_flag);
+      bool ok = true;
+      int T = 0;
+      for (int i = 0; i < n_items && ok; ++i) {
+        const Item it = item_at(i);
+        const int qb = i % C::kQBufs;
+        const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO[qb][0]));
+        const uint32_t t_sfdO = tmem + kColSFdO + 4 * kCv * qb;
+        ok = mbar_wait(&sm.q_full[qb], (i / C::kQBufs) & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after_sync();
-        if (kFp8v) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
-        if (t > 0) {
-          ok = mbar_wait(&sm.sdp_free, (t - 1) & 1, abort_flag);
+        if (kFp8v) {
+          tc_fence_after_sync();
+          sf_copy_tiles<kCv>(t_sfdO, sm.sf_dO[qb]);
+        }
+        for (int t = 0; t < it.n_tiles && ok; ++t) {
+          const int gt = T + t;
+          const int s = gt % kStages, slot = gt & 1;
+          ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
+          if (kFp8v) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
+          if (gt > 0) {
+            ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+          const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
+          issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, t_sfdO,
+                                                                          tmem + kColSFV + 4 * kCv * slot);
+          mma_commit_elect(&sm.sdp_full);
+          mma_commit_elect(&sm.kv_empty[s]);
         }
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
-        issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, tmem + kColSFdO,
-                                                                        tmem + kColSFV + 4 * kCv * slot);
-        mma_commit_elect(&sm.sdp_full);
-        mma_commit_elect(&sm.kv_empty[s]);
+        if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's dO tile has been read
+        T += it.n_tiles;
       }
       if (!ok) {
         int dummy = 0;
@@ -312,6 +378,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     // ------------------------------------------------------------------ dQ issuer
     if (kDQ) {
       bool ok = true;
+      const Item it = item_at(0);                     // the dQ kernel is not persistent: one item
+      const int n_tiles = it.n_tiles;
+      const int n_dq = min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int s = t % kKcStages, slot = t & 1, buf = t & 1;
         ok = mbar_wait(&sm.kc_full[s], (t / kKcStages) & 1, abort_flag);
@@ -349,10 +418,21 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-    const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
+    auto row_of = [&](const Item& it) {
+      return static_cast<size_t>(it.b * p.Hq + it.h) * p.N + it.qt * kTile + row;
+    };
+    bool ok = true;
+    int T = 0;                                        // key steps of the items before this one
+    float lse_next = p.lse[row_of(item_at(0))];
+    for (int i = 0; i < n_items && ok; ++i) {
+    const Item it = item_at(i);
+    const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
+    const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
+    const size_t grow = row_of(it);
     // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
     // to the half ulp the FP32 storage of LSE already carries
-    const float lse_nat = p.lse[grow];
+    const float lse_nat = lse_next;
+    if (kPersist && i + 1 < n_items) lse_next = p.lse[row_of(item_at(i + 1))];   // in flight while this item runs
     const float lse2 = lse_nat * kLog2e;
     const float lse2_lo = fmaf(lse_nat, kLog2e, -lse2) + lse_nat * kLog2eLo;
     const float D = kDQ ? p.delta_in[grow] : 0.f;
@@ -366,11 +446,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       sm.red[grp][2][row] = 0.f;
       sm.red[grp][3][row] = 0.f;
     }
-    bool ok = true;
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 0);
-      ok = mbar_wait(&sm.sdp_full, t & 1, abort_flag);
+      ok = mbar_wait(&sm.sdp_full, (T + t) & 1, abort_flag);
       if (!ok) break;
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 1);
       tc_fence_after_sync();
@@ -477,13 +556,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
-    // combine the row sums of the column groups (fixed order: reproducible)
-    sm.red[grp][0][row] = acc0;
-    sm.red[grp][1][row] = acc1;
+    // combine the row sums of the column groups (fixed order: reproducible).  The persistent
+    // delta kernel alternates between two slots, so that the next item's partial sums do not
+    // overwrite what group 0 may still be reading.
+    const int si = kPersist ? (i & 1) : 0;
+    sm.red[grp][si][row] = acc0;
+    if (kDQ) sm.red[grp][1][row] = acc1;
     named_barrier_sync(1, kSoftmaxThreads);
     if (ok && grp == 0) {
       acc0 = 0.f; acc1 = 0.f;
-      for (int i = 0; i < kGroups; ++i) { acc0 += sm.red[i][0][row]; acc1 += sm.red[i][1][row]; }
+      for (int j = 0; j < kGroups; ++j) {
+        acc0 += sm.red[j][si][row];
+        if (kDQ) acc1 += sm.red[j][1][row];
+      }
       if (!kDQ) {
         p.delta_out[grow] = acc0;
       } else if (p.rowsum && r_tile == 0) {
@@ -491,7 +576,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         p.rowabs[grow] = acc1;
         if (p.post_rowsum) {
           float post0 = 0.f, post1 = 0.f;
-          for (int i = 0; i < kGroups; ++i) { post0 += sm.red[i][2][row]; post1 += sm.red[i][3][row]; }
+          for (int j = 0; j < kGroups; ++j) { post0 += sm.red[j][2][row]; post1 += sm.red[j][3][row]; }
           p.post_rowsum[grow] = post0;
           p.post_rowabs[grow] = post1;
         }
@@ -518,6 +603,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
       }
     }
+    T += n_tiles;
+    }  // items
   }
   __syncwarp();
   tc_fence_before_sync();
@@ -566,6 +653,17 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   const int rq = kDQ ? (s.dqk + 127) / 128 : 1;
   dim3 grid(s.Hq * rq, s.N / kTile, s.B);
+  p.gx = static_cast<int>(grid.x); p.gy = static_cast<int>(grid.y); p.gz = static_cast<int>(grid.z);
+  if (C::kPersist) {
+    // one CTA per SM (the kernel takes a whole SM's shared memory) walks the item list
+    int dev = 0, sms = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess || sms < 1) return fail(ATTN_ERR_CUDA, "bwd q-major: SM count: %s", cudaGetErrorString(e));
+    const long long items = static_cast<long long>(p.gx) * p.gy * p.gz;
+    if (items > 0x7fffffffLL) return fail(ATTN_ERR_UNSUPPORTED, "bwd q-major: %lld work items exceed 2^31 - 1", items);
+    grid = dim3(static_cast<unsigned>(items < sms ? items : sms), 1, 1);
+  }
   if (behind_dkdv) {
     // the key-major kernel ahead in the stream reads what this one reads and writes other buffers:
     // this grid may take the SMs that kernel's last wave leaves idle
