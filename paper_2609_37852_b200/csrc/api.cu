@@ -369,8 +369,9 @@ attn_status_t attn_fp8_read_status(void* workspace, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-  if (e == cudaSuccess && host != 0) {          // reported once: clear it for the calls that follow
-    e = cudaMemsetAsync(workspace, 0, sizeof(int), st);
+  if (e == cudaSuccess && host != 0) {          // reported once: clear the header (status word and the scheduling
+                                                // counters a kernel that gave up may have left) for the calls that follow
+    e = cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   }
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "read_status: %s", cudaGetErrorString(e));

@@ -69,16 +69,16 @@ struct QmCfg {
                                                         // 2 with kEB == 1 is the protected-dP ablation
   static constexpr bool kFp8 = kEB == 1;
   static constexpr bool kFp8v = kEBv == 1;
-  // The delta kernel is persistent: one CTA per SM walks a list of query tiles, with the Q / dO
-  // tiles double-buffered and the K / V ring, the score buffers and their barriers running on
-  // across tile boundaries, so that set-up, pipeline fill and drain are paid once per CTA instead
-  // of once per query tile.  The dQ kernel keeps one query tile per CTA (its accumulator has to
-  // leave tensor memory between tiles, and launched behind the key-major kernel its CTAs start at
-  // different times, which a static tile list cannot balance).
+  // Both kernels are persistent where shared memory allows: a CTA walks a list of query tiles, with
+  // the Q / dO tiles double-buffered and the K / V rings, the score buffers and their barriers
+  // running on across tile boundaries, so that set-up, pipeline fill and most of the drain are paid
+  // once per CTA instead of once per query tile.  The delta kernel takes a static list (all its CTAs
+  // start together).  The dQ kernel is launched behind the key-major kernel, so its CTAs start at
+  // different times: they draw their tiles from a ticket counter in the workspace instead.
   static constexpr int kStep = kTile / kEB;             // keys per step
-  // (where two Q / dO tiles and two K / V stages do not fit in shared memory, the delta kernel is
-  // not persistent either)
-  static constexpr bool kPersist = !kDQ && 2 * (kCq + kCv) * (kTile + kStep) * 128 <= 224 * 1024;
+  static constexpr bool kPersist =
+      2 * (kCq + kCv) * kTile * 128 + 2 * ((kCq + kCv) * kStep * 128 + (kDQ ? kTile * 128 : 0)) <= 216 * 1024;
+  static constexpr bool kTicket = kPersist && kDQ;
   static constexpr int kQBufs = kPersist ? 2 : 1;       // Q / dO tile buffers (and scale-factor slots)
   static constexpr int kGroups = kStep / 32;            // 32-key column groups of a step
   static constexpr int kSoftmaxThreads = 128 * kGroups; // 4 TMEM lane quadrants x column groups
@@ -124,7 +124,9 @@ struct QmSmem {
   uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
   uint64_t sdp_full, sdp_free;
   uint64_t ds_full[2], ds_free[2];
-  uint64_t dq_done;
+  uint64_t dq_done, dq_free;
+  uint64_t item_full[4];        // ticket mode: the producer has published the CTA's i-th work item in item_l[i % 4]
+  int item_l[4];
   uint64_t drain[3];
   uint32_t tmem_base;
   int abort_flag;
@@ -141,6 +143,7 @@ struct QmParams {
   float* post_rowsum;       // optional: row sums of the CAST score gradient (the dQ operand) and of its magnitude
   float* post_rowabs;
   int* status;
+  int* sched;               // ticket mode: {next item, CTAs finished}, both zero between launches
   int N, Hq, Hkv, dqk, dv, causal;
   int gx, gy, gz;           // the (head x column tile, query tile, batch) grid the work items are numbered in
   int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
@@ -155,7 +158,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // declared with the alignment the swizzled operand tiles need, so that the compiler keeps the
   // shared state space of every access derived from it (checked below)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8, kFp8v = C::kFp8v, kPersist = C::kPersist;
+  constexpr bool kDQ = C::kDQ, kFp8 = C::kFp8, kFp8v = C::kFp8v, kPersist = C::kPersist, kTicket = C::kTicket;
   constexpr int kStages = C::kStages, kKcStages = C::kKcStages, kEB = C::kEB, kCq = C::kCq, kCv = C::kCv;
   constexpr int kStep = C::kStep, kGroups = C::kGroups, kSoftmaxThreads = C::kSoftmaxThreads;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColdS = C::kColdS, kColdQ = C::kColdQ, kColSFQ = C::kColSFQ,
@@ -169,36 +172,44 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // Work items are numbered x-fastest over the grid (gx, gy, gz): heads vary fastest and the heaviest
   // (latest) query tiles of all heads come first, so the light tiles fill the tail.  Without
-  // persistence a CTA is its own item.  A persistent CTA takes the items c, 2n-1-c, 2n+c, ... (n CTAs,
-  // c its index): alternate rounds run backwards, so that no CTA collects the heavier item of every
-  // round.
+  // persistence a CTA is its own item.  With a static list a persistent CTA takes the items c,
+  // 2n-1-c, 2n+c, ... (n CTAs, c its index): alternate rounds run backwards, so that no CTA collects
+  // the heavier item of every round.  In ticket mode the producer thread draws item numbers from a
+  // global counter and publishes them to the other warps through shared memory.
   const int rq = kDQ ? (p.dqk + 127) / 128 : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
   const int total_items = p.gx * p.gy * p.gz;
   const int n_cta = static_cast<int>(gridDim.x);
-  const int n_items = !kPersist ? 1
-                                : total_items / n_cta + ((((total_items / n_cta) & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x)
-                                                                                        : static_cast<int>(blockIdx.x)) <
-                                                             total_items % n_cta
-                                                         ? 1 : 0);
-  struct Item { int qt, h, r_tile, b, g, n_tiles; };
-  auto item_at = [&](int i) {
-    int x, y, z;
-    if (kPersist) {
-      const int pos = (i & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
-      const int l = i * n_cta + pos;
-      x = l % p.gx; y = (l / p.gx) % p.gy; z = l / (p.gx * p.gy);
-    } else {
-      x = blockIdx.x; y = blockIdx.y; z = blockIdx.z;
-    }
+  const int n_static = !kPersist ? 1
+                                 : total_items / n_cta + ((((total_items / n_cta) & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x)
+                                                                                         : static_cast<int>(blockIdx.x)) <
+                                                              total_items % n_cta
+                                                          ? 1 : 0);
+  volatile int* abort_flag = &sm.abort_flag;
+  struct Item { int qt, h, r_tile, b, g, n_tiles; bool valid; };
+  auto decode = [&](int x, int y, int z) {
     Item it;
     it.qt = p.causal ? (p.gy - 1 - y) : y;
     it.h = x / rq; it.r_tile = x % rq; it.b = z;
     it.g = it.h / (p.Hq / p.Hkv);
     it.n_tiles = (p.causal ? it.qt + 1 : p.N / kTile) * kEB;       // key steps
+    it.valid = true;
     return it;
   };
+  auto decode_linear = [&](int l) { return decode(l % p.gx, (l / p.gx) % p.gy, l / (p.gx * p.gy)); };
+  // the i-th item of this CTA (valid = false: no more; in ticket mode also when the wait gave up)
+  auto item_at = [&](int i) {
+    Item none; none.valid = false; none.qt = none.h = none.r_tile = none.b = none.g = none.n_tiles = 0;
+    if (!kPersist) return i == 0 ? decode(blockIdx.x, blockIdx.y, blockIdx.z) : none;
+    if (!kTicket) {
+      if (i >= n_static) return none;
+      const int pos = (i & 1) ? n_cta - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
+      return decode_linear(i * n_cta + pos);
+    }
+    if (!mbar_wait(&sm.item_full[i & 3], (i >> 2) & 1, abort_flag)) return none;
+    const int l = *reinterpret_cast<volatile int*>(&sm.item_l[i & 3]);
+    return l >= 0 ? decode_linear(l) : none;
+  };
   const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * C::kEBv / 32;       // 32-byte K steps of the two products
-  volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
     for (int i = 0; i < C::kQBufs; ++i) { mbar_init(&sm.q_full[i], 1); mbar_init(&sm.q_empty[i], 2); }
@@ -208,7 +219,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     for (int s = 0; s < kKcStages; ++s) { mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1); }
     mbar_init(&sm.sdp_full, 2); mbar_init(&sm.sdp_free, kSoftmaxThreads);
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kSoftmaxThreads); mbar_init(&sm.ds_free[i], 1); }
-    mbar_init(&sm.dq_done, 1);
+    mbar_init(&sm.dq_done, 1); mbar_init(&sm.dq_free, kSoftmaxThreads);
+    for (int i = 0; i < 4; ++i) mbar_init(&sm.item_full[i], 1);
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     sm.abort_flag = 0;
     fence_mbar_init();
@@ -231,15 +243,30 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       int issued_kv = 0, issued_kc = 0;
       bool ok = true;
       int T = 0;                                      // key steps of the items before this one
-      for (int i = 0; i < n_items && ok; ++i) {
-        const Item it = item_at(i);
-        const int q_slab = it.b * p.Hq + it.h, kv_slab = it.b * p.Hkv + it.g;
+      int ticket = kTicket ? atomicAdd(p.sched, 1) : 0;
+      for (int i = 0; ok; ++i) {
         const int qb = i % C::kQBufs;
-        if (i >= C::kQBufs) {
-          // both issuers have finished with the item that used this Q / dO buffer
+        if (kPersist && i >= C::kQBufs) {
+          // both issuers have finished with the item that used this Q / dO buffer (and every warp has
+          // long read the slot of the item list that is about to be rewritten)
           ok = mbar_wait(&sm.q_empty[qb], ((i / C::kQBufs) - 1) & 1, abort_flag);
           if (!ok) break;
         }
+        Item it;
+        if (kTicket) {
+          // publish this CTA's i-th item (or the end of the list) to the other warps, and draw the
+          // next ticket now: its latency passes while this item's copies are issued
+          const int l = ticket < total_items ? ticket : -1;
+          sm.item_l[i & 3] = l;
+          mbar_arrive(&sm.item_full[i & 3]);
+          if (l < 0) break;
+          it = decode_linear(l);
+          ticket = atomicAdd(p.sched, 1);
+        } else {
+          it = item_at(i);
+          if (!it.valid) break;
+        }
+        const int q_slab = it.b * p.Hq + it.h, kv_slab = it.b * p.Hkv + it.g;
         mbar_arrive_expect_tx(&sm.q_full[qb], kCq * (kTile * 128 + (kFp8 ? 512 : 0)) + kCv * (kTile * 128 + (kFp8v ? 512 : 0)));
         for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[qb][c], &tm_q, &sm.q_full[qb], 128 * c, q_slab * p.N + it.qt * kTile);
         for (int c = 0; c < kCv; ++c) tma_load_2d(sm.dO[qb][c], &tm_dO, &sm.q_full[qb], 128 * c, q_slab * p.N + it.qt * kTile);
@@ -262,8 +289,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
           ++issued_kv;
           if (kDQ) {
-            const int sc = t % kKcStages;
-            ok = mbar_wait(&sm.kc_empty[sc], ((t / kKcStages) & 1) ^ 1, abort_flag);
+            const int sc = gt % kKcStages;
+            ok = mbar_wait(&sm.kc_empty[sc], ((gt / kKcStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
             mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
             tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * it.r_tile);
@@ -288,8 +315,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     {
       bool ok = true;
       int T = 0;
-      for (int i = 0; i < n_items && ok; ++i) {
+      for (int i = 0; ok; ++i) {
         const Item it = item_at(i);
+        if (!it.valid) break;
         const int qb = i % C::kQBufs;
         const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[qb][0]));
         const uint32_t t_sfq = tmem + kColSFQ + 4 * kCq * qb;
@@ -325,6 +353,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's Q tile has been read
         T += it.n_tiles;
       }
+      if (*abort_flag) ok = false;
       if (!ok) {
         int dummy = 0;
         mma_commit_elect(&sm.drain[0]);
@@ -336,8 +365,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     {
       bool ok = true;
       int T = 0;
-      for (int i = 0; i < n_items && ok; ++i) {
+      for (int i = 0; ok; ++i) {
         const Item it = item_at(i);
+        if (!it.valid) break;
         const int qb = i % C::kQBufs;
         const uint64_t desc_dO = make_desc_sw128(smem_u32(sm.dO[qb][0]));
         const uint32_t t_sfdO = tmem + kColSFdO + 4 * kCv * qb;
@@ -368,6 +398,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's dO tile has been read
         T += it.n_tiles;
       }
+      if (*abort_flag) ok = false;
       if (!ok) {
         int dummy = 0;
         mma_commit_elect(&sm.drain[1]);
@@ -378,34 +409,47 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     // ------------------------------------------------------------------ dQ issuer
     if (kDQ) {
       bool ok = true;
-      const Item it = item_at(0);                     // the dQ kernel is not persistent: one item
-      const int n_tiles = it.n_tiles;
-      const int n_dq = min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % kKcStages, slot = t & 1, buf = t & 1;
-        ok = mbar_wait(&sm.kc_full[s], (t / kKcStages) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-        if (kFp8) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
-        ok = mbar_wait(&sm.ds_full[buf], (t >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-        if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
-        const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          if (kFp8)
-            mma_mxf8_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
-                              make_idesc_mxf8(128, n_dq, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
-                              (t > 0 || kb > 0));
-          else
-            mma_bf16_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
-                              make_idesc_bf16(128, n_dq), (t > 0 || kb > 0));
+      int T = 0;
+      for (int i = 0; ok; ++i) {
+        const Item it = item_at(i);
+        if (!it.valid) break;
+        const int n_tiles = it.n_tiles;
+        const int n_dq = min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
+        if (i > 0) {
+          // the softmax threads have read the previous item's dQ out of tensor memory
+          ok = mbar_wait(&sm.dq_free, (i - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
         }
-        mma_commit_elect(&sm.ds_free[buf]);            // operand and scale bytes of this buffer may be overwritten
-        mma_commit_elect(&sm.kc_empty[s]);
-        if (t == n_tiles - 1) mma_commit_elect(&sm.dq_done);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int gt = T + t;                       // the K^T ring and the dS^ buffers run on across items
+          const int s = gt % kKcStages, slot = gt & 1, buf = gt & 1;
+          ok = mbar_wait(&sm.kc_full[s], (gt / kKcStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          if (kFp8) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+          ok = mbar_wait(&sm.ds_full[buf], (gt >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
+          const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            if (kFp8)
+              mma_mxf8_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+                                make_idesc_mxf8(128, n_dq, kb, kb), tmem + kColSFdS + 4 * buf, tmem + kColSFKc + 4 * slot,
+                                (t > 0 || kb > 0));
+            else
+              mma_bf16_ts_elect(tmem + kColdQ, tmem + kColdS + 32 * buf + 8 * kb, desc_kc + 2 * kb,
+                                make_idesc_bf16(128, n_dq), (t > 0 || kb > 0));
+          }
+          mma_commit_elect(&sm.ds_free[buf]);            // operand and scale bytes of this buffer may be overwritten
+          mma_commit_elect(&sm.kc_empty[s]);
+          if (t == n_tiles - 1) mma_commit_elect(&sm.dq_done);
+        }
+        T += n_tiles;
       }
+      if (*abort_flag) ok = false;
       if (!ok) {
         int dummy = 0;
         mma_commit_elect(&sm.drain[2]);
@@ -423,19 +467,22 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     };
     bool ok = true;
     int T = 0;                                        // key steps of the items before this one
-    float lse_next = p.lse[row_of(item_at(0))];
-    for (int i = 0; i < n_items && ok; ++i) {
-    const Item it = item_at(i);
+    Item it = item_at(0);
+    float lse_next = 0.f, d_next = 0.f;
+    if (it.valid) {
+      lse_next = p.lse[row_of(it)];
+      if (kDQ) d_next = p.delta_in[row_of(it)];
+    }
+    for (int i = 0; ok && it.valid; ++i) {
     const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
     const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
     const size_t grow = row_of(it);
     // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
     // to the half ulp the FP32 storage of LSE already carries
     const float lse_nat = lse_next;
-    if (kPersist && i + 1 < n_items) lse_next = p.lse[row_of(item_at(i + 1))];   // in flight while this item runs
     const float lse2 = lse_nat * kLog2e;
     const float lse2_lo = fmaf(lse_nat, kLog2e, -lse2) + lse_nat * kLog2eLo;
-    const float D = kDQ ? p.delta_in[grow] : 0.f;
+    const float D = d_next;
     const float f_lo = fmaf(-lse2_lo, kLn2, 1.0f);   // 2^-lo to first order (|lo| < 1e-5)
     const float fD = f_lo * D;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
@@ -447,9 +494,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       sm.red[grp][3][row] = 0.f;
     }
     for (int t = 0; t < n_tiles; ++t) {
-      const int buf = t & 1;
+      const int gt = T + t;                           // step index over all items: the dS^ buffers run on
+      const int buf = gt & 1;
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 0);
-      ok = mbar_wait(&sm.sdp_full, (T + t) & 1, abort_flag);
+      ok = mbar_wait(&sm.sdp_full, gt & 1, abort_flag);
       if (!ok) break;
       if (warp == 4 && lane == 0) QM_TRACE(2, t, 1);
       tc_fence_after_sync();
@@ -541,9 +589,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           sm.red[grp][2][row] += ps;
           sm.red[grp][3][row] += pa;
         }
-        if (t >= 2) {
-          // the dQ MMAs of tile t-2 have consumed this buffer's operand and scale bytes
-          ok = mbar_wait(&sm.ds_free[buf], ((t - 2) >> 1) & 1, abort_flag);
+        if (gt >= 2) {
+          // the dQ MMAs of step gt-2 have consumed this buffer's operand and scale bytes
+          ok = mbar_wait(&sm.ds_free[buf], ((gt - 2) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
@@ -556,10 +604,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
+    // the next item (published by now, as a rule): its LSE and D are in flight during this item's epilogue
+    Item nx; nx.valid = false;
+    if (kPersist && ok) {
+      nx = item_at(i + 1);
+      if (nx.valid) {
+        lse_next = p.lse[row_of(nx)];
+        if (kDQ) d_next = p.delta_in[row_of(nx)];
+      }
+    }
     // combine the row sums of the column groups (fixed order: reproducible).  The persistent
     // delta kernel alternates between two slots, so that the next item's partial sums do not
     // overwrite what group 0 may still be reading.
-    const int si = kPersist ? (i & 1) : 0;
+    const int si = (kPersist && !kDQ) ? (i & 1) : 0;   // the dQ kernel uses slots 0 and 1 and a barrier per item
     sm.red[grp][si][row] = acc0;
     if (kDQ) sm.red[grp][1][row] = acc1;
     named_barrier_sync(1, kSoftmaxThreads);
@@ -583,7 +640,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       }
     }
     if (kDQ && ok) {
-      ok = mbar_wait(&sm.dq_done, 0, abort_flag);
+      ok = mbar_wait(&sm.dq_done, i & 1, abort_flag);
       if (ok) {
         tc_fence_after_sync();
         __nv_bfloat16* out_row = p.dq + grow * p.dqk + 128 * r_tile;
@@ -601,9 +658,17 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
 #pragma unroll
           for (int c = 0; c < 4; ++c) dst[c] = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
         }
+        if (kPersist) {
+          // the accumulator may be overwritten by the next item's first dQ MMA
+          tc_fence_before_sync();
+          mbar_arrive(&sm.dq_free);
+        }
       }
     }
+    // the row-sum slots may be overwritten by the next item's partial sums
+    if (kDQ && kPersist) named_barrier_sync(1, kSoftmaxThreads);
     T += n_tiles;
+    it = nx;
     }  // items
   }
   __syncwarp();
@@ -611,6 +676,16 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+  if (kTicket && tid == 0) {
+    // every CTA has drawn its last ticket before it gets here: the last one to arrive puts the two
+    // counters back to zero for the next launch
+    __threadfence();
+    if (atomicAdd(p.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+      p.sched[0] = 0;
+      p.sched[1] = 0;
+      __threadfence();
+    }
+  }
   // This grid may have started while the grid ahead of it was draining.  One CTA, the last in
   // launch order, stays until that grid has completed, so that the completion of this grid
   // implies the completion of both for whatever follows in the stream.
@@ -648,6 +723,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   p.tail_wait = behind_dkdv ? 1 : 0;
+  p.sched = status + 4;                             // bytes 16..23 of the workspace header
   const size_t smem = sizeof(QmSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
