@@ -35,7 +35,7 @@ FP8_OVER_BF16 = 2.0                 # nominal dense FP8 : BF16 tensor ratio on B
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on WORKLOAD, from
 # the ncu captures summarised under profiles/; None where no capture has been taken.
-NCU_TRAFFIC_BYTES = {"quantize": 288.9e6, "fwd": 70.4e6, "bwd_delta": 90.6e6, "bwd_dq": 128.7e6, "bwd_dkdv": 317.9e6}
+NCU_TRAFFIC_BYTES = {"quantize": 288.9e6, "fwd": 70.4e6, "bwd_delta": 90.5e6, "bwd_dq": 126.2e6, "bwd_dkdv": 317.9e6}
 
 # executed matmul products per kernel as (contractions or outputs of width dqk, of width dv): each is
 # 2*width FLOPs per unmasked (i, j) pair and query head
