@@ -493,6 +493,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       sm.red[grp][2][row] = 0.f;
       sm.red[grp][3][row] = 0.f;
     }
+    if (warp == 4 && lane == 0) QM_TRACE(3, i, 0);
     for (int t = 0; t < n_tiles; ++t) {
       const int gt = T + t;                           // step index over all items: the dS^ buffers run on
       const int buf = gt & 1;
@@ -604,6 +605,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
+    if (warp == 4 && lane == 0) QM_TRACE(3, i, 1);
     // the next item (published by now, as a rule): its LSE and D are in flight during this item's epilogue
     Item nx; nx.valid = false;
     if (kPersist && ok) {
@@ -641,6 +643,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     if (kDQ && ok) {
       ok = mbar_wait(&sm.dq_done, i & 1, abort_flag);
+      if (warp == 4 && lane == 0) QM_TRACE(3, i, 2);
       if (ok) {
         tc_fence_after_sync();
         __nv_bfloat16* out_row = p.dq + grow * p.dqk + 128 * r_tile;
@@ -667,6 +670,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     // the row-sum slots may be overwritten by the next item's partial sums
     if (kDQ && kPersist) named_barrier_sync(1, kSoftmaxThreads);
+    if (warp == 4 && lane == 0) QM_TRACE(3, i, 3);
     T += n_tiles;
     it = nx;
     }  // items
