@@ -277,8 +277,8 @@ attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, att
 /* Bytes of workspace the given entry point needs for `p` (attn_ws_kind_t).  The workspace is
  * scratch owned by the caller; one workspace may serve all entry points of a stream.  Its first
  * word is the device-side status word; the rest of its first ATTN_STATUS_WORKSPACE_BYTES bytes holds
- * counters the kernels of one call share (zero between calls: give concurrent streams separate
- * workspaces).  The status is STICKY: kernels only ever set it (a bounded
+ * counters the kernels of one call share (each call clears its own: give concurrent streams
+ * separate workspaces).  The status is STICKY: kernels only ever set it (a bounded
  * wait that gave up, a launch that found its shared memory misaligned), no entry point clears it,
  * so one attn_fp8_read_status at the end of a chain of calls reports a failure of any of them.
  * A workspace must be initialised once before its first use (attn_fp8_workspace_init, or any other

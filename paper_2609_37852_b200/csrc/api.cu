@@ -311,6 +311,12 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
   int* status = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CHECK(prepare_workspace(workspace, workspace_bytes, attn_fp8_workspace_bytes(p, ATTN_WS_BWD), st, &status));
+  if (want_dq) {
+    // the ticket counter of the persistent dQ kernel (bytes 16..31 of the header) starts at zero; cleared
+    // here, ahead of both kernels, so that nothing sits between the key-major launch and the dQ launch
+    cudaError_t e = cudaMemsetAsync(static_cast<char*>(workspace) + 16, 0, 16, st);
+    if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd: cudaMemsetAsync(ticket counter): %s", cudaGetErrorString(e));
+  }
   // Key-major kernel first: its CTAs are few and long, so its last wave leaves SMs idle, which
   // the many short CTAs of the query-major kernel, launched behind it, fill.
   if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));

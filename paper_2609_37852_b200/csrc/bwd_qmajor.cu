@@ -143,7 +143,7 @@ struct QmParams {
   float* post_rowsum;       // optional: row sums of the CAST score gradient (the dQ operand) and of its magnitude
   float* post_rowabs;
   int* status;
-  int* sched;               // ticket mode: {next item, CTAs finished}, both zero between launches
+  int* sched;               // ticket mode: the next item number; the host zeroes it ahead of the launch
   int N, Hq, Hkv, dqk, dv, causal;
   int gx, gy, gz;           // the (head x column tile, query tile, batch) grid the work items are numbered in
   int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
@@ -680,16 +680,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
-  if (kTicket && tid == 0) {
-    // every CTA has drawn its last ticket before it gets here: the last one to arrive puts the two
-    // counters back to zero for the next launch
-    __threadfence();
-    if (atomicAdd(p.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
-      p.sched[0] = 0;
-      p.sched[1] = 0;
-      __threadfence();
-    }
-  }
   // This grid may have started while the grid ahead of it was draining.  One CTA, the last in
   // launch order, stays until that grid has completed, so that the completion of this grid
   // implies the completion of both for whatever follows in the stream.

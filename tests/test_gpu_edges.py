@@ -260,3 +260,26 @@ def test_expired_wait_is_reported_and_the_context_survives():
     B.attn_fp8_workspace_init(raw)
     B.attn_fp8_fwd(params, qq, kq, vq, workspace=raw)
     B.attn_fp8_read_status(raw)
+
+
+def test_header_counters_are_cleared_by_the_call_that_uses_them():
+    """Beyond the status word the workspace header holds the ticket counter of the persistent dQ
+    kernel; the gradient call clears it itself, so whatever an earlier user left there is harmless."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=512)
+    tensors = [x.cuda() for x in workloads.make_inputs(w)]
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, 128, 128, True, w.softmax_scale)
+    (qq, kq, vq, dOq), _ = B.attn_fp8_quantize_batch(tensors)
+    o, lse, ws = B.attn_fp8_fwd(params, qq, kq, vq)
+    delta, ws = B.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
+    ref = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, workspace=ws)
+    B.attn_fp8_read_status(ws)
+    dirty = torch.full((ws.numel(),), 0x5A, dtype=torch.uint8, device="cuda")
+    dirty[:4] = 0                                                       # the status word alone is initialised
+    for call in range(2):
+        got = B.attn_fp8_bwd(params, qq, kq, vq, dOq, lse, delta, workspace=dirty)
+        B.attn_fp8_read_status(dirty)
+        for a, b in zip(got[:3], ref[:3]):
+            assert torch.equal(a, b), f"call {call}"
+        dq_only = B.attn_fp8_bwd_dq(params, qq, kq, vq, dOq, lse, delta, workspace=dirty)
+        assert torch.equal(dq_only[0], ref[0])
