@@ -1,8 +1,10 @@
 // Query-major backward kernels: the matched row correction (Delta-Matching, paper Section 3.3
 // Eq. 4) and the query gradient (paper Appendix "Backward Correction and Gradient Computation").
 //
-// One CTA owns 128 query rows of one (batch, query head) and sweeps the key tiles (128 keys) up to
-// the causal diagonal.  For every key tile the tensor cores recompute
+// A work item is 128 query rows of one (batch, query head); the CTA that has it sweeps the key
+// tiles (128 keys) up to the causal diagonal.  Where shared memory allows, a CTA takes one item
+// after another (one CTA per SM; see QmCfg::kPersist for how the items are handed out).  For every
+// key tile the tensor cores recompute
 //     S  = Q^ K^^T   (row-blocked FP8 copies, contraction over the qk channels)
 //     dP = dO^ V^^T  (row-blocked FP8 copies, contraction over the v channels)
 // into tensor memory; the softmax warps rebuild P = 2^(S*scale*log2e - LSE*log2e) in FP32 from
