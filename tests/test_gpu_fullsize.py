@@ -110,6 +110,15 @@ def test_long_context_sampled():
     _check_sampled(w, tensors, got, heads=[(0, 5)], rows=32, col_groups=2, seed=3)
 
 
+def test_long_context_full_size_sampled():
+    """long64k as configured: B=1, 32/8 heads, N=65536, d=128 (16384 work items per query-major kernel,
+    2.7 GB of operands); about a minute of host-side input generation."""
+    w = workloads.WORKLOADS["long64k"]
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors)
+    _check_sampled(w, tensors, got, heads=[(0, 0), (0, 31)], rows=6, col_groups=2, seed=3)
+
+
 def test_mla_full_size_sampled():
     """mla8k: B=1, 16/16 heads, N=8192, qk head dim 192, v head dim 128."""
     w = workloads.WORKLOADS["mla8k"]
