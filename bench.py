@@ -324,9 +324,12 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
     # per-stage breakdown: the same steps once more with an event at every stage boundary, followed by
     # the two kernels of the gradient pass as separate (serialised) calls
+    stage_sampler = ClockSampler(local_rank)
+    stage_sampler.start()
     for i in range(args.steps):
         step(events[i], split=True)
     torch.cuda.synchronize()
+    stage_clocks = stage_sampler.stop()
     B.attn_fp8_read_status(ws)
     stage_ms = {n: statistics.mean(ev[j].elapsed_time(ev[j + 1]) for ev in events)
                 for j, n in enumerate(("quantize", "fwd", "bwd_delta", "bwd", "bwd_dq", "bwd_dkdv"))}
@@ -431,7 +434,9 @@ def main():
         "stage_ms": stage_ms,
         "stage_timing": "a second loop of the same steps with an event at every stage boundary (the timed region has "
                         "none: an event costs a few microseconds); bwd = the overlapped gradient call, bwd_dq and "
-                        "bwd_dkdv = its two kernels as separate, serialised calls",
+                        "bwd_dkdv = its two kernels as separate, serialised calls; this loop runs later and longer "
+                        "than the timed region, at the clocks sustained load settles to (stage_clocks)",
+        "stage_clocks": stage_clocks,
         # the timed step less the operand preparation (the paper's accounting), and less the forward
         "attn_only_tflops": credited / ((step_ms - stage_ms["quantize"]) * 1e-3) / 1e12,
         "fwd_tflops": fwd_flops / (stage_ms["fwd"] * 1e-3) / 1e12,
