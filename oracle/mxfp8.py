@@ -110,11 +110,12 @@ def fake_quant(x, axis=-1):
 
 def round_bf16(x):
     """Round float64 to the nearest BF16 value (8 significand bits, ties to even);
-    returned as float64.  Overflow and BF16 subnormals are outside the tested range."""
+    returned as float64.  Below 2**-126 the grid is that of the BF16 subnormals (spacing 2**-133,
+    gradual underflow to zero); overflow is outside the tested range."""
     x = np.asarray(x, dtype=np.float64)
     a = np.abs(x)
     _, ex = np.frexp(a)
-    quantum = np.ldexp(1.0, ex - 1 - 7)
+    quantum = np.ldexp(1.0, np.maximum(ex - 1 - 7, -133))
     r = np.rint(a / quantum) * quantum
     r = np.where(a == 0.0, 0.0, r)
     return np.copysign(r, x)

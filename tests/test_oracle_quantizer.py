@@ -153,3 +153,18 @@ def test_round_bf16_matches_torch():
     ours = mxfp8.round_bf16(x32.astype(np.float64))
     theirs = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
     assert np.array_equal(ours, theirs)
+
+
+def test_round_bf16_underflows_gradually_like_torch():
+    """Below 2**-126 BF16 has subnormals of spacing 2**-133: torch's cast is the reference there too, and
+    float64 values far below the format (probabilities of far keys in BF16 mode) round to zero, not NaN."""
+    bits = np.arange(0, 0x01000000, 0x1357, dtype=np.uint32)           # FP32 subnormals and the first normal binades
+    x32 = np.concatenate([bits.view(np.float32), -bits.view(np.float32),
+                          np.float32(2.0) ** np.arange(-149, -120).astype(np.float32) * np.float32(1.5)])
+    ours = mxfp8.round_bf16(x32.astype(np.float64))
+    theirs = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(ours, theirs)
+    tiny = np.array([1e-300, -1e-310, 5e-324, 2.0 ** -135, 2.0 ** -134, 3 * 2.0 ** -135])
+    want = np.array([0.0, -0.0, 0.0, 0.0, 0.0, 2.0 ** -133])            # ties to even; 3/4 of the step rounds up
+    got = mxfp8.round_bf16(tiny)
+    assert np.array_equal(got, want) and not np.isnan(got).any()
