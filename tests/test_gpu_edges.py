@@ -62,6 +62,8 @@ def test_small_and_extreme_shapes(name, kw):
     ("tiny", dict(seqlen=384, heads_q=6, heads_kv=2, causal=True), True),            # BF16 mode at d = 64, groups of 3
     ("long64k", dict(heads_q=2, heads_kv=1, seqlen=1152), False),                    # heavy-tailed channel gains, 9 tiles
     ("gqa8k_outlier", dict(batch=3, heads_q=16, heads_kv=1, seqlen=256), False),     # 16 query heads on one KV head
+    ("gqa8k_outlier", dict(batch=3, heads_q=6, heads_kv=3, seqlen=640), True),       # BF16 mode, outlier scores: far-key
+                                                                                      # probabilities below the BF16 range
 ])
 def test_shape_and_mode_combinations(name, kw, bf16):
     w = workloads.WORKLOADS[name].scaled(**kw)
@@ -283,3 +285,30 @@ def test_header_counters_are_cleared_by_the_call_that_uses_them():
             assert torch.equal(a, b), f"call {call}"
         dq_only = B.attn_fp8_bwd_dq(params, qq, kq, vq, dOq, lse, delta, workspace=dirty)
         assert torch.equal(dq_only[0], ref[0])
+
+
+def test_random_shapes_and_modes():
+    """A seeded sweep over batch, head grouping, sequence length, mask, recipe and operand mode, every
+    case checked against the oracle: the net under the persistent / ticket-scheduled kernels, whose
+    item lists depend on all of these."""
+    import random
+    rnd = random.Random(20260937852)
+    done = 0
+    while done < 16:
+        base = rnd.choice(["tiny", "gqa4k", "gqa8k_outlier", "mla8k", "gqa8k_d256", "long64k"])
+        hkv = rnd.choice([1, 2, 3])
+        kw = dict(batch=rnd.choice([1, 1, 2, 3]), heads_kv=hkv, heads_q=hkv * rnd.choice([1, 2, 4, 5]),
+                  seqlen=128 * rnd.choice([1, 2, 3, 4, 5, 6]), causal=rnd.choice([True, True, False]))
+        w = workloads.WORKLOADS[base].scaled(**kw)
+        if w.batch * w.heads_q * w.seqlen * w.seqlen > 2 * 8 * 768 * 768:
+            continue                                                    # keep the oracle's share to seconds
+        narrow = (w.head_dim_qk, w.head_dim_v) in ((64, 64), (128, 128))
+        bf16 = narrow and rnd.random() < 0.25
+        tensors = workloads.make_inputs(w)
+        if bf16 and w.dtype != "bf16":
+            tensors = tuple(x.to(torch.bfloat16) for x in tensors)
+        try:
+            _check(w, tensors, _full_pass(w, tensors, bf16=bf16), prec="bf16" if bf16 else "mxfp8")
+        except AssertionError as e:
+            raise AssertionError(f"{base} {kw} bf16={bf16}") from e
+        done += 1
