@@ -132,3 +132,42 @@ def test_quantize_batch_single_tile_ring_and_errors():
     with pytest.raises(B.AttnFp8Error) as e:                               # status workspace too small
         B.attn_fp8_quantize_batch([xs[1]], workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 4
+
+
+def test_quantize_batch_random_job_mixes_bit_exact():
+    """Seeded mixes of one to eight tensors with head dims 32 ... 256 (those without a compile-time
+    instance included), both source dtypes, zero columns and random orientations: codes, scale
+    bytes and the zero padding of the scale tiles against the oracle, bit for bit."""
+    import random
+    from paper_2609_37852_b200 import binding as B
+    rnd = random.Random(3)
+    g = torch.Generator().manual_seed(11)
+    for trial in range(8):
+        dt = rnd.choice([torch.bfloat16, torch.float32])
+        xs = []
+        for j in range(rnd.choice([1, 2, 3, 5, 8])):
+            shape = (rnd.choice([1, 2]), rnd.choice([1, 3]), 128 * rnd.choice([1, 2, 3]), 32 * rnd.choice([1, 2, 3, 4, 5, 6, 7, 8]))
+            x = torch.randn(shape, generator=g) * (10.0 ** rnd.uniform(-3, 3))
+            if rnd.random() < 0.3:
+                x[..., ::7] = 0
+            xs.append(x.to(dt).cuda())
+        want = [(rnd.random() < 0.8, True) if rnd.random() < 0.5 else (True, rnd.random() < 0.8) for _ in xs]
+        outs, ws = B.attn_fp8_quantize_batch(xs, want=want)
+        B.attn_fp8_read_status(ws)
+        for x, q, (wr, wc) in zip(xs, outs, want):
+            Bn, H, N, d = x.shape
+            xn = to_np(x)
+            if wr:
+                rc, rs = mxfp8.quantize(xn, axis=-1)
+                assert np.array_equal(q.row_codes.cpu().numpy(), rc), (trial, x.shape)
+                assert np.array_equal(B.unpack_scales(q.row_scales, Bn, H, N, d).cpu().numpy(), rs), (trial, x.shape)
+                assert int(q.row_scales.to(torch.int64).sum()) == int(rs.astype(np.int64).sum())
+            else:
+                assert q.row_codes is None
+            if wc:
+                cc, cs = mxfp8.quantize(xn, axis=-2)
+                assert np.array_equal(q.col_codes.cpu().numpy(), np.swapaxes(cc, -1, -2)), (trial, x.shape)
+                assert np.array_equal(B.unpack_scales(q.col_scales, Bn, H, d, N).cpu().numpy(), np.swapaxes(cs, -1, -2)), (trial, x.shape)
+                assert int(q.col_scales.to(torch.int64).sum()) == int(cs.astype(np.int64).sum())
+            else:
+                assert q.col_codes is None
