@@ -3,10 +3,11 @@
 // tensor or for several in one launch (the four operands of a step: Q, K, V, dO).
 //
 // The tiles (128 tokens x d channels, contiguous in the source) of all tensors form one list.  A
-// persistent grid (two CTAs per SM at d = 128) walks it; each CTA keeps a ring of two source tiles
-// in shared memory (one where two do not fit), filled by bulk asynchronous copies (one instruction per tile, completion counted on an
-// mbarrier), so that the next tile is in flight while the current one is quantised: the short
-// tails and ramps of four separate launches disappear and every SM always has loads outstanding.
+// persistent grid (two CTAs per SM) walks it; each CTA keeps a ring of two source tiles in shared
+// memory (one where two would cost the second CTA), filled by bulk asynchronous copies (one
+// instruction per tile, completion counted on an mbarrier), so that the next tile is in flight
+// while the current one is quantised: the short tails and ramps of four separate launches
+// disappear and every SM always has loads outstanding.
 // Pass 1 walks the tile along channels (row copy), pass 2 along tokens (column copy, staged in
 // shared memory so that it leaves as full 128-byte rows).
 #include <cuda_bf16.h>
