@@ -418,6 +418,18 @@ def main():
                         + ("" if bf16_mode else f" x {FP8_OVER_BF16} (nominal fp8:bf16)")),
         "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (w.name == WORKLOAD and not bf16_mode) else None,
     }
+    # the same figure for every kernel of the step (the operand preparation against the HBM copy bandwidth)
+    rooflines = {}
+    for name, (nq, nv) in PRODUCTS.items():
+        a = pairs2 * (nq * w.head_dim_qk + nv * w.head_dim_v) / (stage_ms[name] * 1e-3) / 1e12
+        rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
+                           "traffic": NCU_TRAFFIC_BYTES.get(name) if (w.name == WORKLOAD and not bf16_mode) else None}
+    n_el = w.batch * w.seqlen * (w.heads_q * (w.head_dim_qk + w.head_dim_v) + w.heads_kv * (w.head_dim_qk + w.head_dim_v))
+    src_bytes = 2 if w.dtype == "bf16" else 4
+    prep_bytes = n_el * (src_bytes + (2 * 2 if bf16_mode else 2 + 2.0 / 32 * 2))      # read once, two copies (+ scales)
+    gbs = prep_bytes / (stage_ms["quantize"] * 1e-3) / 1e9
+    rooflines["quantize"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+                             "traffic": NCU_TRAFFIC_BYTES.get("quantize") if (w.name == WORKLOAD and not bf16_mode) else None}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -447,6 +459,7 @@ def main():
                 "ms_per_step": e2e_ms / e2e_steps if e2e_steps else None},
         "gpu_launches": kernels_per_step * args.steps,
         "roofline": roofline,
+        "rooflines": rooflines,
     }
 
     # ---- row-sum residual of dS (the metric's second half), from one untimed instrumented pass -------
