@@ -37,6 +37,8 @@ attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, i
                                  cudaStream_t stream);
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
                          float* lse, int* status, cudaStream_t stream);
+attn_status_t launch_fwd_interleaved(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
+                                     float* lse, int* status, cudaStream_t stream, int variant);
 attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream);
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,

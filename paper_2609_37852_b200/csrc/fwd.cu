@@ -26,6 +26,7 @@
 // dimension: 128 keys of codes or 64 keys of BF16.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <type_traits>
 
 #include "common.cuh"
@@ -508,6 +509,8 @@ attn_status_t launch_fwd_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t 
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
                          int* status, cudaStream_t stream) {
   const int cq = (s.dqk * s.eb + 127) / 128, rv = (s.dv + 127) / 128;
+  static const int variant = []() { const char* e = getenv("ATTN_FP8_FWD_VARIANT"); return e ? atoi(e) : 2; }();
+  if (s.eb == 1 && cq == 1 && rv == 1 && variant > 0) return launch_fwd_interleaved(s, q, k, v, o, lse, status, stream, variant);
   if (s.eb == 1) {
     if (cq == 1 && rv == 1) return launch_fwd_t<FwdCfg<1, 1, 1>>(s, q, k, v, o, lse, status, stream);
     if (cq == 2 && rv == 1) return launch_fwd_t<FwdCfg<1, 2, 1>>(s, q, k, v, o, lse, status, stream);

@@ -1,0 +1,609 @@
+// Forward attention with block-scaled FP8 operands for head dims up to 128 (paper Appendix
+// "Forward Probability Encoding", re-designed for tcgen05 / tensor memory): the variant in which a
+// softmax thread owns a whole query row of a key step, the key steps of a query tile are dealt
+// round-robin to the softmax warpgroups, and a separate warpgroup keeps the output accumulator's
+// power-of-two unit.
+//
+// One CTA per SM owns 128 query rows of one (batch, query head) and walks the key tiles up to the
+// causal diagonal.  Score tiles of kWG consecutive key steps live in tensor memory at once, one per
+// softmax warpgroup, so the tensor cores compute S of step u+1 while the exponentials of step u run:
+//   warp 0        TMA producer: Q tile once, then K tiles [128 keys x d] and V^T tiles [dv x 128 keys]
+//   warp 1        issues S_u = Q K_u^T into score buffer u % kWG
+//   warp 2        issues O += P^_u V_u (A operand = quantised probabilities read from tensor memory)
+//   warps 4..7    unit keepers: thread <-> query row (see below); they also write O and LSE at the end
+//   warpgroup w   (warps 8+4w .. 11+4w) softmax of the steps u = w, w + kWG, ...: thread <-> query row.
+// A softmax thread keeps a PRIVATE integer shift M and normaliser share l for the steps it sees: the
+// E4M3 codes of a block do not depend on the shift (the block scale absorbs any power of two), and l
+// sums the exponentials before the cast.  It never waits for another softmax thread: it writes the
+// codes to tensor memory, the scale bytes (relative to its M) and M itself to shared memory, and goes
+// on.  What the steps of a row must agree on is only the power of two the output accumulator is
+// expressed in, M_O.  The row's unit keeper holds it in a register and takes the steps in order: it
+// adds M - M_O to the step's scale bytes (exact), hands the step to the P V issuer, and on the rare
+// occasion that M exceeds M_O by more than kLazyUnit it first rescales the accumulator row in tensor
+// memory between two P V products.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "mma_issue.cuh"
+#include "mxfp8_device.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+
+#ifdef ATTN_TRACE
+__device__ long long g_il_trace[5][256][8];
+#define IL_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_il_trace[role][step][ev] = clock64(); } while (0)
+extern "C" int attn_fp8_debug_il_trace(long long* host_out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_il_trace, sizeof(g_il_trace)));
+}
+#else
+#define IL_TRACE(role, step, ev) do { } while (0)
+#endif
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;          // query rows per CTA; keys per K / V tile in shared memory
+constexpr int kStages = 4;          // K ring and V ring depth
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
+constexpr float kLn2Lo = -2.12194440054690583e-4f;
+constexpr int kLazyShift = 8;       // a thread raises its private shift when a step's maximum exceeds it by more
+constexpr int kLazyUnit = 24;       // the accumulator's unit is raised when a step's shift exceeds it by more
+#ifndef ATTN_IL_TURNS
+#define ATTN_IL_TURNS 0
+#endif
+constexpr bool kTurns = ATTN_IL_TURNS != 0;
+#ifndef ATTN_IL_LAG
+#define ATTN_IL_LAG 3
+#endif
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+#ifdef ATTN_IL_VOLATILE
+__device__ __forceinline__ float ex2_il(float x) {
+  float y;
+  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+#else
+#define ex2_il ex2_approx
+#endif
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
+template <int kWG_, int kSW_, int kSplit_>
+struct IlCfg {
+  static constexpr int kWG = kWG_;                      // softmax teams == score buffers in flight
+  static constexpr int kSW = kSW_;                      // keys per step (64 or 128)
+  static constexpr int kSplit = kSplit_;                // threads per query row and step (each takes kSW / kSplit keys)
+  static constexpr int kBlk = kSW / 32;                 // quantisation blocks per step
+  static constexpr int kBlkT = kBlk / kSplit;           // ... per thread
+  static constexpr int kColsT = kSW / kSplit;           // score columns per thread and step
+  static constexpr int kSubPerTile = kTile / kSW;       // steps per K / V tile
+  static constexpr int kSoftmaxThreads = 128 * kWG * kSplit;
+  static constexpr int kThreads = 256 + kSoftmaxThreads;
+  static constexpr int kPCols = kSW / 4;                // columns of one probability buffer
+  static constexpr uint32_t kColS = 0;                  // kWG score buffers
+  static constexpr uint32_t kColO = kWG * kSW;          // output accumulator, up to 128 columns
+  static constexpr uint32_t kColP = kColO + 128;        // kWG probability buffers
+  static constexpr uint32_t kColSFQ = kColP + kWG * kPCols;
+  static constexpr uint32_t kColSFK = kColSFQ + 4;      // 2 slots
+  static constexpr uint32_t kColSFV = kColSFK + 8;      // 2 slots
+  static constexpr uint32_t kColSFP = kColSFV + 8;      // kWG x 4
+  static constexpr uint32_t kColsUsed = kColSFP + 4 * kWG;
+  static_assert(kColsUsed <= 512, "tensor memory exceeded");
+  // registers (the CTA's pool is what it was launched with: 65536 / kThreads per thread, rounded
+  // down to a multiple of 8): the issuing warpgroup and the unit keepers give registers to the
+  // softmax warpgroups
+  static constexpr int kRegsIssue = 40;
+  static constexpr int kRegsKeeper = kSplit == 1 ? 64 : 56;
+  static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
+  static constexpr int kRegsSoftmax = ((kRegsLaunch * kThreads - 128 * (kRegsIssue + kRegsKeeper)) / kSoftmaxThreads) / 8 * 8;
+};
+
+template <class C>
+struct IlSmem {
+  alignas(1024) uint8_t q[kTile * 128];
+  alignas(1024) uint8_t k[kStages][kTile * 128];
+  alignas(1024) uint8_t v[kStages][kTile * 128];
+  alignas(16) uint8_t sf_q[512];
+  alignas(16) uint8_t sf_k[kStages][512];
+  alignas(16) uint8_t sf_v[kStages][512];
+  alignas(16) uint8_t sf_p[C::kWG][512];
+  alignas(16) uint32_t raw_sf[C::kWG][C::kSplit][kTile];    // scale bytes of a step relative to the softmax thread's shift
+  alignas(16) float step_m[C::kWG][C::kSplit][kTile];       // that shift
+  alignas(16) float fin_l[C::kWG * C::kSplit][kTile];       // normaliser shares at the end, and the shifts they are expressed in
+  alignas(16) float fin_m[C::kWG * C::kSplit][kTile];
+  uint64_t q_full;
+  uint64_t k_full[kStages], k_empty[kStages];
+  uint64_t v_full[kStages], v_empty[kStages];
+  uint64_t s_full[C::kWG], s_free[C::kWG];
+  uint64_t p_ready[C::kWG], p_full[C::kWG], p_free[C::kWG];
+  uint64_t o_done, fin;
+  uint64_t turn[C::kWG];
+  uint64_t drain[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct IlParams {
+  const uint8_t* q_sf;      // row scales of Q
+  const uint8_t* k_sf;      // row scales of K
+  const uint8_t* v_sf;      // col scales of V
+  __nv_bfloat16* o;
+  float* lse;
+  int* status;
+  int N, Hq, Hkv, dqk, dv, causal;
+  float scale_log2;         // softmax_scale * log2(e)
+};
+
+// 2^d for an integer-valued d <= 127 (0 below the normal range, -inf included)
+__device__ __forceinline__ float pow2_int(float d) {
+  const int e = d < -126.f ? 0 : 127 + static_cast<int>(d);
+  return __uint_as_float(static_cast<uint32_t>(e) << 23);
+}
+
+template <class C>
+__global__ void __launch_bounds__(C::kThreads, 1)
+fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+              const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  IlSmem<C>& sm = *reinterpret_cast<IlSmem<C>*>(smem_raw);
+  if (smem_u32(smem_raw) & 1023u) {               // never expected: report instead of computing garbage
+    if (threadIdx.x == 0) atomicExch(p.status, static_cast<int>(ATTN_ERR_ALIGNMENT));
+    return;
+  }
+  constexpr int kWG = C::kWG, kSW = C::kSW, kBlk = C::kBlk, kSubPerTile = C::kSubPerTile, kPCols = C::kPCols;
+  constexpr int kSplit = C::kSplit, kBlkT = C::kBlkT, kColsT = C::kColsT;
+  constexpr uint32_t kColS = C::kColS, kColO = C::kColO, kColP = C::kColP, kColSFQ = C::kColSFQ, kColSFK = C::kColSFK,
+                     kColSFV = C::kColSFV, kColSFP = C::kColSFP;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
+  // all heads go first, so the light tiles fill the tail of the launch
+  const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
+  const int h = blockIdx.x, b = blockIdx.z;
+  const int g = h / (p.Hq / p.Hkv);
+  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
+  const int n_steps = n_tiles * kSubPerTile;
+  const int nk_qk = p.dqk / 32;                 // 32-byte K steps of the score MMA
+  volatile int* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
+    }
+    for (int w = 0; w < kWG; ++w) {
+      mbar_init(&sm.s_full[w], 1); mbar_init(&sm.s_free[w], 4 * kSplit);          // one arrival per warp
+      mbar_init(&sm.p_ready[w], 4 * kSplit); mbar_init(&sm.p_full[w], 4); mbar_init(&sm.p_free[w], 1);
+      mbar_init(&sm.turn[w], 4 * kSplit);
+    }
+    mbar_init(&sm.o_done, 1);
+    mbar_init(&sm.fin, 4 * kWG * kSplit);
+    mbar_init(&sm.drain[0], 1); mbar_init(&sm.drain[1], 1);
+    sm.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&sm.tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp < 4) {
+    reg_dealloc<C::kRegsIssue>();
+    if (warp == 0) {
+      // ------------------------------------------------------------------ producer
+      if (lane == 0) {
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+        const int q_row = (b * p.Hq + h) * p.N + qt * kTile;
+        const int tiles_n = p.N / kTile;
+        mbar_arrive_expect_tx(&sm.q_full, kTile * 128 + 512);
+        tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_row);
+        bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(b * p.Hq + h) * tiles_n + qt) * 512, 512, &sm.q_full);
+        const int kv_slab = b * p.Hkv + g;
+        int issued_k = 0, issued_v = 0;
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int s = t % kStages, r = t / kStages;
+          ok = mbar_wait(&sm.k_empty[s], (r & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
+          tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
+          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.k_full[s]);
+          ++issued_k;
+          ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
+          tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
+          bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.v_full[s]);
+          ++issued_v;
+        }
+        if (!ok) {
+          // let the copies already in flight land before the CTA gives its shared memory back
+          int dummy = 0;
+          for (int t = max(0, issued_k - kStages); t < issued_k; ++t)
+            mbar_wait(&sm.k_full[t % kStages], (t / kStages) & 1, &dummy);
+          for (int t = max(0, issued_v - kStages); t < issued_v; ++t)
+            mbar_wait(&sm.v_full[t % kStages], (t / kStages) & 1, &dummy);
+        }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ S = Q K^T issuer
+      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
+      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        sf_copy_tiles<1>(tmem + kColSFQ, sm.sf_q);
+      }
+      for (int u = 0; u < n_steps && ok; ++u) {
+        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1, w = u % kWG;
+        if (sub == 0) {
+          ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          sf_copy_tiles<1>(tmem + kColSFK + 4 * slot, sm.sf_k[s]);
+        }
+        IL_TRACE(0, u, 0);
+        if (u >= kWG) {
+          // warpgroup w has pulled the scores of step u - kWG into registers
+          ok = mbar_wait(&sm.s_free[w], ((u / kWG) - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        IL_TRACE(0, u, 1);
+        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + sub * (kSW * 128 / 16);
+        issue_ss<true, 1, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
+                                                                    tmem + kColSFQ, tmem + kColSFK + 4 * slot + kBlk * sub);
+        mma_commit_elect(&sm.s_full[w]);
+        IL_TRACE(0, u, 2);
+        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit_elect(&sm.drain[0]);
+        mbar_wait(&sm.drain[0], 0, &dummy);
+      }
+    } else if (warp == 2) {
+      // ------------------------------------------------------------------ O += P V issuer
+      bool ok = true;
+      const uint32_t n_dv = static_cast<uint32_t>(p.dv);
+      for (int u = 0; u < n_steps && ok; ++u) {
+        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1, w = u % kWG;
+        if (sub == 0) {
+          ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          sf_copy_tiles<1>(tmem + kColSFV + 4 * slot, sm.sf_v[s]);
+        }
+        IL_TRACE(1, u, 0);
+        ok = mbar_wait(&sm.p_full[w], (u / kWG) & 1, abort_flag);
+        if (!ok) break;
+        IL_TRACE(1, u, 1);
+        tc_fence_after_sync();
+        sf_copy_elect(tmem + kColSFP + 4 * w, make_desc_sf(smem_u32(sm.sf_p[w])));
+        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
+#pragma unroll
+        for (int kb = 0; kb < kBlk; ++kb) {
+          const int kstep = sub * kBlk + kb;              // 32-key block inside the 128-key tile
+          mma_mxf8_ts_elect(tmem + kColO, tmem + kColP + kPCols * w + 8 * kb, desc_v + 2 * kstep,
+                            make_idesc_mxf8(128, n_dv, kb, kstep), tmem + kColSFP + 4 * w, tmem + kColSFV + 4 * slot,
+                            (u > 0 || kb > 0));
+        }
+        IL_TRACE(1, u, 2);
+        mma_commit_elect(&sm.p_free[w]);                  // operand and scale bytes of this buffer consumed; O updated
+        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
+        if (u == n_steps - 1) mma_commit_elect(&sm.o_done);
+      }
+      if (!ok) {
+        int dummy = 0;
+        mma_commit_elect(&sm.drain[1]);
+        mbar_wait(&sm.drain[1], 0, &dummy);
+      }
+    }
+  } else if (warp < 8) {
+    // -------------------------------------------------------------------- unit keepers
+    reg_dealloc<C::kRegsKeeper>();
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                   // row inside the tile == TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    float MO = -INFINITY;                               // the accumulator row is expressed in units of 2^MO
+    bool ok = true;
+    for (int u = 0; u < n_steps; ++u) {
+      const int w = u % kWG, use = u / kWG;
+      if (lane == 0 && quad == 0) IL_TRACE(4, u, 0);
+      ok = mbar_wait(&sm.p_ready[w], use & 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0 && quad == 0) IL_TRACE(4, u, 1);
+      float Mh[kSplit];                                 // -inf: the thread has seen nothing but masked keys
+      uint32_t raw[kSplit];
+#pragma unroll
+      for (int hf = 0; hf < kSplit; ++hf) {
+        Mh[hf] = lds_f32(&sm.step_m[w][hf][row]);
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[hf]) : "r"(smem_u32(&sm.raw_sf[w][hf][row])));
+      }
+      float M = Mh[0];
+#pragma unroll
+      for (int hf = 1; hf < kSplit; ++hf) M = fmaxf(M, Mh[hf]);
+      const bool raise = M > MO + static_cast<float>(kLazyUnit);       // always on step 0
+      if (__any_sync(0xffffffffu, raise)) {
+        if (u > 0) {
+          // rare: the previous P V product must have landed before the accumulator row is rescaled
+          ok = mbar_wait(&sm.p_free[(u - 1) % kWG], ((u - 1) / kWG) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const float factor = raise ? pow2_int(MO - M) : 1.f;
+          for (int c0 = 0; c0 < p.dv; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld16(tmem + kColO + lane_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 16; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
+            tmem_st16(tmem + kColO + lane_addr + c0, r);
+          }
+          tmem_wait_st();
+          tc_fence_before_sync();
+        }
+        if (raise) MO = M;
+      }
+      // scale bytes relative to the accumulator's unit; a block more than 2^-127 below it keeps byte 0
+      uint32_t packed = 0;
+#pragma unroll
+      for (int hf = 0; hf < kSplit; ++hf) {
+        const int shift = Mh[hf] == -INFINITY ? 0 : static_cast<int>(fmaxf(Mh[hf] - MO, -1024.f));
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) {
+          const int byte = static_cast<int>((raw[hf] >> (8 * bk)) & 0xFFu);
+          const int bnew = byte == 0 ? 0 : max(byte + shift, 0);
+          packed |= static_cast<uint32_t>(bnew) << (8 * (hf * kBlkT + bk));
+        }
+      }
+      uint8_t* sf_dst = &sm.sf_p[w][(row & 31) * 16 + (row >> 5) * 4];
+      if (kBlk == 4)
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(sf_dst)), "r"(packed) : "memory");
+      else
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_u32(sf_dst)), "h"(static_cast<uint16_t>(packed)) : "memory");
+      fence_proxy_async_smem();
+      mbar_arrive_warp(&sm.p_full[w]);
+      if (lane == 0 && quad == 0) IL_TRACE(4, u, 2);
+    }
+    // the row's normaliser = sum of the shares of its softmax threads, in the accumulator's unit
+    if (ok) ok = mbar_wait(&sm.fin, 0, abort_flag);
+    if (ok) ok = mbar_wait(&sm.o_done, 0, abort_flag);
+    if (ok) {
+      tc_fence_after_sync();
+      float lt = 0.f;
+#pragma unroll
+      for (int i = 0; i < kWG * kSplit; ++i) lt += lds_f32(&sm.fin_l[i][row]) * pow2_int(lds_f32(&sm.fin_m[i][row]) - MO);   // (0, -inf): no step seen
+      const float inv_l = 1.f / lt;
+      const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
+      __nv_bfloat16* o_row = p.o + grow * p.dv;
+      for (int c0 = 0; c0 < p.dv; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem + kColO + lane_addr + c0, r);
+        tmem_wait_ld();
+        uint32_t packed[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(r[2 * c]) * inv_l, __uint_as_float(r[2 * c + 1]) * inv_l);
+          packed[c] = *reinterpret_cast<uint32_t*>(&v2);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(o_row + c0);
+        dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+      }
+      // LSE = M_O ln2 + ln l with ln2 split so that M_O * ln2_hi is exact: one rounding at the end
+      p.lse[grow] = fmaf(MO, kLn2Hi, fmaf(MO, kLn2Lo, logf(lt)));
+    }
+  } else {
+    // -------------------------------------------------------------------- softmax
+    reg_alloc<C::kRegsSoftmax>();
+    const int w = (warp - 8) / (4 * kSplit);            // team: takes the steps u % kWG == w
+    const int hf = ((warp - 8) >> 2) % kSplit;          // which kColsT keys of a step
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;                   // row inside the tile == TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+    float M = -INFINITY;                                // private integer-valued shift (log2 units)
+    float l = 0.f;                                      // this thread's share of the normaliser, in units of 2^M
+    bool ok = true;
+    for (int u = w; u < n_steps; u += kWG) {
+      const int t = u / kSubPerTile, sub = u % kSubPerTile, use = u / kWG;
+#define SM_TRACE(ev) do { if (lane == 0 && quad == 0 && hf == 0) IL_TRACE(2 + w, u, ev); } while (0)
+      SM_TRACE(0);
+      ok = mbar_wait(&sm.s_full[w], use & 1, abort_flag);
+      if (!ok) break;
+      SM_TRACE(1);
+      tc_fence_after_sync();
+      float sv[kColsT];
+#pragma unroll
+      for (int bk = 0; bk < kBlkT; ++bk)
+        tmem_ld32(tmem + kColS + kSW * w + kColsT * hf + lane_addr + 32 * bk, reinterpret_cast<uint32_t*>(sv + 32 * bk));
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      mbar_arrive_warp(&sm.s_free[w]);                  // the scores are in registers: the next S of this buffer may be issued
+      SM_TRACE(2);
+      // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
+      float mxb[kBlkT];
+      if (p.causal && t == qt) {
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) {
+          const int col0 = sub * kSW + kColsT * hf + 32 * bk;
+          float m = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            if (col0 + c > row) sv[32 * bk + c] = -INFINITY;
+            m = fmaxf(m, sv[32 * bk + c]);
+          }
+          mxb[bk] = m;
+        }
+      } else {
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) {
+          // 16 three-input maxima as a tree of depth 4 (a chain of them is bound by their latency)
+          const float* x = sv + 32 * bk;
+          float a[10];
+#pragma unroll
+          for (int i = 0; i < 10; ++i) a[i] = max3(x[3 * i], x[3 * i + 1], x[3 * i + 2]);
+          const float b0 = max3(a[0], a[1], a[2]), b1 = max3(a[3], a[4], a[5]), b2 = max3(a[6], a[7], a[8]);
+          const float b3 = max3(a[9], x[30], x[31]);
+          mxb[bk] = fmaxf(max3(b0, b1, b2), b3);
+        }
+      }
+      float mx = mxb[0];
+#pragma unroll
+      for (int bk = 1; bk < kBlkT; ++bk) mx = fmaxf(mx, mxb[bk]);
+      // a fully masked step (second half of the diagonal tile for the first 64 rows) gives -inf: it
+      // never raises M and contributes zeros
+      const float mx2 = mx * p.scale_log2;
+      if (mx2 > M + static_cast<float>(kLazyShift)) {     // true on the thread's first unmasked step
+        const float m_new = ceilf(mx2);
+        l *= pow2_int(M - m_new);                         // exact power of two (0 at the start)
+        M = m_new;
+      }
+      SM_TRACE(3);
+      const float neg_m = M == -INFINITY ? 0.f : -M;      // nothing seen yet: every score is -inf, any finite shift gives zeros
+      uint32_t bytes[kBlkT];
+      // The scale 2^e of a block follows from its largest exponential, which is the exponential of
+      // the block's score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the value
+      // the E4M3 cast wants, and the block sum is put back on the thread's scale by one exact
+      // multiplication.
+      float2 nme2[kBlkT];
+#pragma unroll
+      for (int bk = 0; bk < kBlkT; ++bk) {
+        float inv;
+        block_scale_finite(ex2_approx(fmaf(mxb[bk], p.scale_log2, neg_m)), bytes[bk], inv);
+        const float neg_me = neg_m - static_cast<float>(static_cast<int>(bytes[bk]) - 127);
+        nme2[bk] = make_float2(neg_me, neg_me);
+      }
+      uint32_t packed_sf = 0;
+#pragma unroll
+      for (int bk = 0; bk < kBlkT; ++bk) packed_sf |= bytes[bk] << (8 * bk);
+      // The exponentials keep the XU pipe of the SM sub-partition busy by themselves, the rest of a
+      // step does not use it: a warpgroup starts the exponentials of step u once those of step u - 1
+      // are half done, so that the two never fall into step with each other.
+      if (kTurns && u > 0) {
+        ok = mbar_wait(&sm.turn[w], (w == 0 ? use - 1 : use) & 1, abort_flag);
+        if (!ok) break;
+      }
+      // Groups of four keys, the exponentials of group i written kLag groups ahead of the sums and
+      // casts that consume them.  The codes of a block go to tensor memory as soon as it is complete.
+      {
+        constexpr int kGroups = kColsT / 4, kLag = ATTN_IL_LAG;
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+        float2 e01[kGroups], e23[kGroups];
+        float2 bs01[kBlkT], bs23[kBlkT];
+        uint32_t words[kBlkT][8];
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) bs01[bk] = bs23[bk] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < kGroups + kLag; ++i) {
+          if (ATTN_IL_TURNS == 2 && i == kGroups / 2 && u + 1 < n_steps) mbar_arrive_warp(&sm.turn[(u + 1) % kWG]);
+          if (i < kGroups) {
+#ifdef ATTN_IL_NOMATH
+            e01[i] = make_float2(sv[4 * i], sv[4 * i + 1]); e23[i] = make_float2(sv[4 * i + 2], sv[4 * i + 3]);
+#else
+            const float2 a = __ffma2_rn(make_float2(sv[4 * i], sv[4 * i + 1]), sc2, nme2[i / 8]);
+            const float2 c = __ffma2_rn(make_float2(sv[4 * i + 2], sv[4 * i + 3]), sc2, nme2[i / 8]);
+            e01[i] = make_float2(ex2_il(a.x), ex2_il(a.y));
+            e23[i] = make_float2(ex2_il(c.x), ex2_il(c.y));
+#endif
+          }
+          if (i >= kLag) {
+            const int j = i - kLag;
+            bs01[j / 8] = __fadd2_rn(bs01[j / 8], e01[j]);
+            bs23[j / 8] = __fadd2_rn(bs23[j / 8], e23[j]);
+            words[j / 8][j % 8] = cvt_e4m3x4(e01[j].x, e01[j].y, e23[j].x, e23[j].y);
+            if (j == 7) {
+              // The first block is done.  Before anything of this step is stored: the P V MMAs of step
+              // u - kWG have consumed this team's operand buffer (and the unit keepers its scale bytes
+              // and shift before that); that product was issued when the team's previous step ended,
+              // so the wait is over by now as a rule.
+              SM_TRACE(6);
+              if (u >= kWG) {
+                ok = mbar_wait(&sm.p_free[w], (use - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+              }
+              SM_TRACE(7);
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&sm.raw_sf[w][hf][row])), "r"(packed_sf) : "memory");
+              sts_f32(&sm.step_m[w][hf][row], M);
+            }
+            if (j % 8 == 7) tmem_st8(tmem + kColP + kPCols * w + lane_addr + 8 * (hf * kBlkT + j / 8), words[j / 8]);
+          }
+        }
+        if (!ok) break;
+        if (ATTN_IL_TURNS == 1 && u + 1 < n_steps) mbar_arrive_warp(&sm.turn[(u + 1) % kWG]);
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) {
+          const float bs0 = bs01[bk].x + bs01[bk].y, bs1 = bs23[bk].x + bs23[bk].y;
+          l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
+        }
+      }
+      SM_TRACE(4);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive_warp(&sm.p_ready[w]);                 // codes in tensor memory, scale bytes and shift in shared memory
+      SM_TRACE(5);
+    }
+    sts_f32(&sm.fin_l[w * kSplit + hf][row], l);
+    sts_f32(&sm.fin_m[w * kSplit + hf][row], M);
+    mbar_arrive_warp(&sm.fin);
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 512);
+  if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+
+template <class C>
+attn_status_t launch_fwd_il_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o, float* lse,
+                              int* status, cudaStream_t stream) {
+  CUtensorMap tm_q, tm_k, tm_v;
+  attn_status_t st;
+  st = encode_tmap_u8_sw128(&tm_q, q.row_codes, static_cast<uint64_t>(s.dqk), static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
+  if (st != ATTN_OK) return st;
+  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk), static_cast<uint64_t>(s.B) * s.Hkv * s.N, kTile);
+  if (st != ATTN_OK) return st;
+  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.N), static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
+  if (st != ATTN_OK) return st;
+  IlParams p;
+  p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
+  p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
+  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.scale_log2 = s.scale * kLog2e;
+  const size_t smem = sizeof(IlSmem<C>) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(fwd_il_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  dim3 grid(s.Hq, s.N / kTile, s.B);
+  fwd_il_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));
+  return ATTN_OK;
+}
+
+}  // namespace
+
+// FP8 operands, head dims (64,64) and (128,128).  `variant` selects the instantiation.
+attn_status_t launch_fwd_interleaved(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
+                                     float* lse, int* status, cudaStream_t stream, int variant) {
+  if (variant == 2) return launch_fwd_il_t<IlCfg<2, 128, 2>>(s, q, k, v, o, lse, status, stream);
+  return launch_fwd_il_t<IlCfg<2, 128, 1>>(s, q, k, v, o, lse, status, stream);
+}
+
+}  // namespace attnfp8
