@@ -9,9 +9,10 @@ pass and the quantiser earn no credit).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-Prints ONE JSON line (rank 0).  With N > 1 (launched under torchrun) every rank
-runs an independent replica of the workload on its own GPU -- the path has no
-exchange step -- and the value is the aggregate over ranks.
+Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent replica
+of the workload on its own GPU -- the path has no exchange step -- and the value
+is the aggregate over ranks.  ``--gpus N`` without a launcher around it (no
+WORLD_SIZE in the environment) starts the N ranks itself.
 ``--impl reference`` times the CPU oracle on a bounded causal prefix of the
 same workload instead (host cores; rank 0 only).
 """
@@ -35,7 +36,8 @@ FP8_OVER_BF16 = 2.0                 # nominal dense FP8 : BF16 tensor ratio on B
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on WORKLOAD, from
 # the ncu captures summarised under profiles/; None where no capture has been taken.
-NCU_TRAFFIC_BYTES = {"quantize": 288.9e6, "fwd": 70.4e6, "bwd_delta": 90.5e6, "bwd_dq": 126.2e6, "bwd_dkdv": 317.9e6}
+NCU_TRAFFIC_BYTES = {"quantize": 288.9e6, "fwd": 72.5e6, "bwd_delta": 90.5e6, "bwd_dq": 126.2e6, "bwd_dkdv": 317.9e6}
+MACS_PER_CLK_PER_SM_FP8 = 8192      # dense FP8 tensor rate of one SM (the nominal 4.5 PFLOP/s is this at ~1.86 GHz on 148 SMs)
 
 # executed matmul products per kernel as (contractions or outputs of width dqk, of width dv): each is
 # 2*width FLOPs per unmasked (i, j) pair and query head
@@ -218,7 +220,14 @@ def main():
                     help="bf16: the same kernels with BF16 operands and no block scales (reference point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the extra back-to-back loop that shows the settled (power-capped) rate; 0 skips it")
     args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher around this process: start the N ranks (one per GPU) and let rank 0 print the line
+        from paper_2609_37852_b200 import replicas
+        raise SystemExit(replicas.launch_local(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
 
     from paper_2609_37852_b200 import workloads
     w = workloads.WORKLOADS[args.workload]
@@ -334,6 +343,26 @@ def main():
     stage_ms = {n: statistics.mean(ev[j].elapsed_time(ev[j + 1]) for ev in events)
                 for j, n in enumerate(("quantize", "fwd", "bwd_delta", "bwd", "bwd_dq", "bwd_dkdv"))}
 
+    # ---- the same step back to back for a couple of seconds: the rate the part settles to ------------
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / (total_ms / args.steps)))
+        sus_sampler = ClockSampler(local_rank)
+        barrier()
+        sus_sampler.start()
+        s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for i in range(n_sus):
+            step()
+        s1.record(stream)
+        barrier()
+        sus_clocks = sus_sampler.stop()
+        B.attn_fp8_read_status(ws)
+        sustained = {"steps": n_sus, "ms_per_step": s0.elapsed_time(s1) / n_sus, "clocks": sus_clocks}
+
+    # ---- the bare block-scaled FP8 MMA rate of this device (a few ms; see attn_fp8_measure_mma_peak) ----
+    measured_fp8 = None if bf16_mode else B.attn_fp8_measure_mma_peak(ws)
+
     # ---- end to end through the library with host buffers --------------------------------------
     # Host buffers in, host buffers out, every step: copies run on their own streams and overlap the
     # kernels of the neighbouring steps (three slots of device inputs / outputs), as a user pipeline would.
@@ -393,11 +422,13 @@ def main():
     # ---- max over ranks -----------------------------------------------------------------------
     from paper_2609_37852_b200 import replicas
     total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], device=dev)
+    if sustained is not None:
+        sustained["ms_per_step"] = replicas.max_over_ranks([sustained["ms_per_step"]], device=dev)[0]
 
     fwd_flops, bwd_flops = w.credited_flops()
     credited = fwd_flops + bwd_flops
-    value = world * credited * args.steps / (total_ms * 1e-3) / 1e12
-    e2e_value = world * credited * e2e_steps / (e2e_ms * 1e-3) / 1e12 if e2e_steps else None
+    value = replicas.aggregate_rate(credited * args.steps, world, total_ms * 1e-3) / 1e12
+    e2e_value = replicas.aggregate_rate(credited * e2e_steps, world, e2e_ms * 1e-3) / 1e12 if e2e_steps else None
 
     step_ms = total_ms / args.steps
     # ---- roofline of the dominant kernel ------------------------------------------------------
@@ -410,23 +441,34 @@ def main():
     kernel_flops = pairs2 * (n_qk * w.head_dim_qk + n_v * w.head_dim_v)
     achieved = kernel_flops / (stage_ms[dominant] * 1e-3) / 1e12
     ratio = 1.0 if bf16_mode else FP8_OVER_BF16
-    peak = peaks["bf16_sustained"] * ratio
-    roofline = {
-        "kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-        "frac": achieved / peak,
-        "peak_source": (f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s"
-                        + ("" if bf16_mode else f" x {FP8_OVER_BF16} (nominal fp8:bf16)")),
-        "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (w.name == WORKLOAD and not bf16_mode) else None,
-    }
+    # The kernels' durations come from the per-stage loop: the denominator is the measured cuBLAS BF16
+    # figure that goes with the clock that loop ran at -- the burst one when the sampled SM clock stayed
+    # within 5 % of the maximum, the sustained one (taken under the power cap) otherwise.
+    sc = stage_clocks
+    at_boost = bool(sc.get("sm_mhz") and sc.get("sm_max_mhz") and sc["sm_mhz"] >= 0.95 * sc["sm_max_mhz"])
+    which = "burst" if at_boost else "sustained"
+    peak = peaks["bf16_" + which] * ratio
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    clock_peak = (2.0 * MACS_PER_CLK_PER_SM_FP8 / ratio * sms * sc["sm_mhz"] * 1e6 / 1e12) if sc.get("sm_mhz") else None
+
+    def tensor_roofline(a, name):
+        return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
+                "frac_of_nominal_peak": a / (NOMINAL_FP8_TFLOPS / ratio),
+                "frac_of_clock_normalised_peak": a / clock_peak if clock_peak else None,
+                "frac_of_measured_fp8_mma_rate": a / measured_fp8 if measured_fp8 else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(name) if (w.name == WORKLOAD and not bf16_mode) else None}
+    roofline = dict(kernel=dominant, **tensor_roofline(achieved, dominant))
+    roofline["peak_source"] = (f"{peaks['source']} {which} bf16 {peaks['bf16_' + which]} TFLOP/s"
+                               + ("" if bf16_mode else f" x {FP8_OVER_BF16} (nominal fp8:bf16)")
+                               + f"; stage loop ran at a median {sc.get('sm_mhz')} MHz of {sc.get('sm_max_mhz')} MHz")
     # the same figure for every kernel of the step (the operand preparation against the HBM copy bandwidth)
     rooflines = {}
     for name, (nq, nv) in PRODUCTS.items():
         a = pairs2 * (nq * w.head_dim_qk + nv * w.head_dim_v) / (stage_ms[name] * 1e-3) / 1e12
-        rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
-                           "traffic": NCU_TRAFFIC_BYTES.get(name) if (w.name == WORKLOAD and not bf16_mode) else None}
+        rooflines[name] = tensor_roofline(a, name)
     n_el = w.batch * w.seqlen * (w.heads_q * (w.head_dim_qk + w.head_dim_v) + w.heads_kv * (w.head_dim_qk + w.head_dim_v))
     src_bytes = 2 if w.dtype == "bf16" else 4
-    prep_bytes = n_el * (src_bytes + (2 * 2 if bf16_mode else 2 + 2.0 / 32 * 2))      # read once, two copies (+ scales)
+    prep_bytes = n_el * (src_bytes + (2 * 2 if bf16_mode else 2 + 2.0 / 32))          # read once, two copies (+ their scale bytes)
     gbs = prep_bytes / (stage_ms["quantize"] * 1e-3) / 1e9
     rooflines["quantize"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
                              "traffic": NCU_TRAFFIC_BYTES.get("quantize") if (w.name == WORKLOAD and not bf16_mode) else None}
@@ -442,12 +484,18 @@ def main():
                    "step": ("transposed BF16 copies of Q,K,V,dO" if bf16_mode else "quantize(Q,K,V,dO)")
                            + " + fwd + matched delta + dQ + dK/dV"},
         "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
+        "target": "north_star asks for >= 50 % of the nominal dense FP8 peak on this workload: not met",
+        "measured_fp8_mma_tflops": measured_fp8,
+        "pct_of_measured_fp8_mma_rate": (100.0 * value / world / measured_fp8) if measured_fp8 else None,
+        "sustained": (None if sustained is None else dict(
+            sustained, value=replicas.aggregate_rate(credited, world, sustained["ms_per_step"] * 1e-3) / 1e12, unit=UNIT,
+            note="the same step looped back to back for about --sustained-seconds: the rate under the power cap")),
         "pct_of_nominal_peak_of_dtype": 100.0 * value / world / (NOMINAL_FP8_TFLOPS / (FP8_OVER_BF16 if bf16_mode else 1.0)),
         "stage_ms": stage_ms,
-        "stage_timing": "a second loop of the same steps with an event at every stage boundary (the timed region has "
-                        "none: an event costs a few microseconds); bwd = the overlapped gradient call, bwd_dq and "
-                        "bwd_dkdv = its two kernels as separate, serialised calls; this loop runs later and longer "
-                        "than the timed region, at the clocks sustained load settles to (stage_clocks)",
+        "stage_timing": "a second loop of the same steps, after the timed region, with an event at every stage boundary "
+                        "(the timed region has none: an event costs a few microseconds); bwd = the overlapped gradient "
+                        "call, bwd_dq and bwd_dkdv = its two kernels as separate, serialised calls; the rooflines use "
+                        "these durations and the clocks sampled during this loop (stage_clocks)",
         "stage_clocks": stage_clocks,
         # the timed step less the operand preparation (the paper's accounting), and less the forward
         "attn_only_tflops": credited / ((step_ms - stage_ms["quantize"]) * 1e-3) / 1e12,

@@ -151,8 +151,8 @@ typedef struct {
  *   workspace  device, >= ATTN_STATUS_WORKSPACE_BYTES, 16-byte aligned: its status word reports a
  *              copy that never completed (attn_fp8_read_status -> ATTN_ERR_TIMEOUT), as for the
  *              attention entry points; a workspace of those calls may be passed
- * attn_fp8_quantize is this call with one job (its status word lands in the library's built-in
- * scratch, which attn_fp8_read_status does not reach).                                           */
+ * attn_fp8_quantize is this call with one job; its status word lands in the library's built-in
+ * scratch of the current device, which attn_fp8_read_status(NULL, stream) reads.                 */
 attn_status_t attn_fp8_quantize_batch(const attn_quantize_job_t* jobs, int32_t n_jobs, void* workspace,
                                       size_t workspace_bytes, void* stream);
 
@@ -227,7 +227,9 @@ attn_status_t attn_fp8_bwd(const attn_params_t* p, attn_qtensor_t q, attn_qtenso
  *                      reads q.row_*, k.row_*, k.col_*, v.row_*, dO.row_*, lse, delta
  *   attn_fp8_bwd_dkdv  the key-major pass: dK and dV;
  *                      reads q.row_*, q.col_*, k.row_*, v.row_*, dO.row_*, dO.col_*, lse, delta
- * attn_fp8_bwd is exactly the first followed by the second on the same stream.               */
+ * attn_fp8_bwd produces exactly their outputs with one call: it launches the key-major kernel first
+ * and the query-major kernel behind it (the two are independent; the second starts on the SMs the
+ * first one's last wave leaves idle), and both have completed when the stream reaches what follows. */
 attn_status_t attn_fp8_bwd_dq(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                               attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
                               float* diag_rowsum_ds, float* diag_rowsum_abs_ds,
@@ -264,12 +266,14 @@ attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q,
  *   - Problems whose scratch need (attn_fp8_workspace_bytes(p, ATTN_WS_FWD)) exceeds 4096 bytes are
  *     rejected with ATTN_ERR_WORKSPACE and a message naming both sizes.
  *   - The first call on each device looks up the array's device address (a one-time runtime query
- *     made with that device current); make that first call outside of any stream capture.
+ *     made with that device current); make that first call outside of any stream capture.  The
+ *     address is cached per device ordinal for the life of the process: it does not survive a
+ *     cudaDeviceReset of that device (do not reset a device between calls of this library).
  *   - All calls on a device share the one array, and it keeps what earlier calls left; its
  *     status word is only ever set by a kernel that gave up, so nothing has to be cleared between
  *     calls and overlapping calls (different streams) do not disturb one another.
- *   - The device status word lands in the built-in array and is not reported by
- *     attn_fp8_read_status; callers that want the time-out report use attn_fp8_fwd.
+ *   - The device status word lands in the built-in array: attn_fp8_read_status(NULL, stream) reads
+ *     (and, if set, clears) it.
  * Arguments, layouts and error codes are otherwise those of attn_fp8_fwd.                       */
 attn_status_t attn_fp8_fwd_noalloc(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                    void* o_bf16, float* lse, void* stream);
@@ -293,15 +297,27 @@ attn_status_t attn_fp8_workspace_init(void* workspace, size_t workspace_bytes, v
 /* Waits for `stream`, copies the status word of `workspace` to the host and returns it:
  * ATTN_OK, or ATTN_ERR_TIMEOUT / ATTN_ERR_ALIGNMENT if a kernel of any call since the last read (or
  * the initialisation) gave up (outputs of those calls are then undefined).  A non-OK status is
- * cleared by the read.  This is the one call that synchronises.                               */
+ * cleared by the read.  workspace == NULL means the library's built-in scratch array on the current
+ * device, where the entry points without a workspace argument (attn_fp8_quantize,
+ * attn_fp8_fwd_noalloc) report.  This is the one call that synchronises.                        */
 attn_status_t attn_fp8_read_status(void* workspace, void* stream);
 
 /* Self-test of the device-side time-out report: enqueues a one-CTA kernel that waits, with a limit
  * of about 2 ms, on a barrier nothing completes, gives up and sets the status word of `workspace`
  * (>= attn_fp8_workspace_bytes) exactly as an attention kernel whose wait expired would.  A later
  * attn_fp8_read_status(workspace) therefore returns ATTN_ERR_TIMEOUT; the context stays usable.
+ * workspace == NULL (workspace_bytes ignored) targets the built-in scratch array of the current device.
  * For tests of the error path: nothing faults, traps or hangs.                                 */
 attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Measurement aid (the paper has no counterpart): the rate, in TFLOP/s, at which this device executes
+ * the bare block-scaled FP8 tensor-core instruction the attention kernels are built on (E4M3 operands,
+ * E8M0 scales, 128 x 128 x 32 per instruction, three issuing warps per SM, operands resident in shared
+ * memory), written to *tflops (host).  Runs a few milliseconds of such instructions on `stream` three
+ * times (the first warms the clocks up; the faster of the other two counts) and WAITS for them: unlike
+ * the other entry points this one synchronises the stream.  `workspace` as for the attention calls
+ * (status word).  Allocates no device memory.                                                       */
+attn_status_t attn_fp8_measure_mma_peak(double* tflops, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Message for the last non-OK return on this host thread (static storage; never NULL).        */
 const char* attn_fp8_last_error(void);

@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_workspace_init", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
+    "attn_fp8_measure_mma_peak",
 )
 
 
@@ -335,14 +336,27 @@ _lib.attn_fp8_selftest_timeout.restype = _i32
 _lib.attn_fp8_selftest_timeout.argtypes = [_vp, _sz, _vp]
 
 
-def attn_fp8_selftest_timeout(workspace: torch.Tensor, stream=None) -> None:
-    """Enqueues the bounded-wait self-test: the next attn_fp8_read_status(workspace) raises ATTN_ERR_TIMEOUT."""
-    _check(_lib.attn_fp8_selftest_timeout(_ptr(workspace), workspace.numel(), _stream(stream)))
+def attn_fp8_selftest_timeout(workspace: Optional[torch.Tensor], stream=None) -> None:
+    """Enqueues the bounded-wait self-test: the next attn_fp8_read_status(workspace) raises ATTN_ERR_TIMEOUT.
+    ``workspace=None`` targets the library's built-in scratch array on the current device."""
+    _check(_lib.attn_fp8_selftest_timeout(_ptr(workspace), 0 if workspace is None else workspace.numel(), _stream(stream)))
 
 
-def attn_fp8_read_status(workspace: torch.Tensor, stream=None) -> None:
-    """Synchronises ``stream`` and raises if a kernel of the last call reported a timeout."""
+def attn_fp8_read_status(workspace: Optional[torch.Tensor], stream=None) -> None:
+    """Synchronises ``stream`` and raises if a kernel of the last call reported a timeout.
+    ``workspace=None`` reads the built-in scratch array (attn_fp8_quantize, attn_fp8_fwd_noalloc)."""
     _check(_lib.attn_fp8_read_status(_ptr(workspace), _stream(stream)))
+
+
+_lib.attn_fp8_measure_mma_peak.restype = _i32
+_lib.attn_fp8_measure_mma_peak.argtypes = [ctypes.POINTER(ctypes.c_double), _vp, _sz, _vp]
+
+
+def attn_fp8_measure_mma_peak(workspace: torch.Tensor, stream=None) -> float:
+    """TFLOP/s of the bare block-scaled FP8 tensor-core instruction on this device (synchronises)."""
+    out = ctypes.c_double(0.0)
+    _check(_lib.attn_fp8_measure_mma_peak(ctypes.byref(out), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return out.value
 
 
 def attn_fp8_fwd(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, o=None, lse=None, workspace=None,

@@ -81,6 +81,15 @@ static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entr
   if (p->precision != ATTN_PREC_MXFP8 && p->precision != ATTN_PREC_BF16 && p->precision != ATTN_PREC_MXFP8_PROTECTED_DP)
     return fail(ATTN_ERR_INVALID_ARG, "precision %d unknown", p->precision);
   if (p->seqlen % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen must be a multiple of 128");
+  // the kernels form row coordinates of the [B * H * N] and [B * Hkv * d] operand views in 32-bit integers
+  {
+    const long long q_rows = static_cast<long long>(p->batch) * p->heads_q * p->seqlen;
+    const int wide = p->head_dim_qk > p->head_dim_v ? p->head_dim_qk : p->head_dim_v;
+    const long long kv_rows = static_cast<long long>(p->batch) * p->heads_kv * (p->seqlen > wide ? p->seqlen : wide);
+    if (q_rows > 0x7fffffffLL || kv_rows > 0x7fffffffLL)
+      return fail(ATTN_ERR_UNSUPPORTED, "batch * heads * seqlen = %lld exceeds the 2^31 - 1 rows a launch indexes",
+                  q_rows > kv_rows ? q_rows : kv_rows);
+  }
   const int eb = p->precision == ATTN_PREC_BF16 ? 2 : 1;
   if (!dims_supported(entry, eb, p->head_dim_qk, p->head_dim_v))
     return fail(ATTN_ERR_UNSUPPORTED, "head dims (%d, %d) are not built for this entry point in %s mode",
@@ -370,7 +379,10 @@ attn_status_t attn_fp8_workspace_init(void* workspace, size_t workspace_bytes, v
 }
 
 attn_status_t attn_fp8_read_status(void* workspace, void* stream) {
-  if (!workspace) return fail(ATTN_ERR_INVALID_ARG, "workspace is NULL");
+  if (!workspace) {                                  // the built-in scratch array of the current device
+    CHECK(check_device());
+    CHECK(builtin_scratch_for_current_device(&workspace));
+  }
   int host = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -471,6 +483,10 @@ __global__ void wait_selftest_kernel(int* status, long long limit_cycles) {
 
 extern "C" attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes, void* stream) {
   CHECK(check_device());
+  if (!workspace) {                                  // the built-in scratch array of the current device
+    CHECK(builtin_scratch_for_current_device(&workspace));
+    workspace_bytes = kBuiltinScratchBytes;
+  }
   int* status = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
@@ -478,4 +494,13 @@ extern "C" attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t works
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "selftest: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
+}
+
+extern "C" attn_status_t attn_fp8_measure_mma_peak(double* tflops, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!tflops) return fail(ATTN_ERR_INVALID_ARG, "tflops is NULL");
+  CHECK(check_device());
+  int* status = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
+  return measure_mma_peak(tflops, status, st);
 }

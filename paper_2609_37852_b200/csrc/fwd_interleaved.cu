@@ -51,13 +51,6 @@ constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kL
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
 constexpr int kLazyShift = 8;       // a thread raises its private shift when a step's maximum exceeds it by more
 constexpr int kLazyUnit = 24;       // the accumulator's unit is raised when a step's shift exceeds it by more
-#ifndef ATTN_IL_TURNS
-#define ATTN_IL_TURNS 0
-#endif
-constexpr bool kTurns = ATTN_IL_TURNS != 0;
-#ifndef ATTN_IL_LAG
-#define ATTN_IL_LAG 3
-#endif
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
@@ -98,7 +91,7 @@ struct IlCfg {
   static constexpr uint32_t kColO = kWG * kSW;          // output accumulator, up to 128 columns
   static constexpr uint32_t kColP = kColO + 128;        // kWG probability buffers
   static constexpr uint32_t kColSFQ = kColP + kWG * kPCols;
-  static constexpr uint32_t kColSFK = kColSFQ + 4;      // 2 slots
+  static constexpr uint32_t kColSFK = kColSFQ + 8;      // 2 slots (Q: 2 slots)
   static constexpr uint32_t kColSFV = kColSFK + 8;      // 2 slots
   static constexpr uint32_t kColSFP = kColSFV + 8;      // kWG x 4
   static constexpr uint32_t kColsUsed = kColSFP + 4 * kWG;
@@ -114,24 +107,23 @@ struct IlCfg {
 
 template <class C>
 struct IlSmem {
-  alignas(1024) uint8_t q[kTile * 128];
+  alignas(1024) uint8_t q[2][kTile * 128];
   alignas(1024) uint8_t k[kStages][kTile * 128];
   alignas(1024) uint8_t v[kStages][kTile * 128];
-  alignas(16) uint8_t sf_q[512];
+  alignas(16) uint8_t sf_q[2][512];
   alignas(16) uint8_t sf_k[kStages][512];
   alignas(16) uint8_t sf_v[kStages][512];
   alignas(16) uint8_t sf_p[C::kWG][512];
   alignas(16) uint32_t raw_sf[C::kWG][C::kSplit][kTile];    // scale bytes of a step relative to the softmax thread's shift
   alignas(16) float step_m[C::kWG][C::kSplit][kTile];       // that shift
-  alignas(16) float fin_l[C::kWG * C::kSplit][kTile];       // normaliser shares at the end, and the shifts they are expressed in
-  alignas(16) float fin_m[C::kWG * C::kSplit][kTile];
-  uint64_t q_full;
+  alignas(16) float fin_l[4][C::kWG * C::kSplit][kTile];    // normaliser shares at the end of an item (four slots, by item
+  alignas(16) float fin_m[4][C::kWG * C::kSplit][kTile];    // number), and the shifts they are expressed in
+  uint64_t q_full[2], q_empty[2];
   uint64_t k_full[kStages], k_empty[kStages];
   uint64_t v_full[kStages], v_empty[kStages];
   uint64_t s_full[C::kWG], s_free[C::kWG];
   uint64_t p_ready[C::kWG], p_full[C::kWG], p_free[C::kWG];
-  uint64_t o_done, fin;
-  uint64_t turn[C::kWG];
+  uint64_t o_done, o_free;
   uint64_t drain[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -145,6 +137,7 @@ struct IlParams {
   float* lse;
   int* status;
   int N, Hq, Hkv, dqk, dv, causal;
+  int gx, gy, gz;           // the (head, query tile, batch) grid the work items are numbered in
   float scale_log2;         // softmax_scale * log2(e)
 };
 
@@ -169,18 +162,32 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
   constexpr uint32_t kColS = C::kColS, kColO = C::kColO, kColP = C::kColP, kColSFQ = C::kColSFQ, kColSFK = C::kColSFK,
                      kColSFV = C::kColSFV, kColSFP = C::kColSFP;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // blocks are handed out x-fastest: heads vary fastest and the heaviest (latest) query tiles of
-  // all heads go first, so the light tiles fill the tail of the launch
-  const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
-  const int h = blockIdx.x, b = blockIdx.z;
-  const int g = h / (p.Hq / p.Hkv);
-  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
-  const int n_steps = n_tiles * kSubPerTile;
+  // Work items (128 query rows of one head) are numbered x-fastest over (head, query tile, batch):
+  // heads vary fastest and the heaviest (latest) query tiles of all heads come first.  CTA c of n
+  // takes the items c, 2n-1-c, 2n+c, ...: alternate rounds run backwards, so that no CTA collects the
+  // heavier item of every round.  The K / V rings, the score and probability buffers and their
+  // barriers run on across items; Q is double-buffered; the output accumulator is handed from the
+  // unit keepers (who store the finished item) back to the P V issuer once per item.
+  const int n_cta = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
+  const int total_items = p.gx * p.gy * p.gz;
+  struct Item { int qt, h, b, g, n_tiles, n_steps; bool valid; };
+  auto item_at = [&](int i) {
+    Item it;
+    const int l = i * n_cta + ((i & 1) ? n_cta - 1 - cta : cta);
+    it.valid = l < total_items;
+    const int x = l % p.gx, y = (l / p.gx) % p.gy, z = l / (p.gx * p.gy);
+    it.qt = p.causal ? (p.gy - 1 - y) : y;
+    it.h = x; it.b = z;
+    it.g = it.h / (p.Hq / p.Hkv);
+    it.n_tiles = p.causal ? it.qt + 1 : p.N / kTile;
+    it.n_steps = it.n_tiles * kSubPerTile;
+    return it;
+  };
   const int nk_qk = p.dqk / 32;                 // 32-byte K steps of the score MMA
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
-    mbar_init(&sm.q_full, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.q_full[i], 1); mbar_init(&sm.q_empty[i], 1); }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
@@ -188,10 +195,9 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
     for (int w = 0; w < kWG; ++w) {
       mbar_init(&sm.s_full[w], 1); mbar_init(&sm.s_free[w], 4 * kSplit);          // one arrival per warp
       mbar_init(&sm.p_ready[w], 4 * kSplit); mbar_init(&sm.p_full[w], 4); mbar_init(&sm.p_free[w], 1);
-      mbar_init(&sm.turn[w], 4 * kSplit);
     }
     mbar_init(&sm.o_done, 1);
-    mbar_init(&sm.fin, 4 * kWG * kSplit);
+    mbar_init(&sm.o_free, 4);
     mbar_init(&sm.drain[0], 1); mbar_init(&sm.drain[1], 1);
     sm.abort_flag = 0;
     fence_mbar_init();
@@ -211,28 +217,39 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // ------------------------------------------------------------------ producer
       if (lane == 0) {
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-        const int q_row = (b * p.Hq + h) * p.N + qt * kTile;
         const int tiles_n = p.N / kTile;
-        mbar_arrive_expect_tx(&sm.q_full, kTile * 128 + 512);
-        tma_load_2d(sm.q, &tm_q, &sm.q_full, 0, q_row);
-        bulk_load_1d(sm.sf_q, p.q_sf + (static_cast<size_t>(b * p.Hq + h) * tiles_n + qt) * 512, 512, &sm.q_full);
-        const int kv_slab = b * p.Hkv + g;
         int issued_k = 0, issued_v = 0;
+        int T = 0;                                    // key tiles of the items before this one
         bool ok = true;
-        for (int t = 0; t < n_tiles && ok; ++t) {
-          const int s = t % kStages, r = t / kStages;
-          ok = mbar_wait(&sm.k_empty[s], (r & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
-          tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
-          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.k_full[s]);
-          ++issued_k;
-          ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
-          tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
-          bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.v_full[s]);
-          ++issued_v;
+        for (int i = 0; ok; ++i) {
+          const Item it = item_at(i);
+          if (!it.valid) break;
+          const int qb = i & 1;
+          if (i >= 2) {
+            // the S issuer has finished with the item that used this Q buffer
+            ok = mbar_wait(&sm.q_empty[qb], ((i >> 1) - 1) & 1, abort_flag);
+            if (!ok) break;
+          }
+          const int q_slab = it.b * p.Hq + it.h, kv_slab = it.b * p.Hkv + it.g;
+          mbar_arrive_expect_tx(&sm.q_full[qb], kTile * 128 + 512);
+          tma_load_2d(sm.q[qb], &tm_q, &sm.q_full[qb], 0, q_slab * p.N + it.qt * kTile);
+          bulk_load_1d(sm.sf_q[qb], p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + it.qt) * 512, 512, &sm.q_full[qb]);
+          for (int t = 0; t < it.n_tiles && ok; ++t) {
+            const int gt = T + t, s = gt % kStages, r = gt / kStages;
+            ok = mbar_wait(&sm.k_empty[s], (r & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
+            tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.k_full[s]);
+            ++issued_k;
+            ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
+            tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
+            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.v_full[s]);
+            ++issued_v;
+          }
+          T += it.n_tiles;
         }
         if (!ok) {
           // let the copies already in flight land before the CTA gives its shared memory back
@@ -245,35 +262,46 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       }
     } else if (warp == 1) {
       // ------------------------------------------------------------------ S = Q K^T issuer
-      const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q));
-      bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-      if (ok) {
+      bool ok = true;
+      int T = 0, G = 0;                               // key tiles and key steps of the items before this one
+      for (int i = 0; ok; ++i) {
+        const Item it = item_at(i);
+        if (!it.valid) break;
+        const int qb = i & 1;
+        const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[qb]));
+        ok = mbar_wait(&sm.q_full[qb], (i >> 1) & 1, abort_flag);
+        if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_tiles<1>(tmem + kColSFQ, sm.sf_q);
-      }
-      for (int u = 0; u < n_steps && ok; ++u) {
-        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1, w = u % kWG;
-        if (sub == 0) {
-          ok = mbar_wait(&sm.k_full[s], (t / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          sf_copy_tiles<1>(tmem + kColSFK + 4 * slot, sm.sf_k[s]);
+        sf_copy_tiles<1>(tmem + kColSFQ + 4 * qb, sm.sf_q[qb]);
+        for (int u = 0; u < it.n_steps && ok; ++u) {
+          const int gu = G + u, gt = T + u / kSubPerTile;
+          const int sub = u % kSubPerTile, s = gt % kStages, slot = gt & 1, w = gu % kWG;
+          if (sub == 0) {
+            ok = mbar_wait(&sm.k_full[s], (gt / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            sf_copy_tiles<1>(tmem + kColSFK + 4 * slot, sm.sf_k[s]);
+          }
+          IL_TRACE(0, gu, 0);
+          if (gu >= kWG) {
+            // team w has pulled the scores of its previous step into registers
+            ok = mbar_wait(&sm.s_free[w], ((gu / kWG) - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+          IL_TRACE(0, gu, 1);
+          const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + sub * (kSW * 128 / 16);
+          issue_ss<true, 1, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
+                                                                      tmem + kColSFQ + 4 * qb,
+                                                                      tmem + kColSFK + 4 * slot + kBlk * sub);
+          mma_commit_elect(&sm.s_full[w]);
+          IL_TRACE(0, gu, 2);
+          if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
         }
-        IL_TRACE(0, u, 0);
-        if (u >= kWG) {
-          // warpgroup w has pulled the scores of step u - kWG into registers
-          ok = mbar_wait(&sm.s_free[w], ((u / kWG) - 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-        }
-        IL_TRACE(0, u, 1);
-        const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + sub * (kSW * 128 / 16);
-        issue_ss<true, 1, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
-                                                                    tmem + kColSFQ, tmem + kColSFK + 4 * slot + kBlk * sub);
-        mma_commit_elect(&sm.s_full[w]);
-        IL_TRACE(0, u, 2);
-        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
+        if (ok) mma_commit_elect(&sm.q_empty[qb]);       // this item's Q tile has been read
+        T += it.n_tiles; G += it.n_steps;
       }
+      if (*abort_flag) ok = false;
       if (!ok) {
         int dummy = 0;
         mma_commit_elect(&sm.drain[0]);
@@ -283,33 +311,46 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // ------------------------------------------------------------------ O += P V issuer
       bool ok = true;
       const uint32_t n_dv = static_cast<uint32_t>(p.dv);
-      for (int u = 0; u < n_steps && ok; ++u) {
-        const int t = u / kSubPerTile, sub = u % kSubPerTile, s = t % kStages, slot = t & 1, w = u % kWG;
-        if (sub == 0) {
-          ok = mbar_wait(&sm.v_full[s], (t / kStages) & 1, abort_flag);
+      int T = 0, G = 0;
+      for (int i = 0; ok; ++i) {
+        const Item it = item_at(i);
+        if (!it.valid) break;
+        for (int u = 0; u < it.n_steps && ok; ++u) {
+          const int gu = G + u, gt = T + u / kSubPerTile;
+          const int sub = u % kSubPerTile, s = gt % kStages, slot = gt & 1, w = gu % kWG;
+          if (sub == 0) {
+            ok = mbar_wait(&sm.v_full[s], (gt / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            sf_copy_tiles<1>(tmem + kColSFV + 4 * slot, sm.sf_v[s]);
+          }
+          IL_TRACE(1, gu, 0);
+          ok = mbar_wait(&sm.p_full[w], (gu / kWG) & 1, abort_flag);
           if (!ok) break;
+          if (u == 0 && i > 0) {
+            // the unit keepers have read the previous item out of the accumulator
+            ok = mbar_wait(&sm.o_free, (i - 1) & 1, abort_flag);
+            if (!ok) break;
+          }
+          IL_TRACE(1, gu, 1);
           tc_fence_after_sync();
-          sf_copy_tiles<1>(tmem + kColSFV + 4 * slot, sm.sf_v[s]);
-        }
-        IL_TRACE(1, u, 0);
-        ok = mbar_wait(&sm.p_full[w], (u / kWG) & 1, abort_flag);
-        if (!ok) break;
-        IL_TRACE(1, u, 1);
-        tc_fence_after_sync();
-        sf_copy_elect(tmem + kColSFP + 4 * w, make_desc_sf(smem_u32(sm.sf_p[w])));
-        const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
+          sf_copy_elect(tmem + kColSFP + 4 * w, make_desc_sf(smem_u32(sm.sf_p[w])));
+          const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
 #pragma unroll
-        for (int kb = 0; kb < kBlk; ++kb) {
-          const int kstep = sub * kBlk + kb;              // 32-key block inside the 128-key tile
-          mma_mxf8_ts_elect(tmem + kColO, tmem + kColP + kPCols * w + 8 * kb, desc_v + 2 * kstep,
-                            make_idesc_mxf8(128, n_dv, kb, kstep), tmem + kColSFP + 4 * w, tmem + kColSFV + 4 * slot,
-                            (u > 0 || kb > 0));
+          for (int kb = 0; kb < kBlk; ++kb) {
+            const int kstep = sub * kBlk + kb;              // 32-key block inside the 128-key tile
+            mma_mxf8_ts_elect(tmem + kColO, tmem + kColP + kPCols * w + 8 * kb, desc_v + 2 * kstep,
+                              make_idesc_mxf8(128, n_dv, kb, kstep), tmem + kColSFP + 4 * w, tmem + kColSFV + 4 * slot,
+                              (u > 0 || kb > 0));
+          }
+          IL_TRACE(1, gu, 2);
+          mma_commit_elect(&sm.p_free[w]);                  // operand and scale bytes of this buffer consumed; O updated
+          if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
+          if (u == it.n_steps - 1) mma_commit_elect(&sm.o_done);
         }
-        IL_TRACE(1, u, 2);
-        mma_commit_elect(&sm.p_free[w]);                  // operand and scale bytes of this buffer consumed; O updated
-        if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
-        if (u == n_steps - 1) mma_commit_elect(&sm.o_done);
+        T += it.n_tiles; G += it.n_steps;
       }
+      if (*abort_flag) ok = false;
       if (!ok) {
         int dummy = 0;
         mma_commit_elect(&sm.drain[1]);
@@ -322,76 +363,85 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                   // row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-    float MO = -INFINITY;                               // the accumulator row is expressed in units of 2^MO
     bool ok = true;
-    for (int u = 0; u < n_steps; ++u) {
-      const int w = u % kWG, use = u / kWG;
-      if (lane == 0 && quad == 0) IL_TRACE(4, u, 0);
-      ok = mbar_wait(&sm.p_ready[w], use & 1, abort_flag);
-      if (!ok) break;
-      if (lane == 0 && quad == 0) IL_TRACE(4, u, 1);
-      float Mh[kSplit];                                 // -inf: the thread has seen nothing but masked keys
-      uint32_t raw[kSplit];
+    int G = 0;
+    for (int i = 0; ok; ++i) {
+      const Item it = item_at(i);
+      if (!it.valid) break;
+      float MO = -INFINITY;                             // the accumulator row is expressed in units of 2^MO
+      for (int u = 0; u < it.n_steps; ++u) {
+        const int gu = G + u, w = gu % kWG, use = gu / kWG;
+        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 0);
+        ok = mbar_wait(&sm.p_ready[w], use & 1, abort_flag);
+        if (!ok) break;
+        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 1);
+        float Mh[kSplit];                               // -inf: the thread has seen nothing but masked keys
+        uint32_t raw[kSplit];
 #pragma unroll
-      for (int hf = 0; hf < kSplit; ++hf) {
-        Mh[hf] = lds_f32(&sm.step_m[w][hf][row]);
-        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[hf]) : "r"(smem_u32(&sm.raw_sf[w][hf][row])));
-      }
-      float M = Mh[0];
+        for (int hf = 0; hf < kSplit; ++hf) {
+          Mh[hf] = lds_f32(&sm.step_m[w][hf][row]);
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[hf]) : "r"(smem_u32(&sm.raw_sf[w][hf][row])));
+        }
+        float M = Mh[0];
 #pragma unroll
-      for (int hf = 1; hf < kSplit; ++hf) M = fmaxf(M, Mh[hf]);
-      const bool raise = M > MO + static_cast<float>(kLazyUnit);       // always on step 0
-      if (__any_sync(0xffffffffu, raise)) {
-        if (u > 0) {
-          // rare: the previous P V product must have landed before the accumulator row is rescaled
-          ok = mbar_wait(&sm.p_free[(u - 1) % kWG], ((u - 1) / kWG) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const float factor = raise ? pow2_int(MO - M) : 1.f;
-          for (int c0 = 0; c0 < p.dv; c0 += 16) {
-            uint32_t r[16];
-            tmem_ld16(tmem + kColO + lane_addr + c0, r);
-            tmem_wait_ld();
+        for (int hf = 1; hf < kSplit; ++hf) M = fmaxf(M, Mh[hf]);
+        const bool raise = M > MO + static_cast<float>(kLazyUnit);       // always on the item's first step
+        if (__any_sync(0xffffffffu, raise)) {
+          if (u > 0) {
+            // rare: the previous P V product must have landed before the accumulator row is rescaled
+            ok = mbar_wait(&sm.p_free[(gu - 1) % kWG], ((gu - 1) / kWG) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const float factor = raise ? pow2_int(MO - M) : 1.f;
+            for (int c0 = 0; c0 < p.dv; c0 += 16) {
+              uint32_t r[16];
+              tmem_ld16(tmem + kColO + lane_addr + c0, r);
+              tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 16; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
-            tmem_st16(tmem + kColO + lane_addr + c0, r);
+              for (int c = 0; c < 16; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * factor);
+              tmem_st16(tmem + kColO + lane_addr + c0, r);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
           }
-          tmem_wait_st();
-          tc_fence_before_sync();
+          if (raise) MO = M;
         }
-        if (raise) MO = M;
-      }
-      // scale bytes relative to the accumulator's unit; a block more than 2^-127 below it keeps byte 0
-      uint32_t packed = 0;
+        // scale bytes relative to the accumulator's unit; a block more than 2^-127 below it keeps byte 0
+        uint32_t packed = 0;
 #pragma unroll
-      for (int hf = 0; hf < kSplit; ++hf) {
-        const int shift = Mh[hf] == -INFINITY ? 0 : static_cast<int>(fmaxf(Mh[hf] - MO, -1024.f));
+        for (int hf = 0; hf < kSplit; ++hf) {
+          const int shift = Mh[hf] == -INFINITY ? 0 : static_cast<int>(fmaxf(Mh[hf] - MO, -1024.f));
 #pragma unroll
-        for (int bk = 0; bk < kBlkT; ++bk) {
-          const int byte = static_cast<int>((raw[hf] >> (8 * bk)) & 0xFFu);
-          const int bnew = byte == 0 ? 0 : max(byte + shift, 0);
-          packed |= static_cast<uint32_t>(bnew) << (8 * (hf * kBlkT + bk));
+          for (int bk = 0; bk < kBlkT; ++bk) {
+            const int byte = static_cast<int>((raw[hf] >> (8 * bk)) & 0xFFu);
+            const int bnew = byte == 0 ? 0 : max(byte + shift, 0);
+            packed |= static_cast<uint32_t>(bnew) << (8 * (hf * kBlkT + bk));
+          }
         }
+        uint8_t* sf_dst = &sm.sf_p[w][(row & 31) * 16 + (row >> 5) * 4];
+        if (kBlk == 4)
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(sf_dst)), "r"(packed) : "memory");
+        else
+          asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_u32(sf_dst)), "h"(static_cast<uint16_t>(packed)) : "memory");
+        fence_proxy_async_smem();
+        mbar_arrive_warp(&sm.p_full[w]);
+        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 2);
       }
-      uint8_t* sf_dst = &sm.sf_p[w][(row & 31) * 16 + (row >> 5) * 4];
-      if (kBlk == 4)
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(sf_dst)), "r"(packed) : "memory");
-      else
-        asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_u32(sf_dst)), "h"(static_cast<uint16_t>(packed)) : "memory");
-      fence_proxy_async_smem();
-      mbar_arrive_warp(&sm.p_full[w]);
-      if (lane == 0 && quad == 0) IL_TRACE(4, u, 2);
-    }
-    // the row's normaliser = sum of the shares of its softmax threads, in the accumulator's unit
-    if (ok) ok = mbar_wait(&sm.fin, 0, abort_flag);
-    if (ok) ok = mbar_wait(&sm.o_done, 0, abort_flag);
-    if (ok) {
+      // The row's normaliser = sum of the shares of its softmax threads, in the accumulator's unit.  A
+      // team wrote its shares ahead of the arrival that announced its last step of the item (a team
+      // without a step in a one-step item wrote nothing).
+      if (ok) ok = mbar_wait(&sm.o_done, i & 1, abort_flag);
+      if (!ok) break;
       tc_fence_after_sync();
       float lt = 0.f;
 #pragma unroll
-      for (int i = 0; i < kWG * kSplit; ++i) lt += lds_f32(&sm.fin_l[i][row]) * pow2_int(lds_f32(&sm.fin_m[i][row]) - MO);   // (0, -inf): no step seen
+      for (int j = 0; j < kWG * kSplit; ++j) {
+        const int first_u = (j / kSplit + kWG - G % kWG) % kWG;     // the team's first step of this item
+        if (first_u < it.n_steps)
+          lt += lds_f32(&sm.fin_l[i & 3][j][row]) * pow2_int(lds_f32(&sm.fin_m[i & 3][j][row]) - MO);   // M = -inf goes with l = 0
+      }
       const float inv_l = 1.f / lt;
-      const size_t grow = static_cast<size_t>(b * p.Hq + h) * p.N + qt * kTile + row;
+      const size_t grow = static_cast<size_t>(it.b * p.Hq + it.h) * p.N + it.qt * kTile + row;
       __nv_bfloat16* o_row = p.o + grow * p.dv;
       for (int c0 = 0; c0 < p.dv; c0 += 16) {
         uint32_t r[16];
@@ -407,162 +457,164 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
         dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
       }
+      // the accumulator may be overwritten by the next item's first P V product
+      tc_fence_before_sync();
+      mbar_arrive_warp(&sm.o_free);
       // LSE = M_O ln2 + ln l with ln2 split so that M_O * ln2_hi is exact: one rounding at the end
       p.lse[grow] = fmaf(MO, kLn2Hi, fmaf(MO, kLn2Lo, logf(lt)));
+      G += it.n_steps;
     }
   } else {
     // -------------------------------------------------------------------- softmax
     reg_alloc<C::kRegsSoftmax>();
-    const int w = (warp - 8) / (4 * kSplit);            // team: takes the steps u % kWG == w
+    const int w = (warp - 8) / (4 * kSplit);            // team: takes the steps whose running number is w modulo kWG
     const int hf = ((warp - 8) >> 2) % kSplit;          // which kColsT keys of a step
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                   // row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-    float M = -INFINITY;                                // private integer-valued shift (log2 units)
-    float l = 0.f;                                      // this thread's share of the normaliser, in units of 2^M
     bool ok = true;
-    for (int u = w; u < n_steps; u += kWG) {
-      const int t = u / kSubPerTile, sub = u % kSubPerTile, use = u / kWG;
-#define SM_TRACE(ev) do { if (lane == 0 && quad == 0 && hf == 0) IL_TRACE(2 + w, u, ev); } while (0)
-      SM_TRACE(0);
-      ok = mbar_wait(&sm.s_full[w], use & 1, abort_flag);
-      if (!ok) break;
-      SM_TRACE(1);
-      tc_fence_after_sync();
-      float sv[kColsT];
-#pragma unroll
-      for (int bk = 0; bk < kBlkT; ++bk)
-        tmem_ld32(tmem + kColS + kSW * w + kColsT * hf + lane_addr + 32 * bk, reinterpret_cast<uint32_t*>(sv + 32 * bk));
-      tmem_wait_ld();
-      tc_fence_before_sync();
-      mbar_arrive_warp(&sm.s_free[w]);                  // the scores are in registers: the next S of this buffer may be issued
-      SM_TRACE(2);
-      // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
-      float mxb[kBlkT];
-      if (p.causal && t == qt) {
-#pragma unroll
-        for (int bk = 0; bk < kBlkT; ++bk) {
-          const int col0 = sub * kSW + kColsT * hf + 32 * bk;
-          float m = -INFINITY;
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            if (col0 + c > row) sv[32 * bk + c] = -INFINITY;
-            m = fmaxf(m, sv[32 * bk + c]);
-          }
-          mxb[bk] = m;
-        }
-      } else {
-#pragma unroll
-        for (int bk = 0; bk < kBlkT; ++bk) {
-          // 16 three-input maxima as a tree of depth 4 (a chain of them is bound by their latency)
-          const float* x = sv + 32 * bk;
-          float a[10];
-#pragma unroll
-          for (int i = 0; i < 10; ++i) a[i] = max3(x[3 * i], x[3 * i + 1], x[3 * i + 2]);
-          const float b0 = max3(a[0], a[1], a[2]), b1 = max3(a[3], a[4], a[5]), b2 = max3(a[6], a[7], a[8]);
-          const float b3 = max3(a[9], x[30], x[31]);
-          mxb[bk] = fmaxf(max3(b0, b1, b2), b3);
-        }
-      }
-      float mx = mxb[0];
-#pragma unroll
-      for (int bk = 1; bk < kBlkT; ++bk) mx = fmaxf(mx, mxb[bk]);
-      // a fully masked step (second half of the diagonal tile for the first 64 rows) gives -inf: it
-      // never raises M and contributes zeros
-      const float mx2 = mx * p.scale_log2;
-      if (mx2 > M + static_cast<float>(kLazyShift)) {     // true on the thread's first unmasked step
-        const float m_new = ceilf(mx2);
-        l *= pow2_int(M - m_new);                         // exact power of two (0 at the start)
-        M = m_new;
-      }
-      SM_TRACE(3);
-      const float neg_m = M == -INFINITY ? 0.f : -M;      // nothing seen yet: every score is -inf, any finite shift gives zeros
-      uint32_t bytes[kBlkT];
-      // The scale 2^e of a block follows from its largest exponential, which is the exponential of
-      // the block's score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the value
-      // the E4M3 cast wants, and the block sum is put back on the thread's scale by one exact
-      // multiplication.
-      float2 nme2[kBlkT];
-#pragma unroll
-      for (int bk = 0; bk < kBlkT; ++bk) {
-        float inv;
-        block_scale_finite(ex2_approx(fmaf(mxb[bk], p.scale_log2, neg_m)), bytes[bk], inv);
-        const float neg_me = neg_m - static_cast<float>(static_cast<int>(bytes[bk]) - 127);
-        nme2[bk] = make_float2(neg_me, neg_me);
-      }
-      uint32_t packed_sf = 0;
-#pragma unroll
-      for (int bk = 0; bk < kBlkT; ++bk) packed_sf |= bytes[bk] << (8 * bk);
-      // The exponentials keep the XU pipe of the SM sub-partition busy by themselves, the rest of a
-      // step does not use it: a warpgroup starts the exponentials of step u once those of step u - 1
-      // are half done, so that the two never fall into step with each other.
-      if (kTurns && u > 0) {
-        ok = mbar_wait(&sm.turn[w], (w == 0 ? use - 1 : use) & 1, abort_flag);
+    int G = 0;
+    for (int i = 0; ok; ++i) {
+      const Item it = item_at(i);
+      if (!it.valid) break;
+      const int qt = it.qt;
+      float M = -INFINITY;                              // private integer-valued shift (log2 units)
+      float l = 0.f;                                    // this thread's share of the normaliser, in units of 2^M
+      for (int u = (w + kWG - G % kWG) % kWG; u < it.n_steps; u += kWG) {
+        const int gu = G + u, t = u / kSubPerTile, sub = u % kSubPerTile, use = gu / kWG;
+#define SM_TRACE(ev) do { if (lane == 0 && quad == 0 && hf == 0) IL_TRACE(2 + w, gu, ev); } while (0)
+        SM_TRACE(0);
+        ok = mbar_wait(&sm.s_full[w], use & 1, abort_flag);
         if (!ok) break;
-      }
-      // Groups of four keys, the exponentials of group i written kLag groups ahead of the sums and
-      // casts that consume them.  The codes of a block go to tensor memory as soon as it is complete.
-      {
-        constexpr int kGroups = kColsT / 4, kLag = ATTN_IL_LAG;
-        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-        float2 e01[kGroups], e23[kGroups];
-        float2 bs01[kBlkT], bs23[kBlkT];
-        uint32_t words[kBlkT][8];
+        SM_TRACE(1);
+        tc_fence_after_sync();
+        float sv[kColsT];
 #pragma unroll
-        for (int bk = 0; bk < kBlkT; ++bk) bs01[bk] = bs23[bk] = make_float2(0.f, 0.f);
+        for (int bk = 0; bk < kBlkT; ++bk)
+          tmem_ld32(tmem + kColS + kSW * w + kColsT * hf + lane_addr + 32 * bk, reinterpret_cast<uint32_t*>(sv + 32 * bk));
+        tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive_warp(&sm.s_free[w]);                // the scores are in registers: the next S of this buffer may be issued
+        SM_TRACE(2);
+        // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
+        float mxb[kBlkT];
+        if (p.causal && t == qt) {
 #pragma unroll
-        for (int i = 0; i < kGroups + kLag; ++i) {
-          if (ATTN_IL_TURNS == 2 && i == kGroups / 2 && u + 1 < n_steps) mbar_arrive_warp(&sm.turn[(u + 1) % kWG]);
-          if (i < kGroups) {
-#ifdef ATTN_IL_NOMATH
-            e01[i] = make_float2(sv[4 * i], sv[4 * i + 1]); e23[i] = make_float2(sv[4 * i + 2], sv[4 * i + 3]);
-#else
-            const float2 a = __ffma2_rn(make_float2(sv[4 * i], sv[4 * i + 1]), sc2, nme2[i / 8]);
-            const float2 c = __ffma2_rn(make_float2(sv[4 * i + 2], sv[4 * i + 3]), sc2, nme2[i / 8]);
-            e01[i] = make_float2(ex2_il(a.x), ex2_il(a.y));
-            e23[i] = make_float2(ex2_il(c.x), ex2_il(c.y));
-#endif
-          }
-          if (i >= kLag) {
-            const int j = i - kLag;
-            bs01[j / 8] = __fadd2_rn(bs01[j / 8], e01[j]);
-            bs23[j / 8] = __fadd2_rn(bs23[j / 8], e23[j]);
-            words[j / 8][j % 8] = cvt_e4m3x4(e01[j].x, e01[j].y, e23[j].x, e23[j].y);
-            if (j == 7) {
-              // The first block is done.  Before anything of this step is stored: the P V MMAs of step
-              // u - kWG have consumed this team's operand buffer (and the unit keepers its scale bytes
-              // and shift before that); that product was issued when the team's previous step ended,
-              // so the wait is over by now as a rule.
-              SM_TRACE(6);
-              if (u >= kWG) {
-                ok = mbar_wait(&sm.p_free[w], (use - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
-              }
-              SM_TRACE(7);
-              asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&sm.raw_sf[w][hf][row])), "r"(packed_sf) : "memory");
-              sts_f32(&sm.step_m[w][hf][row], M);
+          for (int bk = 0; bk < kBlkT; ++bk) {
+            const int col0 = sub * kSW + kColsT * hf + 32 * bk;
+            float m = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              if (col0 + c > row) sv[32 * bk + c] = -INFINITY;
+              m = fmaxf(m, sv[32 * bk + c]);
             }
-            if (j % 8 == 7) tmem_st8(tmem + kColP + kPCols * w + lane_addr + 8 * (hf * kBlkT + j / 8), words[j / 8]);
+            mxb[bk] = m;
+          }
+        } else {
+#pragma unroll
+          for (int bk = 0; bk < kBlkT; ++bk) {
+            // 16 three-input maxima as a tree of depth 4
+            const float* x = sv + 32 * bk;
+            float a[10];
+#pragma unroll
+            for (int j = 0; j < 10; ++j) a[j] = max3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
+            const float b0 = max3(a[0], a[1], a[2]), b1 = max3(a[3], a[4], a[5]), b2 = max3(a[6], a[7], a[8]);
+            const float b3 = max3(a[9], x[30], x[31]);
+            mxb[bk] = fmaxf(max3(b0, b1, b2), b3);
           }
         }
-        if (!ok) break;
-        if (ATTN_IL_TURNS == 1 && u + 1 < n_steps) mbar_arrive_warp(&sm.turn[(u + 1) % kWG]);
+        float mx = mxb[0];
+#pragma unroll
+        for (int bk = 1; bk < kBlkT; ++bk) mx = fmaxf(mx, mxb[bk]);
+        // a fully masked step (second half of the diagonal tile for the first 64 rows) gives -inf: it
+        // never raises M and contributes zeros
+        const float mx2 = mx * p.scale_log2;
+        if (mx2 > M + static_cast<float>(kLazyShift)) {   // true on the thread's first unmasked step of the item
+          const float m_new = ceilf(mx2);
+          l *= pow2_int(M - m_new);                       // exact power of two (0 at the start)
+          M = m_new;
+        }
+        SM_TRACE(3);
+        const float neg_m = M == -INFINITY ? 0.f : -M;    // nothing seen yet: every score is -inf, any finite shift gives zeros
+        uint32_t bytes[kBlkT];
+        // The scale 2^e of a block follows from its largest exponential, which is the exponential of
+        // the block's score maximum; folding e into the shift makes ex2 deliver p * 2^-e, the value
+        // the E4M3 cast wants, and the block sum is put back on the thread's scale by one exact
+        // multiplication.
+        float2 nme2[kBlkT];
 #pragma unroll
         for (int bk = 0; bk < kBlkT; ++bk) {
-          const float bs0 = bs01[bk].x + bs01[bk].y, bs1 = bs23[bk].x + bs23[bk].y;
-          l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
+          float inv;
+          block_scale_finite(ex2_approx(fmaf(mxb[bk], p.scale_log2, neg_m)), bytes[bk], inv);
+          const float neg_me = neg_m - static_cast<float>(static_cast<int>(bytes[bk]) - 127);
+          nme2[bk] = make_float2(neg_me, neg_me);
         }
+        uint32_t packed_sf = 0;
+#pragma unroll
+        for (int bk = 0; bk < kBlkT; ++bk) packed_sf |= bytes[bk] << (8 * bk);
+        // Groups of four keys, the exponentials of group i written kLag groups ahead of the sums and
+        // casts that consume them.  The codes of a block go to tensor memory as soon as it is complete.
+        {
+          constexpr int kGroups = kColsT / 4, kLag = 3;
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+          float2 e01[kGroups], e23[kGroups];
+          float2 bs01[kBlkT], bs23[kBlkT];
+          uint32_t words[kBlkT][8];
+#pragma unroll
+          for (int bk = 0; bk < kBlkT; ++bk) bs01[bk] = bs23[bk] = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int j0 = 0; j0 < kGroups + kLag; ++j0) {
+            if (j0 < kGroups) {
+              const float2 a = __ffma2_rn(make_float2(sv[4 * j0], sv[4 * j0 + 1]), sc2, nme2[j0 / 8]);
+              const float2 c = __ffma2_rn(make_float2(sv[4 * j0 + 2], sv[4 * j0 + 3]), sc2, nme2[j0 / 8]);
+              e01[j0] = make_float2(ex2_il(a.x), ex2_il(a.y));
+              e23[j0] = make_float2(ex2_il(c.x), ex2_il(c.y));
+            }
+            if (j0 >= kLag) {
+              const int j = j0 - kLag;
+              bs01[j / 8] = __fadd2_rn(bs01[j / 8], e01[j]);
+              bs23[j / 8] = __fadd2_rn(bs23[j / 8], e23[j]);
+              words[j / 8][j % 8] = cvt_e4m3x4(e01[j].x, e01[j].y, e23[j].x, e23[j].y);
+              if (j == 7) {
+                // The first block is done.  Before anything of this step is stored: the P V MMAs of
+                // the team's previous step have consumed its operand buffer (and the unit keepers its
+                // scale bytes and shift before that); that product was issued when the previous step
+                // ended, so the wait is over by now as a rule.
+                SM_TRACE(6);
+                if (gu >= kWG) {
+                  ok = mbar_wait(&sm.p_free[w], (use - 1) & 1, abort_flag);
+                  if (!ok) break;
+                  tc_fence_after_sync();
+                }
+                SM_TRACE(7);
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&sm.raw_sf[w][hf][row])), "r"(packed_sf) : "memory");
+                sts_f32(&sm.step_m[w][hf][row], M);
+              }
+              if (j % 8 == 7) tmem_st8(tmem + kColP + kPCols * w + lane_addr + 8 * (hf * kBlkT + j / 8), words[j / 8]);
+            }
+          }
+          if (!ok) break;
+#pragma unroll
+          for (int bk = 0; bk < kBlkT; ++bk) {
+            const float bs0 = bs01[bk].x + bs01[bk].y, bs1 = bs23[bk].x + bs23[bk].y;
+            l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
+          }
+        }
+        SM_TRACE(4);
+        if (u + kWG >= it.n_steps) {
+          // the team's last step of the item: its normaliser shares go with this arrival (the slot was
+          // last read four items ago)
+          sts_f32(&sm.fin_l[i & 3][w * kSplit + hf][row], l);
+          sts_f32(&sm.fin_m[i & 3][w * kSplit + hf][row], M);
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive_warp(&sm.p_ready[w]);               // codes in tensor memory, scale bytes and shift in shared memory
+        SM_TRACE(5);
       }
-      SM_TRACE(4);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive_warp(&sm.p_ready[w]);                 // codes in tensor memory, scale bytes and shift in shared memory
-      SM_TRACE(5);
+      if (!ok) break;
+      G += it.n_steps;
     }
-    sts_f32(&sm.fin_l[w * kSplit + hf][row], l);
-    sts_f32(&sm.fin_m[w * kSplit + hf][row], M);
-    mbar_arrive_warp(&sm.fin);
   }
   __syncwarp();
   tc_fence_before_sync();
@@ -590,7 +642,15 @@ attn_status_t launch_fwd_il_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   const size_t smem = sizeof(IlSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(fwd_il_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.Hq, s.N / kTile, s.B);
+  p.gx = s.Hq; p.gy = s.N / kTile; p.gz = s.B;
+  const long long items = static_cast<long long>(p.gx) * p.gy * p.gz;
+  if (items > 0x7fffffffLL) return fail(ATTN_ERR_UNSUPPORTED, "fwd: %lld work items exceed 2^31 - 1", items);
+  // one CTA per SM (the kernel takes all of an SM's tensor memory) walks the item list
+  int dev = 0, sms = 0;
+  e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess || sms < 1) return fail(ATTN_ERR_CUDA, "fwd: SM count: %s", cudaGetErrorString(e));
+  dim3 grid(static_cast<unsigned>(items < sms ? items : sms), 1, 1);
   fwd_il_kernel<C><<<grid, C::kThreads, smem, stream>>>(p, tm_q, tm_k, tm_v);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "fwd: launch: %s", cudaGetErrorString(e));

@@ -1,0 +1,100 @@
+// Measurement aid: the rate at which the tensor cores of this device execute the block-scaled FP8
+// instruction the attention kernels are built on (tcgen05.mma.kind::mxf8f6f4.block_scale, E4M3
+// operands with E8M0 scales, M = 128, N = 128, K = 32 per instruction), with nothing else running.
+// Three warps per CTA issue back to back from shared-memory operands into their own accumulators
+// (one warp cannot issue fast enough to keep the pipe busy), one CTA per SM.  The figure is the
+// denominator "measured FP8 peak" of the benchmark's report; the paper has no counterpart.
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attnfp8 {
+namespace {
+
+using namespace sm100;
+
+constexpr int kIssuers = 3;
+
+__global__ void __launch_bounds__(128, 1) mma_peak_kernel(int reps, int* status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* sA = smem_raw;                       // 128 rows x 128 bytes, swizzled layout (the values do not matter)
+  uint8_t* sB = smem_raw + 16384;               // 128 rows x 128 bytes
+  uint8_t* sSF = smem_raw + 32768;              // 512-byte scale tile
+  __shared__ uint64_t bar[kIssuers];
+  __shared__ uint32_t tmem_holder;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (smem_u32(smem_raw) & 1023u) {
+    if (tid == 0) atomicExch(status, static_cast<int>(ATTN_ERR_ALIGNMENT));
+    return;
+  }
+  for (int i = tid; i < 32768 / 4; i += 128) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0x38383838u;   // E4M3 1.0
+  for (int i = tid; i < 512 / 4; i += 128) reinterpret_cast<uint32_t*>(sSF)[i] = 0x7f7f7f7fu;          // scale 2^0
+  if (tid == 0) {
+    for (int i = 0; i < kIssuers; ++i) mbar_init(&bar[i], 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&tmem_holder, 512);
+    tmem_relinquish();
+  }
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_holder;
+  if (warp < kIssuers) {
+    const uint32_t sfa = tmem + 448 + 8 * warp, sfb = sfa + 4;
+    sf_copy_elect(sfa, make_desc_sf(smem_u32(sSF)));
+    sf_copy_elect(sfb, make_desc_sf(smem_u32(sSF)));
+    const uint64_t da = make_desc_sw128(smem_u32(sA)), db = make_desc_sw128(smem_u32(sB));
+    const uint32_t acc = tmem + 128 * warp;
+    for (int r = 0; r < reps; r += 4) {
+#pragma unroll
+      for (int kb = 0; kb < 4; ++kb)
+        mma_mxf8_ss_elect(acc, da + 2 * kb, db + 2 * kb, make_idesc_mxf8(128, 128, kb, kb), sfa, sfb, (r > 0 || kb > 0));
+    }
+    mma_commit_elect(&bar[warp]);
+    mbar_wait(&bar[warp], 0, &abort_flag);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 512);
+  if (tid == 0 && abort_flag) atomicExch(status, static_cast<int>(ATTN_ERR_TIMEOUT));
+}
+
+}  // namespace
+
+attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t stream) {
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess || sms < 1) return fail(ATTN_ERR_CUDA, "mma peak: SM count: %s", cudaGetErrorString(e));
+  const int smem = 32768 + 512;
+  const int reps = 16384;                       // per issuing warp: ~3 ms at the nominal rate
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "mma peak: cudaEventCreate: %s", cudaGetErrorString(e));
+  float best_ms = 0.f;
+  for (int round = 0; round < 3 && e == cudaSuccess; ++round) {      // the first round warms the clocks up
+    cudaEventRecord(e0, stream);
+    mma_peak_kernel<<<sms, 128, smem, stream>>>(reps, status);
+    cudaEventRecord(e1, stream);
+    e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (round > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "mma peak: %s", cudaGetErrorString(e));
+  const double flops = 2.0 * 128 * 128 * 32 * static_cast<double>(reps) * kIssuers * sms;
+  *tflops_out = flops / (best_ms * 1e-3) / 1e12;
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8

@@ -31,3 +31,23 @@ def max_over_ranks(values: Sequence[float], device=None, group=None) -> list:
 def aggregate_rate(work_per_rank: float, world_size: int, seconds_max: float) -> float:
     """Whole-job rate of ``world_size`` replicas that each did ``work_per_rank`` in at most ``seconds_max``."""
     return world_size * work_per_rank / seconds_max
+
+
+def free_port() -> int:
+    """A TCP port that is free on 127.0.0.1 right now (for the rendezvous of a local launch)."""
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def launch_local(n_ranks: int, script: str, argv: Sequence[str], env=None) -> int:
+    """Runs ``script argv`` as ``n_ranks`` processes of one node, one rank per GPU, the way the
+    benchmark is launched for N > 1 (``python -m torch.distributed.run --nnodes=1 --nproc-per-node N``,
+    rendezvous on 127.0.0.1).  Returns the launcher's exit code.  The ranks find RANK, LOCAL_RANK,
+    WORLD_SIZE and MASTER_* in their environment."""
+    import subprocess
+    import sys
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script] + list(argv)
+    return subprocess.call(cmd, env=env)

@@ -86,6 +86,10 @@ def test_validation_errors_without_touching_a_gpu(lib_path):
     p = binding.AttnParams(1, 128, 4, 2, 96, 96, True, 0.1).c_struct()
     st = binding._lib.attn_fp8_fwd(ctypes.byref(p), q, q, q, None, None, None, 0, None)
     assert st == 2
+    # more rows than the kernels' 32-bit row coordinates reach: refused before any launch
+    p = binding.AttnParams(64, 1 << 20, 64, 8, 128, 128, True, 0.1).c_struct()
+    st = binding._lib.attn_fp8_fwd(ctypes.byref(p), q, q, q, None, None, None, 0, None)
+    assert st == 2 and "2^31" in binding.attn_fp8_last_error()
 
 
 def test_batched_quantiser_and_workspace_validation_without_a_gpu(lib_path):
@@ -108,4 +112,8 @@ def test_batched_quantiser_and_workspace_validation_without_a_gpu(lib_path):
     assert lib.attn_fp8_workspace_init(None, 256, None) == 4
     assert lib.attn_fp8_workspace_init(fake, 16, None) == 4
     assert lib.attn_fp8_workspace_init(ctypes.c_void_p(4100), 256, None) == 3
-    assert lib.attn_fp8_read_status(None, None) == 1
+    # a NULL workspace means the built-in scratch array of the current device: without a device the call
+    # stops at the device check (ATTN_ERR_CUDA), with one it reads that array's status word
+    import torch
+    if not torch.cuda.is_available():
+        assert lib.attn_fp8_read_status(None, None) == 6
