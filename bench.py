@@ -169,6 +169,35 @@ def oracle_step(w, sample_tokens, q, k, v, dO, prec="mxfp8"):
     return sum(sub.credited_flops())
 
 
+def residual_statistics(rs, ra, ps, dk):
+    """Row-sum residual statistics of the paper's Appendix "Row-Sum Residuals" / "dS Quantization
+    Residuals" from the outputs of the instrumented dQ pass (rs = sum_j dS, ra = sum_j |dS| before the
+    cast, ps = sum_j dS' after it; [B, Hq, N]) and the key gradient dk [B, Hkv, N, d]: rows i >= 64 with
+    a non-zero denominator, as in the paper."""
+    rs, ra, ps = (t[..., 64:].double().flatten() for t in (rs, ra, ps))
+    live = ra > 0
+    r_pre = rs[live].abs() / ra[live]
+    r_post = ps[live].abs() / ra[live]
+    kappa = (ps[live] - rs[live]) / ra[live]
+    dkf = dk.double()
+    c_k = (dkf.sum(dim=2).norm(dim=-1) / dkf.pow(2).sum(dim=(2, 3)).sqrt()).flatten()
+    def median(t):                                   # the mean of the two middle values when the count is even
+        srt = t.sort().values
+        n = srt.numel()
+        return float(srt[(n - 1) // 2] + srt[n // 2]) / 2.0
+
+    return {
+        "rows": "query rows i >= 64 with a non-zero sum_j |dS_ij|",
+        "r_pre_median": median(r_pre),
+        "r_pre_p99": float(r_pre.sort().values[min(r_pre.numel() - 1, int(0.99 * r_pre.numel()))]),
+        "strict_ok_frac": float((r_pre <= 1e-5).double().mean()),
+        "strict_ok": "share of those rows with |sum_j dS| <= 1e-5 sum_j |dS|",
+        "r_post_median": median(r_post),
+        "kappa_mean": float(kappa.mean()),
+        "key_common_mode_median": median(c_k),
+    }
+
+
 def _cores_used():
     try:
         from threadpoolctl import threadpool_info
@@ -449,11 +478,12 @@ def main():
     which = "burst" if at_boost else "sustained"
     peak = peaks["bf16_" + which] * ratio
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    clock_peak = (2.0 * MACS_PER_CLK_PER_SM_FP8 / ratio * sms * sc["sm_mhz"] * 1e6 / 1e12) if sc.get("sm_mhz") else None
+    dtype_div = FP8_OVER_BF16 if bf16_mode else 1.0           # BF16 mode: half the FP8 rate
+    clock_peak = (2.0 * MACS_PER_CLK_PER_SM_FP8 / dtype_div * sms * sc["sm_mhz"] * 1e6 / 1e12) if sc.get("sm_mhz") else None
 
     def tensor_roofline(a, name):
         return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
-                "frac_of_nominal_peak": a / (NOMINAL_FP8_TFLOPS / ratio),
+                "frac_of_nominal_peak": a / (NOMINAL_FP8_TFLOPS / dtype_div),
                 "frac_of_clock_normalised_peak": a / clock_peak if clock_peak else None,
                 "frac_of_measured_fp8_mma_rate": a / measured_fp8 if measured_fp8 else None,
                 "traffic": NCU_TRAFFIC_BYTES.get(name) if (w.name == WORKLOAD and not bf16_mode) else None}
@@ -514,19 +544,7 @@ def main():
     if rank == 0:
         _, rs, ra, ps, pa, _ = B.attn_fp8_bwd_dq_postcast(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
         B.attn_fp8_read_status(ws)
-        rs, ra, ps = (t[..., 64:].double().flatten() for t in (rs, ra, ps))          # rows i >= 64, as in the paper
-        live = ra > 0
-        r_pre = (rs[live].abs() / ra[live])
-        r_post = (ps[live].abs() / ra[live])
-        kappa = ((ps[live] - rs[live]) / ra[live])
-        dkf = dk.double()
-        c_k = (dkf.sum(dim=2).norm(dim=-1) / dkf.pow(2).sum(dim=(2, 3)).sqrt()).flatten()
-        line["rowsum_ds_residual"] = {
-            "rows": "query rows i >= 64 with a non-zero sum_j |dS_ij|", "delta_mode": "matched",
-            "r_pre_median": float(r_pre.median()), "r_pre_p99": float(r_pre.quantile(0.99)) if r_pre.numel() < 16_000_000 else None,
-            "r_post_median": float(r_post.median()), "kappa_mean": float(kappa.mean()),
-            "key_common_mode_median": float(c_k.median()),
-        }
+        line["rowsum_ds_residual"] = dict(residual_statistics(rs, ra, ps, dk), delta_mode="matched")
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_tokens = 2048

@@ -312,7 +312,7 @@ attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes,
 
 /* Measurement aid (the paper has no counterpart): the rate, in TFLOP/s, at which this device executes
  * the bare block-scaled FP8 tensor-core instruction the attention kernels are built on (E4M3 operands,
- * E8M0 scales, 128 x 128 x 32 per instruction, three issuing warps per SM, operands resident in shared
+ * E8M0 scales, 128 x 224 x 32 per instruction, two issuing warps per SM, operands resident in shared
  * memory), written to *tflops (host).  Runs a few milliseconds of such instructions on `stream` three
  * times (the first warms the clocks up; the faster of the other two counts) and WAITS for them: unlike
  * the other entry points this one synchronises the stream.  `workspace` as for the attention calls

@@ -1,8 +1,9 @@
 // Measurement aid: the rate at which the tensor cores of this device execute the block-scaled FP8
 // instruction the attention kernels are built on (tcgen05.mma.kind::mxf8f6f4.block_scale, E4M3
-// operands with E8M0 scales, M = 128, N = 128, K = 32 per instruction), with nothing else running.
-// Three warps per CTA issue back to back from shared-memory operands into their own accumulators
-// (one warp cannot issue fast enough to keep the pipe busy), one CTA per SM.  The figure is the
+// operands with E8M0 scales, M = 128, N = 224, K = 32 per instruction), with nothing else running.
+// Two warps per CTA issue back to back from shared-memory operands into their own accumulators (one
+// warp cannot issue fast enough to keep the pipe busy; at N = 128 the operand reads from shared
+// memory, 8 KB per 64 tensor cycles, would be the limit instead of the tensor pipe), one CTA per SM.  The figure is the
 // denominator "measured FP8 peak" of the benchmark's report; the paper has no counterpart.
 #include <cuda_runtime.h>
 
@@ -14,13 +15,14 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kIssuers = 3;
+constexpr int kIssuers = 2;
+constexpr int kN = 224;
 
 __global__ void __launch_bounds__(128, 1) mma_peak_kernel(int reps, int* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* sA = smem_raw;                       // 128 rows x 128 bytes, swizzled layout (the values do not matter)
-  uint8_t* sB = smem_raw + 16384;               // 128 rows x 128 bytes
-  uint8_t* sSF = smem_raw + 32768;              // 512-byte scale tile
+  uint8_t* sB = smem_raw + 16384;               // kN rows x 128 bytes (32 KB reserved)
+  uint8_t* sSF = smem_raw + 49152;              // two 512-byte scale tiles
   __shared__ uint64_t bar[kIssuers];
   __shared__ uint32_t tmem_holder;
   __shared__ int abort_flag;
@@ -29,8 +31,8 @@ __global__ void __launch_bounds__(128, 1) mma_peak_kernel(int reps, int* status)
     if (tid == 0) atomicExch(status, static_cast<int>(ATTN_ERR_ALIGNMENT));
     return;
   }
-  for (int i = tid; i < 32768 / 4; i += 128) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0x38383838u;   // E4M3 1.0
-  for (int i = tid; i < 512 / 4; i += 128) reinterpret_cast<uint32_t*>(sSF)[i] = 0x7f7f7f7fu;          // scale 2^0
+  for (int i = tid; i < 49152 / 4; i += 128) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0x38383838u;   // E4M3 1.0
+  for (int i = tid; i < 1024 / 4; i += 128) reinterpret_cast<uint32_t*>(sSF)[i] = 0x7f7f7f7fu;         // scale 2^0
   if (tid == 0) {
     for (int i = 0; i < kIssuers; ++i) mbar_init(&bar[i], 1);
     abort_flag = 0;
@@ -46,15 +48,16 @@ __global__ void __launch_bounds__(128, 1) mma_peak_kernel(int reps, int* status)
   tc_fence_after_sync();
   const uint32_t tmem = tmem_holder;
   if (warp < kIssuers) {
-    const uint32_t sfa = tmem + 448 + 8 * warp, sfb = sfa + 4;
+    const uint32_t sfa = tmem + 2 * kN + 16 * warp, sfb = sfa + 4;       // B: kN / 32 = 7 columns of two tiles
     sf_copy_elect(sfa, make_desc_sf(smem_u32(sSF)));
     sf_copy_elect(sfb, make_desc_sf(smem_u32(sSF)));
+    sf_copy_elect(sfb + 4, make_desc_sf(smem_u32(sSF + 512)));
     const uint64_t da = make_desc_sw128(smem_u32(sA)), db = make_desc_sw128(smem_u32(sB));
-    const uint32_t acc = tmem + 128 * warp;
+    const uint32_t acc = tmem + kN * warp;
     for (int r = 0; r < reps; r += 4) {
 #pragma unroll
       for (int kb = 0; kb < 4; ++kb)
-        mma_mxf8_ss_elect(acc, da + 2 * kb, db + 2 * kb, make_idesc_mxf8(128, 128, kb, kb), sfa, sfb, (r > 0 || kb > 0));
+        mma_mxf8_ss_elect(acc, da + 2 * kb, db + 2 * kb, make_idesc_mxf8(128, kN, kb, kb), sfa, sfb, (r > 0 || kb > 0));
     }
     mma_commit_elect(&bar[warp]);
     mbar_wait(&bar[warp], 0, &abort_flag);
@@ -72,8 +75,10 @@ attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t str
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess || sms < 1) return fail(ATTN_ERR_CUDA, "mma peak: SM count: %s", cudaGetErrorString(e));
-  const int smem = 32768 + 512;
+  const int smem = 49152 + 1024;
   const int reps = 16384;                       // per issuing warp: ~3 ms at the nominal rate
+  e = cudaFuncSetAttribute(mma_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "mma peak: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   e = cudaEventCreate(&e0);
   if (e == cudaSuccess) e = cudaEventCreate(&e1);
@@ -92,7 +97,7 @@ attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t str
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "mma peak: %s", cudaGetErrorString(e));
-  const double flops = 2.0 * 128 * 128 * 32 * static_cast<double>(reps) * kIssuers * sms;
+  const double flops = 2.0 * 128 * kN * 32 * static_cast<double>(reps) * kIssuers * sms;
   *tflops_out = flops / (best_ms * 1e-3) / 1e12;
   return ATTN_OK;
 }

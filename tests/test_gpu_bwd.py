@@ -5,7 +5,7 @@ import torch
 
 from oracle import attention as A
 from paper_2609_37852_b200 import workloads
-from tests.util import rel_fro, to_np
+from tests.util import rel_fro, to_np, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +55,9 @@ def test_matched_backward_matches_oracle(name, kw):
     assert rel_fro(to_np(got["dq"]), dQ) <= TOL_GRAD
     assert rel_fro(to_np(got["dk"]), dK) <= TOL_GRAD
     assert rel_fro(to_np(got["dv"]), dV) <= TOL_GRAD
+    # and no single row of substance is far off (ten times the tensor tolerance)
+    for n_, ref in (("dq", dQ), ("dk", dK), ("dv", dV)):
+        assert worst_row_error(to_np(got[n_]), ref) <= 10 * TOL_GRAD, n_
     # pre-cast row statistics
     assert rel_fro(to_np(got["ra"]), ra) <= 1e-3
     # zero-row-sum invariant on the GPU's own statistics: |sum_j dS| <= 1e-5 sum_j |dS|, plus the
@@ -95,6 +98,8 @@ def _check_backward(w, q, k, v, dO, got, prec):
     assert rel_fro(to_np(got["dq"]), dQ) <= TOL_GRAD
     assert rel_fro(to_np(got["dk"]), dK) <= TOL_GRAD
     assert rel_fro(to_np(got["dv"]), dV) <= TOL_GRAD
+    for n_, ref in (("dq", dQ), ("dk", dK), ("dv", dV)):
+        assert worst_row_error(to_np(got[n_]), ref) <= 10 * TOL_GRAD, n_
     assert rel_fro(to_np(got["ra"]), ra) <= 1e-3
     g_rs, g_ra = to_np(got["rs"]), to_np(got["ra"])
     live = g_ra[..., 64:] > 0
@@ -250,3 +255,52 @@ def test_backward_is_reproducible():
     b = run_all(w, q, k, v, dO)
     for key in ("delta", "dq", "dk", "dv", "rs", "ra"):
         assert torch.equal(a[key], b[key]), key
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("gqa4k", dict(batch=1, heads_q=4, heads_kv=2, seqlen=384)),
+    ("gqa8k_outlier", dict(heads_q=4, heads_kv=2, seqlen=512)),
+])
+def test_whole_chain_against_an_oracle_that_never_sees_gpu_values(name, kw):
+    """The other backward tests hand the GPU's saved LSE and D to the oracle's gradient pass (as the GPU
+    gradient pass gets them).  Here the oracle runs its own chain end to end -- forward, its LSE into its
+    correction pass, its D into its gradient pass -- and the GPU's outputs are compared with that."""
+    w = workloads.WORKLOADS[name].scaled(**kw)
+    q, k, v, dO = workloads.make_inputs(w)
+    got = run_all(w, q, k, v, dO)
+    qn, kn, vn, dOn = (to_np(x) for x in (q, k, v, dO))
+    O, LSE = A.emu_forward(qn, kn, vn, w.softmax_scale, w.causal)
+    D = A.emu_delta(qn, kn, vn, dOn, LSE, w.softmax_scale, w.causal)
+    dQ, dK, dV, _, _ = A.emu_backward(qn, kn, vn, dOn, LSE, D, w.softmax_scale, w.causal)
+    assert rel_fro(to_np(got["o"]), O) <= 2e-3 and rel_fro(to_np(got["lse"]), LSE) <= 2e-3
+    assert rel_fro(to_np(got["delta"]), D) <= TOL_DELTA
+    for n_, ref in (("dq", dQ), ("dk", dK), ("dv", dV)):
+        assert rel_fro(to_np(got[n_]), ref) <= TOL_GRAD, n_
+        assert worst_row_error(to_np(got[n_]), ref) <= 10 * TOL_GRAD, n_
+
+
+def test_bench_residual_statistics_match_the_oracle_helpers():
+    """bench.py forms r_pre, r_post, kappa and c_K from the instrumented dQ pass with torch; the same
+    numbers from the oracle's (pinned) helpers, on the same kernel outputs."""
+    import bench
+    from paper_2609_37852_b200 import binding
+    w = workloads.WORKLOADS["gqa8k_outlier"].scaled(heads_q=4, heads_kv=2, seqlen=512)
+    q, k, v, dO = workloads.make_inputs(w)
+    params = binding.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                                w.softmax_scale)
+    qq, kq, vq, dOq = (binding.attn_fp8_quantize(x.cuda()) for x in (q, k, v, dO))
+    o, lse, ws = binding.attn_fp8_fwd(params, qq, kq, vq)
+    delta, ws = binding.attn_fp8_bwd_delta(params, qq, kq, vq, dOq, lse, workspace=ws)
+    dq, rs, ra, ps, pa, ws = binding.attn_fp8_bwd_dq_postcast(params, qq, kq, vq, dOq, lse, delta, workspace=ws)
+    dk, dv, ws = binding.attn_fp8_bwd_dkdv(params, qq, kq, vq, dOq, lse, delta, workspace=ws)
+    binding.attn_fp8_read_status(ws)
+    stats = bench.residual_statistics(rs, ra, ps, dk)
+    rsn, ran, psn, pan = (to_np(t)[..., 64:].ravel() for t in (rs, ra, ps, pa))
+    live = ran > 0
+    r_post, r_own, kappa = A.postcast_residuals(rsn[live], ran[live], psn[live], pan[live])
+    r_pre = A.residual_ratio(rsn[live], ran[live])
+    assert np.isclose(stats["r_pre_median"], np.median(r_pre), rtol=1e-12, atol=0)
+    assert np.isclose(stats["r_post_median"], np.median(r_post), rtol=1e-12, atol=0)
+    assert np.isclose(stats["kappa_mean"], np.mean(kappa), rtol=1e-9, atol=1e-18)
+    assert np.isclose(stats["key_common_mode_median"], np.median(A.key_common_mode(to_np(dk))), rtol=1e-12, atol=0)
+    assert np.isclose(stats["strict_ok_frac"], np.mean(r_pre <= 1e-5), rtol=0, atol=1e-12)

@@ -6,7 +6,7 @@ import torch
 from oracle import attention as A
 from oracle import mxfp8
 from paper_2609_37852_b200 import workloads
-from tests.util import rel_fro, to_np
+from tests.util import rel_fro, to_np, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +36,9 @@ def _check(w, tensors, got, prec="mxfp8"):
     assert rel_fro(to_np(got["dq"]), dQ) <= 5e-3
     assert rel_fro(to_np(got["dk"]), dK) <= 5e-3
     assert rel_fro(to_np(got["dv"]), dV) <= 5e-3
+    assert worst_row_error(to_np(got["o"]), O) <= 2e-2
+    for n_, ref in (("dq", dQ), ("dk", dK), ("dv", dV)):
+        assert worst_row_error(to_np(got[n_]), ref) <= 5e-2, n_
 
 
 @pytest.mark.parametrize("name,kw", [
