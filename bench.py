@@ -169,11 +169,25 @@ def oracle_step(w, sample_tokens, q, k, v, dO, prec="mxfp8"):
     return sum(sub.credited_flops())
 
 
-def residual_statistics(rs, ra, ps, dk):
+def residual_statistics(rs, ra, ps, dk, lse=None, dust=None):
     """Row-sum residual statistics of the paper's Appendix "Row-Sum Residuals" / "dS Quantization
     Residuals" from the outputs of the instrumented dQ pass (rs = sum_j dS, ra = sum_j |dS| before the
     cast, ps = sum_j dS' after it; [B, Hq, N]) and the key gradient dk [B, Hkv, N, d]: rows i >= 64 with
     a non-zero denominator, as in the paper."""
+    import torch
+    extra = {}
+    if lse is not None and dust is not None:
+        # the per-row acceptance on EVERY row: 1e-5 of sum |dS| plus the dust the FP32 storage of LSE leaves of
+        # delta_i (1 - sum_j P_ij), (ulp(LSE_i) + 2^-20) * sum_j P_ij |dP^_ij|
+        a = lse.abs()
+        ulp = (torch.nextafter(a, torch.full_like(a, float("inf"))) - a).double()
+        keys = torch.arange(1, rs.shape[-1] + 1, device=rs.device, dtype=torch.float64)      # keys a causal row sees
+        c = 2.0 ** -20 * torch.clamp(keys / 8192.0, min=1.0)                                 # FP32 summation over the row
+        ok = rs.double().abs() <= 1e-5 * ra.double() + (ulp + c) * dust.double()
+        extra = {"bound_with_lse_dust_ok_frac_all_rows": float(ok.double().mean()),
+                 "bound_with_lse_dust_ok_frac_rows_ge_64": float(ok[..., 64:].double().mean()),
+                 "bound_with_lse_dust": "|sum_j dS| <= 1e-5 sum_j |dS| + (ulp(LSE_i) + 2^-20 max(1, keys / 8192)) "
+                                        "sum_j P |dP^|, every row"}
     rs, ra, ps = (t[..., 64:].double().flatten() for t in (rs, ra, ps))
     live = ra > 0
     r_pre = rs[live].abs() / ra[live]
@@ -195,6 +209,7 @@ def residual_statistics(rs, ra, ps, dk):
         "r_post_median": median(r_post),
         "kappa_mean": float(kappa.mean()),
         "key_common_mode_median": median(c_k),
+        **extra,
     }
 
 
@@ -544,7 +559,9 @@ def main():
     if rank == 0:
         _, rs, ra, ps, pa, _ = B.attn_fp8_bwd_dq_postcast(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
         B.attn_fp8_read_status(ws)
-        line["rowsum_ds_residual"] = dict(residual_statistics(rs, ra, ps, dk), delta_mode="matched")
+        _, _, _, dust, _ = B.attn_fp8_bwd_dq_rowprobe(params, qq, kq, vq, dOq, lse, delta, dq=dq, workspace=ws)
+        B.attn_fp8_read_status(ws)
+        line["rowsum_ds_residual"] = dict(residual_statistics(rs, ra, ps, dk, lse=lse, dust=dust), delta_mode="matched")
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_tokens = 2048

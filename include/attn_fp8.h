@@ -252,6 +252,20 @@ attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q,
                                        float* diag_post_rowsum_ds, float* diag_post_rowsum_abs_ds,
                                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* attn_fp8_bwd_dq with the quantities the per-row acceptance of the zero-row-sum invariant needs (paper
+ * Section 3.3 Eq. 5; Appendix "Row-Sum Residuals").  With the matched correction the row sum of dS is, in
+ * exact arithmetic, delta_i (1 - sum_j P_ij): zero up to the rounding of the FP32-stored LSE, which leaves
+ * dust of size ulp(LSE_i) * sum_j P_ij |dP^_ij|.  Besides the pre-cast pair the call writes that last sum,
+ *   diag_p_abs_dp   sum_j P_ij |dP^_ij|   [B, Hq, N] FP32,
+ * so that a caller can test |sum_j dS| <= 1e-5 sum_j |dS| + (ulp(LSE_i) + c) * diag_p_abs_dp on EVERY row, c = 2^-20
+ * for rows of up to 8192 keys (the FP32 summation of the normaliser and of delta), growing in proportion to
+ * the key count beyond (rows that see one key, or are one-hot, have sum_j |dS| -> 0 and only the dust).  All three diagnostic
+ * pointers are required; dQ is identical to attn_fp8_bwd_dq's.                                        */
+attn_status_t attn_fp8_bwd_dq_rowprobe(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                       attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                                       float* diag_rowsum_ds, float* diag_rowsum_abs_ds, float* diag_p_abs_dp,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* Forward without a workspace argument (the paper has no counterpart; this is a packaging variant
  * of attn_fp8_fwd and computes exactly the same O and LSE).
  *

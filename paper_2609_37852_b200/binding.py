@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "attn_fp8_scale_offset", "attn_fp8_scale_bytes", "attn_fp8_quantize", "attn_fp8_quantize_fused", "attn_fp8_prepare_bf16", "attn_fp8_fwd", "attn_fp8_bwd_delta",
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_workspace_init", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
-    "attn_fp8_measure_mma_peak",
+    "attn_fp8_measure_mma_peak", "attn_fp8_bwd_dq_rowprobe",
 )
 
 
@@ -448,6 +448,28 @@ def attn_fp8_bwd_dq_postcast(params: AttnParams, q: QTensor, k: QTensor, v: QTen
     workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
     c = params.c_struct()
     _check(_lib.attn_fp8_bwd_dq_postcast(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),
+                                         _ptr(lse), _ptr(delta), _ptr(dq), *(_ptr(t) for t in stats), _ptr(workspace),
+                                         workspace.numel(), _stream(stream)))
+    return (dq, *stats, workspace)
+
+
+_lib.attn_fp8_bwd_dq_rowprobe.restype = _i32
+_lib.attn_fp8_bwd_dq_rowprobe.argtypes = [ctypes.POINTER(_Params), _QTensor, _QTensor, _QTensor, _QTensor, _vp, _vp, _vp,
+                                          _vp, _vp, _vp, _vp, _sz, _vp]
+
+
+def attn_fp8_bwd_dq_rowprobe(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTensor, lse, delta, dq=None,
+                             workspace=None, stream=None):
+    """dQ plus what the per-row acceptance of the zero-row-sum invariant needs.  Returns
+    (dQ, rowsum_dS, rowsum_abs_dS, rowsum_P_abs_dP, workspace)."""
+    dev = lse.device
+    B, N = params.batch, params.seqlen
+    if dq is None:
+        dq = torch.empty((B, params.heads_q, N, params.head_dim_qk), dtype=torch.bfloat16, device=dev)
+    stats = [torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev) for _ in range(3)]
+    workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_bwd_dq_rowprobe(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),
                                          _ptr(lse), _ptr(delta), _ptr(dq), *(_ptr(t) for t in stats), _ptr(workspace),
                                          workspace.numel(), _stream(stream)))
     return (dq, *stats, workspace)

@@ -297,7 +297,7 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
                               attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16, void* dk_bf16,
                               void* dv_bf16, float* diag_rowsum_ds, float* diag_rowsum_abs_ds, void* workspace,
                               size_t workspace_bytes, void* stream, bool want_dq, bool want_dkdv,
-                              float* post_rowsum = nullptr, float* post_rowabs = nullptr) {
+                              float* post_rowsum = nullptr, float* post_rowabs = nullptr, float* p_abs_dp = nullptr) {
   AttnShape s;
   if (want_dq) CHECK(check_params(p, &s, kEntryDq));
   if (want_dkdv) CHECK(check_params(p, &s, kEntryDkdv));
@@ -311,6 +311,8 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
       return fail(ATTN_ERR_INVALID_ARG, "the two diagnostic outputs must be given together");
     if ((post_rowsum == nullptr) != (post_rowabs == nullptr) || (post_rowsum && !diag_rowsum_ds))
       return fail(ATTN_ERR_INVALID_ARG, "the post-cast outputs come as a pair and need the pre-cast pair as well");
+    if (p_abs_dp && !diag_rowsum_ds) return fail(ATTN_ERR_INVALID_ARG, "diag_p_abs_dp needs the pre-cast pair as well");
+    if (p_abs_dp) CHECK(check_ptr(p_abs_dp, "diag_p_abs_dp"));
   }
   if (want_dkdv) {
     CHECK_OPERAND(q, col, fp8); CHECK_OPERAND(dO, col, fp8);
@@ -331,7 +333,7 @@ static attn_status_t bwd_impl(const attn_params_t* p, attn_qtensor_t q, attn_qte
   if (want_dkdv) CHECK(launch_bwd_dkdv(s, q, k, v, dO, lse, delta, dk_bf16, dv_bf16, status, st));
   if (want_dq)
     CHECK(launch_bwd_dq(s, q, k, v, dO, lse, delta, dq_bf16, diag_rowsum_ds, diag_rowsum_abs_ds, post_rowsum, post_rowabs,
-                        status, st, /*behind_dkdv=*/want_dkdv));
+                        status, st, /*behind_dkdv=*/want_dkdv, p_abs_dp));
   return ATTN_OK;
 }
 
@@ -360,6 +362,16 @@ attn_status_t attn_fp8_bwd_dq_postcast(const attn_params_t* p, attn_qtensor_t q,
     return fail(ATTN_ERR_INVALID_ARG, "attn_fp8_bwd_dq_postcast needs all four diagnostic outputs");
   return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, nullptr, nullptr, diag_rowsum_ds, diag_rowsum_abs_ds,
                   workspace, workspace_bytes, stream, true, false, diag_post_rowsum_ds, diag_post_rowsum_abs_ds);
+}
+
+attn_status_t attn_fp8_bwd_dq_rowprobe(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
+                                       attn_qtensor_t dO, const float* lse, const float* delta, void* dq_bf16,
+                                       float* diag_rowsum_ds, float* diag_rowsum_abs_ds, float* diag_p_abs_dp,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  if (!diag_rowsum_ds || !diag_rowsum_abs_ds || !diag_p_abs_dp)
+    return fail(ATTN_ERR_INVALID_ARG, "attn_fp8_bwd_dq_rowprobe needs all three diagnostic outputs");
+  return bwd_impl(p, q, k, v, dO, lse, delta, dq_bf16, nullptr, nullptr, diag_rowsum_ds, diag_rowsum_abs_ds,
+                  workspace, workspace_bytes, stream, true, false, nullptr, nullptr, diag_p_abs_dp);
 }
 
 attn_status_t attn_fp8_bwd_dkdv(const attn_params_t* p, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,

@@ -120,7 +120,7 @@ struct QmSmem {
   alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
   alignas(16) uint8_t sf_kc[C::kKcStages][512];
   alignas(16) uint8_t sf_ds[2][512];
-  alignas(16) float red[C::kGroups][4][kTile];   // partial row sums of every column group
+  alignas(16) float red[C::kGroups][5][kTile];   // partial row sums of every column group
   uint64_t q_full[C::kQBufs], q_empty[C::kQBufs];
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
@@ -144,6 +144,7 @@ struct QmParams {
   float* rowabs;
   float* post_rowsum;       // optional: row sums of the CAST score gradient (the dQ operand) and of its magnitude
   float* post_rowabs;
+  float* p_abs_dp;          // optional (with rowsum): sum_j P_ij |dP^_ij|, the scale of the rounding dust of a row sum
   int* status;
   int* sched;               // ticket mode: the next item number; the host zeroes it ahead of the launch
   int N, Hq, Hkv, dqk, dv, causal;
@@ -488,6 +489,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float f_lo = fmaf(-lse2_lo, kLn2, 1.0f);   // 2^-lo to first order (|lo| < 1e-5)
     const float fD = f_lo * D;
     float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
+    float acc2 = 0.f;                                 // kDQ with statistics: sum P |dP| (without the factor f_lo)
     // kDQ, on request: sum dS', sum |dS'| of the cast values, kept in shared memory so that the
     // common path carries no extra registers
     const bool want_post = kDQ && p.post_rowsum != nullptr;
@@ -541,6 +543,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             if (kStats) {
               acc0 += d2.x + d2.y;
               acc1 += fabsf(d2.x) + fabsf(d2.y);
+              acc2 = fmaf(pr2.x, fabsf(dp2.x), fmaf(pr2.y, fabsf(dp2.y), acc2));
             }
           } else {
             part2 = __ffma2_rn(pr2, dp2, part2);
@@ -623,6 +626,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const int si = (kPersist && !kDQ) ? (i & 1) : 0;   // the dQ kernel uses slots 0 and 1 and a barrier per item
     sm.red[grp][si][row] = acc0;
     if (kDQ) sm.red[grp][1][row] = acc1;
+    if (kDQ && p.p_abs_dp) sm.red[grp][4][row] = acc2 * f_lo;
     named_barrier_sync(1, kSoftmaxThreads);
     if (ok && grp == 0) {
       acc0 = 0.f; acc1 = 0.f;
@@ -635,6 +639,11 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       } else if (p.rowsum && r_tile == 0) {
         p.rowsum[grow] = acc0;
         p.rowabs[grow] = acc1;
+        if (p.p_abs_dp) {
+          float dust = 0.f;
+          for (int j = 0; j < kGroups; ++j) dust += sm.red[j][4][row];
+          p.p_abs_dp[grow] = dust;
+        }
         if (p.post_rowsum) {
           float post0 = 0.f, post1 = 0.f;
           for (int j = 0; j < kGroups; ++j) { post0 += sm.red[j][2][row]; post1 += sm.red[j][3][row]; }
@@ -693,7 +702,7 @@ template <class C>
 attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                               const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
                               float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
-                              bool behind_dkdv) {
+                              bool behind_dkdv, float* p_abs_dp) {
   constexpr bool kDQ = C::kDQ;
   static_assert(sizeof(QmSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
@@ -715,7 +724,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.q_sf = q.row_scales; p.dO_sf = dO.row_scales; p.k_sf = k.row_scales; p.v_sf = v.row_scales;
   p.kc_sf = kDQ ? k.col_scales : nullptr;
   p.lse = lse; p.delta_in = delta_in; p.delta_out = delta_out;
-  p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.status = status;
+  p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.p_abs_dp = p_abs_dp; p.status = status;
   p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   p.tail_wait = behind_dkdv ? 1 : 0;
@@ -759,12 +768,12 @@ template <bool kDQ>
 attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta_in, float* delta_out, void* dq, float* rowsum,
                             float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
-                            bool behind_dkdv = false) {
+                            bool behind_dkdv = false, float* p_abs_dp = nullptr) {
   const int cq = (s.dqk * s.eb + 127) / 128, cv = (s.dv * s.ebv + 127) / 128;
 #define ATTN_QM_CASE(EB, CQ, CV, EBV)                                                                         \
   if (s.eb == EB && s.ebv == EBV && cq == CQ && cv == CV)                                                     \
     return launch_qmajor_t<QmCfg<kDQ, EB, CQ, CV, EBV>>(s, q, k, v, dO, lse, delta_in, delta_out, dq, rowsum, rowabs, \
-                                                       post_rowsum, post_rowabs, status, stream, behind_dkdv);
+                                                       post_rowsum, post_rowabs, status, stream, behind_dkdv, p_abs_dp);
   ATTN_QM_CASE(1, 1, 1, 1)
   ATTN_QM_CASE(1, 2, 1, 1)
   ATTN_QM_CASE(1, 2, 2, 1)
@@ -853,9 +862,10 @@ attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtenso
 
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                             const float* lse, const float* delta, void* dq, float* rowsum, float* rowabs,
-                            float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream, bool behind_dkdv) {
+                            float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream, bool behind_dkdv,
+                            float* p_abs_dp) {
   return launch_qmajor<true>(s, q, k, v, dO, lse, delta, nullptr, dq, rowsum, rowabs, post_rowsum, post_rowabs, status, stream,
-                             behind_dkdv);
+                             behind_dkdv, p_abs_dp);
 }
 
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,

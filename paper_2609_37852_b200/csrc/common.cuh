@@ -38,7 +38,7 @@ attn_status_t launch_bf16_copies(const void* src, int src_dtype, int B, int H, i
 attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
                          float* lse, int* status, cudaStream_t stream);
 attn_status_t launch_fwd_interleaved(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
-                                     float* lse, int* status, cudaStream_t stream, int variant);
+                                     float* lse, int* status, cudaStream_t stream);
 attn_status_t launch_bwd_delta(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                                attn_qtensor_t dO, const float* lse, float* delta, int* status, cudaStream_t stream);
 attn_status_t launch_stale_delta(const AttnShape& s, const void* dO_bf16, const void* o_bf16, float* delta,
@@ -48,7 +48,7 @@ attn_status_t launch_consistent_delta(const AttnShape& s, attn_qtensor_t dO, con
 attn_status_t launch_bwd_dq(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                             attn_qtensor_t dO, const float* lse, const float* delta, void* dq, float* rowsum,
                             float* rowabs, float* post_rowsum, float* post_rowabs, int* status, cudaStream_t stream,
-                            bool behind_dkdv = false);
+                            bool behind_dkdv = false, float* p_abs_dp = nullptr);
 attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v,
                               attn_qtensor_t dO, const float* lse, const float* delta, void* dk, void* dv,
                               int* status, cudaStream_t stream);

@@ -30,16 +30,6 @@
 
 namespace attnfp8 {
 
-#ifdef ATTN_TRACE
-__device__ long long g_il_trace[5][256][8];
-#define IL_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_il_trace[role][step][ev] = clock64(); } while (0)
-extern "C" int attn_fp8_debug_il_trace(long long* host_out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_il_trace, sizeof(g_il_trace)));
-}
-#else
-#define IL_TRACE(role, step, ev) do { } while (0)
-#endif
-
 namespace {
 
 using namespace sm100;
@@ -57,15 +47,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-#ifdef ATTN_IL_VOLATILE
-__device__ __forceinline__ float ex2_il(float x) {
-  float y;
-  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-#else
-#define ex2_il ex2_approx
-#endif
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -193,8 +174,9 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
     for (int w = 0; w < kWG; ++w) {
-      mbar_init(&sm.s_full[w], 1); mbar_init(&sm.s_free[w], 4 * kSplit);          // one arrival per warp
-      mbar_init(&sm.p_ready[w], 4 * kSplit); mbar_init(&sm.p_full[w], 4); mbar_init(&sm.p_free[w], 1);
+      // every thread arrives for itself (one elected arrival per warp behind a warp barrier measured slower)
+      mbar_init(&sm.s_full[w], 1); mbar_init(&sm.s_free[w], 128 * kSplit);
+      mbar_init(&sm.p_ready[w], 128 * kSplit); mbar_init(&sm.p_full[w], 128); mbar_init(&sm.p_free[w], 1);
     }
     mbar_init(&sm.o_done, 1);
     mbar_init(&sm.o_free, 4);
@@ -282,20 +264,17 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             tc_fence_after_sync();
             sf_copy_tiles<1>(tmem + kColSFK + 4 * slot, sm.sf_k[s]);
           }
-          IL_TRACE(0, gu, 0);
           if (gu >= kWG) {
             // team w has pulled the scores of its previous step into registers
             ok = mbar_wait(&sm.s_free[w], ((gu / kWG) - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
-          IL_TRACE(0, gu, 1);
           const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + sub * (kSW * 128 / 16);
           issue_ss<true, 1, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
                                                                       tmem + kColSFQ + 4 * qb,
                                                                       tmem + kColSFK + 4 * slot + kBlk * sub);
           mma_commit_elect(&sm.s_full[w]);
-          IL_TRACE(0, gu, 2);
           if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
         }
         if (ok) mma_commit_elect(&sm.q_empty[qb]);       // this item's Q tile has been read
@@ -324,7 +303,6 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             tc_fence_after_sync();
             sf_copy_tiles<1>(tmem + kColSFV + 4 * slot, sm.sf_v[s]);
           }
-          IL_TRACE(1, gu, 0);
           ok = mbar_wait(&sm.p_full[w], (gu / kWG) & 1, abort_flag);
           if (!ok) break;
           if (u == 0 && i > 0) {
@@ -332,7 +310,6 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             ok = mbar_wait(&sm.o_free, (i - 1) & 1, abort_flag);
             if (!ok) break;
           }
-          IL_TRACE(1, gu, 1);
           tc_fence_after_sync();
           sf_copy_elect(tmem + kColSFP + 4 * w, make_desc_sf(smem_u32(sm.sf_p[w])));
           const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s]));
@@ -343,7 +320,6 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
                               make_idesc_mxf8(128, n_dv, kb, kstep), tmem + kColSFP + 4 * w, tmem + kColSFV + 4 * slot,
                               (u > 0 || kb > 0));
           }
-          IL_TRACE(1, gu, 2);
           mma_commit_elect(&sm.p_free[w]);                  // operand and scale bytes of this buffer consumed; O updated
           if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
           if (u == it.n_steps - 1) mma_commit_elect(&sm.o_done);
@@ -371,10 +347,8 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       float MO = -INFINITY;                             // the accumulator row is expressed in units of 2^MO
       for (int u = 0; u < it.n_steps; ++u) {
         const int gu = G + u, w = gu % kWG, use = gu / kWG;
-        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 0);
         ok = mbar_wait(&sm.p_ready[w], use & 1, abort_flag);
         if (!ok) break;
-        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 1);
         float Mh[kSplit];                               // -inf: the thread has seen nothing but masked keys
         uint32_t raw[kSplit];
 #pragma unroll
@@ -424,8 +398,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         else
           asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_u32(sf_dst)), "h"(static_cast<uint16_t>(packed)) : "memory");
         fence_proxy_async_smem();
-        mbar_arrive_warp(&sm.p_full[w]);
-        if (lane == 0 && quad == 0) IL_TRACE(4, gu, 2);
+        mbar_arrive(&sm.p_full[w]);
       }
       // The row's normaliser = sum of the shares of its softmax threads, in the accumulator's unit.  A
       // team wrote its shares ahead of the arrival that announced its last step of the item (a team
@@ -482,11 +455,8 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       float l = 0.f;                                    // this thread's share of the normaliser, in units of 2^M
       for (int u = (w + kWG - G % kWG) % kWG; u < it.n_steps; u += kWG) {
         const int gu = G + u, t = u / kSubPerTile, sub = u % kSubPerTile, use = gu / kWG;
-#define SM_TRACE(ev) do { if (lane == 0 && quad == 0 && hf == 0) IL_TRACE(2 + w, gu, ev); } while (0)
-        SM_TRACE(0);
         ok = mbar_wait(&sm.s_full[w], use & 1, abort_flag);
         if (!ok) break;
-        SM_TRACE(1);
         tc_fence_after_sync();
         float sv[kColsT];
 #pragma unroll
@@ -494,8 +464,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
           tmem_ld32(tmem + kColS + kSW * w + kColsT * hf + lane_addr + 32 * bk, reinterpret_cast<uint32_t*>(sv + 32 * bk));
         tmem_wait_ld();
         tc_fence_before_sync();
-        mbar_arrive_warp(&sm.s_free[w]);                // the scores are in registers: the next S of this buffer may be issued
-        SM_TRACE(2);
+        mbar_arrive(&sm.s_free[w]);                // the scores are in registers: the next S of this buffer may be issued
         // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
         float mxb[kBlkT];
         if (p.causal && t == qt) {
@@ -534,7 +503,6 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
           l *= pow2_int(M - m_new);                       // exact power of two (0 at the start)
           M = m_new;
         }
-        SM_TRACE(3);
         const float neg_m = M == -INFINITY ? 0.f : -M;    // nothing seen yet: every score is -inf, any finite shift gives zeros
         uint32_t bytes[kBlkT];
         // The scale 2^e of a block follows from its largest exponential, which is the exponential of
@@ -567,8 +535,8 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             if (j0 < kGroups) {
               const float2 a = __ffma2_rn(make_float2(sv[4 * j0], sv[4 * j0 + 1]), sc2, nme2[j0 / 8]);
               const float2 c = __ffma2_rn(make_float2(sv[4 * j0 + 2], sv[4 * j0 + 3]), sc2, nme2[j0 / 8]);
-              e01[j0] = make_float2(ex2_il(a.x), ex2_il(a.y));
-              e23[j0] = make_float2(ex2_il(c.x), ex2_il(c.y));
+              e01[j0] = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+              e23[j0] = make_float2(ex2_approx(c.x), ex2_approx(c.y));
             }
             if (j0 >= kLag) {
               const int j = j0 - kLag;
@@ -580,13 +548,11 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
                 // the team's previous step have consumed its operand buffer (and the unit keepers its
                 // scale bytes and shift before that); that product was issued when the previous step
                 // ended, so the wait is over by now as a rule.
-                SM_TRACE(6);
                 if (gu >= kWG) {
                   ok = mbar_wait(&sm.p_free[w], (use - 1) & 1, abort_flag);
                   if (!ok) break;
                   tc_fence_after_sync();
                 }
-                SM_TRACE(7);
                 asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_u32(&sm.raw_sf[w][hf][row])), "r"(packed_sf) : "memory");
                 sts_f32(&sm.step_m[w][hf][row], M);
               }
@@ -600,7 +566,6 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             l = fmaf(bs0 + bs1, __uint_as_float(bytes[bk] << 23), l);   // 2^e (0 for an all-masked block, whose sum is 0)
           }
         }
-        SM_TRACE(4);
         if (u + kWG >= it.n_steps) {
           // the team's last step of the item: its normaliser shares go with this arrival (the slot was
           // last read four items ago)
@@ -609,8 +574,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive_warp(&sm.p_ready[w]);               // codes in tensor memory, scale bytes and shift in shared memory
-        SM_TRACE(5);
+        mbar_arrive(&sm.p_ready[w]);               // codes in tensor memory, scale bytes and shift in shared memory
       }
       if (!ok) break;
       G += it.n_steps;
@@ -659,11 +623,10 @@ attn_status_t launch_fwd_il_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
 
 }  // namespace
 
-// FP8 operands, head dims (64,64) and (128,128).  `variant` selects the instantiation.
+// FP8 operands, head dims (64,64) and (128,128): two teams, 128-key steps, two threads per row and step.
 attn_status_t launch_fwd_interleaved(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
-                                     float* lse, int* status, cudaStream_t stream, int variant) {
-  if (variant == 2) return launch_fwd_il_t<IlCfg<2, 128, 2>>(s, q, k, v, o, lse, status, stream);
-  return launch_fwd_il_t<IlCfg<2, 128, 1>>(s, q, k, v, o, lse, status, stream);
+                                     float* lse, int* status, cudaStream_t stream) {
+  return launch_fwd_il_t<IlCfg<2, 128, 2>>(s, q, k, v, o, lse, status, stream);
 }
 
 }  // namespace attnfp8
