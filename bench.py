@@ -407,6 +407,16 @@ def main():
     # ---- the bare block-scaled FP8 MMA rate of this device (a few ms; see attn_fp8_measure_mma_peak) ----
     measured_fp8 = None if bf16_mode else B.attn_fp8_measure_mma_peak(ws)
 
+    # ---- what the FP32 reduction of dQ alone would cost in a merged key-major gradient pass (see
+    #      attn_fp8_measure_dq_reduction): a design question kept measurable, outside every timed region
+    dq_reduction = None
+    if not bf16_mode and rank == 0 and w.head_dim_qk <= 128:
+        scratch = torch.empty((w.batch, w.heads_q, w.seqlen, w.head_dim_qk), dtype=torch.float32, device=dev)
+        red_ms, red_bytes = B.attn_fp8_measure_dq_reduction(params, scratch)
+        del scratch
+        dq_reduction = {"ms": red_ms, "GB": red_bytes / 1e9, "TB_per_s": red_bytes / (red_ms * 1e-3) / 1e12,
+                        "note": "FP32 adds a merged dQ/dK/dV pass would send to L2; compare stage_ms.bwd_dq"}
+
     # ---- end to end through the library with host buffers --------------------------------------
     # Host buffers in, host buffers out, every step: copies run on their own streams and overlap the
     # kernels of the neighbouring steps (three slots of device inputs / outputs), as a user pipeline would.
@@ -531,6 +541,7 @@ def main():
         "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
         "target": "north_star asks for >= 50 % of the nominal dense FP8 peak on this workload: not met",
         "measured_fp8_mma_tflops": measured_fp8,
+        "merged_pass_dq_reduction": dq_reduction,
         "pct_of_measured_fp8_mma_rate": (100.0 * value / world / measured_fp8) if measured_fp8 else None,
         "sustained": (None if sustained is None else dict(
             sustained, value=replicas.aggregate_rate(credited, world, sustained["ms_per_step"] * 1e-3) / 1e12, unit=UNIT,

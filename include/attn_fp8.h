@@ -333,6 +333,17 @@ attn_status_t attn_fp8_selftest_timeout(void* workspace, size_t workspace_bytes,
  * (status word).  Allocates no device memory.                                                       */
 attn_status_t attn_fp8_measure_mma_peak(double* tflops, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Measurement aid for one design question (the paper's Limitations name a fused gradient pass as open
+ * engineering; it has no such kernel): what the FP32 reduction of dQ alone would cost if the key-major
+ * kernel also produced dQ.  Issues, with no other work, the adds such a pass would make for the shape `p`
+ * (one [64 x head_dim_qk] FP32 partial per key tile of 128 and query sub-tile of 64 that the mask keeps,
+ * red.global.add.v4.f32 of ones, one CTA per (KV head, key tile, batch)) into `dq_f32`
+ * ([B, Hq, N, head_dim_qk] FP32, device, >= that many bytes; cleared by the call), three times, and WAITS:
+ * *ms = the faster of the last two passes, *bytes = the bytes added per pass.  Afterwards element
+ * (b, h, i, c) holds the number of key tiles row i sees.  Allocates nothing.                           */
+attn_status_t attn_fp8_measure_dq_reduction(const attn_params_t* p, float* dq_f32, size_t dq_f32_bytes, double* ms,
+                                            double* bytes, void* stream);
+
 /* Message for the last non-OK return on this host thread (static storage; never NULL).        */
 const char* attn_fp8_last_error(void);
 

@@ -36,6 +36,7 @@ EXPORTED_SYMBOLS = (
     "attn_fp8_bwd", "attn_fp8_bwd_dq", "attn_fp8_bwd_dq_postcast", "attn_fp8_bwd_dkdv", "attn_fp8_fwd_noalloc",
     "attn_fp8_quantize_batch", "attn_fp8_workspace_bytes", "attn_fp8_workspace_init", "attn_fp8_read_status", "attn_fp8_last_error", "attn_fp8_selftest_timeout",
     "attn_fp8_measure_mma_peak", "attn_fp8_bwd_dq_rowprobe",
+    "attn_fp8_measure_dq_reduction",
 )
 
 
@@ -350,6 +351,21 @@ def attn_fp8_read_status(workspace: Optional[torch.Tensor], stream=None) -> None
 
 _lib.attn_fp8_measure_mma_peak.restype = _i32
 _lib.attn_fp8_measure_mma_peak.argtypes = [ctypes.POINTER(ctypes.c_double), _vp, _sz, _vp]
+
+
+_lib.attn_fp8_measure_dq_reduction.restype = _i32
+_lib.attn_fp8_measure_dq_reduction.argtypes = [ctypes.POINTER(_Params), _vp, _sz, ctypes.POINTER(ctypes.c_double),
+                                               ctypes.POINTER(ctypes.c_double), _vp]
+
+
+def attn_fp8_measure_dq_reduction(params: "AttnParams", dq_f32: torch.Tensor, stream=None):
+    """(milliseconds, bytes added) of the FP32 dQ reduction a merged key-major gradient pass would issue
+    for ``params``; ``dq_f32`` is an FP32 [B, Hq, N, dqk] device tensor (overwritten).  Synchronises."""
+    ms, nbytes = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    c = params.c_struct()
+    _check(_lib.attn_fp8_measure_dq_reduction(ctypes.byref(c), _ptr(dq_f32), dq_f32.numel() * dq_f32.element_size(),
+                                              ctypes.byref(ms), ctypes.byref(nbytes), _stream(stream)))
+    return ms.value, nbytes.value
 
 
 def attn_fp8_measure_mma_peak(workspace: torch.Tensor, stream=None) -> float:

@@ -516,3 +516,15 @@ extern "C" attn_status_t attn_fp8_measure_mma_peak(double* tflops, void* workspa
   CHECK(prepare_workspace(workspace, workspace_bytes, kWorkspaceHeaderBytes, st, &status));
   return measure_mma_peak(tflops, status, st);
 }
+
+extern "C" attn_status_t attn_fp8_measure_dq_reduction(const attn_params_t* p, float* dq_f32, size_t dq_f32_bytes, double* ms,
+                                                        double* bytes, void* stream) {
+  AttnShape s;
+  CHECK(check_params(p, &s, kEntryDq));
+  if (!ms || !bytes) return fail(ATTN_ERR_INVALID_ARG, "ms / bytes is NULL");
+  CHECK(check_ptr(dq_f32, "dq_f32"));
+  const size_t need = static_cast<size_t>(s.B) * s.Hq * s.N * s.dqk * sizeof(float);
+  if (dq_f32_bytes < need) return fail(ATTN_ERR_WORKSPACE, "dq_f32 of %zu bytes needed, %zu given", need, dq_f32_bytes);
+  CHECK(check_device());
+  return measure_dq_reduction(s, dq_f32, ms, bytes, static_cast<cudaStream_t>(stream));
+}

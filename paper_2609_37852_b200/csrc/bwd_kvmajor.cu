@@ -37,17 +37,6 @@
 
 namespace attnfp8 {
 
-#ifdef ATTN_TRACE
-// Debug build only: clock stamps of one CTA (roles x steps x events), read back by the host.
-__device__ long long g_kv_trace[4][256][4];
-#define KV_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_kv_trace[role][step][ev] = clock64(); } while (0)
-extern "C" int attn_fp8_debug_kv_trace(long long* host_out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_kv_trace, sizeof(g_kv_trace)));
-}
-#else
-#define KV_TRACE(role, step, ev) do { } while (0)
-#endif
-
 namespace {
 
 using namespace sm100;
@@ -314,19 +303,16 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * slot, st.sf_q);
         }
-        KV_TRACE(0, u, 0);
         if (u > 0) {
           // the team of the previous sub-tile has pulled S and dP into registers
           ok = mbar_wait(&sm.sdp_free[(u - 1) % kTeams], ((u - 1) / kTeams) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        KV_TRACE(0, u, 1);
         const uint64_t desc_q = make_desc_sw128(smem_u32(st.q[0])) + sub_r * (kSub * 128 / 16);
         issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColS, desc_k, desc_q, nk_qk, tmem + kColSFK, tmem + kColSFQ + 4 * kCq * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
-        KV_TRACE(0, u, 2);
       }
       if (!ok) {
         int dummy = 0;
@@ -393,10 +379,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             if (kHasDk) sf_copy_tiles<kRq>(tmem + kColSFQc + 4 * kRq * slot, st.sf_qc);
           }
         }
-        KV_TRACE(1, u, 0);
         ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
-        KV_TRACE(1, u, 1);
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
         if (u % kSubPerRow == kSubPerRow - 1 && lane == 0) mbar_arrive(&sm.row_empty[(u / kSubPerRow) % kRowStages]);
@@ -415,7 +399,6 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         // operands and scale bytes of this buffer may be overwritten once these MMAs have run; the
         // col stage may be refilled after its last sub-tile
         mma_commit_elect(&sm.pds_free[buf]);
-        KV_TRACE(1, u, 2);
         if (sub_c == kSubPerCol - 1) mma_commit_elect(&sm.col_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.done);
       }
@@ -437,10 +420,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
     for (int u = team; u < n_sub; u += kTeams) {
       const int half = u & 1, buf = u & 1, ri = u / kSubPerRow, s = ri % kRowStages;
-      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 0);
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
-      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 1);
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];                       // S then P; dP then dS (in place)
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
@@ -448,7 +429,6 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
-      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 2);
       ok = mbar_wait(&sm.lse_ready[s], (ri / kRowStages) & 1, abort_flag);
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
@@ -548,7 +528,6 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.pds_full[buf]);
-      if (quad == 0 && lane == 0 && grp == 0) KV_TRACE(2, u, 3);
       it = (it + 1 == tiles_n) ? it0 : it + 1;        // next tile of this head, or the first tile of the next head
     }
     // the epilogue is done by team 0 (group 0 stores dV, group 1 stores dK)

@@ -39,17 +39,6 @@
 
 namespace attnfp8 {
 
-#ifdef ATTN_TRACE
-// Debug build only: clock stamps of one CTA (roles x tiles x events), read back by the host.
-__device__ long long g_qm_trace[4][128][4];
-#define QM_TRACE(role, tile, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (tile) < 128) g_qm_trace[role][tile][ev] = clock64(); } while (0)
-extern "C" int attn_fp8_debug_qm_trace(long long* host_out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_qm_trace, sizeof(g_qm_trace)));
-}
-#else
-#define QM_TRACE(role, tile, ev) do { } while (0)
-#endif
-
 namespace {
 
 using namespace sm100;
@@ -282,7 +271,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           const int s = gt % kStages, u = gt / kStages;
           ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
           if (!ok) break;
-          QM_TRACE(0, t, 0);
           mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
           for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
           for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
@@ -335,23 +323,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           const int s = gt % kStages, slot = gt & 1;
           ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
-          QM_TRACE(1, t, 0);
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
-          QM_TRACE(1, t, 1);
           if (gt > 0) {
             // the softmax threads have pulled the previous S and dP into registers
             ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
-          QM_TRACE(1, t, 2);
           const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
           issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, t_sfq,
                                                                           tmem + kColSFK + 4 * kCq * slot);
           mma_commit_elect(&sm.sdp_full);
           mma_commit_elect(&sm.kv_empty[s]);
-          QM_TRACE(1, t, 3);
         }
         if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's Q tile has been read
         T += it.n_tiles;
@@ -497,14 +481,11 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       sm.red[grp][2][row] = 0.f;
       sm.red[grp][3][row] = 0.f;
     }
-    if (warp == 4 && lane == 0) QM_TRACE(3, i, 0);
     for (int t = 0; t < n_tiles; ++t) {
       const int gt = T + t;                           // step index over all items: the dS^ buffers run on
       const int buf = gt & 1;
-      if (warp == 4 && lane == 0) QM_TRACE(2, t, 0);
       ok = mbar_wait(&sm.sdp_full, gt & 1, abort_flag);
       if (!ok) break;
-      if (warp == 4 && lane == 0) QM_TRACE(2, t, 1);
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
       tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
@@ -512,7 +493,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free);
-      if (warp == 4 && lane == 0) QM_TRACE(2, t, 2);
       // column, inside the query tile's own key range, of this thread's first element (negative
       // before the diagonal tile)
       const int col0 = t * kStep - qt * kTile + 32 * grp;
@@ -610,7 +590,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.ds_full[buf]);
       }
     }
-    if (warp == 4 && lane == 0) QM_TRACE(3, i, 1);
     // the next item (published by now, as a rule): its LSE and D are in flight during this item's epilogue
     Item nx; nx.valid = false;
     if (kPersist && ok) {
@@ -654,7 +633,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     if (kDQ && ok) {
       ok = mbar_wait(&sm.dq_done, i & 1, abort_flag);
-      if (warp == 4 && lane == 0) QM_TRACE(3, i, 2);
       if (ok) {
         tc_fence_after_sync();
         __nv_bfloat16* out_row = p.dq + grow * p.dqk + 128 * r_tile;
@@ -681,7 +659,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     // the row-sum slots may be overwritten by the next item's partial sums
     if (kDQ && kPersist) named_barrier_sync(1, kSoftmaxThreads);
-    if (warp == 4 && lane == 0) QM_TRACE(3, i, 3);
     T += n_tiles;
     it = nx;
     }  // items

@@ -54,6 +54,7 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
                               int* status, cudaStream_t stream);
 
 attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t stream);
+attn_status_t measure_dq_reduction(const AttnShape& s, float* dq_f32, double* ms_out, double* bytes_out, cudaStream_t stream);
 
 inline size_t scale_tiles_per_slab(int64_t rows, int64_t cols) {
   return static_cast<size_t>((rows + 127) / 128) * static_cast<size_t>((cols / 32 + 3) / 4);

@@ -36,17 +36,6 @@
 
 namespace attnfp8 {
 
-#ifdef ATTN_TRACE
-// Debug build only: clock stamps of one CTA (roles x steps x events), read back by the host.
-__device__ long long g_fw_trace[4][256][8];
-#define FW_TRACE(role, step, ev) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 256) g_fw_trace[role][step][ev] = clock64(); } while (0)
-extern "C" int attn_fp8_debug_fw_trace(long long* host_out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_fw_trace, sizeof(g_fw_trace)));
-}
-#else
-#define FW_TRACE(role, step, ev) do { } while (0)
-#endif
-
 namespace {
 
 using namespace sm100;
@@ -232,19 +221,16 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
         }
-        FW_TRACE(0, u, 0);
         if (u > 0) {
           // the softmax threads have pulled the previous scores into registers
           ok = mbar_wait(&sm.s_free, (u - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
-        FW_TRACE(0, u, 1);
         const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0])) + sub * (kSub * 128 / 16);
         issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, C::kTileKeys * 128 / 16>(
             tmem + kColS, desc_q, desc_k, nk_qk, tmem + kColSFQ, tmem + kColSFK + 4 * kCq * slot + 2 * sub);
         mma_commit_elect(&sm.s_full);
-        FW_TRACE(0, u, 2);
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
       }
       if (!ok) {
@@ -265,17 +251,14 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           tc_fence_after_sync();
           if (kFp8) sf_copy_tiles<kRv>(tmem + kColSFV + 4 * kRv * slot, sm.sf_v[s]);
         }
-        FW_TRACE(1, u, 0);
         ok = mbar_wait(&sm.p_full[buf], (u >> 1) & 1, abort_flag);
         if (!ok) break;
-        FW_TRACE(1, u, 1);
         tc_fence_after_sync();
         if (kFp8) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
         // 64 keys = 2 (codes) or 4 (BF16) steps of 32 bytes; the V^T operand is taken 128 rows at a time
         issue_ts<kFp8, kEB, kRv>(tmem + kColO, tmem + kColP + kPCols * buf, make_desc_sw128(smem_u32(sm.v[s])), p.dv, sub,
                                  tmem + kColSFP + 4 * buf, tmem + kColSFV + 4 * kRv * slot, u > 0);
         mma_commit_elect(&sm.p_free[buf]);              // operand (and scale bytes) of this buffer consumed; O updated
-        FW_TRACE(1, u, 2);
         if (sub == kSubPerTile - 1) mma_commit_elect(&sm.v_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.o_done);
       }
@@ -302,11 +285,8 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     bool ok = true;
     for (int u = 0; u < n_sub; ++u) {
       const int t = u >> 1, half = u & 1, buf = u & 1;
-#define SM_TRACE(ev) do { if (lane == 0 && (warp == 4 || warp == 8)) FW_TRACE(warp == 4 ? 2 : 3, u, ev); } while (0)
-      SM_TRACE(0);
       ok = mbar_wait(&sm.s_full, u & 1, abort_flag);
       if (!ok) break;
-      SM_TRACE(1);
       tc_fence_after_sync();
       float sv[32 * kBpt];
 #pragma unroll
@@ -315,7 +295,6 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.s_free);
-      SM_TRACE(2);
       // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
       float mxb[kBpt];
       if (p.causal && t == qt) {
@@ -348,7 +327,6 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         if (!ok) break;
         mx = fmaxf(mx, lds_f32(&sm.xch[u & 1][grp ^ 1][row]));
       }
-      SM_TRACE(3);
       // a fully masked sub-tile (second half of the diagonal tile for the first 64 rows) gives -inf:
       // it never raises M and contributes zeros
       const float m_new = ceilf(mx * p.scale_log2);
@@ -416,14 +394,12 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
           l += bs0 + bs1;
         }
       }
-      SM_TRACE(4);
       if (u >= 2) {
         // the P V MMAs of sub-tile u-2 have consumed this buffer's operand and scale bytes
         ok = mbar_wait(&sm.p_free[buf], ((u - 2) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
-      SM_TRACE(5);
 #pragma unroll
       for (int bk = 0; bk < kBpt; ++bk) {
 #pragma unroll
@@ -435,7 +411,6 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(&sm.p_full[buf]);
-      SM_TRACE(6);
     }
     // total normaliser of the row = sum of the shares of its threads
     if (ok && kSplit == 2) {

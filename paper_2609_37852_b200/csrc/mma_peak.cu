@@ -68,6 +68,23 @@ __global__ void __launch_bounds__(128, 1) mma_peak_kernel(int reps, int* status)
   if (tid == 0 && abort_flag) atomicExch(status, static_cast<int>(ATTN_ERR_TIMEOUT));
 }
 
+// What the FP32 reduction of dQ would cost in a merged key-major gradient pass (the shape the paper's
+// Limitations name as open engineering: one pass that forms dS once and produces dQ, dK and dV): every
+// (key tile of 128, query sub-tile of 64) pair of the workload adds a [64 x dqk] FP32 partial into an FP32
+// dQ of the whole problem.  This kernel issues exactly those adds (red.global.add.v4.f32, the partial is
+// all ones) and nothing else, one CTA per (KV head, key tile, batch) in the order the key-major kernel
+// uses; the result is checkable (element (h, i, c) ends up as the number of key tiles row i sees).
+__global__ void __launch_bounds__(256, 1) dq_reduction_kernel(float* dq, int N, int Hq, int Hkv, int dqk, int causal) {
+  const int jt = blockIdx.y, g = blockIdx.x, b = blockIdx.z, G = Hq / Hkv, tiles = N / 128;
+  for (int h = g * G; h < (g + 1) * G; ++h)
+    for (int it = causal ? jt : 0; it < tiles; ++it)
+      for (int half = 0; half < 2; ++half) {
+        float* dst = dq + (static_cast<size_t>(b * Hq + h) * N + it * 128 + half * 64) * dqk;
+        for (int e = threadIdx.x * 4; e < 64 * dqk; e += 256 * 4)
+          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + e), "f"(1.f), "f"(1.f), "f"(1.f), "f"(1.f) : "memory");
+      }
+}
+
 }  // namespace
 
 attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t stream) {
@@ -99,6 +116,39 @@ attn_status_t measure_mma_peak(double* tflops_out, int* status, cudaStream_t str
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "mma peak: %s", cudaGetErrorString(e));
   const double flops = 2.0 * 128 * kN * 32 * static_cast<double>(reps) * kIssuers * sms;
   *tflops_out = flops / (best_ms * 1e-3) / 1e12;
+  return ATTN_OK;
+}
+
+}  // namespace attnfp8
+
+namespace attnfp8 {
+
+attn_status_t measure_dq_reduction(const AttnShape& s, float* dq_f32, double* ms_out, double* bytes_out, cudaStream_t stream) {
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "dq reduction: cudaEventCreate: %s", cudaGetErrorString(e));
+  const size_t n = static_cast<size_t>(s.B) * s.Hq * s.N * s.dqk;
+  const dim3 grid(s.Hkv, s.N / 128, s.B);
+  float best_ms = 0.f;
+  for (int round = 0; round < 3 && e == cudaSuccess; ++round) {     // the last round leaves the checkable result
+    e = cudaMemsetAsync(dq_f32, 0, n * sizeof(float), stream);
+    cudaEventRecord(e0, stream);
+    dq_reduction_kernel<<<grid, 256, 0, stream>>>(dq_f32, s.N, s.Hq, s.Hkv, s.dqk, s.causal);
+    cudaEventRecord(e1, stream);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (round > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "dq reduction: %s", cudaGetErrorString(e));
+  const double tiles = s.N / 128;
+  const double pairs = static_cast<double>(s.B) * s.Hq * (s.causal ? tiles * (tiles + 1) / 2 : tiles * tiles) * 2;
+  *ms_out = best_ms;
+  *bytes_out = pairs * 64 * s.dqk * sizeof(float);
   return ATTN_OK;
 }
 

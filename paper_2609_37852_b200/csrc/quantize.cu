@@ -37,7 +37,7 @@ struct Producer {
 };
 
 // One rotated channel: x*cos -+ partner*sin with one rounding for the product and a fused
-// multiply-add, then BF16 (the order the oracle writes out).
+// multiply-add, then BF16 (the order the header of attn_fp8_quantize_fused states).
 __device__ __forceinline__ float rotate_bf16(float x, float partner, float c, float s, bool upper) {
   const float t = __fmul_rn(partner, s);
   const float r = __fmaf_rn(x, c, upper ? t : -t);

@@ -315,3 +315,19 @@ def test_random_shapes_and_modes():
         except AssertionError as e:
             raise AssertionError(f"{base} {kw} bf16={bf16}") from e
         done += 1
+
+
+def test_measurement_aids():
+    """The two measurement entry points of the benchmark: the bare block-scaled MMA rate (a plausible
+    number, status word clean) and the dQ-reduction probe (its adds land where they should)."""
+    from paper_2609_37852_b200 import binding as B
+    ws = B.new_workspace(256, torch.device("cuda"))
+    tflops = B.attn_fp8_measure_mma_peak(ws)
+    B.attn_fp8_read_status(ws)
+    assert 1000.0 < tflops < 6000.0, tflops
+    params = B.AttnParams(1, 1024, 4, 2, 128, 128, True, 0.1)
+    dq = torch.empty((1, 4, 1024, 128), dtype=torch.float32, device="cuda")
+    ms, nbytes = B.attn_fp8_measure_dq_reduction(params, dq)
+    assert ms > 0 and nbytes == 4 * (8 * 9 // 2) * 2 * 64 * 128 * 4
+    want = (torch.arange(1024, device="cuda") // 128 + 1).float()          # key tiles a causal row sees
+    assert torch.equal(dq, want[None, None, :, None].expand_as(dq))
