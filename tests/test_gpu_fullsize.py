@@ -17,7 +17,7 @@ from tests.util import rel_fro, to_np
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, tensors, prec="mxfp8"):
+def _run(w, tensors, prec="mxfp8", strict_floor=0.999):
     from paper_2609_37852_b200 import binding as B
     params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
                           w.softmax_scale, precision=B.ATTN_PREC_BF16 if prec == "bf16" else B.ATTN_PREC_MXFP8)
@@ -34,16 +34,22 @@ def _run(w, tensors, prec="mxfp8"):
     B.attn_fp8_read_status(ws)
     assert torch.equal(dq2, dq) and torch.equal(rs2, rs) and torch.equal(ra2, ra)
     got = dict(o=o, lse=lse, delta=delta, dq=dq, dk=dk, dv=dv, rs=rs, ra=ra, dust=dust)
-    _assert_row_sum_invariant_on_every_row(got)
+    _assert_row_sum_invariant_on_every_row(got, strict_floor)
     return got
 
 
-def _assert_row_sum_invariant_on_every_row(got):
+def _assert_row_sum_invariant_on_every_row(got, strict_floor):
     """|sum_j dS| <= 1e-5 sum_j |dS| + (ulp(LSE_i) + c_i) sum_j P |dP^| on EVERY row of every head.  The
     second term is what is left of delta_i (1 - sum_j P_ij): the FP32 storage of LSE (one ulp), and the FP32
     summation of the normaliser and of delta over the row's keys, c_i = 2^-20 up to 8192 keys and growing
     in proportion to the key count beyond (the worst case of a sum of 2^-24 roundings, one per 32-key block).
-    It is all there is on rows whose dS vanishes analytically."""
+    It is all there is on rows whose dS vanishes analytically.
+
+    The strict form without the second term is also counted, on rows i >= 64 with a non-zero
+    sum_j |dS|: its share must reach ``strict_floor``, a floor per workload a little under what the
+    kernels measure (1.0 on the diffuse recipes; 0.908 on the outlier-channel recipe and 0.990-0.996 on
+    the heavy-tailed one, whose nearly one-hot rows have dS -> 0 and keep only the second term), and
+    the median of the ratio must stay under 1e-5 everywhere."""
     rs, ra, dust, lse = (got[n].double() for n in ("rs", "ra", "dust", "lse"))
     a = got["lse"].abs()
     ulp = (torch.nextafter(a, torch.full_like(a, float("inf"))) - a).double()
@@ -51,6 +57,11 @@ def _assert_row_sum_invariant_on_every_row(got):
     c = 2.0 ** -20 * torch.clamp(keys / 8192.0, min=1.0)
     ok = rs.abs() <= 1e-5 * ra + (ulp + c) * dust
     assert bool(ok.all()), f"{int((~ok).sum())} of {ok.numel()} rows break the bound"
+    rs64, ra64 = rs[..., 64:], ra[..., 64:]
+    ratio = (rs64.abs() / ra64)[ra64 > 0]
+    share = float((ratio <= 1e-5).double().mean())
+    assert share >= strict_floor, f"strict form holds on {share:.4f} of the rows, floor {strict_floor}"
+    assert float(ratio.median()) <= 1e-5
 
 
 def _check_sampled(w, tensors, got, heads, rows, col_groups, seed, prec="mxfp8"):
@@ -110,7 +121,7 @@ def test_bench_workload_full_size_sampled():
     """gqa8k_outlier: B=1, 32/8 heads, N=8192, d=128 -- the workload bench.py times."""
     w = workloads.WORKLOADS["gqa8k_outlier"]
     tensors = workloads.make_inputs(w)
-    got = _run(w, tensors)
+    got = _run(w, tensors, strict_floor=0.90)
     _check_sampled(w, tensors, got, heads=[(0, 0), (0, 13), (0, 31)], rows=48, col_groups=3, seed=1)
 
 
@@ -127,7 +138,7 @@ def test_long_context_sampled():
     65536; the kernels have no size-dependent path beyond the tile loop counts)."""
     w = workloads.WORKLOADS["long64k"].scaled(seqlen=16384, heads_q=8, heads_kv=2)
     tensors = workloads.make_inputs(w)
-    got = _run(w, tensors)
+    got = _run(w, tensors, strict_floor=0.99)
     _check_sampled(w, tensors, got, heads=[(0, 5)], rows=32, col_groups=2, seed=3)
 
 
@@ -142,7 +153,7 @@ def test_long_context_full_size_sampled():
     full = os.environ.get("ATTN_FP8_FULL_SAMPLE") == "1"
     w = workloads.WORKLOADS["long64k"]
     tensors = workloads.make_inputs(w)
-    got = _run(w, tensors)
+    got = _run(w, tensors, strict_floor=0.98)
     heads = [(0, 0), (0, 9), (0, 22), (0, 31)] if full else [(0, 0), (0, 31)]    # the cost is per sampled head
     _check_sampled(w, tensors, got, heads=heads, rows=64 if full else 32, col_groups=16 if full else 8, seed=3)
 
@@ -167,5 +178,5 @@ def test_bench_workload_bf16_mode_sampled():
     """gqa8k_outlier in BF16 mode (the reference-point configuration bench.py --precision bf16 times)."""
     w = workloads.WORKLOADS["gqa8k_outlier"]
     tensors = workloads.make_inputs(w)
-    got = _run(w, tensors, prec="bf16")
+    got = _run(w, tensors, prec="bf16", strict_floor=0.90)
     _check_sampled(w, tensors, got, heads=[(0, 6), (0, 31)], rows=32, col_groups=2, seed=6, prec="bf16")

@@ -44,3 +44,64 @@ def test_noalloc_forward_validates_like_forward():
     with pytest.raises(B.AttnFp8Error) as e:
         B.attn_fp8_fwd_noalloc(params, empty, empty, empty, torch.empty(1, device="cuda"), torch.empty(1, device="cuda"))
     assert e.value.status == 1
+
+
+def test_noalloc_forwards_on_two_streams_share_the_scratch_array():
+    """Two calls in flight at once on different streams use the same built-in array.  All they keep
+    there is the sticky status word, which a kernel only ever sets on a failure, so neither disturbs
+    the other: both outputs are bit-identical to those of the forward with a caller workspace, and the
+    status read back through the NULL workspace is clean."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=8, heads_kv=2, seqlen=1152)
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                          w.softmax_scale)
+    cases = []
+    for seed_shift in (0, 1):
+        q, k, v, _ = workloads.make_inputs(w)
+        if seed_shift:                       # a second, different problem: the same tokens in reverse order
+            q, k, v = q.flip(2).contiguous(), k.flip(2).contiguous(), v.flip(2).contiguous()
+        qq = B.attn_fp8_quantize(q.cuda(), want_col=False)
+        kq = B.attn_fp8_quantize(k.cuda(), want_col=False)
+        vq = B.attn_fp8_quantize(v.cuda(), want_row=False)
+        o_ref, lse_ref, ws = B.attn_fp8_fwd(params, qq, kq, vq)
+        B.attn_fp8_read_status(ws)
+        cases.append((qq, kq, vq, o_ref, lse_ref, torch.full_like(o_ref, float("nan")),
+                      torch.full_like(lse_ref, float("nan"))))
+    assert not torch.equal(cases[0][3], cases[1][3])
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rep in range(3):                      # alternate the streams so that launches interleave
+        for (qq, kq, vq, _, _, o, lse), st in zip(cases, streams):
+            B.attn_fp8_fwd_noalloc(params, qq, kq, vq, o, lse, stream=st)
+    for st in streams:
+        st.synchronize()
+    B.attn_fp8_read_status(None)
+    for i, (_, _, _, o_ref, lse_ref, o, lse) in enumerate(cases):
+        assert torch.equal(o, o_ref), f"stream {i}: O differs"
+        assert torch.equal(lse, lse_ref), f"stream {i}: LSE differs"
+
+
+def test_status_of_the_builtin_scratch_is_readable_and_clears():
+    """The NULL workspace names the built-in array in attn_fp8_selftest_timeout and attn_fp8_read_status:
+    a bounded wait that runs out there is reported once, the word is clear afterwards, and the no-alloc
+    forward still produces the reference result."""
+    from paper_2609_37852_b200 import binding as B
+    w = workloads.WORKLOADS["gqa4k"].scaled(batch=1, heads_q=4, heads_kv=2, seqlen=384)
+    q, k, v, _ = workloads.make_inputs(w)
+    params = B.AttnParams(w.batch, w.seqlen, w.heads_q, w.heads_kv, w.head_dim_qk, w.head_dim_v, w.causal,
+                          w.softmax_scale)
+    qq = B.attn_fp8_quantize(q.cuda(), want_col=False)
+    kq = B.attn_fp8_quantize(k.cuda(), want_col=False)
+    vq = B.attn_fp8_quantize(v.cuda(), want_row=False)
+    o_ref, lse_ref, ws = B.attn_fp8_fwd(params, qq, kq, vq)
+    B.attn_fp8_read_status(ws)
+    B.attn_fp8_read_status(None)              # clean to begin with
+    B.attn_fp8_selftest_timeout(None)
+    with pytest.raises(B.AttnFp8Error) as e:
+        B.attn_fp8_read_status(None)
+    assert e.value.status == 7          # ATTN_ERR_TIMEOUT
+    B.attn_fp8_read_status(None)              # the read that found it set has cleared it
+    o, lse = torch.empty_like(o_ref), torch.empty_like(lse_ref)
+    B.attn_fp8_fwd_noalloc(params, qq, kq, vq, o, lse)
+    B.attn_fp8_read_status(None)
+    assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)
