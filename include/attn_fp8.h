@@ -33,7 +33,7 @@
  *
  * Supported shapes: seqlen a multiple of 128 (Nq == Nk, causal means key j <= query i);
  * heads_q a multiple of heads_kv; head dims (qk, v): (64,64), (128,128), (192,128), (256,256) for
- * every attention entry point in FP8 mode, (64,64) and (128,128) in BF16 mode and with protected dP;
+ * every attention entry point in FP8 and in BF16 mode, (64,64) and (128,128) with protected dP;
  * the quantiser accepts any d that is a multiple of 32 up to 256.  Anything else returns
  * ATTN_ERR_UNSUPPORTED.
  *

@@ -65,10 +65,10 @@ enum Entry { kEntryFwd = 0, kEntryDelta = 1, kEntryDq = 2, kEntryDkdv = 3 };
 
 // Head-dimension pairs each kernel family is built for, per operand width.
 static bool dims_supported(int entry, int eb, int dqk, int dv) {
-  (void)entry;
+  (void)entry; (void)eb;
   const bool narrow = (dqk == 64 && dv == 64) || (dqk == 128 && dv == 128);
   const bool wide = (dqk == 192 && dv == 128) || (dqk == 256 && dv == 256);
-  return narrow || (eb == 1 && wide);
+  return narrow || wide;
 }
 
 static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entry) {

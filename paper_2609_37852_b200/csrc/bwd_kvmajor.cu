@@ -52,7 +52,7 @@ constexpr int kSmemLimit = 232448;              // dynamic shared memory a CTA m
 enum KvMode { kBoth = 0, kDvOnly = 1, kDkOnly = 2 };
 
 // Operand geometry, ring depths and tensor-memory map of one instantiation.
-template <int kEB_, int kCq_, int kCv_, int kMode_, int kEBv_ = kEB_>
+template <int kEB_, int kCq_, int kCv_, int kMode_, int kEBv_ = kEB_, int kDkTile_ = -1>
 struct KvCfg {
   static constexpr int kEB = kEB_, kCq = kCq_, kCv = kCv_, kMode = kMode_;
   static constexpr int kEBv = kEBv_;                   // bytes per element of the V / dO row operands (dP^T only):
@@ -63,6 +63,10 @@ struct KvCfg {
   static constexpr bool kHasDk = kMode != kDvOnly;     // accumulates dK (needs dP^T, D, dS^)
   static constexpr int kRq = kCq / kEB > 0 ? (kCq + kEB - 1) / kEB : 1;   // 128-row tiles of the Q^c operand (dqk / 128, rounded up)
   static constexpr int kRv = (kCv + kEBv - 1) / kEBv;                     // 128-row tiles of the dO^c operand
+  // BF16 at head dim 256: K, V and one row stage fill shared memory, so a dK pass takes one 128-column
+  // tile of dK (kDkTile = 0, 1) and the launcher runs one pass per tile
+  static constexpr int kDkTile = kDkTile_;
+  static constexpr int kRqAcc = kDkTile >= 0 ? 1 : kRq;                   // 128-row tiles of Q^c a pass accumulates into dK
   // Per query tile the CTA streams a 'row' set (Q and dO row copies, their scales, LSE, D: read by
   // the S^T / dP^T MMAs and the softmax) and a 'col' set (Q and dO column copies: read by the dV /
   // dK MMAs).  The row set is released early and gets the deeper ring, so that a reload never sits
@@ -72,10 +76,13 @@ struct KvCfg {
   static constexpr int kSubPerRow = kRowTok / kSub, kSubPerCol = kColTok / kSub;
   static constexpr int kKvBytes = (kCq + (kHasDk ? kCv : 0)) * kTile * 128;
   static constexpr int kRowBytes = (kCq + (kHasDk ? kCv : 0)) * kRowTok * 128;
-  static constexpr int kColBytes = ((kHasDk ? kRq : 0) + (kHasDv ? kRv : 0)) * kTile * 128;
-  static constexpr int kColStages = 2;
+  static constexpr int kColBytes = ((kHasDk ? kRqAcc : 0) + (kHasDv ? kRv : 0)) * kTile * 128;
+  // rings shrink to one stage where two do not fit (wide heads in BF16 mode): loads and MMAs of
+  // successive steps then no longer overlap
+  static constexpr int kColStages = kKvBytes + 2 * kRowBytes + 2 * kColBytes <= 210 * 1024 ? 2 : 1;
   static constexpr int kRowRaw = (216 * 1024 - kKvBytes - kColStages * kColBytes) / kRowBytes;
-  static constexpr int kRowStages = kRowRaw < 2 ? 2 : (kRowRaw > 3 ? 3 : kRowRaw);
+  static constexpr bool kTwoRowsFit = kKvBytes + kColStages * kColBytes + 2 * kRowBytes <= 214 * 1024;
+  static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > 3 ? 3 : kRowRaw);
   // tensor memory
   static constexpr int kOpCols = 16 * kEB;             // columns of one P^ / dS^ buffer (64 queries)
   static constexpr uint32_t kColS = 0;
@@ -84,7 +91,7 @@ struct KvCfg {
   static constexpr uint32_t kColdS = kColP + (kHasDv ? 2 * kOpCols : 0);
   static constexpr uint32_t kColdV = kColdS + (kHasDk ? 2 * kOpCols : 0);
   static constexpr uint32_t kColdK = kColdV + (kHasDv ? 128 * kRv : 0);
-  static constexpr uint32_t kColSFK = kColdK + (kHasDk ? 128 * kRq : 0);
+  static constexpr uint32_t kColSFK = kColdK + (kHasDk ? 128 * kRqAcc : 0);
   static constexpr uint32_t kColSFV = kColSFK + 4 * kCq;
   static constexpr uint32_t kColSFQ = kColSFV + (kHasDk && kFp8v ? 4 * kCv : 0);   // 2 slots
   static constexpr uint32_t kColSFdO = kColSFQ + 8 * kCq;                      // 2 slots
@@ -92,7 +99,7 @@ struct KvCfg {
   static constexpr uint32_t kColSFdS = kColSFP + (kHasDv ? 8 : 0);             // 2 x 4
   static constexpr uint32_t kColSFdOc = kColSFdS + (kHasDk ? 8 : 0);           // 2 slots x row tiles
   static constexpr uint32_t kColSFQc = kColSFdOc + (kHasDv ? 8 * kRv : 0);     // 2 slots x row tiles
-  static constexpr uint32_t kColsUsed = kFp8 ? kColSFQc + (kHasDk ? 8 * kRq : 0) : kColSFK;
+  static constexpr uint32_t kColsUsed = kFp8 ? kColSFQc + (kHasDk ? 8 * kRqAcc : 0) : kColSFK;
   static constexpr uint32_t kTmemCols = 512;
   static_assert(kColsUsed <= 512, "tensor memory exceeded");
 };
@@ -109,9 +116,9 @@ struct KvRowStage {
 };
 template <class C>
 struct KvColStage {
-  alignas(1024) uint8_t qc[C::kHasDk ? C::kRq * kTile * 128 : 16];      // Q col copy  [dqk][queries]
+  alignas(1024) uint8_t qc[C::kHasDk ? C::kRqAcc * kTile * 128 : 16];   // Q col copy  [dqk][queries]
   alignas(1024) uint8_t dOc[C::kHasDv ? C::kRv * kTile * 128 : 16];     // dO col copy [dv][queries]
-  alignas(16) uint8_t sf_qc[C::kRq * 512];
+  alignas(16) uint8_t sf_qc[C::kRqAcc * 512];
   alignas(16) uint8_t sf_dOc[C::kRv * 512];
 };
 
@@ -157,7 +164,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   // shared state space of every access derived from it (checked below)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   constexpr bool kFp8 = C::kFp8, kFp8v = C::kFp8v, kHasDv = C::kHasDv, kHasDk = C::kHasDk;
-  constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRq, kRv = C::kRv;
+  constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRqAcc, kRv = C::kRv;
   constexpr int kRowStages = C::kRowStages, kColStages = C::kColStages, kRowTok = C::kRowTok;
   constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
@@ -181,6 +188,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   const int n_qtiles = G * tiles_per_head;          // query tiles this CTA walks
   const int n_sub = 2 * n_qtiles;
   const int nk_qk = p.dqk * kEB / 32, nk_v = p.dv * C::kEBv / 32;   // 32-byte K steps of S^T and dP^T
+  // columns of dK (rows of Q^c) this pass accumulates: all of them, or one tile of 128
+  const int dk_col0 = C::kDkTile >= 0 ? 128 * C::kDkTile : 0;
+  const int dk_cols = C::kDkTile >= 0 ? min(128, p.dqk - dk_col0) : p.dqk;
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
@@ -255,10 +265,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           ok = mbar_wait(&sm.col_empty[cs], ((ci / kColStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
           KvColStage<C>& c = sm.cst[cs];
-          mbar_arrive_expect_tx(&sm.col_full[cs], (kHasDk ? p.dqk * 128 + (kFp8 ? kRq * 512 : 0) : 0) +
+          mbar_arrive_expect_tx(&sm.col_full[cs], (kHasDk ? dk_cols * 128 + (kFp8 ? kRq * 512 : 0) : 0) +
                                                       (kHasDv ? p.dv * 128 + (kFp8 ? kRv * 512 : 0) : 0));
           if (kHasDk) {
-            tma_load_2d(c.qc, &tm_qc, &sm.col_full[cs], x0, q_slab * p.dqk);
+            tma_load_2d(c.qc, &tm_qc, &sm.col_full[cs], x0, q_slab * p.dqk + dk_col0);
             if (kFp8)
               for (int r = 0; r < kRq; ++r)
                 bulk_load_1d(c.sf_qc + 512 * r, p.qc_sf + ((static_cast<size_t>(q_slab) * kRq + r) * tiles_n + it) * 512, 512,
@@ -394,7 +404,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           issue_ts<kFp8, kEB, kRv>(tmem + kColdV, tmem + kColP + kOpCols * buf, make_desc_sw128(smem_u32(st.dOc)), p.dv,
                                    sub_c, tmem + kColSFP + 4 * buf, tmem + kColSFdOc + 4 * kRv * slot, u > 0);
         if (kHasDk)
-          issue_ts<kFp8, kEB, kRq>(tmem + kColdK, tmem + kColdS + kOpCols * buf, make_desc_sw128(smem_u32(st.qc)), p.dqk,
+          issue_ts<kFp8, kEB, kRq>(tmem + kColdK, tmem + kColdS + kOpCols * buf, make_desc_sw128(smem_u32(st.qc)), dk_cols,
                                    sub_c, tmem + kColSFdS + 4 * buf, tmem + kColSFQc + 4 * kRq * slot, u > 0);
         // operands and scale bytes of this buffer may be overwritten once these MMAs have run; the
         // col stage may be refilled after its last sub-tile
@@ -539,9 +549,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       const size_t grow = static_cast<size_t>(b * p.Hkv + g) * p.N + jt * kTile + row;
       const uint32_t col = grp == 0 ? kColdV : kColdK;
       const int width = grp == 0 ? p.dv : p.dqk;
+      const int first = grp == 0 ? 0 : dk_col0, count = grp == 0 ? p.dv : dk_cols;   // columns this pass holds
       const float mul = grp == 0 ? 1.f : p.scale;
-      __nv_bfloat16* out_row = (grp == 0 ? p.dv_out : p.dk) + grow * width;
-      for (int c0 = 0; c0 < width; c0 += 32) {
+      __nv_bfloat16* out_row = (grp == 0 ? p.dv_out : p.dk) + grow * width + first;
+      for (int c0 = 0; c0 < count; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem + col + lane_addr + c0, r);
         tmem_wait_ld();
@@ -577,7 +588,8 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * ebv, q_rows, C::kRowTok)) != ATTN_OK) return st;
-  if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, s.dqk)) != ATTN_OK) return st;
+  const int qc_rows = C::kDkTile >= 0 ? (s.dqk - 128 * C::kDkTile < 128 ? s.dqk - 128 * C::kDkTile : 128) : s.dqk;
+  if ((st = encode_tmap_u8_sw128(&tm_qc, q.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dqk, qc_rows)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_dOc, dO.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hq * s.dv, s.dv)) != ATTN_OK) return st;
   KvParams p;
   p.k_sf = k.row_scales; p.v_sf = v.row_scales; p.q_sf = q.row_scales; p.dO_sf = dO.row_scales;
@@ -625,6 +637,18 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
     attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
     return launch_kvmajor_t<KvCfg<1, 2, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  }
+  if (s.eb == 2 && cq == 3 && cv == 2) {
+    attn_status_t st = launch_kvmajor_t<KvCfg<2, 3, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (st != ATTN_OK) return st;
+    return launch_kvmajor_t<KvCfg<2, 3, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+  }
+  if (s.eb == 2 && cq == 4 && cv == 4) {
+    attn_status_t st = launch_kvmajor_t<KvCfg<2, 4, 4, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (st != ATTN_OK) return st;
+    st = launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 0>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    if (st != ATTN_OK) return st;
+    return launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 1>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   }
   return fail(ATTN_ERR_UNSUPPORTED, "bwd kv-major: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv,
               s.eb);

@@ -80,7 +80,10 @@ struct QmCfg {
   static constexpr int kKvBytes = (kCq + kCv) * kStep * 128;
   static constexpr int kKcBytes = kDQ ? kTile * 128 : 0;
   static constexpr int kRaw = ((kPersist ? 216 : 224) * 1024 - kFixedBytes - kKcBytes) / (kKvBytes + kKcBytes);
-  static constexpr int kStages = kRaw < 2 ? 2 : (kRaw > 4 ? 4 : kRaw);
+  // (BF16 at head dim 256: the Q / dO tiles alone take 128 KB and a K / V step 64 KB, so the ring is
+  // a single stage there: loads and MMAs of successive steps no longer overlap)
+  static constexpr bool kTwoFit = kFixedBytes + 2 * kKvBytes + kKcBytes <= 212 * 1024;
+  static constexpr int kStages = kRaw < 2 ? (kTwoFit ? 2 : 1) : (kRaw > 4 ? 4 : kRaw);
   static constexpr int kKcStages = !kDQ ? 1 : (kRaw < 2 ? 1 : kStages);
   // tensor memory
   static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* 2 x 32 */, kColdQ = 2 * kStep + 64;
@@ -102,7 +105,7 @@ struct QmSmem {
   alignas(1024) uint8_t dO[C::kQBufs][C::kCv][kTile * 128];
   alignas(1024) uint8_t k[kStages][C::kCq][C::kStep * 128];
   alignas(1024) uint8_t v[kStages][C::kCv][C::kStep * 128];
-  alignas(1024) uint8_t kc[C::kKcStages][kTile * 128];
+  alignas(1024) uint8_t kc[C::kKcStages][C::kDQ ? kTile * 128 : 1024];   // K^c tiles of the dQ product
   alignas(16) uint8_t sf_q[C::kQBufs][C::kCq * 512];
   alignas(16) uint8_t sf_dO[C::kQBufs][C::kCv * 512];
   alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
@@ -756,6 +759,8 @@ attn_status_t launch_qmajor(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t
   ATTN_QM_CASE(1, 2, 2, 1)
   ATTN_QM_CASE(2, 1, 1, 2)
   ATTN_QM_CASE(2, 2, 2, 2)
+  ATTN_QM_CASE(2, 3, 2, 2)
+  ATTN_QM_CASE(2, 4, 4, 2)
   ATTN_QM_CASE(1, 1, 1, 2)   // protected dP, d = 64
   ATTN_QM_CASE(1, 1, 2, 2)   // protected dP, d = 128
 #undef ATTN_QM_CASE

@@ -492,6 +492,8 @@ attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k,
   } else {
     if (cq == 1 && rv == 1) return launch_fwd_t<FwdCfg<2, 1, 1>>(s, q, k, v, o, lse, status, stream);
     if (cq == 2 && rv == 1) return launch_fwd_t<FwdCfg<2, 2, 1>>(s, q, k, v, o, lse, status, stream);
+    if (cq == 3 && rv == 1) return launch_fwd_t<FwdCfg<2, 3, 1>>(s, q, k, v, o, lse, status, stream);
+    if (cq == 4 && rv == 2) return launch_fwd_t<FwdCfg<2, 4, 2>>(s, q, k, v, o, lse, status, stream);
   }
   return fail(ATTN_ERR_UNSUPPORTED, "fwd: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv, s.eb);
 }

@@ -126,6 +126,9 @@ def test_backward_wide_heads_matches_oracle(name, kw):
     ("tiny", dict(causal=True, seqlen=384)),
     ("gqa4k", dict(batch=2, heads_q=4, heads_kv=2, seqlen=640)),
     ("gqa8k_outlier", dict(heads_q=4, heads_kv=1, seqlen=768)),
+    ("mla8k", dict(heads_q=4, heads_kv=2, seqlen=640)),              # (192, 128): dV and dK in separate passes
+    ("gqa8k_d256", dict(heads_q=4, heads_kv=2, seqlen=640)),         # (256, 256): dK in two column passes
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=2, seqlen=384, causal=False)),
 ])
 def test_backward_bf16_mode_matches_oracle(name, kw):
     """BF16 mode against the oracle's BF16-operand path."""

@@ -67,6 +67,9 @@ def test_small_and_extreme_shapes(name, kw):
     ("gqa8k_outlier", dict(batch=3, heads_q=16, heads_kv=1, seqlen=256), False),     # 16 query heads on one KV head
     ("gqa8k_outlier", dict(batch=3, heads_q=6, heads_kv=3, seqlen=640), True),       # BF16 mode, outlier scores: far-key
                                                                                       # probabilities below the BF16 range
+    ("mla8k", dict(batch=2, heads_q=6, heads_kv=3, seqlen=384), True),               # BF16 mode at (192, 128)
+    ("mla8k", dict(heads_q=2, heads_kv=1, seqlen=256, causal=False), True),
+    ("gqa8k_d256", dict(batch=2, heads_q=4, heads_kv=2, seqlen=384), True),          # BF16 mode at (256, 256)
 ])
 def test_shape_and_mode_combinations(name, kw, bf16):
     w = workloads.WORKLOADS[name].scaled(**kw)
@@ -137,6 +140,8 @@ def test_zero_output_gradient_gives_zero_gradients():
     ("gqa4k", dict(batch=1, heads_q=2, heads_kv=1, seqlen=256), True),
     ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=256), False),
     ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=256), False),
+    ("mla8k", dict(heads_q=2, heads_kv=2, seqlen=256), True),
+    ("gqa8k_d256", dict(heads_q=2, heads_kv=1, seqlen=256), True),
 ])
 def test_every_output_element_is_written(name, kw, bf16):
     """Outputs pre-filled with NaN: a region no CTA writes would survive the call."""
@@ -305,8 +310,7 @@ def test_random_shapes_and_modes():
         w = workloads.WORKLOADS[base].scaled(**kw)
         if w.batch * w.heads_q * w.seqlen * w.seqlen > 2 * 8 * 768 * 768:
             continue                                                    # keep the oracle's share to seconds
-        narrow = (w.head_dim_qk, w.head_dim_v) in ((64, 64), (128, 128))
-        bf16 = narrow and rnd.random() < 0.25
+        bf16 = rnd.random() < 0.25
         tensors = workloads.make_inputs(w)
         if bf16 and w.dtype != "bf16":
             tensors = tuple(x.to(torch.bfloat16) for x in tensors)

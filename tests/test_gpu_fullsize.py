@@ -180,3 +180,17 @@ def test_bench_workload_bf16_mode_sampled():
     tensors = workloads.make_inputs(w)
     got = _run(w, tensors, prec="bf16", strict_floor=0.90)
     _check_sampled(w, tensors, got, heads=[(0, 6), (0, 31)], rows=32, col_groups=2, seed=6, prec="bf16")
+
+
+def test_wide_heads_bf16_mode_sampled():
+    """The two wide-head configurations in BF16 mode at N = 8192 (their reference points): (192, 128)
+    with 4 of the 16 heads and (256, 256) with 2 query heads on one KV head, enough for every tile
+    count and pass of the full configuration."""
+    w = workloads.WORKLOADS["mla8k"].scaled(heads_q=4, heads_kv=4)
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors, prec="bf16")
+    _check_sampled(w, tensors, got, heads=[(0, 2)], rows=24, col_groups=2, seed=7, prec="bf16")
+    w = workloads.WORKLOADS["gqa8k_d256"].scaled(heads_q=2, heads_kv=1)
+    tensors = workloads.make_inputs(w)
+    got = _run(w, tensors, prec="bf16")
+    _check_sampled(w, tensors, got, heads=[(0, 1)], rows=24, col_groups=2, seed=8, prec="bf16")
