@@ -31,7 +31,8 @@
  *   - Results of quantize, fwd, bwd_delta and bwd are bitwise reproducible run to run.
  *   - Changing delta_mode changes only `delta`, dQ and dK -- never O, LSE or dV.
  *
- * Supported shapes: seqlen a multiple of 128 (Nq == Nk, causal means key j <= query i);
+ * Supported shapes: seqlen a multiple of 128 (causal means key j <= query i; a caller that holds
+ * a shard of the queries against a longer key sequence says so with seqlen_k / q_start below);
  * heads_q a multiple of heads_kv; head dims (qk, v): (64,64), (128,128), (192,128), (256,256) for
  * every attention entry point in FP8 and in BF16 mode, (64,64) and (128,128) with protected dP;
  * the quantiser accepts any d that is a multiple of 32 up to 256.  Anything else returns
@@ -81,14 +82,26 @@ typedef enum { ATTN_WS_FWD = 0, ATTN_WS_BWD_DELTA = 1, ATTN_WS_BWD = 2 } attn_ws
 
 /* Problem description shared by the attention entry points.
  * Tensors: Q, dO, O, dQ are [batch, heads_q, seqlen, dim]; K, V, dK, dV are
- * [batch, heads_kv, seqlen, dim]; LSE, delta and the diagnostics are [batch, heads_q, seqlen].
- * Query head h reads KV head h / (heads_q / heads_kv).                                        */
+ * [batch, heads_kv, seqlen_k, dim]; LSE, delta and the diagnostics are [batch, heads_q, seqlen].
+ * Query head h reads KV head h / (heads_q / heads_kv).
+ *
+ * Sequence shards (the paper's Limitations name a context-parallel exchange of FP8 K / V as the
+ * next step; this is the per-shard problem such a scheme runs).  With seqlen_k == 0 the problem is
+ * square: seqlen keys, query i at position i.  Otherwise the caller holds `seqlen` consecutive
+ * queries that start at position q_start of a sequence and `seqlen_k` keys from position 0 on:
+ * under the causal mask key j is visible to local query i iff j <= q_start + i.  seqlen_k and
+ * q_start are multiples of 128; with causal == 1, seqlen_k must equal q_start + seqlen (keys past
+ * the last query are not part of the shard's problem); with causal == 0, q_start is ignored.
+ * dK / dV are the shard's contribution for all seqlen_k keys (a sum over shards gives the
+ * gradient).  Rows of O, LSE, delta and dQ are bit-identical to those of the unsharded problem. */
 typedef struct {
   int32_t batch, seqlen, heads_q, heads_kv, head_dim_qk, head_dim_v;
   int32_t causal;          /* 0 or 1                                                          */
   float   softmax_scale;   /* multiplies the FP32 score accumulator; NOT folded into Q         */
   int32_t precision;       /* attn_precision_t                                                 */
   int32_t delta_mode;      /* attn_delta_mode_t (read by attn_fp8_bwd_delta only)              */
+  int32_t seqlen_k;        /* keys; 0 means seqlen (square problem, q_start must be 0)         */
+  int32_t q_start;         /* position of query row 0 in the key sequence                      */
 } attn_params_t;
 
 /* One quantised tensor X [B, H, N, d] (caller-allocated device memory).

@@ -50,7 +50,7 @@ class _Params(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("seqlen", ctypes.c_int32), ("heads_q", ctypes.c_int32),
                 ("heads_kv", ctypes.c_int32), ("head_dim_qk", ctypes.c_int32), ("head_dim_v", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("precision", ctypes.c_int32),
-                ("delta_mode", ctypes.c_int32)]
+                ("delta_mode", ctypes.c_int32), ("seqlen_k", ctypes.c_int32), ("q_start", ctypes.c_int32)]
 
 
 class _QTensor(ctypes.Structure):
@@ -120,10 +120,17 @@ class AttnParams:
     softmax_scale: float
     precision: int = ATTN_PREC_MXFP8
     delta_mode: int = ATTN_DELTA_MATCHED
+    seqlen_k: int = 0            # keys; 0 = seqlen (square problem)
+    q_start: int = 0             # position of query row 0 in the key sequence (a shard of the queries)
+
+    @property
+    def keys(self) -> int:
+        return self.seqlen_k or self.seqlen
 
     def c_struct(self) -> _Params:
         return _Params(self.batch, self.seqlen, self.heads_q, self.heads_kv, self.head_dim_qk, self.head_dim_v,
-                       int(self.causal), float(self.softmax_scale), self.precision, self.delta_mode)
+                       int(self.causal), float(self.softmax_scale), self.precision, self.delta_mode, self.seqlen_k,
+                       self.q_start)
 
 
 @dataclass
@@ -413,9 +420,9 @@ def attn_fp8_bwd(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO: QTe
     if dq is None:
         dq = torch.empty((B, params.heads_q, N, params.head_dim_qk), **bf)
     if dk is None:
-        dk = torch.empty((B, params.heads_kv, N, params.head_dim_qk), **bf)
+        dk = torch.empty((B, params.heads_kv, params.keys, params.head_dim_qk), **bf)
     if dv is None:
-        dv = torch.empty((B, params.heads_kv, N, params.head_dim_v), **bf)
+        dv = torch.empty((B, params.heads_kv, params.keys, params.head_dim_v), **bf)
     rs = ra = None
     if diagnostics:
         rs = torch.empty((B, params.heads_q, N), dtype=torch.float32, device=dev)
@@ -498,9 +505,9 @@ def attn_fp8_bwd_dkdv(params: AttnParams, q: QTensor, k: QTensor, v: QTensor, dO
     bf = dict(dtype=torch.bfloat16, device=dev)
     B, N = params.batch, params.seqlen
     if dk is None:
-        dk = torch.empty((B, params.heads_kv, N, params.head_dim_qk), **bf)
+        dk = torch.empty((B, params.heads_kv, params.keys, params.head_dim_qk), **bf)
     if dv is None:
-        dv = torch.empty((B, params.heads_kv, N, params.head_dim_v), **bf)
+        dv = torch.empty((B, params.heads_kv, params.keys, params.head_dim_v), **bf)
     workspace = _workspace(params, ATTN_WS_BWD, workspace, dev)
     c = params.c_struct()
     _check(_lib.attn_fp8_bwd_dkdv(ctypes.byref(c), q.c_struct(), k.c_struct(), v.c_struct(), dO.c_struct(),

@@ -81,11 +81,19 @@ static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entr
   if (p->precision != ATTN_PREC_MXFP8 && p->precision != ATTN_PREC_BF16 && p->precision != ATTN_PREC_MXFP8_PROTECTED_DP)
     return fail(ATTN_ERR_INVALID_ARG, "precision %d unknown", p->precision);
   if (p->seqlen % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen must be a multiple of 128");
+  if (p->seqlen_k < 0 || p->q_start < 0) return fail(ATTN_ERR_INVALID_ARG, "seqlen_k and q_start must not be negative");
+  if (p->seqlen_k == 0 && p->q_start != 0) return fail(ATTN_ERR_INVALID_ARG, "q_start needs seqlen_k");
+  const int seqlen_k = p->seqlen_k ? p->seqlen_k : p->seqlen;
+  const int q_start = p->causal ? p->q_start : 0;
+  if (seqlen_k % 128 || p->q_start % 128) return fail(ATTN_ERR_UNSUPPORTED, "seqlen_k and q_start must be multiples of 128");
+  if (p->causal && static_cast<long long>(q_start) + p->seqlen != seqlen_k)
+    return fail(ATTN_ERR_UNSUPPORTED, "causal shard: seqlen_k (%d) must equal q_start + seqlen (%d + %d)", seqlen_k, q_start,
+                p->seqlen);
   // the kernels form row coordinates of the [B * H * N] and [B * Hkv * d] operand views in 32-bit integers
   {
     const long long q_rows = static_cast<long long>(p->batch) * p->heads_q * p->seqlen;
     const int wide = p->head_dim_qk > p->head_dim_v ? p->head_dim_qk : p->head_dim_v;
-    const long long kv_rows = static_cast<long long>(p->batch) * p->heads_kv * (p->seqlen > wide ? p->seqlen : wide);
+    const long long kv_rows = static_cast<long long>(p->batch) * p->heads_kv * (seqlen_k > wide ? seqlen_k : wide);
     if (q_rows > 0x7fffffffLL || kv_rows > 0x7fffffffLL)
       return fail(ATTN_ERR_UNSUPPORTED, "batch * heads * seqlen = %lld exceeds the 2^31 - 1 rows a launch indexes",
                   q_rows > kv_rows ? q_rows : kv_rows);
@@ -99,7 +107,7 @@ static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entr
   if (protect && !((p->head_dim_qk == 64 && p->head_dim_v == 64) || (p->head_dim_qk == 128 && p->head_dim_v == 128)))
     return fail(ATTN_ERR_UNSUPPORTED, "protected dP is built for head dims (64,64) and (128,128)");
   *s = AttnShape{p->batch, p->seqlen, p->heads_q, p->heads_kv, p->head_dim_qk, p->head_dim_v, p->causal,
-                 p->softmax_scale, eb, protect ? 2 : eb};
+                 p->softmax_scale, eb, protect ? 2 : eb, seqlen_k, q_start / 128};
   return ATTN_OK;
 }
 
@@ -521,6 +529,7 @@ extern "C" attn_status_t attn_fp8_measure_dq_reduction(const attn_params_t* p, f
                                                         double* bytes, void* stream) {
   AttnShape s;
   CHECK(check_params(p, &s, kEntryDq));
+  if (s.Nk != s.N || s.q0t) return fail(ATTN_ERR_UNSUPPORTED, "dq reduction probe: square problems only");
   if (!ms || !bytes) return fail(ATTN_ERR_INVALID_ARG, "ms / bytes is NULL");
   CHECK(check_ptr(dq_f32, "dq_f32"));
   const size_t need = static_cast<size_t>(s.B) * s.Hq * s.N * s.dqk * sizeof(float);

@@ -151,7 +151,7 @@ struct KvParams {
   __nv_bfloat16* dk;
   __nv_bfloat16* dv_out;
   int* status;
-  int N, Hq, Hkv, dqk, dv, causal;
+  int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
   float scale, scale_log2;
 };
 
@@ -182,8 +182,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   const int jt = blockIdx.y;
   const int g = blockIdx.x, b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
-  const int tiles_n = p.N / kTile;
-  const int it0 = p.causal ? jt : 0;                // first query tile that sees these keys
+  const int tiles_n = p.N / kTile, tiles_nk = p.Nk / kTile;
+  const int it0 = p.causal ? max(jt - p.q0t, 0) : 0;   // first query tile that sees these keys
   const int tiles_per_head = tiles_n - it0;
   const int n_qtiles = G * tiles_per_head;          // query tiles this CTA walks
   const int n_sub = 2 * n_qtiles;
@@ -227,11 +227,11 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       const int kv_slab = b * p.Hkv + g;
       mbar_arrive_expect_tx(&sm.kv_full, kCq * (kTile * 128 + (kFp8 ? 512 : 0)) +
                                              (kHasDk ? kCv * (kTile * 128 + (kFp8v ? 512 : 0)) : 0));
-      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[c], &tm_k, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
-      if (kFp8) bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCq * 512, kCq * 512, &sm.kv_full);
+      for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[c], &tm_k, &sm.kv_full, 128 * c, kv_slab * p.Nk + jt * kTile);
+      if (kFp8) bulk_load_1d(sm.sf_k, p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + jt) * kCq * 512, kCq * 512, &sm.kv_full);
       if (kHasDk) {
-        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[c], &tm_v, &sm.kv_full, 128 * c, kv_slab * p.N + jt * kTile);
-        if (kFp8v) bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + jt) * kCv * 512, kCv * 512, &sm.kv_full);
+        for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[c], &tm_v, &sm.kv_full, 128 * c, kv_slab * p.Nk + jt * kTile);
+        if (kFp8v) bulk_load_1d(sm.sf_v, p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + jt) * kCv * 512, kCv * 512, &sm.kv_full);
       }
       int issued_row = 0, issued_col = 0;
       bool ok = true;
@@ -481,7 +481,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           }
         }
       };
-      if (p.causal && it == jt) body(std::true_type{}); else body(std::false_type{});
+      if (p.causal && it + p.q0t == jt) body(std::true_type{}); else body(std::false_type{});
       uint32_t byte_p = 0, byte_s = 0;
       float inv_p = 1.f, inv_s = 1.f;
       if (kFp8) {
@@ -546,7 +546,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     if (ok) ok = mbar_wait(&sm.done, 0, abort_flag);
     if (ok) {
       tc_fence_after_sync();
-      const size_t grow = static_cast<size_t>(b * p.Hkv + g) * p.N + jt * kTile + row;
+      const size_t grow = static_cast<size_t>(b * p.Hkv + g) * p.Nk + jt * kTile + row;
       const uint32_t col = grp == 0 ? kColdV : kColdK;
       const int width = grp == 0 ? p.dv : p.dqk;
       const int first = grp == 0 ? 0 : dk_col0, count = grp == 0 ? p.dv : dk_cols;   // columns this pass holds
@@ -583,7 +583,7 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   CUtensorMap tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc;
   attn_status_t st;
   const uint64_t eb = C::kEB, ebv = C::kEBv;
-  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
+  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.Nk;
   if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, C::kRowTok)) != ATTN_OK) return st;
@@ -596,12 +596,12 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   p.qc_sf = q.col_scales; p.dOc_sf = dO.col_scales;
   p.lse = lse; p.delta = delta;
   p.dk = static_cast<__nv_bfloat16*>(dk); p.dv_out = static_cast<__nv_bfloat16*>(dv); p.status = status;
-  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   const size_t smem = sizeof(KvSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  dim3 grid(s.Hkv, s.N / kTile, s.B);
+  dim3 grid(s.Hkv, s.Nk / kTile, s.B);
   kvmajor_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));

@@ -139,7 +139,7 @@ struct QmParams {
   float* p_abs_dp;          // optional (with rowsum): sum_j P_ij |dP^_ij|, the scale of the rounding dust of a row sum
   int* status;
   int* sched;               // ticket mode: the next item number; the host zeroes it ahead of the launch
-  int N, Hq, Hkv, dqk, dv, causal;
+  int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
   int gx, gy, gz;           // the (head x column tile, query tile, batch) grid the work items are numbered in
   int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
   float scale, scale_log2;
@@ -186,7 +186,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     it.qt = p.causal ? (p.gy - 1 - y) : y;
     it.h = x / rq; it.r_tile = x % rq; it.b = z;
     it.g = it.h / (p.Hq / p.Hkv);
-    it.n_tiles = (p.causal ? it.qt + 1 : p.N / kTile) * kEB;       // key steps
+    it.n_tiles = (p.causal ? it.qt + p.q0t + 1 : p.Nk / kTile) * kEB;       // key steps
     it.valid = true;
     return it;
   };
@@ -234,7 +234,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     if (lane == 0) {
       prefetch_tmap(&tm_q); prefetch_tmap(&tm_dO); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
       if (kDQ) prefetch_tmap(&tm_kc);
-      const int tiles_n = p.N / kTile;
+      const int tiles_n = p.N / kTile, tiles_nk = p.Nk / kTile;
       int issued_kv = 0, issued_kc = 0;
       bool ok = true;
       int T = 0;                                      // key steps of the items before this one
@@ -275,12 +275,12 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           ok = mbar_wait(&sm.kv_empty[s], (u & 1) ^ 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
-          for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
-          for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.N + t * kStep);
+          for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.Nk + t * kStep);
+          for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.Nk + t * kStep);
           if (kFp8)
-            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
           if (kFp8v)
-            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
+            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
           ++issued_kv;
           if (kDQ) {
             const int sc = gt % kKcStages;
@@ -289,7 +289,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
             tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * it.r_tile);
             if (kFp8)
-              bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + it.r_tile) * tiles_n + t) * 512, 512,
+              bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + it.r_tile) * tiles_nk + t) * 512, 512,
                            &sm.kc_full[sc]);
             ++issued_kc;
           }
@@ -498,7 +498,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       mbar_arrive(&sm.sdp_free);
       // column, inside the query tile's own key range, of this thread's first element (negative
       // before the diagonal tile)
-      const int col0 = t * kStep - qt * kTile + 32 * grp;
+      const int col0 = t * kStep - (qt + p.q0t) * kTile + 32 * grp;
       float ds[32];
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
       // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
@@ -533,7 +533,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           }
         }
       };
-      const bool diag = p.causal && t * kStep >= qt * kTile;
+      const bool diag = p.causal && t * kStep >= (qt + p.q0t) * kTile;
       if (kDQ && p.rowsum != nullptr) {
         if (diag) body(std::true_type{}, std::true_type{}); else body(std::false_type{}, std::true_type{});
       } else {
@@ -688,13 +688,13 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   CUtensorMap tm_q, tm_dO, tm_k, tm_v, tm_kc;
   attn_status_t st;
   const uint64_t eb = C::kEB, ebv = C::kEBv;
-  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.N;
+  const uint64_t q_rows = static_cast<uint64_t>(s.B) * s.Hq * s.N, kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.Nk;
   if ((st = encode_tmap_u8_sw128(&tm_q, q.row_codes, s.dqk * eb, q_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_dO, dO.row_codes, s.dv * ebv, q_rows, kTile)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_k, k.row_codes, s.dqk * eb, kv_rows, C::kStep)) != ATTN_OK) return st;
   if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, C::kStep)) != ATTN_OK) return st;
   if (kDQ) {
-    if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.N * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
+    if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.Nk * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
                                    s.dqk < 128 ? s.dqk : 128)) != ATTN_OK)
       return st;
   } else {
@@ -705,7 +705,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.kc_sf = kDQ ? k.col_scales : nullptr;
   p.lse = lse; p.delta_in = delta_in; p.delta_out = delta_out;
   p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.p_abs_dp = p_abs_dp; p.status = status;
-  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   p.tail_wait = behind_dkdv ? 1 : 0;
   p.sched = status + 4;                             // bytes 16..23 of the workspace header

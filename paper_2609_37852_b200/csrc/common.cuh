@@ -22,10 +22,12 @@ attn_status_t encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t 
                                    uint32_t box_rows);
 
 struct AttnShape {
-  int B, N, Hq, Hkv, dqk, dv, causal;
+  int B, N, Hq, Hkv, dqk, dv, causal;   // N: query rows (the length of Q, dO, O, dQ, LSE, delta)
   float scale;
   int eb;   // bytes per operand element: 1 = E4M3 codes with E8M0 block scales, 2 = BF16 without scales
   int ebv;  // the same for the row copies of dO and V, the operands of dP alone (2 with eb == 1: protected dP)
+  int Nk;   // keys (the length of K, V, dK, dV); == N unless the caller holds a shard of the queries
+  int q0t;  // 128-row tile index of query row 0 in the key sequence: key j is visible to query i iff j <= 128 * q0t + i
 };
 
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).

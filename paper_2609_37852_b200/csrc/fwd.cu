@@ -105,7 +105,7 @@ struct FwdParams {
   __nv_bfloat16* o;
   float* lse;
   int* status;
-  int N, Hq, Hkv, dqk, dv, causal;
+  int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
   float scale_log2;         // softmax_scale * log2(e)
 };
 
@@ -133,7 +133,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
   const int qt = p.causal ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y;
   const int h = blockIdx.x, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
-  const int n_tiles = p.causal ? qt + 1 : p.N / kTile;
+  const int n_tiles = p.causal ? qt + p.q0t + 1 : p.Nk / kTile;
   const int n_sub = 2 * n_tiles;
   const int n_stage_tiles = n_tiles * kEB;      // K / V stages to stream
   const int nk_qk = p.dqk * kEB / 32;           // 32-byte K steps of the score MMA
@@ -167,7 +167,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
     if (lane == 0) {
       prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
       const int q_row = (b * p.Hq + h) * p.N + qt * kTile;
-      const int tiles_n = p.N / kTile;
+      const int tiles_n = p.N / kTile, tiles_nk = p.Nk / kTile;
       mbar_arrive_expect_tx(&sm.q_full, kCq * kTile * 128 + (kFp8 ? kCq * 512 : 0));
       for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[c], &tm_q, &sm.q_full, 128 * c, q_row);
       if (kFp8)
@@ -181,9 +181,9 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         if (!ok) break;
         mbar_arrive_expect_tx(&sm.k_full[s], kCq * C::kTileKeys * 128 + (kFp8 ? kCq * 512 : 0));
         for (int c = 0; c < kCq; ++c)
-          tma_load_2d(sm.k[s][c], &tm_k, &sm.k_full[s], 128 * c, kv_slab * p.N + t * C::kTileKeys);
+          tma_load_2d(sm.k[s][c], &tm_k, &sm.k_full[s], 128 * c, kv_slab * p.Nk + t * C::kTileKeys);
         if (kFp8)
-          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * kCq * 512, kCq * 512, &sm.k_full[s]);
+          bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCq * 512, kCq * 512, &sm.k_full[s]);
         ++issued_k;
         ok = mbar_wait(&sm.v_empty[s], (u & 1) ^ 1, abort_flag);
         if (!ok) break;
@@ -191,7 +191,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
         tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
         if (kFp8)
           for (int r = 0; r < kRv; ++r)
-            bulk_load_1d(sm.sf_v[s] + 512 * r, p.v_sf + ((static_cast<size_t>(kv_slab) * kRv + r) * tiles_n + t) * 512, 512,
+            bulk_load_1d(sm.sf_v[s] + 512 * r, p.v_sf + ((static_cast<size_t>(kv_slab) * kRv + r) * tiles_nk + t) * 512, 512,
                          &sm.v_full[s]);
         ++issued_v;
       }
@@ -297,7 +297,7 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       mbar_arrive(&sm.s_free);
       // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
       float mxb[kBpt];
-      if (p.causal && t == qt) {
+      if (p.causal && t == qt + p.q0t) {
 #pragma unroll
         for (int bk = 0; bk < kBpt; ++bk) {
           const int col0 = half * kSub + 32 * (blk0 + bk);
@@ -459,15 +459,15 @@ attn_status_t launch_fwd_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t 
   constexpr int eb = C::kEB;
   st = encode_tmap_u8_sw128(&tm_q, q.row_codes, static_cast<uint64_t>(s.dqk) * eb, static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.N,
+  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.Nk,
                             C::kTileKeys);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.N) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
+  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.Nk) * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
   if (st != ATTN_OK) return st;
   FwdParams p;
   p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
   p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
-  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale_log2 = s.scale * kLog2e;
   const size_t smem = sizeof(FwdSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(fwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));

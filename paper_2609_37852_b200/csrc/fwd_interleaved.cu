@@ -117,7 +117,7 @@ struct IlParams {
   __nv_bfloat16* o;
   float* lse;
   int* status;
-  int N, Hq, Hkv, dqk, dv, causal;
+  int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
   int gx, gy, gz;           // the (head, query tile, batch) grid the work items are numbered in
   float scale_log2;         // softmax_scale * log2(e)
 };
@@ -160,7 +160,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
     it.qt = p.causal ? (p.gy - 1 - y) : y;
     it.h = x; it.b = z;
     it.g = it.h / (p.Hq / p.Hkv);
-    it.n_tiles = p.causal ? it.qt + 1 : p.N / kTile;
+    it.n_tiles = p.causal ? it.qt + p.q0t + 1 : p.Nk / kTile;
     it.n_steps = it.n_tiles * kSubPerTile;
     return it;
   };
@@ -199,7 +199,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // ------------------------------------------------------------------ producer
       if (lane == 0) {
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-        const int tiles_n = p.N / kTile;
+        const int tiles_n = p.N / kTile, tiles_nk = p.Nk / kTile;
         int issued_k = 0, issued_v = 0;
         int T = 0;                                    // key tiles of the items before this one
         bool ok = true;
@@ -221,14 +221,14 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             ok = mbar_wait(&sm.k_empty[s], (r & 1) ^ 1, abort_flag);
             if (!ok) break;
             mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
-            tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.N + t * kTile);
-            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.k_full[s]);
+            tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.Nk + t * kTile);
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * 512, 512, &sm.k_full[s]);
             ++issued_k;
             ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
             if (!ok) break;
             mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
             tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
-            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_n + t) * 512, 512, &sm.v_full[s]);
+            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * 512, 512, &sm.v_full[s]);
             ++issued_v;
           }
           T += it.n_tiles;
@@ -467,7 +467,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         mbar_arrive(&sm.s_free[w]);                // the scores are in registers: the next S of this buffer may be issued
         // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
         float mxb[kBlkT];
-        if (p.causal && t == qt) {
+        if (p.causal && t == qt + p.q0t) {
 #pragma unroll
           for (int bk = 0; bk < kBlkT; ++bk) {
             const int col0 = sub * kSW + kColsT * hf + 32 * bk;
@@ -594,14 +594,14 @@ attn_status_t launch_fwd_il_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   attn_status_t st;
   st = encode_tmap_u8_sw128(&tm_q, q.row_codes, static_cast<uint64_t>(s.dqk), static_cast<uint64_t>(s.B) * s.Hq * s.N, kTile);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk), static_cast<uint64_t>(s.B) * s.Hkv * s.N, kTile);
+  st = encode_tmap_u8_sw128(&tm_k, k.row_codes, static_cast<uint64_t>(s.dqk), static_cast<uint64_t>(s.B) * s.Hkv * s.Nk, kTile);
   if (st != ATTN_OK) return st;
-  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.N), static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
+  st = encode_tmap_u8_sw128(&tm_v, v.col_codes, static_cast<uint64_t>(s.Nk), static_cast<uint64_t>(s.B) * s.Hkv * s.dv, s.dv);
   if (st != ATTN_OK) return st;
   IlParams p;
   p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
   p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
-  p.N = s.N; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale_log2 = s.scale * kLog2e;
   const size_t smem = sizeof(IlSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(fwd_il_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
