@@ -508,6 +508,7 @@ def main():
 
     def tensor_roofline(a, name):
         return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
+                "frac_of_cublas_bf16_x2": a / peak,       # the same as frac, under the name of what the peak is
                 "frac_of_nominal_peak": a / (NOMINAL_FP8_TFLOPS / dtype_div),
                 "frac_of_clock_normalised_peak": a / clock_peak if clock_peak else None,
                 "frac_of_measured_fp8_mma_rate": a / measured_fp8 if measured_fp8 else None,
