@@ -152,6 +152,7 @@ struct KvParams {
   __nv_bfloat16* dv_out;
   int* status;
   int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
+  int tail_wait;            // launched behind another key-major pass of the same call (see launch_kvmajor_t)
   float scale, scale_log2;
 };
 
@@ -573,12 +574,22 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
   if (tid == 0 && sm.abort_flag) atomicExch(p.status, static_cast<int>(ATTN_ERR_TIMEOUT));
+  // This grid may have started while the pass ahead of it was draining.  One CTA, the last in launch
+  // order, stays until that grid has completed, so that the completion of this grid implies the
+  // completion of both for whatever follows in the stream.
+  if (p.tail_wait && tid == 0 && blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1 && blockIdx.z == gridDim.z - 1)
+    griddep_wait();
 }
 
+// `behind`: the launch follows another key-major pass of the same call, which writes another output
+// (dV or dK, or another column tile of dK) from the same inputs.  With few KV heads a pass has fewer
+// CTAs than the GPU has SMs, or a long tail behind its heaviest CTAs; programmatic stream serialisation
+// lets this pass's CTAs take the SMs the pass ahead leaves idle (every key-major CTA executes
+// griddepcontrol.launch_dependents once set up).
 template <class C>
 attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, attn_qtensor_t dO,
                                const float* lse, const float* delta, void* dk, void* dv, int* status,
-                               cudaStream_t stream) {
+                               cudaStream_t stream, bool behind = false) {
   static_assert(sizeof(KvSmem<C>) + 1024 <= kSmemLimit, "shared memory exceeded");
   CUtensorMap tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc;
   attn_status_t st;
@@ -598,11 +609,23 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   p.dk = static_cast<__nv_bfloat16*>(dk); p.dv_out = static_cast<__nv_bfloat16*>(dv); p.status = status;
   p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
+  p.tail_wait = behind ? 1 : 0;
   const size_t smem = sizeof(KvSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(kvmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   dim3 grid(s.Hkv, s.Nk / kTile, s.B);
-  kvmajor_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
+  if (behind) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kvmajor_kernel<C>, p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
+    if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));
+  } else {
+    kvmajor_kernel<C><<<grid, kThreads, smem, stream>>>(p, tm_k, tm_v, tm_q, tm_dO, tm_qc, tm_dOc);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd kv-major: launch: %s", cudaGetErrorString(e));
   return ATTN_OK;
@@ -627,28 +650,29 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
     return launch_kvmajor_t<KvCfg<2, 1, 1, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   if (s.eb == 2 && cq == 2 && cv == 2)
     return launch_kvmajor_t<KvCfg<2, 2, 2, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
-  // qk head dim above 128: dV and dK do not fit in tensor memory together; one pass each
+  // qk head dim above 128: dV and dK do not fit in tensor memory together; one pass each, the
+  // heavier dK pass first and the dV pass launched behind it (see launch_kvmajor_t)
   if (s.eb == 1 && cq == 2 && cv == 1) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 1, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 1, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<1, 2, 1, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    return launch_kvmajor_t<KvCfg<1, 2, 1, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
   }
   if (s.eb == 1 && cq == 2 && cv == 2) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<1, 2, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    return launch_kvmajor_t<KvCfg<1, 2, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
   }
   if (s.eb == 2 && cq == 3 && cv == 2) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<2, 3, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    attn_status_t st = launch_kvmajor_t<KvCfg<2, 3, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<2, 3, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    return launch_kvmajor_t<KvCfg<2, 3, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
   }
   if (s.eb == 2 && cq == 4 && cv == 4) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<2, 4, 4, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    attn_status_t st = launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 0>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
-    st = launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 0>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    st = launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 1>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
     if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 1>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
+    return launch_kvmajor_t<KvCfg<2, 4, 4, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
   }
   return fail(ATTN_ERR_UNSUPPORTED, "bwd kv-major: no kernel for head dims (%d, %d) at %d bytes per element", s.dqk, s.dv,
               s.eb);
