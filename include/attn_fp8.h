@@ -93,7 +93,16 @@ typedef enum { ATTN_WS_FWD = 0, ATTN_WS_BWD_DELTA = 1, ATTN_WS_BWD = 2 } attn_ws
  * q_start are multiples of 128; with causal == 1, seqlen_k must equal q_start + seqlen (keys past
  * the last query are not part of the shard's problem); with causal == 0, q_start is ignored.
  * dK / dV are the shard's contribution for all seqlen_k keys (a sum over shards gives the
- * gradient).  Rows of O, LSE, delta and dQ are bit-identical to those of the unsharded problem. */
+ * gradient).  Rows of O, LSE, delta and dQ are bit-identical to those of the unsharded problem.
+ *
+ * Ragged lengths.  Tensors are always allocated, and quantised, at a multiple of 128 tokens: a caller
+ * with fewer tokens pads Q, K, V and dO with zero rows (zero blocks quantise to zero codes, and a
+ * partly filled 32-token block takes the scale of its real tokens).  keys_valid says how many of the
+ * seqlen_k keys are real (0: all of them; otherwise seqlen_k - 128 < keys_valid <= seqlen_k): without
+ * the causal mask the keys from keys_valid on are masked out of every row; under the causal mask real
+ * queries never see them, and keys_valid is not needed.  Rows of the outputs that belong to padded
+ * queries hold finite values the caller ignores; because their dO rows are zero they add nothing to
+ * dK and dV, and the dK / dV rows of padded keys come out as zeros.                               */
 typedef struct {
   int32_t batch, seqlen, heads_q, heads_kv, head_dim_qk, head_dim_v;
   int32_t causal;          /* 0 or 1                                                          */
@@ -102,6 +111,7 @@ typedef struct {
   int32_t delta_mode;      /* attn_delta_mode_t (read by attn_fp8_bwd_delta only)              */
   int32_t seqlen_k;        /* keys; 0 means seqlen (square problem, q_start must be 0)         */
   int32_t q_start;         /* position of query row 0 in the key sequence                      */
+  int32_t keys_valid;      /* real keys among the seqlen_k allocated ones; 0 means all         */
 } attn_params_t;
 
 /* One quantised tensor X [B, H, N, d] (caller-allocated device memory).

@@ -50,7 +50,8 @@ class _Params(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("seqlen", ctypes.c_int32), ("heads_q", ctypes.c_int32),
                 ("heads_kv", ctypes.c_int32), ("head_dim_qk", ctypes.c_int32), ("head_dim_v", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("precision", ctypes.c_int32),
-                ("delta_mode", ctypes.c_int32), ("seqlen_k", ctypes.c_int32), ("q_start", ctypes.c_int32)]
+                ("delta_mode", ctypes.c_int32), ("seqlen_k", ctypes.c_int32), ("q_start", ctypes.c_int32),
+                ("keys_valid", ctypes.c_int32)]
 
 
 class _QTensor(ctypes.Structure):
@@ -122,6 +123,7 @@ class AttnParams:
     delta_mode: int = ATTN_DELTA_MATCHED
     seqlen_k: int = 0            # keys; 0 = seqlen (square problem)
     q_start: int = 0             # position of query row 0 in the key sequence (a shard of the queries)
+    keys_valid: int = 0          # real keys among the allocated ones (zero-padded ragged sequence); 0 = all
 
     @property
     def keys(self) -> int:
@@ -130,7 +132,7 @@ class AttnParams:
     def c_struct(self) -> _Params:
         return _Params(self.batch, self.seqlen, self.heads_q, self.heads_kv, self.head_dim_qk, self.head_dim_v,
                        int(self.causal), float(self.softmax_scale), self.precision, self.delta_mode, self.seqlen_k,
-                       self.q_start)
+                       self.q_start, self.keys_valid)
 
 
 @dataclass
@@ -153,6 +155,18 @@ def protect_dp_operand(qt: QTensor, src_bf16: torch.Tensor) -> QTensor:
     if src_bf16.dtype != torch.bfloat16 or not src_bf16.is_contiguous() or tuple(src_bf16.shape) != tuple(qt.shape):
         raise ValueError("src_bf16 must be a contiguous bfloat16 tensor of the operand's shape")
     return QTensor(shape=qt.shape, row_codes=src_bf16, row_scales=None, col_codes=qt.col_codes, col_scales=qt.col_scales)
+
+
+def pad_tokens(x: torch.Tensor, multiple: int = 128) -> torch.Tensor:
+    """``x`` [B, H, N, d] with zero rows appended up to the next multiple of ``multiple`` tokens (the form in
+    which a ragged sequence is handed to the library; see attn_params_t.keys_valid)."""
+    n = x.shape[2]
+    pad = (-n) % multiple
+    if pad == 0:
+        return x.contiguous()
+    out = torch.zeros((x.shape[0], x.shape[1], n + pad, x.shape[3]), dtype=x.dtype, device=x.device)
+    out[:, :, :n] = x
+    return out
 
 
 def attn_fp8_scale_offset(row: int, block: int, n_blocks: int) -> int:

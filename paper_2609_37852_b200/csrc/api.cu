@@ -106,8 +106,12 @@ static attn_status_t check_params(const attn_params_t* p, AttnShape* s, int entr
   const bool protect = p->precision == ATTN_PREC_MXFP8_PROTECTED_DP && entry != kEntryFwd;
   if (protect && !((p->head_dim_qk == 64 && p->head_dim_v == 64) || (p->head_dim_qk == 128 && p->head_dim_v == 128)))
     return fail(ATTN_ERR_UNSUPPORTED, "protected dP is built for head dims (64,64) and (128,128)");
+  if (p->keys_valid < 0 || p->keys_valid > seqlen_k || (p->keys_valid && p->keys_valid <= seqlen_k - 128))
+    return fail(ATTN_ERR_INVALID_ARG, "keys_valid (%d) must be 0 or lie in the last 128-key tile of seqlen_k (%d)",
+                p->keys_valid, seqlen_k);
+  const int kv_lim = p->keys_valid ? p->keys_valid - 1 - (seqlen_k - 128) : 127;
   *s = AttnShape{p->batch, p->seqlen, p->heads_q, p->heads_kv, p->head_dim_qk, p->head_dim_v, p->causal,
-                 p->softmax_scale, eb, protect ? 2 : eb, seqlen_k, q_start / 128};
+                 p->softmax_scale, eb, protect ? 2 : eb, seqlen_k, q_start / 128, kv_lim};
   return ATTN_OK;
 }
 

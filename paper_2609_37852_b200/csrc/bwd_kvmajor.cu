@@ -152,6 +152,7 @@ struct KvParams {
   __nv_bfloat16* dv_out;
   int* status;
   int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
+  int kv_lim;               // without the causal mask: last real key of the last key tile (127: all real)
   int tail_wait;            // launched behind another key-major pass of the same call (see launch_kvmajor_t)
   float scale, scale_log2;
 };
@@ -451,6 +452,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
       // bound by instruction issue, not by a pipe
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), minus1 = make_float2(-1.f, -1.f);
+      // masked sub-tiles: those of the diagonal tile under the causal mask (key `row` after query col0 + c);
+      // without it, all sub-tiles of the last key tile when the sequence ends inside it (key `row` after kv_lim)
+      const int mask_at = p.causal ? col0 : p.kv_lim, mask_step = p.causal ? 1 : 0;
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
@@ -463,9 +467,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             const int c = c4 + e;
             const float2 lv2 = e == 0 ? make_float2(l4.x, l4.y) : make_float2(l4.z, l4.w);
             float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, lv2);
-            if (kDiag) {                                      // key after the query
-              if (row > col0 + c) x2.x = -INFINITY;
-              if (row > col0 + c + 1) x2.y = -INFINITY;
+            if (kDiag) {                                      // key after the query, or after the last real key
+              if (row > mask_at + mask_step * c) x2.x = -INFINITY;
+              if (row > mask_at + mask_step * (c + 1)) x2.y = -INFINITY;
             }
             const float2 p2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
             sr[c] = __float_as_uint(p2.x);
@@ -482,7 +486,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           }
         }
       };
-      if (p.causal && it + p.q0t == jt) body(std::true_type{}); else body(std::false_type{});
+      if (p.causal ? it + p.q0t == jt : (p.kv_lim < kTile - 1 && jt == tiles_nk - 1)) body(std::true_type{});
+      else body(std::false_type{});
       uint32_t byte_p = 0, byte_s = 0;
       float inv_p = 1.f, inv_s = 1.f;
       if (kFp8) {
@@ -607,7 +612,7 @@ attn_status_t launch_kvmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtenso
   p.qc_sf = q.col_scales; p.dOc_sf = dO.col_scales;
   p.lse = lse; p.delta = delta;
   p.dk = static_cast<__nv_bfloat16*>(dk); p.dv_out = static_cast<__nv_bfloat16*>(dv); p.status = status;
-  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.kv_lim = s.kv_lim; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   p.tail_wait = behind ? 1 : 0;
   const size_t smem = sizeof(KvSmem<C>) + 1024;

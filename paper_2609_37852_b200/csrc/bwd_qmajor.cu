@@ -140,6 +140,7 @@ struct QmParams {
   int* status;
   int* sched;               // ticket mode: the next item number; the host zeroes it ahead of the launch
   int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
+  int kv_lim;               // without the causal mask: last real key of the last key tile (127: all real)
   int gx, gy, gz;           // the (head x column tile, query tile, batch) grid the work items are numbered in
   int tail_wait;            // launched behind the key-major kernel of the same call (see launch_bwd_dq)
   float scale, scale_log2;
@@ -498,7 +499,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       mbar_arrive(&sm.sdp_free);
       // column, inside the query tile's own key range, of this thread's first element (negative
       // before the diagonal tile)
-      const int col0 = t * kStep - (qt + p.q0t) * kTile + 32 * grp;
+      // (without the causal mask: inside the last key tile, where a ragged sequence ends)
+      const int col0 = t * kStep - (p.causal ? (qt + p.q0t) * kTile : p.Nk - kTile) + 32 * grp;
+      const int lim = p.causal ? row : p.kv_lim;        // last visible column
       float ds[32];
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
       // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
@@ -514,8 +517,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         for (int c = 0; c < 32; c += 2) {
           float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nl2);
           if (kDiag) {
-            if (col0 + c > row) x2.x = -INFINITY;
-            if (col0 + c + 1 > row) x2.y = -INFINITY;
+            if (col0 + c > lim) x2.x = -INFINITY;
+            if (col0 + c + 1 > lim) x2.y = -INFINITY;
           }
           const float2 pr2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
           const float2 dp2 = make_float2(__uint_as_float(dpr[c]), __uint_as_float(dpr[c + 1]));
@@ -533,7 +536,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           }
         }
       };
-      const bool diag = p.causal && t * kStep >= (qt + p.q0t) * kTile;
+      const bool diag = p.causal ? t * kStep >= (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 && t * kStep >= p.Nk - kTile);
       if (kDQ && p.rowsum != nullptr) {
         if (diag) body(std::true_type{}, std::true_type{}); else body(std::false_type{}, std::true_type{});
       } else {
@@ -705,7 +708,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   p.kc_sf = kDQ ? k.col_scales : nullptr;
   p.lse = lse; p.delta_in = delta_in; p.delta_out = delta_out;
   p.dq = static_cast<__nv_bfloat16*>(dq); p.rowsum = rowsum; p.rowabs = rowabs; p.post_rowsum = post_rowsum; p.post_rowabs = post_rowabs; p.p_abs_dp = p_abs_dp; p.status = status;
-  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.kv_lim = s.kv_lim; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale = s.scale; p.scale_log2 = s.scale * kLog2e;
   p.tail_wait = behind_dkdv ? 1 : 0;
   p.sched = status + 4;                             // bytes 16..23 of the workspace header

@@ -28,6 +28,7 @@ struct AttnShape {
   int ebv;  // the same for the row copies of dO and V, the operands of dP alone (2 with eb == 1: protected dP)
   int Nk;   // keys (the length of K, V, dK, dV); == N unless the caller holds a shard of the queries
   int q0t;  // 128-row tile index of query row 0 in the key sequence: key j is visible to query i iff j <= 128 * q0t + i
+  int kv_lim;  // last real key inside the last key tile (127: the tile is full); read without the causal mask only
 };
 
 // Kernel launchers (each validates nothing: the C-ABI layer has done so).

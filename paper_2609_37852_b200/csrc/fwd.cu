@@ -106,6 +106,7 @@ struct FwdParams {
   float* lse;
   int* status;
   int N, Nk, q0t, Hq, Hkv, dqk, dv, causal;   // N query rows, Nk keys, q0t: tile offset of the causal diagonal
+  int kv_lim;               // without the causal mask: last real key of the last key tile (127: all real)
   float scale_log2;         // softmax_scale * log2(e)
 };
 
@@ -297,14 +298,16 @@ fwd_kernel(const FwdParams p, const __grid_constant__ CUtensorMap tm_q, const __
       mbar_arrive(&sm.s_free);
       // maxima of the raw accumulators per block (the scale is positive), masked on the diagonal tile
       float mxb[kBpt];
-      if (p.causal && t == qt + p.q0t) {
+      // masked tiles: the diagonal one under the causal mask, else the last one when the sequence ends inside it
+      if (p.causal ? t == qt + p.q0t : (p.kv_lim < kTile - 1 && t == n_tiles - 1)) {
+        const int lim = p.causal ? row : p.kv_lim;
 #pragma unroll
         for (int bk = 0; bk < kBpt; ++bk) {
           const int col0 = half * kSub + 32 * (blk0 + bk);
           float m = -INFINITY;
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
-            if (col0 + c > row) sv[32 * bk + c] = -INFINITY;
+            if (col0 + c > lim) sv[32 * bk + c] = -INFINITY;
             m = fmaxf(m, sv[32 * bk + c]);
           }
           mxb[bk] = m;
@@ -467,7 +470,7 @@ attn_status_t launch_fwd_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t 
   FwdParams p;
   p.q_sf = q.row_scales; p.k_sf = k.row_scales; p.v_sf = v.col_scales;
   p.o = static_cast<__nv_bfloat16*>(o); p.lse = lse; p.status = status;
-  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
+  p.N = s.N; p.Nk = s.Nk; p.q0t = s.q0t; p.kv_lim = s.kv_lim; p.Hq = s.Hq; p.Hkv = s.Hkv; p.dqk = s.dqk; p.dv = s.dv; p.causal = s.causal;
   p.scale_log2 = s.scale * kLog2e;
   const size_t smem = sizeof(FwdSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(fwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
