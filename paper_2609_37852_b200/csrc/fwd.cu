@@ -1,6 +1,6 @@
 // Forward attention (paper Appendix "Forward Probability Encoding", re-designed for tcgen05 / tensor
 // memory) for the operand widths the row-owner kernel of fwd_interleaved.cu does not cover: FP8 operands
-// at head dims above 128, and BF16 mode.
+// at v head dim 256, and BF16 mode.
 //
 // One CTA owns 128 query rows of one (batch, query head) and walks the keys up to the causal
 // diagonal, 64 keys at a time; it uses 256 of the 512 tensor-memory columns and under half of the
@@ -488,7 +488,8 @@ attn_status_t launch_fwd(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k,
                          int* status, cudaStream_t stream) {
   const int cq = (s.dqk * s.eb + 127) / 128, rv = (s.dv + 127) / 128;
   // FP8 operands at head dims up to 128: the kernel with a row-owning thread per half step (fwd_interleaved.cu)
-  if (s.eb == 1 && cq == 1 && rv == 1) return launch_fwd_interleaved(s, q, k, v, o, lse, status, stream);
+  // (and at qk head dim 192 with v head dim 128, where two chunks per Q / K row still leave tensor memory for it)
+  if (s.eb == 1 && cq <= 2 && rv == 1) return launch_fwd_interleaved(s, q, k, v, o, lse, status, stream);
   if (s.eb == 1) {
     if (cq == 2 && rv == 1) return launch_fwd_t<FwdCfg<1, 2, 1>>(s, q, k, v, o, lse, status, stream);
     if (cq == 2 && rv == 2) return launch_fwd_t<FwdCfg<1, 2, 2>>(s, q, k, v, o, lse, status, stream);

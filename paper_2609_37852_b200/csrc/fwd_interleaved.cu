@@ -1,4 +1,4 @@
-// Forward attention with block-scaled FP8 operands for head dims up to 128 (paper Appendix
+// Forward attention with block-scaled FP8 operands for v head dims up to 128 and qk head dims up to 192 (paper Appendix
 // "Forward Probability Encoding", re-designed for tcgen05 / tensor memory): the variant in which a
 // softmax thread owns a whole query row of a key step, the key steps of a query tile are dealt
 // round-robin to the softmax warpgroups, and a separate warpgroup keeps the output accumulator's
@@ -35,7 +35,6 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;          // query rows per CTA; keys per K / V tile in shared memory
-constexpr int kStages = 4;          // K ring and V ring depth
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2Hi = 0.693359375f;             // ln 2 = kLn2Hi + kLn2Lo, kLn2Hi has 8 significant bits
 constexpr float kLn2Lo = -2.12194440054690583e-4f;
@@ -56,8 +55,10 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 
-template <int kWG_, int kSW_, int kSplit_>
+template <int kWG_, int kSW_, int kSplit_, int kCq_ = 1>
 struct IlCfg {
+  static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row (2: qk head dim 192)
+  static constexpr int kStages = kCq == 1 ? 4 : 2;      // K ring and V ring depth (what shared memory holds)
   static constexpr int kWG = kWG_;                      // softmax teams == score buffers in flight
   static constexpr int kSW = kSW_;                      // keys per step (64 or 128)
   static constexpr int kSplit = kSplit_;                // threads per query row and step (each takes kSW / kSplit keys)
@@ -72,8 +73,8 @@ struct IlCfg {
   static constexpr uint32_t kColO = kWG * kSW;          // output accumulator, up to 128 columns
   static constexpr uint32_t kColP = kColO + 128;        // kWG probability buffers
   static constexpr uint32_t kColSFQ = kColP + kWG * kPCols;
-  static constexpr uint32_t kColSFK = kColSFQ + 8;      // 2 slots (Q: 2 slots)
-  static constexpr uint32_t kColSFV = kColSFK + 8;      // 2 slots
+  static constexpr uint32_t kColSFK = kColSFQ + 8 * kCq;   // 2 slots (Q: 2 slots), 4 columns per chunk
+  static constexpr uint32_t kColSFV = kColSFK + 8 * kCq;   // 2 slots
   static constexpr uint32_t kColSFP = kColSFV + 8;      // kWG x 4
   static constexpr uint32_t kColsUsed = kColSFP + 4 * kWG;
   static_assert(kColsUsed <= 512, "tensor memory exceeded");
@@ -88,11 +89,12 @@ struct IlCfg {
 
 template <class C>
 struct IlSmem {
-  alignas(1024) uint8_t q[2][kTile * 128];
-  alignas(1024) uint8_t k[kStages][kTile * 128];
+  static constexpr int kStages = C::kStages;
+  alignas(1024) uint8_t q[2][C::kCq][kTile * 128];
+  alignas(1024) uint8_t k[kStages][C::kCq][kTile * 128];
   alignas(1024) uint8_t v[kStages][kTile * 128];
-  alignas(16) uint8_t sf_q[2][512];
-  alignas(16) uint8_t sf_k[kStages][512];
+  alignas(16) uint8_t sf_q[2][C::kCq * 512];
+  alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
   alignas(16) uint8_t sf_v[kStages][512];
   alignas(16) uint8_t sf_p[C::kWG][512];
   alignas(16) uint32_t raw_sf[C::kWG][C::kSplit][kTile];    // scale bytes of a step relative to the softmax thread's shift
@@ -165,6 +167,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
     it.n_steps = it.n_tiles * kSubPerTile;
     return it;
   };
+  constexpr int kStages = C::kStages, kCq = C::kCq;
   const int nk_qk = p.dqk / 32;                 // 32-byte K steps of the score MMA
   volatile int* abort_flag = &sm.abort_flag;
 
@@ -214,16 +217,18 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             if (!ok) break;
           }
           const int q_slab = it.b * p.Hq + it.h, kv_slab = it.b * p.Hkv + it.g;
-          mbar_arrive_expect_tx(&sm.q_full[qb], kTile * 128 + 512);
-          tma_load_2d(sm.q[qb], &tm_q, &sm.q_full[qb], 0, q_slab * p.N + it.qt * kTile);
-          bulk_load_1d(sm.sf_q[qb], p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + it.qt) * 512, 512, &sm.q_full[qb]);
+          mbar_arrive_expect_tx(&sm.q_full[qb], kCq * (kTile * 128 + 512));
+          for (int c = 0; c < kCq; ++c) tma_load_2d(sm.q[qb][c], &tm_q, &sm.q_full[qb], 128 * c, q_slab * p.N + it.qt * kTile);
+          bulk_load_1d(sm.sf_q[qb], p.q_sf + (static_cast<size_t>(q_slab) * tiles_n + it.qt) * kCq * 512, kCq * 512,
+                       &sm.q_full[qb]);
           for (int t = 0; t < it.n_tiles && ok; ++t) {
             const int gt = T + t, s = gt % kStages, r = gt / kStages;
             ok = mbar_wait(&sm.k_empty[s], (r & 1) ^ 1, abort_flag);
             if (!ok) break;
-            mbar_arrive_expect_tx(&sm.k_full[s], kTile * 128 + 512);
-            tma_load_2d(sm.k[s], &tm_k, &sm.k_full[s], 0, kv_slab * p.Nk + t * kTile);
-            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * 512, 512, &sm.k_full[s]);
+            mbar_arrive_expect_tx(&sm.k_full[s], kCq * (kTile * 128 + 512));
+            for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.k_full[s], 128 * c, kv_slab * p.Nk + t * kTile);
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCq * 512, kCq * 512,
+                         &sm.k_full[s]);
             ++issued_k;
             ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
             if (!ok) break;
@@ -251,11 +256,11 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         const Item it = item_at(i);
         if (!it.valid) break;
         const int qb = i & 1;
-        const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[qb]));
+        const uint64_t desc_q = make_desc_sw128(smem_u32(sm.q[qb][0]));
         ok = mbar_wait(&sm.q_full[qb], (i >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        sf_copy_tiles<1>(tmem + kColSFQ + 4 * qb, sm.sf_q[qb]);
+        sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * qb, sm.sf_q[qb]);
         for (int u = 0; u < it.n_steps && ok; ++u) {
           const int gu = G + u, gt = T + u / kSubPerTile;
           const int sub = u % kSubPerTile, s = gt % kStages, slot = gt & 1, w = gu % kWG;
@@ -263,7 +268,7 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             ok = mbar_wait(&sm.k_full[s], (gt / kStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
-            sf_copy_tiles<1>(tmem + kColSFK + 4 * slot, sm.sf_k[s]);
+            sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
           }
           if (gu >= kWG) {
             // team w has pulled the scores of its previous step into registers
@@ -271,10 +276,10 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             if (!ok) break;
             tc_fence_after_sync();
           }
-          const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s])) + sub * (kSW * 128 / 16);
-          issue_ss<true, 1, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
-                                                                      tmem + kColSFQ + 4 * qb,
-                                                                      tmem + kColSFK + 4 * slot + kBlk * sub);
+          const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0])) + sub * (kSW * 128 / 16);
+          issue_ss<true, kCq, kSW, kTile * 128 / 16, kTile * 128 / 16>(tmem + kColS + kSW * w, desc_q, desc_k, nk_qk,
+                                                                        tmem + kColSFQ + 4 * kCq * qb,
+                                                                        tmem + kColSFK + 4 * kCq * slot + kBlk * sub);
           mma_commit_elect(&sm.s_full[w]);
           if (sub == kSubPerTile - 1) mma_commit_elect(&sm.k_empty[s]);
         }
@@ -630,6 +635,7 @@ attn_status_t launch_fwd_il_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
 // FP8 operands, head dims (64,64) and (128,128): two teams, 128-key steps, two threads per row and step.
 attn_status_t launch_fwd_interleaved(const AttnShape& s, attn_qtensor_t q, attn_qtensor_t k, attn_qtensor_t v, void* o,
                                      float* lse, int* status, cudaStream_t stream) {
+  if (s.dqk > 128) return launch_fwd_il_t<IlCfg<2, 128, 2, 2>>(s, q, k, v, o, lse, status, stream);
   return launch_fwd_il_t<IlCfg<2, 128, 2>>(s, q, k, v, o, lse, status, stream);
 }
 
