@@ -67,6 +67,14 @@ struct QmCfg {
   // start together).  The dQ kernel is launched behind the key-major kernel, so its CTAs start at
   // different times: they draw their tiles from a ticket counter in the workspace instead.
   static constexpr int kStep = kTile / kEB;             // keys per step
+  // FP8 at (192, 128): the whole dQ row (192 columns) stays in one CTA, which then runs S, dP and the
+  // softmax once per item instead of once per 128-column tile of dQ.  Tensor memory holds it exactly when
+  // the dS^ operand and every scale-factor slot are single: S 128 + dP 128 + dS^ 32 + dQ 192 + SF 32 = 512.
+  static constexpr bool kOneCta = kDQ && kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 1;
+  static constexpr int kDsBufs = kOneCta ? 1 : 2;       // dS^ operand buffers (and their scale-byte slots)
+  static constexpr int kSfSlots = kOneCta ? 1 : 2;      // scale-factor slots of the K, V and K^c stages
+  static constexpr int kKcRows = kOneCta ? 192 : 128;   // rows (dQ columns) of a K^c stage
+  static constexpr int kDqCols = kOneCta ? 192 : 128;
   static constexpr bool kPersist =
       2 * (kCq + kCv) * kTile * 128 + 2 * ((kCq + kCv) * kStep * 128 + (kDQ ? kTile * 128 : 0)) <= 216 * 1024;
   static constexpr bool kTicket = kPersist && kDQ;
@@ -78,7 +86,7 @@ struct QmCfg {
   // the K^T ring of the dQ product falls back to one stage when two do not fit
   static constexpr int kFixedBytes = kQBufs * (kCq + kCv) * kTile * 128;
   static constexpr int kKvBytes = (kCq + kCv) * kStep * 128;
-  static constexpr int kKcBytes = kDQ ? kTile * 128 : 0;
+  static constexpr int kKcBytes = kDQ ? kKcRows * 128 : 0;
   static constexpr int kRaw = ((kPersist ? 216 : 224) * 1024 - kFixedBytes - kKcBytes) / (kKvBytes + kKcBytes);
   // (BF16 at head dim 256: the Q / dO tiles alone take 128 KB and a K / V step 64 KB, so the ring is
   // a single stage there: loads and MMAs of successive steps no longer overlap)
@@ -86,14 +94,14 @@ struct QmCfg {
   static constexpr int kStages = kRaw < 2 ? (kTwoFit ? 2 : 1) : (kRaw > 4 ? 4 : kRaw);
   static constexpr int kKcStages = !kDQ ? 1 : (kRaw < 2 ? 1 : kStages);
   // tensor memory
-  static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* 2 x 32 */, kColdQ = 2 * kStep + 64;
-  static constexpr uint32_t kColSFQ = kDQ ? kColdQ + 128 : 2 * kStep;   // kQBufs slots (no dS^ / dQ columns without dQ)
+  static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* kDsBufs x 32 */, kColdQ = 2 * kStep + 32 * kDsBufs;
+  static constexpr uint32_t kColSFQ = kDQ ? kColdQ + kDqCols : 2 * kStep;   // kQBufs slots (no dS^ / dQ columns without dQ)
   static constexpr uint32_t kColSFdO = kColSFQ + 4 * kCq * kQBufs;   // kQBufs slots
-  static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv * kQBufs;   // 2 slots
-  static constexpr uint32_t kColSFV = kColSFK + 8 * kCq;     // 2 slots
-  static constexpr uint32_t kColSFdS = kColSFV + 8 * kCv;    // 2 x 4
-  static constexpr uint32_t kColSFKc = kColSFdS + 8;         // 2 x 4
-  static constexpr uint32_t kColsUsed = kFp8 ? kColSFKc + 8 : kColSFQ;
+  static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv * kQBufs;   // kSfSlots slots
+  static constexpr uint32_t kColSFV = kColSFK + 4 * kSfSlots * kCq;
+  static constexpr uint32_t kColSFdS = kColSFV + 4 * kSfSlots * kCv; // kDsBufs x 4
+  static constexpr uint32_t kColSFKc = kColSFdS + 4 * kDsBufs;       // kSfSlots x 4 (one row tile of K^c at a time)
+  static constexpr uint32_t kColsUsed = kFp8 ? kColSFKc + 4 * kSfSlots : kColSFQ;
   static constexpr uint32_t kTmemCols = 512;
   static_assert(kColsUsed <= 512, "tensor memory exceeded");
 };
@@ -105,12 +113,12 @@ struct QmSmem {
   alignas(1024) uint8_t dO[C::kQBufs][C::kCv][kTile * 128];
   alignas(1024) uint8_t k[kStages][C::kCq][C::kStep * 128];
   alignas(1024) uint8_t v[kStages][C::kCv][C::kStep * 128];
-  alignas(1024) uint8_t kc[C::kKcStages][C::kDQ ? kTile * 128 : 1024];   // K^c tiles of the dQ product
+  alignas(1024) uint8_t kc[C::kKcStages][C::kDQ ? C::kKcRows * 128 : 1024];   // K^c tiles of the dQ product
   alignas(16) uint8_t sf_q[C::kQBufs][C::kCq * 512];
   alignas(16) uint8_t sf_dO[C::kQBufs][C::kCv * 512];
   alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
   alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
-  alignas(16) uint8_t sf_kc[C::kKcStages][512];
+  alignas(16) uint8_t sf_kc[C::kKcStages][C::kOneCta ? 1024 : 512];
   alignas(16) uint8_t sf_ds[2][512];
   alignas(16) float red[C::kGroups][5][kTile];   // partial row sums of every column group
   uint64_t q_full[C::kQBufs], q_empty[C::kQBufs];
@@ -172,7 +180,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // 2n-1-c, 2n+c, ... (n CTAs, c its index): alternate rounds run backwards, so that no CTA collects
   // the heavier item of every round.  In ticket mode the producer thread draws item numbers from a
   // global counter and publishes them to the other warps through shared memory.
-  const int rq = kDQ ? (p.dqk + 127) / 128 : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
+  constexpr bool kOneCta = C::kOneCta;
+  constexpr int kDsBufs = C::kDsBufs, kSfSlots = C::kSfSlots;
+  const int rq_sf = (p.dqk + 127) / 128;                   // 128-row tiles of the K^c scale tensor
+  const int rq = (kDQ && !kOneCta) ? rq_sf : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
   const int total_items = p.gx * p.gy * p.gz;
   const int n_cta = static_cast<int>(gridDim.x);
   const int n_static = !kPersist ? 1
@@ -287,11 +298,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             const int sc = gt % kKcStages;
             ok = mbar_wait(&sm.kc_empty[sc], ((gt / kKcStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
-            mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
-            tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * it.r_tile);
-            if (kFp8)
-              bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq + it.r_tile) * tiles_nk + t) * 512, 512,
-                           &sm.kc_full[sc]);
+            if (kOneCta) {
+              mbar_arrive_expect_tx(&sm.kc_full[sc], C::kKcRows * 128 + 2 * 512);
+              tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk);
+              for (int r = 0; r < 2; ++r)
+                bulk_load_1d(sm.sf_kc[sc] + 512 * r, p.kc_sf + ((static_cast<size_t>(kv_slab) * rq_sf + r) * tiles_nk + t) * 512, 512,
+                             &sm.kc_full[sc]);
+            } else {
+              mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
+              tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk + 128 * it.r_tile);
+              if (kFp8)
+                bulk_load_1d(sm.sf_kc[sc], p.kc_sf + ((static_cast<size_t>(kv_slab) * rq_sf + it.r_tile) * tiles_nk + t) * 512, 512,
+                             &sm.kc_full[sc]);
+            }
             ++issued_kc;
           }
         }
@@ -324,17 +343,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < it.n_tiles && ok; ++t) {
           const int gt = T + t;
-          const int s = gt % kStages, slot = gt & 1;
+          const int s = gt % kStages, slot = gt % kSfSlots;
           ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
+          if (kFp8 && kSfSlots == 2) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
           if (gt > 0) {
             // the softmax threads have pulled the previous S and dP into registers
             ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
+          // a single scale slot is rewritten only now that the product that read it has been consumed
+          if (kFp8 && kSfSlots == 1) sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k[s]);
           const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
           issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, t_sfq,
                                                                           tmem + kColSFK + 4 * kCq * slot);
@@ -370,16 +391,17 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < it.n_tiles && ok; ++t) {
           const int gt = T + t;
-          const int s = gt % kStages, slot = gt & 1;
+          const int s = gt % kStages, slot = gt % kSfSlots;
           ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8v) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
+          if (kFp8v && kSfSlots == 2) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
           if (gt > 0) {
             ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
+          if (kFp8v && kSfSlots == 1) sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v[s]);
           const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
           issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, t_sfdO,
                                                                           tmem + kColSFV + 4 * kCv * slot);
@@ -405,7 +427,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         const Item it = item_at(i);
         if (!it.valid) break;
         const int n_tiles = it.n_tiles;
-        const int n_dq = min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
+        const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
         if (i > 0) {
           // the softmax threads have read the previous item's dQ out of tensor memory
           ok = mbar_wait(&sm.dq_free, (i - 1) & 1, abort_flag);
@@ -414,16 +436,30 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int gt = T + t;                       // the K^T ring and the dS^ buffers run on across items
-          const int s = gt % kKcStages, slot = gt & 1, buf = gt & 1;
+          const int s = gt % kKcStages, slot = gt % kSfSlots, buf = gt % kDsBufs;
           ok = mbar_wait(&sm.kc_full[s], (gt / kKcStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
-          ok = mbar_wait(&sm.ds_full[buf], (gt >> 1) & 1, abort_flag);
+          if (kFp8 && !kOneCta) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+          ok = mbar_wait(&sm.ds_full[buf], (gt / kDsBufs) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
           const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
+          if (kOneCta) {
+            // The 192 dQ columns are two row tiles of K^c (128 + 64), one after the other through the one
+            // scale slot: copies and MMAs of one thread run in the order issued.  The step before has
+            // completed (its commit released the single dS^ buffer this step's operand came through).
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              sf_copy_elect(tmem + kColSFKc, make_desc_sf(smem_u32(sm.sf_kc[s] + 512 * r)));
+#pragma unroll
+              for (int kb = 0; kb < 4; ++kb)
+                mma_mxf8_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
+                                  make_idesc_mxf8(128, r == 0 ? 128 : n_dq - 128, kb, kb), tmem + kColSFdS, tmem + kColSFKc,
+                                  (t > 0 || kb > 0));
+            }
+          } else
 #pragma unroll
           for (int kb = 0; kb < 4; ++kb) {
             if (kFp8)
@@ -466,7 +502,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     for (int i = 0; ok && it.valid; ++i) {
     const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
-    const int n_dq = min(128, p.dqk - 128 * r_tile);         // dQ columns of this CTA
+    const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
     const size_t grow = row_of(it);
     // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
     // to the half ulp the FP32 storage of LSE already carries
@@ -487,7 +523,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     for (int t = 0; t < n_tiles; ++t) {
       const int gt = T + t;                           // step index over all items: the dS^ buffers run on
-      const int buf = gt & 1;
+      const int buf = gt % kDsBufs;
       ok = mbar_wait(&sm.sdp_full, gt & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
@@ -581,9 +617,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           sm.red[grp][2][row] += ps;
           sm.red[grp][3][row] += pa;
         }
-        if (gt >= 2) {
-          // the dQ MMAs of step gt-2 have consumed this buffer's operand and scale bytes
-          ok = mbar_wait(&sm.ds_free[buf], ((gt - 2) >> 1) & 1, abort_flag);
+        if (gt >= kDsBufs) {
+          // the dQ MMAs of the step that last used this buffer have consumed its operand and scale bytes
+          ok = mbar_wait(&sm.ds_free[buf], ((gt - kDsBufs) / kDsBufs) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
@@ -698,7 +734,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, C::kStep)) != ATTN_OK) return st;
   if (kDQ) {
     if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.Nk * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
-                                   s.dqk < 128 ? s.dqk : 128)) != ATTN_OK)
+                                   C::kOneCta ? C::kKcRows : (s.dqk < 128 ? s.dqk : 128))) != ATTN_OK)
       return st;
   } else {
     tm_kc = tm_k;
@@ -715,7 +751,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   const size_t smem = sizeof(QmSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  const int rq = kDQ ? (s.dqk + 127) / 128 : 1;
+  const int rq = (kDQ && !C::kOneCta) ? (s.dqk + 127) / 128 : 1;
   dim3 grid(s.Hq * rq, s.N / kTile, s.B);
   p.gx = static_cast<int>(grid.x); p.gy = static_cast<int>(grid.y); p.gz = static_cast<int>(grid.z);
   if (C::kPersist) {
