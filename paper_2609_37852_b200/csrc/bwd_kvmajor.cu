@@ -82,24 +82,32 @@ struct KvCfg {
   static constexpr int kColStages = kKvBytes + 2 * kRowBytes + 2 * kColBytes <= 210 * 1024 ? 2 : 1;
   static constexpr int kRowRaw = (216 * 1024 - kKvBytes - kColStages * kColBytes) / kRowBytes;
   static constexpr bool kTwoRowsFit = kKvBytes + kColStages * kColBytes + 2 * kRowBytes <= 214 * 1024;
-  static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > 3 ? 3 : kRowRaw);
+  static constexpr int kRowCap = (kEB == 1 && kEBv == 1 && kMode_ == kBoth && kCq == 2 && kCv == 1) ? 2 : 3;   // (192,128) in one pass: shared memory
+  static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > kRowCap ? kRowCap : kRowRaw);
   // tensor memory
+  // FP8 at (192, 128) with both gradients in one pass: dV 128 + dK 192 columns beside the score tiles
+  // fill tensor memory exactly when the P^ / dS^ operands and every scale-factor slot are single and the
+  // scale columns of the two gradient products are shared (they are used one after the other by one
+  // issuing thread): 64 + 64 + 16 + 16 + 128 + 192 + SF 32 = 512.
+  static constexpr bool kTight = kFp8 && kFp8v && kMode == kBoth && kCq == 2 && kCv == 1;
+  static constexpr int kOpBufs = kTight ? 1 : 2;       // P^ / dS^ operand buffers
+  static constexpr int kSl = kTight ? 1 : 2;           // scale-factor slots per streamed stage
   static constexpr int kOpCols = 16 * kEB;             // columns of one P^ / dS^ buffer (64 queries)
   static constexpr uint32_t kColS = 0;
   static constexpr uint32_t kColdP = 64;
   static constexpr uint32_t kColP = kColdP + (kHasDk ? 64 : 0);
-  static constexpr uint32_t kColdS = kColP + (kHasDv ? 2 * kOpCols : 0);
-  static constexpr uint32_t kColdV = kColdS + (kHasDk ? 2 * kOpCols : 0);
+  static constexpr uint32_t kColdS = kColP + (kHasDv ? kOpBufs * kOpCols : 0);
+  static constexpr uint32_t kColdV = kColdS + (kHasDk ? kOpBufs * kOpCols : 0);
   static constexpr uint32_t kColdK = kColdV + (kHasDv ? 128 * kRv : 0);
-  static constexpr uint32_t kColSFK = kColdK + (kHasDk ? 128 * kRqAcc : 0);
+  static constexpr uint32_t kColSFK = kColdK + (kHasDk ? (kTight ? 192 : 128 * kRqAcc) : 0);
   static constexpr uint32_t kColSFV = kColSFK + 4 * kCq;
-  static constexpr uint32_t kColSFQ = kColSFV + (kHasDk && kFp8v ? 4 * kCv : 0);   // 2 slots
-  static constexpr uint32_t kColSFdO = kColSFQ + 8 * kCq;                      // 2 slots
-  static constexpr uint32_t kColSFP = kColSFdO + (kHasDk && kFp8v ? 8 * kCv : 0);  // 2 x 4
-  static constexpr uint32_t kColSFdS = kColSFP + (kHasDv ? 8 : 0);             // 2 x 4
-  static constexpr uint32_t kColSFdOc = kColSFdS + (kHasDk ? 8 : 0);           // 2 slots x row tiles
-  static constexpr uint32_t kColSFQc = kColSFdOc + (kHasDv ? 8 * kRv : 0);     // 2 slots x row tiles
-  static constexpr uint32_t kColsUsed = kFp8 ? kColSFQc + (kHasDk ? 8 * kRqAcc : 0) : kColSFK;
+  static constexpr uint32_t kColSFQ = kColSFV + (kHasDk && kFp8v ? 4 * kCv : 0);   // kSl slots
+  static constexpr uint32_t kColSFdO = kColSFQ + 4 * kSl * kCq;                // kSl slots
+  static constexpr uint32_t kColSFP = kColSFdO + (kHasDk && kFp8v ? 4 * kSl * kCv : 0);  // kOpBufs x 4
+  static constexpr uint32_t kColSFdS = kTight ? kColSFP : kColSFP + (kHasDv ? 8 : 0);   // kOpBufs x 4
+  static constexpr uint32_t kColSFdOc = kColSFdS + (kTight ? 4 : (kHasDk ? 8 : 0));     // kSl slots x row tiles
+  static constexpr uint32_t kColSFQc = kTight ? kColSFdOc : kColSFdOc + (kHasDv ? 8 * kRv : 0);   // kSl slots x row tiles
+  static constexpr uint32_t kColsUsed = kFp8 ? (kTight ? kColSFQc + 4 : kColSFQc + (kHasDk ? 8 * kRqAcc : 0)) : kColSFK;
   static constexpr uint32_t kTmemCols = 512;
   static_assert(kColsUsed <= 512, "tensor memory exceeded");
 };
@@ -169,6 +177,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   constexpr int kEB = C::kEB, kCq = C::kCq, kCv = C::kCv, kRq = C::kRqAcc, kRv = C::kRv;
   constexpr int kRowStages = C::kRowStages, kColStages = C::kColStages, kRowTok = C::kRowTok;
   constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
+  constexpr bool kTight = C::kTight;
+  constexpr int kOpBufs = C::kOpBufs, kSl = C::kSl;
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
                      kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
                      kColSFdO = C::kColSFdO, kColSFP = C::kColSFP, kColSFdS = C::kColSFdS, kColSFdOc = C::kColSFdOc,
@@ -307,13 +317,13 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k);
       }
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri & 1, sub_r = u % kSubPerRow;
+        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri % kSl, sub_r = u % kSubPerRow;
         KvRowStage<C>& st = sm.rst[s];
         if (sub_r == 0) {
           ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8) sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * slot, st.sf_q);
+          if (kFp8 && kSl == 2) sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * slot, st.sf_q);
         }
         if (u > 0) {
           // the team of the previous sub-tile has pulled S and dP into registers
@@ -321,6 +331,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           if (!ok) break;
           tc_fence_after_sync();
         }
+        // a single scale slot is rewritten only now that the product that read it has been consumed
+        if (kFp8 && kSl == 1 && sub_r == 0) sf_copy_tiles<kCq>(tmem + kColSFQ, st.sf_q);
         const uint64_t desc_q = make_desc_sw128(smem_u32(st.q[0])) + sub_r * (kSub * 128 / 16);
         issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColS, desc_k, desc_q, nk_qk, tmem + kColSFK, tmem + kColSFQ + 4 * kCq * slot + 2 * half);
@@ -341,7 +353,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v);
     }
     for (int u = 0; u < n_sub && ok; ++u) {
-      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri & 1, sub_r = u % kSubPerRow;
+      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri % kSl, sub_r = u % kSubPerRow;
       KvRowStage<C>& st = sm.rst[s];
       if (sub_r == 0) {
         ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
@@ -353,7 +365,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
               make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
         }
         mbar_arrive_warp(&sm.lse_ready[s]);
-        if (kFp8v && kHasDk) {
+        if (kFp8v && kHasDk && kSl == 2) {
           tc_fence_after_sync();
           sf_copy_tiles<kCv>(tmem + kColSFdO + 4 * kCv * slot, st.sf_dO);
         }
@@ -364,6 +376,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           if (!ok) break;
         }
         tc_fence_after_sync();
+        if (kFp8v && kSl == 1 && sub_r == 0) sf_copy_tiles<kCv>(tmem + kColSFdO, st.sf_dO);
         const uint64_t desc_dO = make_desc_sw128(smem_u32(st.dO[0])) + sub_r * (kSub * 128 / 16);
         issue_ss<kFp8v, kCv, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColdP, desc_v, desc_dO, nk_v, tmem + kColSFV, tmem + kColSFdO + 4 * kCv * slot + 2 * half);
@@ -380,27 +393,44 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int buf = u & 1, ci = u / kSubPerCol, s = ci % kColStages, slot = ci & 1, sub_c = u % kSubPerCol;
+        const int buf = u % kOpBufs, ci = u / kSubPerCol, s = ci % kColStages, slot = ci % kSl, sub_c = u % kSubPerCol;
         KvColStage<C>& st = sm.cst[s];
         if (sub_c == 0) {
           ok = mbar_wait(&sm.col_full[s], (ci / kColStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8) {
+          if (kFp8 && !kTight) {
             if (kHasDv) sf_copy_tiles<kRv>(tmem + kColSFdOc + 4 * kRv * slot, st.sf_dOc);
             if (kHasDk) sf_copy_tiles<kRq>(tmem + kColSFQc + 4 * kRq * slot, st.sf_qc);
           }
         }
-        ok = mbar_wait(&sm.pds_full[buf], (u >> 1) & 1, abort_flag);
+        ok = mbar_wait(&sm.pds_full[buf], (u / kOpBufs) & 1, abort_flag);
         if (!ok) break;
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
         if (u % kSubPerRow == kSubPerRow - 1 && lane == 0) mbar_arrive(&sm.row_empty[(u / kSubPerRow) % kRowStages]);
         tc_fence_after_sync();
-        if (kFp8) {
+        if (kFp8 && !kTight) {
           if (kHasDv) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
           if (kHasDk) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         }
+        if (kTight) {
+          // One operand buffer, one pair of scale slots: the scales of P^ and dO^c, the dV product, then the
+          // scales of dS^ and of each row tile of Q^c in the same columns and the dK product of that tile.
+          // Copies and MMAs of one thread run in the order issued.
+          const uint64_t desc_qc = make_desc_sw128(smem_u32(st.qc));
+          sf_copy_elect(tmem + kColSFP, make_desc_sf(smem_u32(sm.sf_p[0])));
+          sf_copy_elect(tmem + kColSFdOc, make_desc_sf(smem_u32(st.sf_dOc)));
+          issue_ts<true, 1, 1>(tmem + kColdV, tmem + kColP, make_desc_sw128(smem_u32(st.dOc)), p.dv, sub_c, tmem + kColSFP,
+                               tmem + kColSFdOc, u > 0);
+          sf_copy_elect(tmem + kColSFdS, make_desc_sf(smem_u32(sm.sf_ds[0])));
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            sf_copy_elect(tmem + kColSFQc, make_desc_sf(smem_u32(st.sf_qc + 512 * r)));
+            issue_ts<true, 1, 1>(tmem + kColdK + 128 * r, tmem + kColdS, desc_qc + r * (128 * 128 / 16), r == 0 ? 128 : dk_cols - 128,
+                                 sub_c, tmem + kColSFdS, tmem + kColSFQc, u > 0);
+          }
+        } else {
         // 64 queries = 2 (codes) or 4 (BF16) steps of 32 bytes; the B operands are taken 128 rows at a time
         if (kHasDv)
           issue_ts<kFp8, kEB, kRv>(tmem + kColdV, tmem + kColP + kOpCols * buf, make_desc_sw128(smem_u32(st.dOc)), p.dv,
@@ -408,6 +438,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (kHasDk)
           issue_ts<kFp8, kEB, kRq>(tmem + kColdK, tmem + kColdS + kOpCols * buf, make_desc_sw128(smem_u32(st.qc)), dk_cols,
                                    sub_c, tmem + kColSFdS + 4 * buf, tmem + kColSFQc + 4 * kRq * slot, u > 0);
+        }
         // operands and scale bytes of this buffer may be overwritten once these MMAs have run; the
         // col stage may be refilled after its last sub-tile
         mma_commit_elect(&sm.pds_free[buf]);
@@ -431,7 +462,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
     for (int u = team; u < n_sub; u += kTeams) {
-      const int half = u & 1, buf = u & 1, ri = u / kSubPerRow, s = ri % kRowStages;
+      const int half = u & 1, buf = u % kOpBufs, ri = u / kSubPerRow, s = ri % kRowStages;
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
@@ -494,9 +525,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (kHasDv) block_scale_finite(amax_p, byte_p, inv_p);
         if (kHasDk) block_scale_finite(max_s, byte_s, inv_s);
       }
-      if (u >= 2) {
-        // the dV / dK MMAs of sub-tile u-2 have consumed this buffer's operands and scale bytes
-        ok = mbar_wait(&sm.pds_free[buf], ((u - 2) >> 1) & 1, abort_flag);
+      if (u >= kOpBufs) {
+        // the dV / dK MMAs of the sub-tile that last used this buffer have consumed its operands and scale bytes
+        ok = mbar_wait(&sm.pds_free[buf], ((u - kOpBufs) / kOpBufs) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
@@ -657,11 +688,9 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
     return launch_kvmajor_t<KvCfg<2, 2, 2, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   // qk head dim above 128: dV and dK do not fit in tensor memory together; one pass each, the
   // heavier dK pass first and the dV pass launched behind it (see launch_kvmajor_t)
-  if (s.eb == 1 && cq == 2 && cv == 1) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 1, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
-    if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<1, 2, 1, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
-  }
+  // (at (192,128) both fit when every operand buffer and scale slot is single: KvCfg::kTight)
+  if (s.eb == 1 && cq == 2 && cv == 1)
+    return launch_kvmajor_t<KvCfg<1, 2, 1, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   if (s.eb == 1 && cq == 2 && cv == 2) {
     attn_status_t st = launch_kvmajor_t<KvCfg<1, 2, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;
