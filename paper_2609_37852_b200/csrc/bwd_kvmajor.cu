@@ -317,7 +317,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k);
       }
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri % kSl, sub_r = u % kSubPerRow;
+        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
         KvRowStage<C>& st = sm.rst[s];
         if (sub_r == 0) {
           ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
@@ -353,7 +353,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v);
     }
     for (int u = 0; u < n_sub && ok; ++u) {
-      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = ri % kSl, sub_r = u % kSubPerRow;
+      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
       KvRowStage<C>& st = sm.rst[s];
       if (sub_r == 0) {
         ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
@@ -393,7 +393,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     {
       bool ok = true;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int buf = u % kOpBufs, ci = u / kSubPerCol, s = ci % kColStages, slot = ci % kSl, sub_c = u % kSubPerCol;
+        const int buf = kOpBufs == 2 ? (u & 1) : 0, ci = u / kSubPerCol, s = ci % kColStages, slot = kSl == 2 ? (ci & 1) : 0, sub_c = u % kSubPerCol;
         KvColStage<C>& st = sm.cst[s];
         if (sub_c == 0) {
           ok = mbar_wait(&sm.col_full[s], (ci / kColStages) & 1, abort_flag);
@@ -404,7 +404,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             if (kHasDk) sf_copy_tiles<kRq>(tmem + kColSFQc + 4 * kRq * slot, st.sf_qc);
           }
         }
-        ok = mbar_wait(&sm.pds_full[buf], (u / kOpBufs) & 1, abort_flag);
+        ok = mbar_wait(&sm.pds_full[buf], (kOpBufs == 2 ? u >> 1 : u) & 1, abort_flag);
         if (!ok) break;
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
@@ -462,7 +462,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
     for (int u = team; u < n_sub; u += kTeams) {
-      const int half = u & 1, buf = u % kOpBufs, ri = u / kSubPerRow, s = ri % kRowStages;
+      const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0, ri = u / kSubPerRow, s = ri % kRowStages;
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
@@ -483,11 +483,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
       // bound by instruction issue, not by a pipe
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), minus1 = make_float2(-1.f, -1.f);
-      // masked sub-tiles: those of the diagonal tile under the causal mask (key `row` after query col0 + c);
-      // without it, all sub-tiles of the last key tile when the sequence ends inside it (key `row` after kv_lim)
-      const int mask_at = p.causal ? col0 : p.kv_lim, mask_step = p.causal ? 1 : 0;
+      // masked sub-tiles: those of the diagonal tile under the causal mask (tag 1: key `row` after query col0 + c);
+      // without it, all sub-tiles of the last key tile when the sequence ends inside it (tag 2: key `row` after kv_lim)
       auto body = [&](auto diag_tag) {
-        constexpr bool kDiag = decltype(diag_tag)::value;
+        constexpr int kDiag = decltype(diag_tag)::value;
 #pragma unroll
         for (int c4 = 0; c4 < 32; c4 += 4) {
           const float4 l4 = lds_f4(&s_lse[c4]);
@@ -498,9 +497,12 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             const int c = c4 + e;
             const float2 lv2 = e == 0 ? make_float2(l4.x, l4.y) : make_float2(l4.z, l4.w);
             float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, lv2);
-            if (kDiag) {                                      // key after the query, or after the last real key
-              if (row > mask_at + mask_step * c) x2.x = -INFINITY;
-              if (row > mask_at + mask_step * (c + 1)) x2.y = -INFINITY;
+            if (kDiag == 1) {                                 // key after the query
+              if (row > col0 + c) x2.x = -INFINITY;
+              if (row > col0 + c + 1) x2.y = -INFINITY;
+            }
+            if (kDiag == 2) {                                 // key after the last real key
+              if (row > p.kv_lim) x2.x = x2.y = -INFINITY;
             }
             const float2 p2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
             sr[c] = __float_as_uint(p2.x);
@@ -517,8 +519,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           }
         }
       };
-      if (p.causal ? it + p.q0t == jt : (p.kv_lim < kTile - 1 && jt == tiles_nk - 1)) body(std::true_type{});
-      else body(std::false_type{});
+      if (p.causal && it + p.q0t == jt) body(std::integral_constant<int, 1>{});
+      else if (__builtin_expect(!p.causal && p.kv_lim < kTile - 1 && jt == p.Nk / kTile - 1, 0)) body(std::integral_constant<int, 2>{});
+      else body(std::integral_constant<int, 0>{});
       uint32_t byte_p = 0, byte_s = 0;
       float inv_p = 1.f, inv_s = 1.f;
       if (kFp8) {
@@ -527,7 +530,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       }
       if (u >= kOpBufs) {
         // the dV / dK MMAs of the sub-tile that last used this buffer have consumed its operands and scale bytes
-        ok = mbar_wait(&sm.pds_free[buf], ((u - kOpBufs) / kOpBufs) & 1, abort_flag);
+        ok = mbar_wait(&sm.pds_free[buf], (kOpBufs == 2 ? (u - 2) >> 1 : u - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }

@@ -343,7 +343,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < it.n_tiles && ok; ++t) {
           const int gt = T + t;
-          const int s = gt % kStages, slot = gt % kSfSlots;
+          const int s = gt % kStages, slot = kSfSlots == 2 ? (gt & 1) : 0;
           ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
@@ -391,7 +391,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < it.n_tiles && ok; ++t) {
           const int gt = T + t;
-          const int s = gt % kStages, slot = gt % kSfSlots;
+          const int s = gt % kStages, slot = kSfSlots == 2 ? (gt & 1) : 0;
           ok = mbar_wait(&sm.kv_full[s], (gt / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
@@ -436,12 +436,12 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int gt = T + t;                       // the K^T ring and the dS^ buffers run on across items
-          const int s = gt % kKcStages, slot = gt % kSfSlots, buf = gt % kDsBufs;
+          const int s = gt % kKcStages, slot = kSfSlots == 2 ? (gt & 1) : 0, buf = kDsBufs == 2 ? (gt & 1) : 0;
           ok = mbar_wait(&sm.kc_full[s], (gt / kKcStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8 && !kOneCta) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
-          ok = mbar_wait(&sm.ds_full[buf], (gt / kDsBufs) & 1, abort_flag);
+          ok = mbar_wait(&sm.ds_full[buf], (kDsBufs == 2 ? gt >> 1 : gt) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
@@ -504,6 +504,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
     const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
     const size_t grow = row_of(it);
+    // first key of the masked tile (the diagonal one; without the causal mask the last one, when the sequence
+    // ends inside it) and the last visible column inside it
+    const int mask_from = p.causal ? (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 ? p.Nk - kTile : 0x7fffffff);
+    const int lim = p.causal ? row : p.kv_lim;
     // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
     // to the half ulp the FP32 storage of LSE already carries
     const float lse_nat = lse_next;
@@ -523,7 +527,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     for (int t = 0; t < n_tiles; ++t) {
       const int gt = T + t;                           // step index over all items: the dS^ buffers run on
-      const int buf = gt % kDsBufs;
+      const int buf = kDsBufs == 2 ? (gt & 1) : 0;
       ok = mbar_wait(&sm.sdp_full, gt & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
@@ -536,8 +540,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       // column, inside the query tile's own key range, of this thread's first element (negative
       // before the diagonal tile)
       // (without the causal mask: inside the last key tile, where a ragged sequence ends)
-      const int col0 = t * kStep - (p.causal ? (qt + p.q0t) * kTile : p.Nk - kTile) + 32 * grp;
-      const int lim = p.causal ? row : p.kv_lim;        // last visible column
+      const int col0 = t * kStep - mask_from + 32 * grp;
       float ds[32];
       // P = 2^(x - lo) = 2^x * f with x = S*scale*log2e - hi and f = 2^-lo folded into the factors
       // that multiply P; the causal mask only exists on the diagonal tile, so the other tiles run
@@ -572,7 +575,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           }
         }
       };
-      const bool diag = p.causal ? t * kStep >= (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 && t * kStep >= p.Nk - kTile);
+      const bool diag = t * kStep >= mask_from;
       if (kDQ && p.rowsum != nullptr) {
         if (diag) body(std::true_type{}, std::true_type{}); else body(std::false_type{}, std::true_type{});
       } else {
@@ -619,7 +622,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         }
         if (gt >= kDsBufs) {
           // the dQ MMAs of the step that last used this buffer have consumed its operand and scale bytes
-          ok = mbar_wait(&sm.ds_free[buf], ((gt - kDsBufs) / kDsBufs) & 1, abort_flag);
+          ok = mbar_wait(&sm.ds_free[buf], (kDsBufs == 2 ? (gt - 2) >> 1 : gt - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
         }
