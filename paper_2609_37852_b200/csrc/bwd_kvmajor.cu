@@ -461,6 +461,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     bool ok = true;
     int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
+    // last real key of this tile: 127 unless the sequence ends inside it and no causal mask hides the padding
+    const int key_lim = (!p.causal && jt == p.Nk / kTile - 1) ? p.kv_lim : kTile - 1;
     for (int u = team; u < n_sub; u += kTeams) {
       const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0, ri = u / kSubPerRow, s = ri % kRowStages;
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
@@ -483,10 +485,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
       // bound by instruction issue, not by a pipe
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), minus1 = make_float2(-1.f, -1.f);
-      // masked sub-tiles: those of the diagonal tile under the causal mask (tag 1: key `row` after query col0 + c);
-      // without it, all sub-tiles of the last key tile when the sequence ends inside it (tag 2: key `row` after kv_lim)
       auto body = [&](auto diag_tag) {
-        constexpr int kDiag = decltype(diag_tag)::value;
+        constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
         for (int c4 = 0; c4 < 32; c4 += 4) {
           const float4 l4 = lds_f4(&s_lse[c4]);
@@ -497,12 +497,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             const int c = c4 + e;
             const float2 lv2 = e == 0 ? make_float2(l4.x, l4.y) : make_float2(l4.z, l4.w);
             float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, lv2);
-            if (kDiag == 1) {                                 // key after the query
+            if (kDiag) {                                      // key after the query
               if (row > col0 + c) x2.x = -INFINITY;
               if (row > col0 + c + 1) x2.y = -INFINITY;
-            }
-            if (kDiag == 2) {                                 // key after the last real key
-              if (row > p.kv_lim) x2.x = x2.y = -INFINITY;
             }
             const float2 p2 = make_float2(ex2_approx(x2.x), ex2_approx(x2.y));
             sr[c] = __float_as_uint(p2.x);
@@ -519,9 +516,14 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           }
         }
       };
-      if (p.causal && it + p.q0t == jt) body(std::integral_constant<int, 1>{});
-      else if (__builtin_expect(!p.causal && p.kv_lim < kTile - 1 && jt == p.Nk / kTile - 1, 0)) body(std::integral_constant<int, 2>{});
-      else body(std::integral_constant<int, 0>{});
+      if (p.causal && it + p.q0t == jt) body(std::true_type{}); else body(std::false_type{});
+      if (__builtin_expect(row > key_lim, 0)) {
+        // a padded key of a ragged sequence (no causal mask): its probabilities and score gradients are zero
+#pragma unroll
+        for (int c = 0; c < 32; ++c) { sr[c] = 0u; dpr[c] = 0u; }
+        amax_p = 0.f;
+        max_s = 0.f;
+      }
       uint32_t byte_p = 0, byte_s = 0;
       float inv_p = 1.f, inv_s = 1.f;
       if (kFp8) {

@@ -505,9 +505,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
     const size_t grow = row_of(it);
     // first key of the masked tile (the diagonal one; without the causal mask the last one, when the sequence
-    // ends inside it) and the last visible column inside it
+    // ends inside it)
     const int mask_from = p.causal ? (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 ? p.Nk - kTile : 0x7fffffff);
-    const int lim = p.causal ? row : p.kv_lim;
     // LSE * log2(e) as an unevaluated sum hi + lo, so that rebuilding P adds no rounding of its own
     // to the half ulp the FP32 storage of LSE already carries
     const float lse_nat = lse_next;
@@ -552,6 +551,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       auto body = [&](auto diag_tag, auto stats_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
         constexpr bool kStats = decltype(stats_tag)::value;      // pre-cast row statistics requested
+        const int lim = p.causal ? row : p.kv_lim;               // last visible column of the masked tile
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           float2 x2 = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, nl2);
