@@ -461,8 +461,6 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     bool ok = true;
     int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
-    // last real key of this tile: 127 unless the sequence ends inside it and no causal mask hides the padding
-    const int key_lim = (!p.causal && jt == p.Nk / kTile - 1) ? p.kv_lim : kTile - 1;
     for (int u = team; u < n_sub; u += kTeams) {
       const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0, ri = u / kSubPerRow, s = ri % kRowStages;
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
@@ -517,7 +515,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         }
       };
       if (p.causal && it + p.q0t == jt) body(std::true_type{}); else body(std::false_type{});
-      if (__builtin_expect(row > key_lim, 0)) {
+      if (__builtin_expect(!p.causal && row > p.kv_lim && jt == p.Nk / kTile - 1, 0)) {
         // a padded key of a ragged sequence (no causal mask): its probabilities and score gradients are zero
 #pragma unroll
         for (int c = 0; c < 32; ++c) { sr[c] = 0u; dpr[c] = 0u; }

@@ -515,8 +515,13 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     const float D = d_next;
     const float f_lo = fmaf(-lse2_lo, kLn2, 1.0f);   // 2^-lo to first order (|lo| < 1e-5)
     const float fD = f_lo * D;
-    float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP; kDQ: sum dS, sum |dS|
-    float acc2 = 0.f;                                 // kDQ with statistics: sum P |dP| (without the factor f_lo)
+    float acc0 = 0.f, acc1 = 0.f;                     // kDelta: sum P dP (kDQ: used by the final sum only)
+    // kDQ with statistics: sum dS and sum |dS| live in shared memory (slots 0 and 1), a step's share added
+    // after the step, so that the common path carries no register for them
+    if (kDQ && p.rowsum) { sm.red[grp][0][row] = 0.f; sm.red[grp][1][row] = 0.f; }
+    // kDQ with statistics, on request: sum P |dP| (without the factor f_lo), kept in shared memory like the
+    // post-cast sums so that the common path carries no extra register
+    if (kDQ && p.p_abs_dp) sm.red[grp][4][row] = 0.f;
     // kDQ, on request: sum dS', sum |dS'| of the cast values, kept in shared memory so that the
     // common path carries no extra registers
     const bool want_post = kDQ && p.post_rowsum != nullptr;
@@ -548,6 +553,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nl2 = make_float2(-lse2, -lse2);
       const float2 fl2 = make_float2(f_lo, f_lo), nfd2 = make_float2(-fD, -fD);
       float2 part2 = make_float2(0.f, 0.f);
+      float a2 = 0.f;                                  // this step's share of sum P |dP| (statistics only)
+      float s0 = 0.f, s1 = 0.f;                        // ... of sum dS and sum |dS|
       auto body = [&](auto diag_tag, auto stats_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
         constexpr bool kStats = decltype(stats_tag)::value;      // pre-cast row statistics requested
@@ -566,9 +573,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             ds[c] = d2.x;
             ds[c + 1] = d2.y;
             if (kStats) {
-              acc0 += d2.x + d2.y;
-              acc1 += fabsf(d2.x) + fabsf(d2.y);
-              acc2 = fmaf(pr2.x, fabsf(dp2.x), fmaf(pr2.y, fabsf(dp2.y), acc2));
+              s0 += d2.x + d2.y;
+              s1 += fabsf(d2.x) + fabsf(d2.y);
+              a2 = fmaf(pr2.x, fabsf(dp2.x), fmaf(pr2.y, fabsf(dp2.y), a2));
             }
           } else {
             part2 = __ffma2_rn(pr2, dp2, part2);
@@ -578,6 +585,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       const bool diag = t * kStep >= mask_from;
       if (kDQ && p.rowsum != nullptr) {
         if (diag) body(std::true_type{}, std::true_type{}); else body(std::false_type{}, std::true_type{});
+        sm.red[grp][0][row] += s0;
+        sm.red[grp][1][row] += s1;
+        if (p.p_abs_dp) sm.red[grp][4][row] += a2;
       } else {
         if (diag) body(std::true_type{}, std::false_type{}); else body(std::false_type{}, std::false_type{});
       }
@@ -648,9 +658,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     // delta kernel alternates between two slots, so that the next item's partial sums do not
     // overwrite what group 0 may still be reading.
     const int si = (kPersist && !kDQ) ? (i & 1) : 0;   // the dQ kernel uses slots 0 and 1 and a barrier per item
-    sm.red[grp][si][row] = acc0;
-    if (kDQ) sm.red[grp][1][row] = acc1;
-    if (kDQ && p.p_abs_dp) sm.red[grp][4][row] = acc2 * f_lo;
+    if (!kDQ) sm.red[grp][si][row] = acc0;
+    if (kDQ && p.p_abs_dp) sm.red[grp][4][row] *= f_lo;
     named_barrier_sync(1, kSoftmaxThreads);
     if (ok && grp == 0) {
       acc0 = 0.f; acc1 = 0.f;
