@@ -316,11 +316,16 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         tc_fence_after_sync();
         sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k);
       }
+      // the row ring is walked with a running (stage, phase) pair: a division by a ring depth of 3 in every
+      // iteration is felt in the issue rate
+      int s = 0;
+      uint32_t s_phase = 0;
       for (int u = 0; u < n_sub && ok; ++u) {
-        const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
+        const int half = u & 1, ri = u / kSubPerRow, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
+        if (u > 0 && sub_r == 0 && ++s == kRowStages) { s = 0; s_phase ^= 1u; }
         KvRowStage<C>& st = sm.rst[s];
         if (sub_r == 0) {
-          ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
+          ok = mbar_wait(&sm.row_full[s], s_phase, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8 && kSl == 2) sf_copy_tiles<kCq>(tmem + kColSFQ + 4 * kCq * slot, st.sf_q);
@@ -352,11 +357,14 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tc_fence_after_sync();
       sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v);
     }
+    int s = 0;                                        // running (stage, phase) of the row ring
+    uint32_t s_phase = 0;
     for (int u = 0; u < n_sub && ok; ++u) {
-      const int half = u & 1, ri = u / kSubPerRow, s = ri % kRowStages, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
+      const int half = u & 1, ri = u / kSubPerRow, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
+      if (u > 0 && sub_r == 0 && ++s == kRowStages) { s = 0; s_phase ^= 1u; }
       KvRowStage<C>& st = sm.rst[s];
       if (sub_r == 0) {
-        ok = mbar_wait(&sm.row_full[s], (ri / kRowStages) & 1, abort_flag);
+        ok = mbar_wait(&sm.row_full[s], s_phase, abort_flag);
         if (!ok) break;
         // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
         if (4 * lane < kRowTok) {
@@ -392,6 +400,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // ------------------------------------------------------------------ dV / dK issuer
     {
       bool ok = true;
+      int rs_done = 0;                                // row stage whose queries go through the softmax next
       for (int u = 0; u < n_sub && ok; ++u) {
         const int buf = kOpBufs == 2 ? (u & 1) : 0, ci = u / kSubPerCol, s = ci % kColStages, slot = kSl == 2 ? (ci & 1) : 0, sub_c = u % kSubPerCol;
         KvColStage<C>& st = sm.cst[s];
@@ -408,7 +417,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (!ok) break;
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
-        if (u % kSubPerRow == kSubPerRow - 1 && lane == 0) mbar_arrive(&sm.row_empty[(u / kSubPerRow) % kRowStages]);
+        if (u % kSubPerRow == kSubPerRow - 1) {
+          if (lane == 0) mbar_arrive(&sm.row_empty[rs_done]);
+          if (++rs_done == kRowStages) rs_done = 0;
+        }
         tc_fence_after_sync();
         if (kFp8 && !kTight) {
           if (kHasDv) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
@@ -461,8 +473,17 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     bool ok = true;
     int it = it0;                                     // query tile of the current sub-tile (kTeams == 2: one tile per iteration)
     static_assert(kTeams == 2, "a team advances by one query tile per iteration");
+    // running (stage, phase) of the row ring: the team's first sub-tile is in row stage team / kSubPerRow and
+    // it advances by kTeams / kSubPerRow stages per iteration
+    int s = (team / kSubPerRow) % kRowStages;
+    uint32_t s_phase = ((team / kSubPerRow) / kRowStages) & 1;
     for (int u = team; u < n_sub; u += kTeams) {
-      const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0, ri = u / kSubPerRow, s = ri % kRowStages;
+      const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0;
+      if (u != team) {
+#pragma unroll
+        for (int a = 0; a < kTeams / kSubPerRow; ++a)
+          if (++s == kRowStages) { s = 0; s_phase ^= 1u; }
+      }
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
@@ -472,7 +493,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
-      ok = mbar_wait(&sm.lse_ready[s], (ri / kRowStages) & 1, abort_flag);
+      ok = mbar_wait(&sm.lse_ready[s], s_phase, abort_flag);
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
       const int st0 = (u % kSubPerRow) * kSub + 32 * grp;   // the same inside the row stage
