@@ -213,6 +213,22 @@ def residual_statistics(rs, ra, ps, dk, lse=None, dust=None):
     }
 
 
+def roofline_peaks(stage_clocks, peaks, bf16_mode, sms):
+    """Denominators of the tensor rooflines.  The kernels' durations come from the per-stage loop, so the
+    measured cuBLAS BF16 figure that applies is the one that goes with the clock that loop ran at: the burst
+    figure when the sampled SM clock stayed within 5 % of the maximum, the sustained one (taken under the
+    power cap) otherwise; doubled for FP8 (nominal ratio).  Returns (peak TFLOP/s, "burst" | "sustained",
+    clock-normalised peak or None, divisor that turns FP8 figures into those of the mode's dtype)."""
+    sc = stage_clocks
+    at_boost = bool(sc.get("sm_mhz") and sc.get("sm_max_mhz") and sc["sm_mhz"] >= 0.95 * sc["sm_max_mhz"])
+    which = "burst" if at_boost else "sustained"
+    ratio = 1.0 if bf16_mode else FP8_OVER_BF16
+    peak = peaks["bf16_" + which] * ratio
+    dtype_div = FP8_OVER_BF16 if bf16_mode else 1.0           # BF16 mode: half the FP8 rate
+    clock_peak = (2.0 * MACS_PER_CLK_PER_SM_FP8 / dtype_div * sms * sc["sm_mhz"] * 1e6 / 1e12) if sc.get("sm_mhz") else None
+    return peak, which, clock_peak, dtype_div
+
+
 def _cores_used():
     try:
         from threadpoolctl import threadpool_info
@@ -494,17 +510,9 @@ def main():
     n_qk, n_v = PRODUCTS[dominant]
     kernel_flops = pairs2 * (n_qk * w.head_dim_qk + n_v * w.head_dim_v)
     achieved = kernel_flops / (stage_ms[dominant] * 1e-3) / 1e12
-    ratio = 1.0 if bf16_mode else FP8_OVER_BF16
-    # The kernels' durations come from the per-stage loop: the denominator is the measured cuBLAS BF16
-    # figure that goes with the clock that loop ran at -- the burst one when the sampled SM clock stayed
-    # within 5 % of the maximum, the sustained one (taken under the power cap) otherwise.
     sc = stage_clocks
-    at_boost = bool(sc.get("sm_mhz") and sc.get("sm_max_mhz") and sc["sm_mhz"] >= 0.95 * sc["sm_max_mhz"])
-    which = "burst" if at_boost else "sustained"
-    peak = peaks["bf16_" + which] * ratio
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    dtype_div = FP8_OVER_BF16 if bf16_mode else 1.0           # BF16 mode: half the FP8 rate
-    clock_peak = (2.0 * MACS_PER_CLK_PER_SM_FP8 / dtype_div * sms * sc["sm_mhz"] * 1e6 / 1e12) if sc.get("sm_mhz") else None
+    peak, which, clock_peak, dtype_div = roofline_peaks(sc, peaks, bf16_mode, sms)
 
     def tensor_roofline(a, name):
         return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
