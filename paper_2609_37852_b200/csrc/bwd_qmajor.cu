@@ -503,7 +503,6 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     for (int i = 0; ok && it.valid; ++i) {
     const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
     const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
-    const size_t grow = row_of(it);
     // first key of the masked tile (the diagonal one; without the causal mask the last one, when the sequence
     // ends inside it)
     const int mask_from = p.causal ? (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 ? p.Nk - kTile : 0x7fffffff);
@@ -654,6 +653,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (kDQ) d_next = p.delta_in[row_of(nx)];
       }
     }
+    const size_t grow = row_of(it);                   // (formed here: not a register of the step loop)
     // combine the row sums of the column groups (fixed order: reproducible).  The persistent
     // delta kernel alternates between two slots, so that the next item's partial sums do not
     // overwrite what group 0 may still be reading.
