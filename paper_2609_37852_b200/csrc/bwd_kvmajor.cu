@@ -89,7 +89,8 @@ struct KvCfg {
   // fill tensor memory exactly when the P^ / dS^ operands and every scale-factor slot are single and the
   // scale columns of the two gradient products are shared (they are used one after the other by one
   // issuing thread): 64 + 64 + 16 + 16 + 128 + 192 + SF 32 = 512.
-  static constexpr bool kTight = kFp8 && kFp8v && kMode == kBoth && kCq == 2 && kCv == 1;
+  // (BF16 at the same head dims: no scale factors, 64 + 64 + 32 + 32 + 128 + 192 = 512 with single operand buffers)
+  static constexpr bool kTight = kMode == kBoth && ((kFp8 && kFp8v && kCq == 2 && kCv == 1) || (kEB == 2 && kEBv == 2 && kCq == 3 && kCv == 2));
   static constexpr int kOpBufs = kTight ? 1 : 2;       // P^ / dS^ operand buffers
   static constexpr int kSl = kTight ? 1 : 2;           // scale-factor slots per streamed stage
   static constexpr int kOpCols = 16 * kEB;             // columns of one P^ / dS^ buffer (64 queries)
@@ -426,7 +427,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           if (kHasDv) sf_copy_elect(tmem + kColSFP + 4 * buf, make_desc_sf(smem_u32(sm.sf_p[buf])));
           if (kHasDk) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
         }
-        if (kTight) {
+        if (kTight && kFp8) {
           // One operand buffer, one pair of scale slots: the scales of P^ and dO^c, the dV product, then the
           // scales of dS^ and of each row tile of Q^c in the same columns and the dK product of that tile.
           // Copies and MMAs of one thread run in the order issued.
@@ -720,11 +721,8 @@ attn_status_t launch_bwd_dkdv(const AttnShape& s, attn_qtensor_t q, attn_qtensor
     if (st != ATTN_OK) return st;
     return launch_kvmajor_t<KvCfg<1, 2, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
   }
-  if (s.eb == 2 && cq == 3 && cv == 2) {
-    attn_status_t st = launch_kvmajor_t<KvCfg<2, 3, 2, kDkOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
-    if (st != ATTN_OK) return st;
-    return launch_kvmajor_t<KvCfg<2, 3, 2, kDvOnly>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream, true);
-  }
+  if (s.eb == 2 && cq == 3 && cv == 2)
+    return launch_kvmajor_t<KvCfg<2, 3, 2, kBoth>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
   if (s.eb == 2 && cq == 4 && cv == 4) {
     attn_status_t st = launch_kvmajor_t<KvCfg<2, 4, 4, kDkOnly, 2, 0>>(s, q, k, v, dO, lse, delta, dk, dv, status, stream);
     if (st != ATTN_OK) return st;

@@ -70,7 +70,8 @@ struct QmCfg {
   // FP8 at (192, 128): the whole dQ row (192 columns) stays in one CTA, which then runs S, dP and the
   // softmax once per item instead of once per 128-column tile of dQ.  Tensor memory holds it exactly when
   // the dS^ operand and every scale-factor slot are single: S 128 + dP 128 + dS^ 32 + dQ 192 + SF 32 = 512.
-  static constexpr bool kOneCta = kDQ && kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 1;
+  // (BF16 at the same head dims has no scale factors and fits with room to spare; it takes the same path)
+  static constexpr bool kOneCta = kDQ && ((kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 1) || (kEB == 2 && kEBv == 2 && kCq == 3 && kCv == 2));
   static constexpr int kDsBufs = kOneCta ? 1 : 2;       // dS^ operand buffers (and their scale-byte slots)
   static constexpr int kSfSlots = kOneCta ? 1 : 2;      // scale-factor slots of the K, V and K^c stages
   static constexpr int kKcRows = kOneCta ? 192 : 128;   // rows (dQ columns) of a K^c stage
@@ -299,9 +300,9 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             ok = mbar_wait(&sm.kc_empty[sc], ((gt / kKcStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
             if (kOneCta) {
-              mbar_arrive_expect_tx(&sm.kc_full[sc], C::kKcRows * 128 + 2 * 512);
+              mbar_arrive_expect_tx(&sm.kc_full[sc], C::kKcRows * 128 + (kFp8 ? 2 * 512 : 0));
               tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk);
-              for (int r = 0; r < 2; ++r)
+              for (int r = 0; kFp8 && r < 2; ++r)
                 bulk_load_1d(sm.sf_kc[sc] + 512 * r, p.kc_sf + ((static_cast<size_t>(kv_slab) * rq_sf + r) * tiles_nk + t) * 512, 512,
                              &sm.kc_full[sc]);
             } else {
@@ -452,12 +453,17 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
             // completed (its commit released the single dS^ buffer this step's operand came through).
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-              sf_copy_elect(tmem + kColSFKc, make_desc_sf(smem_u32(sm.sf_kc[s] + 512 * r)));
+              if (kFp8) sf_copy_elect(tmem + kColSFKc, make_desc_sf(smem_u32(sm.sf_kc[s] + 512 * r)));
 #pragma unroll
-              for (int kb = 0; kb < 4; ++kb)
-                mma_mxf8_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
-                                  make_idesc_mxf8(128, r == 0 ? 128 : n_dq - 128, kb, kb), tmem + kColSFdS, tmem + kColSFKc,
-                                  (t > 0 || kb > 0));
+              for (int kb = 0; kb < 4; ++kb) {
+                if (kFp8)
+                  mma_mxf8_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
+                                    make_idesc_mxf8(128, r == 0 ? 128 : n_dq - 128, kb, kb), tmem + kColSFdS, tmem + kColSFKc,
+                                    (t > 0 || kb > 0));
+                else
+                  mma_bf16_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
+                                    make_idesc_bf16(128, r == 0 ? 128 : n_dq - 128), (t > 0 || kb > 0));
+              }
             }
           } else
 #pragma unroll
