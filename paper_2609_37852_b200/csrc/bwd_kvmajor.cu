@@ -372,6 +372,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
           *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
               make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
+          if (kHasDk) {                                 // and the row correction into its negative, in place
+            const float4 d = *reinterpret_cast<const float4*>(&st.delta[4 * lane]);
+            *reinterpret_cast<float4*>(&st.delta[4 * lane]) = make_float4(-d.x, -d.y, -d.z, -d.w);
+          }
         }
         mbar_arrive_warp(&sm.lse_ready[s]);
         if (kFp8v && kHasDk && kSl == 2) {
@@ -504,7 +508,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       const float* s_delta = &st.delta[st0];
       // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
       // bound by instruction issue, not by a pipe
-      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), minus1 = make_float2(-1.f, -1.f);
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
       auto body = [&](auto diag_tag) {
         constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
@@ -527,7 +531,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             amax_p = fmaxf(amax_p, fmaxf(p2.x, p2.y));
             if (kHasDk) {
               const float2 dv2 = e == 0 ? make_float2(d4.x, d4.y) : make_float2(d4.z, d4.w);
-              const float2 t2 = __ffma2_rn(dv2, minus1, make_float2(__uint_as_float(dpr[c]), __uint_as_float(dpr[c + 1])));
+              const float2 t2 = __fadd2_rn(make_float2(__uint_as_float(dpr[c]), __uint_as_float(dpr[c + 1])), dv2);   // dP - D (dv2 holds -D)
               const float2 ds2 = __fmul2_rn(p2, t2);          // dS = P (dP - D)
               dpr[c] = __float_as_uint(ds2.x);
               dpr[c + 1] = __float_as_uint(ds2.y);
