@@ -66,7 +66,11 @@ struct QmCfg {
   // once per CTA instead of once per query tile.  The delta kernel takes a static list (all its CTAs
   // start together).  The dQ kernel is launched behind the key-major kernel, so its CTAs start at
   // different times: they draw their tiles from a ticket counter in the workspace instead.
-  static constexpr int kStep = kTile / kEB;             // keys per step
+  // FP8 at (256, 256) takes 64 keys per step: the whole dQ row (256 columns) then fits in tensor memory
+  // next to S and dP (64 + 64 + 2 x 32 + 256 + 64 columns of scale factors = 512), and one CTA owns it
+  static constexpr bool kHalf = kDQ && kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 2;
+  static constexpr int kStep = kHalf ? 64 : kTile / kEB; // keys per step
+  static constexpr int kStepsPerTile = kTile / kStep;
   // FP8 at (192, 128): the whole dQ row (192 columns) stays in one CTA, which then runs S, dP and the
   // softmax once per item instead of once per 128-column tile of dQ.  Tensor memory holds it exactly when
   // the dS^ operand and every scale-factor slot are single: S 128 + dP 128 + dS^ 32 + dQ 192 + SF 32 = 512.
@@ -74,8 +78,10 @@ struct QmCfg {
   static constexpr bool kOneCta = kDQ && ((kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 1) || (kEB == 2 && kEBv == 2 && kCq == 3 && kCv == 2));
   static constexpr int kDsBufs = kOneCta ? 1 : 2;       // dS^ operand buffers (and their scale-byte slots)
   static constexpr int kSfSlots = kOneCta ? 1 : 2;      // scale-factor slots of the K, V and K^c stages
-  static constexpr int kKcRows = kOneCta ? 192 : 128;   // rows (dQ columns) of a K^c stage
-  static constexpr int kDqCols = kOneCta ? 192 : 128;
+  static constexpr bool kWhole = kOneCta || kHalf;      // one CTA holds every dQ column of its rows
+  static constexpr int kKcRows = kOneCta ? 192 : (kHalf ? 256 : 128);   // rows (dQ columns) of a K^c stage
+  static constexpr int kDqCols = kKcRows;
+  static constexpr int kKb = kStep * kEB / 32;          // 32-byte K steps of the dQ product per key step
   static constexpr bool kPersist =
       2 * (kCq + kCv) * kTile * 128 + 2 * ((kCq + kCv) * kStep * 128 + (kDQ ? kTile * 128 : 0)) <= 216 * 1024;
   static constexpr bool kTicket = kPersist && kDQ;
@@ -119,7 +125,7 @@ struct QmSmem {
   alignas(16) uint8_t sf_dO[C::kQBufs][C::kCv * 512];
   alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
   alignas(16) uint8_t sf_v[kStages][C::kCv * 512];
-  alignas(16) uint8_t sf_kc[C::kKcStages][C::kOneCta ? 1024 : 512];
+  alignas(16) uint8_t sf_kc[C::kKcStages][C::kWhole ? 1024 : 512];
   alignas(16) uint8_t sf_ds[2][512];
   alignas(16) float red[C::kGroups][5][kTile];   // partial row sums of every column group
   uint64_t q_full[C::kQBufs], q_empty[C::kQBufs];
@@ -181,10 +187,10 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // 2n-1-c, 2n+c, ... (n CTAs, c its index): alternate rounds run backwards, so that no CTA collects
   // the heavier item of every round.  In ticket mode the producer thread draws item numbers from a
   // global counter and publishes them to the other warps through shared memory.
-  constexpr bool kOneCta = C::kOneCta;
+  constexpr bool kOneCta = C::kOneCta, kHalf = C::kHalf, kWhole = C::kWhole;
   constexpr int kDsBufs = C::kDsBufs, kSfSlots = C::kSfSlots;
   const int rq_sf = (p.dqk + 127) / 128;                   // 128-row tiles of the K^c scale tensor
-  const int rq = (kDQ && !kOneCta) ? rq_sf : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
+  const int rq = (kDQ && !kWhole) ? rq_sf : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
   const int total_items = p.gx * p.gy * p.gz;
   const int n_cta = static_cast<int>(gridDim.x);
   const int n_static = !kPersist ? 1
@@ -199,7 +205,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     it.qt = p.causal ? (p.gy - 1 - y) : y;
     it.h = x / rq; it.r_tile = x % rq; it.b = z;
     it.g = it.h / (p.Hq / p.Hkv);
-    it.n_tiles = (p.causal ? it.qt + p.q0t + 1 : p.Nk / kTile) * kEB;       // key steps
+    it.n_tiles = (p.causal ? it.qt + p.q0t + 1 : p.Nk / kTile) * C::kStepsPerTile;       // key steps
     it.valid = true;
     return it;
   };
@@ -290,20 +296,22 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           mbar_arrive_expect_tx(&sm.kv_full[s], kCq * (kStep * 128 + (kFp8 ? 512 : 0)) + kCv * (kStep * 128 + (kFp8v ? 512 : 0)));
           for (int c = 0; c < kCq; ++c) tma_load_2d(sm.k[s][c], &tm_k, &sm.kv_full[s], 128 * c, kv_slab * p.Nk + t * kStep);
           for (int c = 0; c < kCv; ++c) tma_load_2d(sm.v[s][c], &tm_v, &sm.kv_full[s], 128 * c, kv_slab * p.Nk + t * kStep);
+          // (64-key steps: both halves of a key tile load the tile's scale bytes and its K^c chunk)
+          const int tt = kHalf ? t >> 1 : t;          // 128-key tile of the scale tensors / 128-byte chunk of K^c
           if (kFp8)
-            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCq * 512, kCq * 512, &sm.kv_full[s]);
+            bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + tt) * kCq * 512, kCq * 512, &sm.kv_full[s]);
           if (kFp8v)
-            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCv * 512, kCv * 512, &sm.kv_full[s]);
+            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + tt) * kCv * 512, kCv * 512, &sm.kv_full[s]);
           ++issued_kv;
           if (kDQ) {
             const int sc = gt % kKcStages;
             ok = mbar_wait(&sm.kc_empty[sc], ((gt / kKcStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
-            if (kOneCta) {
+            if (kWhole) {
               mbar_arrive_expect_tx(&sm.kc_full[sc], C::kKcRows * 128 + (kFp8 ? 2 * 512 : 0));
-              tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], t * 128, kv_slab * p.dqk);
+              tma_load_2d(sm.kc[sc], &tm_kc, &sm.kc_full[sc], tt * 128, kv_slab * p.dqk);
               for (int r = 0; kFp8 && r < 2; ++r)
-                bulk_load_1d(sm.sf_kc[sc] + 512 * r, p.kc_sf + ((static_cast<size_t>(kv_slab) * rq_sf + r) * tiles_nk + t) * 512, 512,
+                bulk_load_1d(sm.sf_kc[sc] + 512 * r, p.kc_sf + ((static_cast<size_t>(kv_slab) * rq_sf + r) * tiles_nk + tt) * 512, 512,
                              &sm.kc_full[sc]);
             } else {
               mbar_arrive_expect_tx(&sm.kc_full[sc], min(128, p.dqk) * 128 + (kFp8 ? 512 : 0));
@@ -359,7 +367,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           if (kFp8 && kSfSlots == 1) sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k[s]);
           const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
           issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, t_sfq,
-                                                                          tmem + kColSFK + 4 * kCq * slot);
+                                                                          tmem + kColSFK + 4 * kCq * slot + (kHalf ? 2 * (t & 1) : 0));
           mma_commit_elect(&sm.sdp_full);
           mma_commit_elect(&sm.kv_empty[s]);
         }
@@ -405,7 +413,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           if (kFp8v && kSfSlots == 1) sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v[s]);
           const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
           issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, t_sfdO,
-                                                                          tmem + kColSFV + 4 * kCv * slot);
+                                                                          tmem + kColSFV + 4 * kCv * slot + (kHalf ? 2 * (t & 1) : 0));
           mma_commit_elect(&sm.sdp_full);
           mma_commit_elect(&sm.kv_empty[s]);
         }
@@ -428,7 +436,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
         const Item it = item_at(i);
         if (!it.valid) break;
         const int n_tiles = it.n_tiles;
-        const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
+        const int n_dq = kWhole ? p.dqk : min(128, p.dqk - 128 * it.r_tile);   // dQ columns of this CTA
         if (i > 0) {
           // the softmax threads have read the previous item's dQ out of tensor memory
           ok = mbar_wait(&sm.dq_free, (i - 1) & 1, abort_flag);
@@ -441,28 +449,34 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           ok = mbar_wait(&sm.kc_full[s], (gt / kKcStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          if (kFp8 && !kOneCta) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
+          if (kFp8 && !kWhole) sf_copy_elect(tmem + kColSFKc + 4 * slot, make_desc_sf(smem_u32(sm.sf_kc[s])));
           ok = mbar_wait(&sm.ds_full[buf], (kDsBufs == 2 ? gt >> 1 : gt) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8) sf_copy_elect(tmem + kColSFdS + 4 * buf, make_desc_sf(smem_u32(sm.sf_ds[buf])));
           const uint64_t desc_kc = make_desc_sw128(smem_u32(sm.kc[s]));
-          if (kOneCta) {
-            // The 192 dQ columns are two row tiles of K^c (128 + 64), one after the other through the one
-            // scale slot: copies and MMAs of one thread run in the order issued.  The step before has
-            // completed (its commit released the single dS^ buffer this step's operand came through).
+          if (kWhole) {
+            // The dQ columns are two row tiles of K^c (128 + 64, or 128 + 128), one after the other.  With a
+            // single scale slot both go through it: copies and MMAs of one thread run in the order issued,
+            // and the step before has completed (its commit released the single dS^ buffer this step's
+            // operand came through).  With 64-key steps the operand is half of the 128-byte chunk (K steps
+            // koff, koff + 1), each row tile has a scale slot of its own and the dS^ buffers alternate.
+            const int koff = kHalf ? 2 * (t & 1) : 0;
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-              if (kFp8) sf_copy_elect(tmem + kColSFKc, make_desc_sf(smem_u32(sm.sf_kc[s] + 512 * r)));
+              const uint32_t t_sfkc = tmem + kColSFKc + (kHalf ? 4 * r : 0);
+              if (kFp8) sf_copy_elect(t_sfkc, make_desc_sf(smem_u32(sm.sf_kc[s] + 512 * r)));
 #pragma unroll
-              for (int kb = 0; kb < 4; ++kb) {
+              for (int kb = 0; kb < C::kKb; ++kb) {
                 if (kFp8)
-                  mma_mxf8_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
-                                    make_idesc_mxf8(128, r == 0 ? 128 : n_dq - 128, kb, kb), tmem + kColSFdS, tmem + kColSFKc,
-                                    (t > 0 || kb > 0));
+                  mma_mxf8_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 32 * buf + 8 * kb,
+                                    desc_kc + (r * (128 * 128 / 16) + 2 * (koff + kb)),
+                                    make_idesc_mxf8(128, r == 0 ? 128 : n_dq - 128, kb, koff + kb), tmem + kColSFdS + 4 * buf,
+                                    t_sfkc, (t > 0 || kb > 0));
                 else
-                  mma_bf16_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 8 * kb, desc_kc + (r * (128 * 128 / 16) + 2 * kb),
-                                    make_idesc_bf16(128, r == 0 ? 128 : n_dq - 128), (t > 0 || kb > 0));
+                  mma_bf16_ts_elect(tmem + kColdQ + 128 * r, tmem + kColdS + 32 * buf + 8 * kb,
+                                    desc_kc + (r * (128 * 128 / 16) + 2 * kb), make_idesc_bf16(128, r == 0 ? 128 : n_dq - 128),
+                                    (t > 0 || kb > 0));
               }
             }
           } else
@@ -508,7 +522,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     }
     for (int i = 0; ok && it.valid; ++i) {
     const int qt = it.qt, r_tile = it.r_tile, n_tiles = it.n_tiles;
-    const int n_dq = kOneCta ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
+    const int n_dq = kWhole ? p.dqk : min(128, p.dqk - 128 * r_tile);   // dQ columns of this CTA
     // first key of the masked tile (the diagonal one; without the causal mask the last one, when the sequence
     // ends inside it)
     const int mask_from = p.causal ? (qt + p.q0t) * kTile : (p.kv_lim < kTile - 1 ? p.Nk - kTile : 0x7fffffff);
@@ -752,7 +766,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   if ((st = encode_tmap_u8_sw128(&tm_v, v.row_codes, s.dv * ebv, kv_rows, C::kStep)) != ATTN_OK) return st;
   if (kDQ) {
     if ((st = encode_tmap_u8_sw128(&tm_kc, k.col_codes, s.Nk * eb, static_cast<uint64_t>(s.B) * s.Hkv * s.dqk,
-                                   C::kOneCta ? C::kKcRows : (s.dqk < 128 ? s.dqk : 128))) != ATTN_OK)
+                                   C::kWhole ? C::kKcRows : (s.dqk < 128 ? s.dqk : 128))) != ATTN_OK)
       return st;
   } else {
     tm_kc = tm_k;
@@ -769,7 +783,7 @@ attn_status_t launch_qmajor_t(const AttnShape& s, attn_qtensor_t q, attn_qtensor
   const size_t smem = sizeof(QmSmem<C>) + 1024;
   cudaError_t e = cudaFuncSetAttribute(qmajor_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "bwd q-major: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  const int rq = (kDQ && !C::kOneCta) ? (s.dqk + 127) / 128 : 1;
+  const int rq = (kDQ && !C::kWhole) ? (s.dqk + 127) / 128 : 1;
   dim3 grid(s.Hq * rq, s.N / kTile, s.B);
   p.gx = static_cast<int>(grid.x); p.gy = static_cast<int>(grid.y); p.gz = static_cast<int>(grid.z);
   if (C::kPersist) {
