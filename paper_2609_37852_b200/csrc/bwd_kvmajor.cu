@@ -146,7 +146,12 @@ struct KvSmem {
   uint64_t col_full[C::kColStages], col_empty[C::kColStages];
   uint64_t lse_ready[C::kRowStages];
   uint64_t sdp_full[kTeams], sdp_free[kTeams];
+  // P^ / dS^ hand-off.  "free" barriers are per softmax team (the team that writes the buffer next waits on its
+  // own: a team takes every other sub-tile, and a parity wait on a barrier that completes once per sub-tile
+  // would pass at once for a waiter a whole phase behind).  With a single operand buffer P^ and dS^ are handed
+  // over separately (p_full / p_free for P^), so that the next P^ is written while the dK MMAs still run.
   uint64_t pds_full[2], pds_free[2];
+  uint64_t p_full, p_free[2];
   uint64_t done;
   uint64_t drain[3];
   uint32_t tmem_base;
@@ -180,6 +185,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
   constexpr bool kTight = C::kTight;
   constexpr int kOpBufs = C::kOpBufs, kSl = C::kSl;
+  constexpr bool kSplit = kOpBufs == 1;          // single operand buffer: P^ and dS^ are handed over separately
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
                      kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
                      kColSFdO = C::kColSFdO, kColSFP = C::kColSFP, kColSFdS = C::kColSFdS, kColSFdOc = C::kColSFdOc,
@@ -214,7 +220,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     }
     for (int s = 0; s < kColStages; ++s) { mbar_init(&sm.col_full[s], 1); mbar_init(&sm.col_empty[s], 1); }
     for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], kHasDk ? 2 : 1); mbar_init(&sm.sdp_free[t], kTeamThreads); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); mbar_init(&sm.p_free[i], 1); }
+    mbar_init(&sm.p_full, kTeamThreads);
     for (int i = 0; i < 3; ++i) mbar_init(&sm.drain[i], 1);
     mbar_init(&sm.done, 1);
     sm.abort_flag = 0;
@@ -418,7 +425,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             if (kHasDk) sf_copy_tiles<kRq>(tmem + kColSFQc + 4 * kRq * slot, st.sf_qc);
           }
         }
-        ok = mbar_wait(&sm.pds_full[buf], (kOpBufs == 2 ? u >> 1 : u) & 1, abort_flag);
+        // (single operand buffer: P^ comes first, dS^ is waited for ahead of the dK product)
+        ok = kSplit ? mbar_wait(&sm.p_full, u & 1, abort_flag) : mbar_wait(&sm.pds_full[buf], (kOpBufs == 2 ? u >> 1 : u) & 1, abort_flag);
         if (!ok) break;
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
@@ -440,6 +448,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           sf_copy_elect(tmem + kColSFdOc, make_desc_sf(smem_u32(st.sf_dOc)));
           issue_ts<true, 1, 1>(tmem + kColdV, tmem + kColP, make_desc_sw128(smem_u32(st.dOc)), p.dv, sub_c, tmem + kColSFP,
                                tmem + kColSFdOc, u > 0);
+          mma_commit_elect(&sm.p_free[(u + 1) & 1]);      // P^ and its scale bytes may be rewritten (by the other team)
+          ok = mbar_wait(&sm.pds_full[0], u & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
           sf_copy_elect(tmem + kColSFdS, make_desc_sf(smem_u32(sm.sf_ds[0])));
 #pragma unroll
           for (int r = 0; r < 2; ++r) {
@@ -452,13 +464,19 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (kHasDv)
           issue_ts<kFp8, kEB, kRv>(tmem + kColdV, tmem + kColP + kOpCols * buf, make_desc_sw128(smem_u32(st.dOc)), p.dv,
                                    sub_c, tmem + kColSFP + 4 * buf, tmem + kColSFdOc + 4 * kRv * slot, u > 0);
+        if (kSplit) {
+          mma_commit_elect(&sm.p_free[(u + 1) & 1]);
+          ok = mbar_wait(&sm.pds_full[0], u & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
         if (kHasDk)
           issue_ts<kFp8, kEB, kRq>(tmem + kColdK, tmem + kColdS + kOpCols * buf, make_desc_sw128(smem_u32(st.qc)), dk_cols,
                                    sub_c, tmem + kColSFdS + 4 * buf, tmem + kColSFQc + 4 * kRq * slot, u > 0);
         }
         // operands and scale bytes of this buffer may be overwritten once these MMAs have run; the
         // col stage may be refilled after its last sub-tile
-        mma_commit_elect(&sm.pds_free[buf]);
+        mma_commit_elect(&sm.pds_free[kOpBufs == 2 ? buf : ((u + 1) & 1)]);   // indexed by the team that writes next
         if (sub_c == kSubPerCol - 1) mma_commit_elect(&sm.col_empty[s]);
         if (u == n_sub - 1) mma_commit_elect(&sm.done);
       }
@@ -556,7 +574,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       }
       if (u >= kOpBufs) {
         // the dV / dK MMAs of the sub-tile that last used this buffer have consumed its operands and scale bytes
-        ok = mbar_wait(&sm.pds_free[buf], (kOpBufs == 2 ? (u - 2) >> 1 : u - 1) & 1, abort_flag);
+        // (single buffer: the dV MMAs have consumed P^; dS^ is waited for below)
+        ok = mbar_wait(kSplit ? &sm.p_free[team] : &sm.pds_free[team], ((u - kOpBufs) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
       }
@@ -578,6 +597,19 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
 #pragma unroll
         for (int i = 0; i < kEB; ++i) tmem_st8(tmem + kColP + kOpCols * buf + lane_addr + 8 * kEB * grp + 8 * i, words + 8 * i);
       }
+      if (kSplit) {
+        // hand P^ over, then wait for the dK MMAs of the sub-tile before to have consumed dS^
+        if (kFp8) sts_u8(&sm.sf_p[0][(row & 31) * 16 + (row >> 5) * 4 + grp], byte_p);
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&sm.p_full);
+        if (u >= 1) {
+          ok = mbar_wait(&sm.pds_free[team], ((u - 1) >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+      }
       if (kHasDk) {
         if (kFp8) {
           const float2 inv2 = make_float2(inv_s, inv_s);
@@ -597,7 +629,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       }
       if (kFp8) {
         const int sf_at = (row & 31) * 16 + (row >> 5) * 4 + grp;
-        if (kHasDv) sts_u8(&sm.sf_p[buf][sf_at], byte_p);
+        if (kHasDv && !kSplit) sts_u8(&sm.sf_p[buf][sf_at], byte_p);
         if (kHasDk) sts_u8(&sm.sf_ds[buf][sf_at], byte_s);
       }
       tmem_wait_st();
