@@ -76,13 +76,17 @@ struct KvCfg {
   static constexpr int kSubPerRow = kRowTok / kSub, kSubPerCol = kColTok / kSub;
   static constexpr int kKvBytes = (kCq + (kHasDk ? kCv : 0)) * kTile * 128;
   static constexpr int kRowBytes = (kCq + (kHasDk ? kCv : 0)) * kRowTok * 128;
-  static constexpr int kColBytes = ((kHasDk ? kRqAcc : 0) + (kHasDv ? kRv : 0)) * kTile * 128;
+  // (192,128) with both gradients in one pass (see kTight below): the Q^c stage holds the 192 rows it is
+  // loaded with, not two full row tiles, which leaves room for a third row stage
+  static constexpr bool kTightDims = kMode_ == kBoth && ((kEB == 1 && kEBv == 1 && kCq == 2 && kCv == 1) || (kEB == 2 && kEBv == 2 && kCq == 3 && kCv == 2));
+  static constexpr int kQcRows = kTightDims ? 192 : kRqAcc * kTile;
+  static constexpr int kColBytes = ((kHasDk ? kQcRows : 0) + (kHasDv ? kRv * kTile : 0)) * 128;
   // rings shrink to one stage where two do not fit (wide heads in BF16 mode): loads and MMAs of
   // successive steps then no longer overlap
   static constexpr int kColStages = kKvBytes + 2 * kRowBytes + 2 * kColBytes <= 210 * 1024 ? 2 : 1;
   static constexpr int kRowRaw = (216 * 1024 - kKvBytes - kColStages * kColBytes) / kRowBytes;
   static constexpr bool kTwoRowsFit = kKvBytes + kColStages * kColBytes + 2 * kRowBytes <= 214 * 1024;
-  static constexpr int kRowCap = (kEB == 1 && kEBv == 1 && kMode_ == kBoth && kCq == 2 && kCv == 1) ? 2 : 3;   // (192,128) in one pass: shared memory
+  static constexpr int kRowCap = 3;
   static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > kRowCap ? kRowCap : kRowRaw);
   // tensor memory
   // FP8 at (192, 128) with both gradients in one pass: dV 128 + dK 192 columns beside the score tiles
@@ -125,7 +129,7 @@ struct KvRowStage {
 };
 template <class C>
 struct KvColStage {
-  alignas(1024) uint8_t qc[C::kHasDk ? C::kRqAcc * kTile * 128 : 16];   // Q col copy  [dqk][queries]
+  alignas(1024) uint8_t qc[C::kHasDk ? C::kQcRows * 128 : 16];   // Q col copy  [dqk][queries]
   alignas(1024) uint8_t dOc[C::kHasDv ? C::kRv * kTile * 128 : 16];     // dO col copy [dv][queries]
   alignas(16) uint8_t sf_qc[C::kRqAcc * 512];
   alignas(16) uint8_t sf_dOc[C::kRv * 512];
