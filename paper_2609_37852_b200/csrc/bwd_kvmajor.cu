@@ -189,6 +189,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   constexpr int kSubPerRow = C::kSubPerRow, kSubPerCol = C::kSubPerCol, kOpCols = C::kOpCols;
   constexpr bool kTight = C::kTight;
   constexpr int kOpBufs = C::kOpBufs, kSl = C::kSl;
+  // 64-query row stages: LSE and D of a stage are fetched by the preparation warp with plain loads, one stage
+  // ahead, instead of two more bulk copies per stage by the producer thread (which paces the kernel there)
+  constexpr bool kPrepLoads = C::kRowTok == kSub;
   constexpr bool kSplit = kOpBufs == 1;          // single operand buffer: P^ and dS^ are handed over separately
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
                      kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
@@ -272,14 +275,14 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
           KvRowStage<C>& r = sm.rst[rs];
           mbar_arrive_expect_tx(&sm.row_full[rs], kCq * (kRowTok * 128 + (kFp8 ? 512 : 0)) +
                                                       (kHasDk ? kCv * (kRowTok * 128 + (kFp8v ? 512 : 0)) : 0) +
-                                                      (kHasDk ? 2 : 1) * kRowTok * 4);
+                                                      (kPrepLoads ? 0 : (kHasDk ? 2 : 1) * kRowTok * 4));
           for (int c = 0; c < kCq; ++c) tma_load_2d(r.q[c], &tm_q, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
           if (kFp8) bulk_load_1d(r.sf_q, p.q_sf + sf_tile * kCq * 512, kCq * 512, &sm.row_full[rs]);
-          bulk_load_1d(r.lse, p.lse + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
+          if (!kPrepLoads) bulk_load_1d(r.lse, p.lse + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
           if (kHasDk) {
             for (int c = 0; c < kCv; ++c) tma_load_2d(r.dO[c], &tm_dO, &sm.row_full[rs], 128 * c, q_slab * p.N + tok0);
             if (kFp8v) bulk_load_1d(r.sf_dO, p.dO_sf + sf_tile * kCv * 512, kCv * 512, &sm.row_full[rs]);
-            bulk_load_1d(r.delta, p.delta + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
+            if (!kPrepLoads) bulk_load_1d(r.delta, p.delta + static_cast<size_t>(q_slab) * p.N + tok0, kRowTok * 4, &sm.row_full[rs]);
           }
           ++issued_row;
         }
@@ -371,6 +374,18 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     }
     int s = 0;                                        // running (stage, phase) of the row ring
     uint32_t s_phase = 0;
+    // kPrepLoads: LSE and D of the next row stage (= sub-tile), in flight while this one is handled
+    int pf_h = g * G, pf_it = it0;                    // (head, query tile) of the stage fetched next
+    float4 pf_l = make_float4(0.f, 0.f, 0.f, 0.f), pf_d = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto prefetch = [&](int uu) {
+      if (4 * lane < kRowTok) {
+        const size_t at = static_cast<size_t>(b * p.Hq + pf_h) * p.N + pf_it * kTile + (uu & 1) * kSub + 4 * lane;
+        pf_l = *reinterpret_cast<const float4*>(p.lse + at);
+        if (kHasDk) pf_d = *reinterpret_cast<const float4*>(p.delta + at);
+      }
+      if ((uu & 1) && ++pf_it == tiles_n) { pf_it = it0; ++pf_h; }
+    };
+    if (kPrepLoads && n_sub > 0) prefetch(0);
     for (int u = 0; u < n_sub && ok; ++u) {
       const int half = u & 1, ri = u / kSubPerRow, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
       if (u > 0 && sub_r == 0 && ++s == kRowStages) { s = 0; s_phase ^= 1u; }
@@ -378,6 +393,14 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       if (sub_r == 0) {
         ok = mbar_wait(&sm.row_full[s], s_phase, abort_flag);
         if (!ok) break;
+        if (kPrepLoads) {
+          if (4 * lane < kRowTok) {
+            *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
+                make_float4(-pf_l.x * kLog2e, -pf_l.y * kLog2e, -pf_l.z * kLog2e, -pf_l.w * kLog2e);
+            if (kHasDk) *reinterpret_cast<float4*>(&st.delta[4 * lane]) = make_float4(-pf_d.x, -pf_d.y, -pf_d.z, -pf_d.w);
+          }
+          if (u + 1 < n_sub) prefetch(u + 1);
+        } else
         // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
         if (4 * lane < kRowTok) {
           const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
