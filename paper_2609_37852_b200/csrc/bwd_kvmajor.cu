@@ -191,7 +191,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   constexpr int kOpBufs = C::kOpBufs, kSl = C::kSl;
   // 64-query row stages: LSE and D of a stage are fetched by the preparation warp with plain loads, one stage
   // ahead, instead of two more bulk copies per stage by the producer thread (which paces the kernel there)
-  constexpr bool kPrepLoads = C::kRowTok == kSub;
+  // (FP8 only: in BF16 mode the producer is not what paces the kernel, and the change cost 5 % there)
+  constexpr bool kPrepLoads = kFp8 && C::kRowTok == kSub;
   constexpr bool kSplit = kOpBufs == 1;          // single operand buffer: P^ and dS^ are handed over separately
   constexpr uint32_t kColS = C::kColS, kColdP = C::kColdP, kColP = C::kColP, kColdS = C::kColdS, kColdV = C::kColdV,
                      kColdK = C::kColdK, kColSFK = C::kColSFK, kColSFV = C::kColSFV, kColSFQ = C::kColSFQ,
