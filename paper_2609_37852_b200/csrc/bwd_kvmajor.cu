@@ -88,6 +88,14 @@ struct KvCfg {
   static constexpr bool kTwoRowsFit = kKvBytes + kColStages * kColBytes + 2 * kRowBytes <= 214 * 1024;
   static constexpr int kRowCap = 3;
   static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > kRowCap ? kRowCap : kRowRaw);
+  // FP8 with 64-query row stages (one sub-tile each): -LSE*log2(e) and -D of a sub-tile live in a small ring
+  // of their own, written by the preparation warp, so that the operand part of a row stage is released as soon
+  // as the S^T / dP^T MMAs that read it have run, not when the softmax is done with the sub-tile: the reload is
+  // in flight a whole softmax step earlier.  Slot reuse is safe kRowStages + 3 sub-tiles later (the row load
+  // that precedes the rewrite waits for the MMAs of sub-tile u + 3, which are issued after the team of u has
+  // taken S of u + 2, i.e. finished u); an even count keeps each slot with one team.
+  static constexpr bool kEarly = kEB == 1 && kRowTok == kSub;
+  static constexpr int kLseSlots = kEarly ? ((kRowStages + 4) & ~1) : kRowStages;
   // tensor memory
   // FP8 at (192, 128) with both gradients in one pass: dV 128 + dK 192 columns beside the score tiles
   // fill tensor memory exactly when the P^ / dS^ operands and every scale-factor slot are single and the
@@ -148,7 +156,9 @@ struct KvSmem {
   uint64_t kv_full;
   uint64_t row_full[C::kRowStages], row_empty[C::kRowStages];
   uint64_t col_full[C::kColStages], col_empty[C::kColStages];
-  uint64_t lse_ready[C::kRowStages];
+  uint64_t lse_ready[C::kLseSlots];
+  alignas(16) float lse_ring[C::kEarly ? C::kLseSlots : 1][kSub];     // kEarly: -LSE * log2(e) of a sub-tile
+  alignas(16) float delta_ring[C::kEarly ? C::kLseSlots : 1][kSub];   // kEarly: -D
   uint64_t sdp_full[kTeams], sdp_free[kTeams];
   // P^ / dS^ hand-off.  "free" barriers are per softmax team (the team that writes the buffer next waits on its
   // own: a team takes every other sub-tile, and a parity wait on a barrier that completes once per sub-tile
@@ -223,9 +233,10 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < kRowStages; ++s) {
-      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], 1);      // released once the softmax teams are done with the rows
-      mbar_init(&sm.lse_ready[s], 1);                 // one arrival by the prep warp
+      // released once the softmax teams are done with the rows (kEarly: once the S^T and dP^T MMAs have read them)
+      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], C::kEarly ? (kHasDk ? 2 : 1) : 1);
     }
+    for (int s = 0; s < C::kLseSlots; ++s) mbar_init(&sm.lse_ready[s], 1);   // one arrival by the prep warp
     for (int s = 0; s < kColStages; ++s) { mbar_init(&sm.col_full[s], 1); mbar_init(&sm.col_empty[s], 1); }
     for (int t = 0; t < kTeams; ++t) { mbar_init(&sm.sdp_full[t], kHasDk ? 2 : 1); mbar_init(&sm.sdp_free[t], kTeamThreads); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.pds_full[i], kTeamThreads); mbar_init(&sm.pds_free[i], 1); mbar_init(&sm.p_free[i], 1); }
@@ -358,6 +369,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         issue_ss<kFp8, kCq, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColS, desc_k, desc_q, nk_qk, tmem + kColSFK, tmem + kColSFQ + 4 * kCq * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
+        if (C::kEarly) mma_commit_elect(&sm.row_empty[s]);   // the row operands of this sub-tile have been read
       }
       if (!ok) {
         int dummy = 0;
@@ -387,6 +399,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       if ((uu & 1) && ++pf_it == tiles_n) { pf_it = it0; ++pf_h; }
     };
     if (kPrepLoads && n_sub > 0) prefetch(0);
+    int ls = 0;                                       // kEarly: slot of the LSE / D ring (sub-tile u modulo its depth)
     for (int u = 0; u < n_sub && ok; ++u) {
       const int half = u & 1, ri = u / kSubPerRow, slot = kSl == 2 ? (ri & 1) : 0, sub_r = u % kSubPerRow;
       if (u > 0 && sub_r == 0 && ++s == kRowStages) { s = 0; s_phase ^= 1u; }
@@ -396,9 +409,9 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (!ok) break;
         if (kPrepLoads) {
           if (4 * lane < kRowTok) {
-            *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
+            *reinterpret_cast<float4*>(&sm.lse_ring[ls][4 * lane]) =
                 make_float4(-pf_l.x * kLog2e, -pf_l.y * kLog2e, -pf_l.z * kLog2e, -pf_l.w * kLog2e);
-            if (kHasDk) *reinterpret_cast<float4*>(&st.delta[4 * lane]) = make_float4(-pf_d.x, -pf_d.y, -pf_d.z, -pf_d.w);
+            if (kHasDk) *reinterpret_cast<float4*>(&sm.delta_ring[ls][4 * lane]) = make_float4(-pf_d.x, -pf_d.y, -pf_d.z, -pf_d.w);
           }
           if (u + 1 < n_sub) prefetch(u + 1);
         } else
@@ -412,7 +425,8 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
             *reinterpret_cast<float4*>(&st.delta[4 * lane]) = make_float4(-d.x, -d.y, -d.z, -d.w);
           }
         }
-        mbar_arrive_warp(&sm.lse_ready[s]);
+        mbar_arrive_warp(&sm.lse_ready[kPrepLoads ? ls : s]);
+        if (++ls == C::kLseSlots) ls = 0;
         if (kFp8v && kHasDk && kSl == 2) {
           tc_fence_after_sync();
           sf_copy_tiles<kCv>(tmem + kColSFdO + 4 * kCv * slot, st.sf_dO);
@@ -429,6 +443,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         issue_ss<kFp8v, kCv, kSub, kTile * 128 / 16, kRowTok * 128 / 16>(
             tmem + kColdP, desc_v, desc_dO, nk_v, tmem + kColSFV, tmem + kColSFdO + 4 * kCv * slot + 2 * half);
         mma_commit_elect(&sm.sdp_full[u % kTeams]);
+        if (C::kEarly) mma_commit_elect(&sm.row_empty[s]);
       }
     }
     if (!ok && kHasDk) {
@@ -458,7 +473,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         if (!ok) break;
         // all queries of a row stage have been through the softmax: the stage (score operands,
         // LSE, D) is no longer read
-        if (u % kSubPerRow == kSubPerRow - 1) {
+        if (!C::kEarly && u % kSubPerRow == kSubPerRow - 1) {
           if (lane == 0) mbar_arrive(&sm.row_empty[rs_done]);
           if (++rs_done == kRowStages) rs_done = 0;
         }
@@ -528,12 +543,15 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     // it advances by kTeams / kSubPerRow stages per iteration
     int s = (team / kSubPerRow) % kRowStages;
     uint32_t s_phase = ((team / kSubPerRow) / kRowStages) & 1;
+    int ls = team;                                    // kEarly: running (slot, phase) of the LSE / D ring
+    uint32_t ls_phase = 0;
     for (int u = team; u < n_sub; u += kTeams) {
       const int half = u & 1, buf = kOpBufs == 2 ? (u & 1) : 0;
       if (u != team) {
 #pragma unroll
         for (int a = 0; a < kTeams / kSubPerRow; ++a)
           if (++s == kRowStages) { s = 0; s_phase ^= 1u; }
+        if ((ls += kTeams) >= C::kLseSlots) { ls -= C::kLseSlots; ls_phase ^= 1u; }
       }
       ok = mbar_wait(&sm.sdp_full[team], (u / kTeams) & 1, abort_flag);
       if (!ok) break;
@@ -544,14 +562,14 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(&sm.sdp_free[team]);
-      ok = mbar_wait(&sm.lse_ready[s], s_phase, abort_flag);
+      ok = C::kEarly ? mbar_wait(&sm.lse_ready[ls], ls_phase, abort_flag) : mbar_wait(&sm.lse_ready[s], s_phase, abort_flag);
       if (!ok) break;
       const int col0 = half * kSub + 32 * grp;        // query row (inside the tile) of this thread's first column
       const int st0 = (u % kSubPerRow) * kSub + 32 * grp;   // the same inside the row stage
       const KvRowStage<C>& st = sm.rst[s];
       float amax_p = 0.f, max_s = 0.f;
-      const float* s_lse = &st.neg_lse2[st0];
-      const float* s_delta = &st.delta[st0];
+      const float* s_lse = C::kEarly ? &sm.lse_ring[ls][32 * grp] : &st.neg_lse2[st0];
+      const float* s_delta = C::kEarly ? &sm.delta_ring[ls][32 * grp] : &st.delta[st0];
       // two elements per instruction (fma / mul .f32x2) wherever the arithmetic allows: the loop is
       // bound by instruction issue, not by a pipe
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
