@@ -88,13 +88,17 @@ struct KvCfg {
   static constexpr bool kTwoRowsFit = kKvBytes + kColStages * kColBytes + 2 * kRowBytes <= 214 * 1024;
   static constexpr int kRowCap = 3;
   static constexpr int kRowStages = kRowRaw < 2 ? (kTwoRowsFit ? 2 : 1) : (kRowRaw > kRowCap ? kRowCap : kRowRaw);
-  // FP8 with 64-query row stages (one sub-tile each): -LSE*log2(e) and -D of a sub-tile live in a small ring
+  // 64-query row stages (one sub-tile each): -LSE*log2(e) and -D of a sub-tile live in a small ring
   // of their own, written by the preparation warp, so that the operand part of a row stage is released as soon
   // as the S^T / dP^T MMAs that read it have run, not when the softmax is done with the sub-tile: the reload is
   // in flight a whole softmax step earlier.  Slot reuse is safe kRowStages + 3 sub-tiles later (the row load
   // that precedes the rewrite waits for the MMAs of sub-tile u + 3, which are issued after the team of u has
   // taken S of u + 2, i.e. finished u); an even count keeps each slot with one team.
-  static constexpr bool kEarly = kEB == 1 && kRowTok == kSub;
+  // (not at (192,128) in BF16 mode, one pass: a single column stage paces that kernel and the change cost 5 %)
+  static constexpr bool kEarly = kRowTok == kSub && !(kEB == 2 && kTightDims);
+  // arrivals that release a row stage: the commits behind the S^T and dP^T MMAs; without dP^T, in BF16 mode
+  // (LSE arrives in the stage by a bulk copy), the preparation warp once it has read LSE out of the stage
+  static constexpr int kRowReleases = !kEarly ? 1 : (kHasDk ? 2 : (kEB == 1 ? 1 : 2));
   static constexpr int kLseSlots = kEarly ? ((kRowStages + 4) & ~1) : kRowStages;
   // tensor memory
   // FP8 at (192, 128) with both gradients in one pass: dV 128 + dK 192 columns beside the score tiles
@@ -234,7 +238,7 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < kRowStages; ++s) {
       // released once the softmax teams are done with the rows (kEarly: once the S^T and dP^T MMAs have read them)
-      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], C::kEarly ? (kHasDk ? 2 : 1) : 1);
+      mbar_init(&sm.row_full[s], 1); mbar_init(&sm.row_empty[s], C::kRowReleases);
     }
     for (int s = 0; s < C::kLseSlots; ++s) mbar_init(&sm.lse_ready[s], 1);   // one arrival by the prep warp
     for (int s = 0; s < kColStages; ++s) { mbar_init(&sm.col_full[s], 1); mbar_init(&sm.col_empty[s], 1); }
@@ -418,14 +422,15 @@ kvmajor_kernel(const KvParams p, const __grid_constant__ CUtensorMap tm_k, const
         // every lane turns four LSE values into -LSE*log2(e) for the softmax teams
         if (4 * lane < kRowTok) {
           const float4 l = *reinterpret_cast<const float4*>(&st.lse[4 * lane]);
-          *reinterpret_cast<float4*>(&st.neg_lse2[4 * lane]) =
+          *reinterpret_cast<float4*>(C::kEarly ? &sm.lse_ring[ls][4 * lane] : &st.neg_lse2[4 * lane]) =
               make_float4(-l.x * kLog2e, -l.y * kLog2e, -l.z * kLog2e, -l.w * kLog2e);
-          if (kHasDk) {                                 // and the row correction into its negative, in place
+          if (kHasDk) {                                 // and the row correction into its negative (in place, or into the ring)
             const float4 d = *reinterpret_cast<const float4*>(&st.delta[4 * lane]);
-            *reinterpret_cast<float4*>(&st.delta[4 * lane]) = make_float4(-d.x, -d.y, -d.z, -d.w);
+            *reinterpret_cast<float4*>(C::kEarly ? &sm.delta_ring[ls][4 * lane] : &st.delta[4 * lane]) = make_float4(-d.x, -d.y, -d.z, -d.w);
           }
         }
-        mbar_arrive_warp(&sm.lse_ready[kPrepLoads ? ls : s]);
+        if (C::kEarly && !kPrepLoads && !kHasDk) mbar_arrive_warp(&sm.row_empty[s]);   // LSE has been read out of the stage
+        mbar_arrive_warp(&sm.lse_ready[C::kEarly ? ls : s]);
         if (++ls == C::kLseSlots) ls = 0;
         if (kFp8v && kHasDk && kSl == 2) {
           tc_fence_after_sync();
