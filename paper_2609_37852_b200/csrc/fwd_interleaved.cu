@@ -58,7 +58,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
 template <int kWG_, int kSW_, int kSplit_, int kCq_ = 1>
 struct IlCfg {
   static constexpr int kCq = kCq_;                      // 128-byte chunks per Q / K row (2: qk head dim 192)
-  static constexpr int kStages = kCq == 1 ? 4 : 2;      // K ring and V ring depth (what shared memory holds)
+  // Ring depths (what shared memory holds).  A V stage is held from its copy until the P V product of its tile,
+  // about two steps after the score product that frees the K stage of the same tile, so the V ring is the one
+  // that needs the depth: at qk head dim 192, two K stages and four V stages (0.278 -> 0.224 ms on mla8k against
+  // two and two, where every third step waited a step's time for V).
+  static constexpr int kStages = kCq == 1 ? 4 : 2;      // K ring depth
+  static constexpr int kVStages = 4;                    // V ring depth
   static constexpr int kWG = kWG_;                      // softmax teams == score buffers in flight
   static constexpr int kSW = kSW_;                      // keys per step (64 or 128)
   static constexpr int kSplit = kSplit_;                // threads per query row and step (each takes kSW / kSplit keys)
@@ -92,10 +97,10 @@ struct IlSmem {
   static constexpr int kStages = C::kStages;
   alignas(1024) uint8_t q[2][C::kCq][kTile * 128];
   alignas(1024) uint8_t k[kStages][C::kCq][kTile * 128];
-  alignas(1024) uint8_t v[kStages][kTile * 128];
+  alignas(1024) uint8_t v[C::kVStages][kTile * 128];
   alignas(16) uint8_t sf_q[2][C::kCq * 512];
   alignas(16) uint8_t sf_k[kStages][C::kCq * 512];
-  alignas(16) uint8_t sf_v[kStages][512];
+  alignas(16) uint8_t sf_v[C::kVStages][512];
   alignas(16) uint8_t sf_p[C::kWG][512];
   alignas(16) uint32_t raw_sf[C::kWG][C::kSplit][kTile];    // scale bytes of a step relative to the softmax thread's shift
   alignas(16) float step_m[C::kWG][C::kSplit][kTile];       // that shift
@@ -103,7 +108,7 @@ struct IlSmem {
   alignas(16) float fin_m[4][C::kWG * C::kSplit][kTile];    // number), and the shifts they are expressed in
   uint64_t q_full[2], q_empty[2];
   uint64_t k_full[kStages], k_empty[kStages];
-  uint64_t v_full[kStages], v_empty[kStages];
+  uint64_t v_full[C::kVStages], v_empty[C::kVStages];
   uint64_t s_full[C::kWG], s_free[C::kWG];
   uint64_t p_ready[C::kWG], p_full[C::kWG], p_free[C::kWG];
   uint64_t o_done, o_free;
@@ -167,16 +172,14 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
     it.n_steps = it.n_tiles * kSubPerTile;
     return it;
   };
-  constexpr int kStages = C::kStages, kCq = C::kCq;
+  constexpr int kStages = C::kStages, kVStages = C::kVStages, kCq = C::kCq;
   const int nk_qk = p.dqk / 32;                 // 32-byte K steps of the score MMA
   volatile int* abort_flag = &sm.abort_flag;
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.q_full[i], 1); mbar_init(&sm.q_empty[i], 1); }
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
-      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
-    }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kVStages; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
     for (int w = 0; w < kWG; ++w) {
       // every thread arrives for itself (one elected arrival per warp behind a warp barrier measured slower)
       mbar_init(&sm.s_full[w], 1); mbar_init(&sm.s_free[w], 128 * kSplit);
@@ -230,11 +233,12 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
             bulk_load_1d(sm.sf_k[s], p.k_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * kCq * 512, kCq * 512,
                          &sm.k_full[s]);
             ++issued_k;
-            ok = mbar_wait(&sm.v_empty[s], (r & 1) ^ 1, abort_flag);
+            const int sv = gt % kVStages, rv = gt / kVStages;
+            ok = mbar_wait(&sm.v_empty[sv], (rv & 1) ^ 1, abort_flag);
             if (!ok) break;
-            mbar_arrive_expect_tx(&sm.v_full[s], p.dv * 128 + 512);
-            tma_load_2d(sm.v[s], &tm_v, &sm.v_full[s], t * 128, kv_slab * p.dv);
-            bulk_load_1d(sm.sf_v[s], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * 512, 512, &sm.v_full[s]);
+            mbar_arrive_expect_tx(&sm.v_full[sv], p.dv * 128 + 512);
+            tma_load_2d(sm.v[sv], &tm_v, &sm.v_full[sv], t * 128, kv_slab * p.dv);
+            bulk_load_1d(sm.sf_v[sv], p.v_sf + (static_cast<size_t>(kv_slab) * tiles_nk + t) * 512, 512, &sm.v_full[sv]);
             ++issued_v;
           }
           T += it.n_tiles;
@@ -244,8 +248,8 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
           int dummy = 0;
           for (int t = max(0, issued_k - kStages); t < issued_k; ++t)
             mbar_wait(&sm.k_full[t % kStages], (t / kStages) & 1, &dummy);
-          for (int t = max(0, issued_v - kStages); t < issued_v; ++t)
-            mbar_wait(&sm.v_full[t % kStages], (t / kStages) & 1, &dummy);
+          for (int t = max(0, issued_v - kVStages); t < issued_v; ++t)
+            mbar_wait(&sm.v_full[t % kVStages], (t / kVStages) & 1, &dummy);
         }
       }
     } else if (warp == 1) {
@@ -302,9 +306,9 @@ fwd_il_kernel(const IlParams p, const __grid_constant__ CUtensorMap tm_q, const 
         if (!it.valid) break;
         for (int u = 0; u < it.n_steps && ok; ++u) {
           const int gu = G + u, gt = T + u / kSubPerTile;
-          const int sub = u % kSubPerTile, s = gt % kStages, slot = gt & 1, w = gu % kWG;
+          const int sub = u % kSubPerTile, s = gt % kVStages, slot = gt & 1, w = gu % kWG;
           if (sub == 0) {
-            ok = mbar_wait(&sm.v_full[s], (gt / kStages) & 1, abort_flag);
+            ok = mbar_wait(&sm.v_full[s], (gt / kVStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
             sf_copy_tiles<1>(tmem + kColSFV + 4 * slot, sm.sf_v[s]);
