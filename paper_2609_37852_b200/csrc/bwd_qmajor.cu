@@ -101,8 +101,14 @@ struct QmCfg {
   static constexpr int kStages = kRaw < 2 ? (kTwoFit ? 2 : 1) : (kRaw > 4 ? 4 : kRaw);
   static constexpr int kKcStages = !kDQ ? 1 : (kRaw < 2 ? 1 : kStages);
   // tensor memory
-  static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = 2 * kStep /* kDsBufs x 32 */, kColdQ = 2 * kStep + 32 * kDsBufs;
-  static constexpr uint32_t kColSFQ = kDQ ? kColdQ + kDqCols : 2 * kStep;   // kQBufs slots (no dS^ / dQ columns without dQ)
+  // BF16 mode has no scale-factor columns and 64-key steps: a second S / dP pair fits, so the products of the
+  // next step are issued while the softmax threads still work on this one (with one pair the 8 MMAs of a 64-key
+  // step, their completion, the wake-up, the load and the release ran one after the other: 1175 cycles a step in
+  // the correction pass at head dim 128, 0.683 -> 0.598 ms on the 8K workload; the wide head dims gain nothing)
+  static constexpr int kSBufs = (kEB == 2 && kEBv == 2 && kCq == 2 && kCv == 2) ? 2 : 1;
+  static constexpr uint32_t kSdp = 2 * kStep;           // columns of an S / dP pair
+  static constexpr uint32_t kColS = 0, kColdP = kStep, kColdS = kSdp * kSBufs /* kDsBufs x 32 */, kColdQ = kColdS + 32 * kDsBufs;
+  static constexpr uint32_t kColSFQ = kDQ ? kColdQ + kDqCols : kSdp * kSBufs;   // kQBufs slots (no dS^ / dQ columns without dQ)
   static constexpr uint32_t kColSFdO = kColSFQ + 4 * kCq * kQBufs;   // kQBufs slots
   static constexpr uint32_t kColSFK = kColSFdO + 4 * kCv * kQBufs;   // kSfSlots slots
   static constexpr uint32_t kColSFV = kColSFK + 4 * kSfSlots * kCq;
@@ -131,7 +137,7 @@ struct QmSmem {
   uint64_t q_full[C::kQBufs], q_empty[C::kQBufs];
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t kc_full[C::kKcStages], kc_empty[C::kKcStages];
-  uint64_t sdp_full, sdp_free;
+  uint64_t sdp_full[2], sdp_free[2];   // per S / dP pair
   uint64_t ds_full[2], ds_free[2];
   uint64_t dq_done, dq_free;
   uint64_t item_full[4];        // ticket mode: the producer has published the CTA's i-th work item in item_l[i % 4]
@@ -188,6 +194,8 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
   // the heavier item of every round.  In ticket mode the producer thread draws item numbers from a
   // global counter and publishes them to the other warps through shared memory.
   constexpr bool kOneCta = C::kOneCta, kHalf = C::kHalf, kWhole = C::kWhole;
+  constexpr int kSBufs = C::kSBufs;
+  constexpr uint32_t kSdp = C::kSdp;
   constexpr int kDsBufs = C::kDsBufs, kSfSlots = C::kSfSlots;
   const int rq_sf = (p.dqk + 127) / 128;                   // 128-row tiles of the K^c scale tensor
   const int rq = (kDQ && !kWhole) ? rq_sf : 1;            // dQ column tiles (128 wide) of one head, neighbours in x
@@ -231,7 +239,7 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
       mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 2);   // released by the S and the dP issuer
     }
     for (int s = 0; s < kKcStages; ++s) { mbar_init(&sm.kc_full[s], 1); mbar_init(&sm.kc_empty[s], 1); }
-    mbar_init(&sm.sdp_full, 2); mbar_init(&sm.sdp_free, kSoftmaxThreads);
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.sdp_full[i], 2); mbar_init(&sm.sdp_free[i], kSoftmaxThreads); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.ds_full[i], kSoftmaxThreads); mbar_init(&sm.ds_free[i], 1); }
     mbar_init(&sm.dq_done, 1); mbar_init(&sm.dq_free, kSoftmaxThreads);
     for (int i = 0; i < 4; ++i) mbar_init(&sm.item_full[i], 1);
@@ -357,18 +365,19 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8 && kSfSlots == 2) sf_copy_tiles<kCq>(tmem + kColSFK + 4 * kCq * slot, sm.sf_k[s]);
-          if (gt > 0) {
-            // the softmax threads have pulled the previous S and dP into registers
-            ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
+          const int sb = kSBufs == 2 ? (gt & 1) : 0;   // S / dP pair of this step
+          if (gt >= kSBufs) {
+            // the softmax threads have pulled the S and dP that last used this pair into registers
+            ok = mbar_wait(&sm.sdp_free[sb], (kSBufs == 2 ? (gt >> 1) - 1 : gt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
           // a single scale slot is rewritten only now that the product that read it has been consumed
           if (kFp8 && kSfSlots == 1) sf_copy_tiles<kCq>(tmem + kColSFK, sm.sf_k[s]);
           const uint64_t desc_k = make_desc_sw128(smem_u32(sm.k[s][0]));
-          issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS, desc_q, desc_k, nk_qk, t_sfq,
+          issue_ss<kFp8, kCq, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColS + kSdp * sb, desc_q, desc_k, nk_qk, t_sfq,
                                                                           tmem + kColSFK + 4 * kCq * slot + (kHalf ? 2 * (t & 1) : 0));
-          mma_commit_elect(&sm.sdp_full);
+          mma_commit_elect(&sm.sdp_full[sb]);
           mma_commit_elect(&sm.kv_empty[s]);
         }
         if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's Q tile has been read
@@ -405,16 +414,17 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
           if (!ok) break;
           tc_fence_after_sync();
           if (kFp8v && kSfSlots == 2) sf_copy_tiles<kCv>(tmem + kColSFV + 4 * kCv * slot, sm.sf_v[s]);
-          if (gt > 0) {
-            ok = mbar_wait(&sm.sdp_free, (gt - 1) & 1, abort_flag);
+          const int sb = kSBufs == 2 ? (gt & 1) : 0;
+          if (gt >= kSBufs) {
+            ok = mbar_wait(&sm.sdp_free[sb], (kSBufs == 2 ? (gt >> 1) - 1 : gt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
           }
           if (kFp8v && kSfSlots == 1) sf_copy_tiles<kCv>(tmem + kColSFV, sm.sf_v[s]);
           const uint64_t desc_v = make_desc_sw128(smem_u32(sm.v[s][0]));
-          issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP, desc_dO, desc_v, nk_v, t_sfdO,
+          issue_ss<kFp8v, kCv, kStep, kTile * 128 / 16, kStep * 128 / 16>(tmem + kColdP + kSdp * sb, desc_dO, desc_v, nk_v, t_sfdO,
                                                                           tmem + kColSFV + 4 * kCv * slot + (kHalf ? 2 * (t & 1) : 0));
-          mma_commit_elect(&sm.sdp_full);
+          mma_commit_elect(&sm.sdp_full[sb]);
           mma_commit_elect(&sm.kv_empty[s]);
         }
         if (kPersist && ok) mma_commit_elect(&sm.q_empty[qb]);     // this item's dO tile has been read
@@ -551,15 +561,16 @@ qmajor_kernel(const QmParams p, const __grid_constant__ CUtensorMap tm_q, const 
     for (int t = 0; t < n_tiles; ++t) {
       const int gt = T + t;                           // step index over all items: the dS^ buffers run on
       const int buf = kDsBufs == 2 ? (gt & 1) : 0;
-      ok = mbar_wait(&sm.sdp_full, gt & 1, abort_flag);
+      const int sb = kSBufs == 2 ? (gt & 1) : 0;
+      ok = mbar_wait(&sm.sdp_full[sb], (kSBufs == 2 ? gt >> 1 : gt) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
       uint32_t sr[32], dpr[32];
-      tmem_ld32(tmem + kColS + lane_addr + 32 * grp, sr);
-      tmem_ld32(tmem + kColdP + lane_addr + 32 * grp, dpr);
+      tmem_ld32(tmem + kColS + kSdp * sb + lane_addr + 32 * grp, sr);
+      tmem_ld32(tmem + kColdP + kSdp * sb + lane_addr + 32 * grp, dpr);
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(&sm.sdp_free);
+      mbar_arrive(&sm.sdp_free[sb]);
       // column, inside the query tile's own key range, of this thread's first element (negative
       // before the diagonal tile)
       // (without the causal mask: inside the last key tile, where a ragged sequence ends)
